@@ -1,0 +1,86 @@
+"""Pins for the oracle's pack (no GPU): a slow per-row search in pure Python on tiny inputs, and
+the properties that hold at any size."""
+import numpy as np
+import pytest
+
+from workloads import SchedParams, complete_catalog, tree_topology
+from workloads.demand import demand_from_routing, moe_routing
+
+import torch
+
+
+def _case(oracle_lib, T, topk, E, hidden, seed, rank, drop=False):
+    cat = complete_catalog(tree_topology(1))
+    oc = oracle_lib.OracleCatalog(cat.topology.blob(), cat.blob())
+    N = oc.N
+    row_bytes = hidden * 2
+    idx = moe_routing(T * N, E, topk, 1.2, seed)
+    src = torch.repeat_interleave(torch.arange(N), T)
+    D = demand_from_routing(idx, src, N, E, row_bytes).numpy()
+    mine = idx[rank * T:(rank + 1) * T].numpy().copy()
+    if drop:                                   # dropped copies (negative ids) are not part of the demand
+        mine[::3, 0] = -1
+        D[rank] = 0
+        for t in range(T):
+            for s in range(topk):
+                if mine[t, s] >= 0 and mine[t, s] // (E // N) != rank:
+                    D[rank, mine[t, s] // (E // N)] += row_bytes
+    plan = oc.schedule(D, SchedParams(granule_bytes=row_bytes).resolved(N))
+    assert plan["status"] == 0
+    rows = np.random.default_rng(seed).integers(0, 65536, size=(T, hidden), dtype=np.uint16)
+    return oc, plan, mine, rows, D, row_bytes, E // N
+
+
+@pytest.mark.parametrize("rank,drop", [(0, False), (5, False), (3, True)])
+def test_pack_matches_per_row_search(oracle_lib, rank, drop):
+    oc, plan, idx, rows, D, row_bytes, epr = _case(oracle_lib, T=37, topk=4, E=32, hidden=24, seed=7,
+                                                   rank=rank, drop=drop)
+    R = int(D[rank].sum() // row_bytes)
+    staged, src_map, st = oc.pack(plan, rank, idx, epr, rows, R)
+    assert st == 0
+    T, topk = idx.shape
+    # slow definition: staged row r belongs to the step whose [send_off[k], send_off[k+1]) holds it;
+    # it is the p-th row of that step, i.e. the (rows sent to that destination in earlier steps + p)-th
+    # copy, in ascending (token, slot), among the copies routed to the step's destination.
+    for r in range(R):
+        k = max(kk for kk in range(int(plan["n_steps"])) if plan["send_off"][kk][rank] <= r * row_bytes
+                and plan["lane_dst"][kk][rank] >= 0 and plan["send_off"][kk][rank] < plan["send_off"][kk + 1][rank])
+        j = int(plan["lane_dst"][k][rank])
+        earlier = sum(int(plan["lane_bytes"][kk][rank]) // row_bytes for kk in range(k)
+                      if plan["lane_dst"][kk][rank] == j)
+        p = r - int(plan["send_off"][k][rank]) // row_bytes
+        copies = [(t, s) for t in range(T) for s in range(topk)
+                  if idx[t, s] >= 0 and idx[t, s] // epr == j]
+        t, s = copies[earlier + p]
+        assert src_map[r] == t * topk + s
+        assert (staged[r].view(np.uint16) == rows[t]).all()
+
+
+def test_pack_properties(oracle_lib):
+    oc, plan, idx, rows, D, row_bytes, epr = _case(oracle_lib, T=400, topk=8, E=64, hidden=16, seed=3, rank=2)
+    rank = 2
+    R = int(D[rank].sum() // row_bytes)
+    staged, src_map, st = oc.pack(plan, rank, idx, epr, rows, R + 5)
+    assert st == 0
+    topk = idx.shape[1]
+    remote = sorted(e for e in range(idx.size) if idx.flat[e] // epr != rank)
+    assert sorted(src_map[:R].tolist()) == remote            # a permutation of the remote copies
+    assert (src_map[R:] == -1).all() and not staged[R:].any()  # nothing beyond the plan's bytes
+    for k in range(int(plan["n_steps"])):
+        lo, hi = (int(plan["send_off"][k + x][rank]) // row_bytes for x in (0, 1))
+        chunk = src_map[lo:hi]
+        assert (np.diff(chunk) > 0).all()                     # ascending (token, slot) inside a step
+        if hi > lo:
+            assert (idx.flat[chunk] // epr == plan["lane_dst"][k][rank]).all()
+    assert (staged[:R].view(np.uint16) == rows[src_map[:R] // topk]).all()
+
+
+def test_pack_error_statuses(oracle_lib):
+    oracle = oracle_lib
+    oc, plan, idx, rows, D, row_bytes, epr = _case(oracle_lib, T=50, topk=4, E=32, hidden=8, seed=9, rank=1)
+    R = int(D[1].sum() // row_bytes)
+    assert oc.pack(plan, 1, idx, epr, rows, R - 1)[2] == oracle.ST_PACK_CAPACITY
+    other = idx.copy()
+    other[0, 0] = (other[0, 0] + epr) % 32                    # routing no longer matches the plan
+    assert oc.pack(plan, 1, other, epr, rows, R)[2] & oracle.ST_PACK_MISMATCH
+    assert oc.pack(plan, 1, idx, epr, rows, R)[2] == 0
