@@ -1,0 +1,223 @@
+/*
+ * variopath.h - C ABI of the B200 (sm_100a) VarioPath online scheduler and
+ * send-buffer pack.
+ *
+ * The library implements the demand-dependent half of the method: for every
+ * AlltoAllv invocation, decompose the N x N integer demand matrix over an
+ * offline catalog of contention-free channel families into a sequence of
+ * channel activations (Algorithm 2, Section 4.2), and lay one rank's token rows
+ * out in the send buffer in activation x destination order (Section 5,
+ * "Device-resident buffer layout").  Everything runs in CUDA kernels on one
+ * GPU; there is no CPU fallback.
+ *
+ * Conventions
+ *  - Every call returns 0 (VP_OK) or a negative VP_E_* code; nothing throws,
+ *    traps or aborts.  Per-matrix problems are reported as bit flags in
+ *    status[b] (VP_ST_*), never by faulting.
+ *  - "device" pointers are plain CUDA global-memory addresses on the
+ *    catalog's device, owned by the caller; "host" pointers are ordinary host
+ *    memory.  The library allocates device memory only in vp_load_catalog; all
+ *    scratch is passed in by the caller (see the *_workspace_bytes calls).
+ *  - Kernels are enqueued on the caller's stream (a cudaStream_t passed as
+ *    void*; NULL = the default stream) and the device-pointer calls return
+ *    without synchronising.
+ *  - Ranks of group a are a*g .. a*g+g-1 (Section 4.1: N = G*g switch-local
+ *    groups).  All volumes are bytes held in int64.
+ *  - Results are deterministic: the same inputs give the same bytes whatever
+ *    the batch size or launch geometry.
+ */
+#ifndef VARIOPATH_H
+#define VARIOPATH_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* ---- return codes ------------------------------------------------------ */
+#define VP_OK               0
+#define VP_E_BAD_ARG      (-1)  /* NULL pointer, non-positive size, parameter out of range      */
+#define VP_E_BAD_CATALOG  (-2)  /* blob truncated / malformed, or violates Eq. (3) / Eq. (4)      */
+#define VP_E_NOMEM        (-3)  /* host or device allocation failed in vp_load_catalog            */
+#define VP_E_CUDA         (-4)  /* a CUDA runtime call failed; the extension may be unusable      */
+#define VP_E_WORKSPACE    (-5)  /* workspace NULL, misaligned (256 B) or smaller than required    */
+#define VP_E_UNSUPPORTED  (-6)  /* group size > 4, N > 256, more than 8 distinct path rates ...   */
+
+/* ---- per-matrix status bits (status[b]); 0 = a complete valid schedule ---- */
+#define VP_ST_NEGATIVE        1   /* some D_ij < 0                                               */
+#define VP_ST_OVERFLOW_RISK   2   /* some D_ij >= 2^40                                           */
+#define VP_ST_DIAG_NONZERO    4   /* some D_ii != 0 (Section 3: self traffic is omitted)          */
+#define VP_ST_NOT_GRANULE     8   /* some D_ij not a multiple of granule_bytes                    */
+#define VP_ST_BAD_TAU        16   /* tau_ns_in[b] < 0 or > 2^40                                   */
+#define VP_ST_UNCOVERED      32   /* residual demand left but every shape scores 0 (Eq. 6)        */
+#define VP_ST_NO_PROGRESS    64   /* best candidate carries 0 bytes (only if n_start < g)         */
+#define VP_ST_STEP_LIMIT    128   /* k_max activations emitted, residual demand left              */
+#define VP_ST_PACK_MISMATCH 256   /* vp_pack: routed copies disagree with the plan's byte counts  */
+#define VP_ST_PACK_CAPACITY 512   /* vp_pack: staged buffer smaller than the plan's send volume   */
+/* Bits 1..16 reject the matrix before scheduling: n_steps[b] = 0 and an empty plan. */
+
+typedef struct vp_catalog vp_catalog;   /* opaque, owned by the library */
+
+typedef struct vp_info {
+    int32_t N, G, g;              /* ranks, groups, ranks per group                              */
+    int32_t groups_per_node;
+    int32_t n_resources;          /* directed shared resources (the set U of Section 3)           */
+    int32_t n_instances;          /* group-level path instances                                   */
+    int32_t n_shapes, n_families; /* catalog size (Table 3 columns)                               */
+    int32_t max_nnz;              /* largest number of non-zero group pairs of a shape            */
+    int32_t max_bucket;           /* largest number of families realising one shape               */
+    int32_t covered;              /* 1 if every group pair that can carry demand is in some shape */
+    int32_t node_symmetric;       /* 1 if every shape is invariant under a shift of the node index:
+                                     Eq. (6) is then evaluated on per-node-offset sums of D-hat   */
+    int64_t rate_lcm;             /* lcm of all path rates (utilities are compared exactly)       */
+} vp_info;
+
+/*
+ * Scheduler parameters (Algorithm 2 "Require": tau, lambda, N_start, I_AA;
+ * Section 5 "Global execution granularity": K_target).
+ */
+typedef struct vp_sched_params {
+    int64_t lambda_ns;      /* per-activation overhead of Eq. (2)/(10), 0 <= lambda < 2^40        */
+    int64_t granule_bytes;  /* every D_ij must be a multiple; lane capacities are rounded down to
+                               it (at least one granule).  Use the row size when packing.  >= 1   */
+    int32_t k_target;       /* target round count, 0 -> 2N                                        */
+    int32_t n_start;        /* AA starts, 0 -> g; start t rotates every group's in-slots by t      */
+    int32_t i_aa;           /* AA sweep limit, 0 -> 3                                             */
+    int32_t k_max;          /* capacity of the plan arrays in activations, > 0                    */
+} vp_sched_params;
+
+/*
+ * vp_load_catalog - parse, validate and upload a topology + channel catalog
+ * (Section 4.1: rank groups, path instances, shapes, families, buckets).
+ *
+ * topology, channels: host, little-endian blobs.
+ *   topology: u32 magic 'VPTP', u32 version(1), u32 N, u32 G, u32 g,
+ *     u32 groups_per_node, u32 n_resources, u32 n_instances; then per instance
+ *     20 bytes: u16 src_group, u16 dst_group, u8 kind, u8 n_res (<=4), u16 mult
+ *     (lanes of one family that may share it), u32 bw (bytes/ns), u16 res[4].
+ *     Instance id = position; ids must be sorted by (src_group, dst_group).
+ *   channels: u32 magic 'VPCH', u32 version(1), u32 N, u32 n_shapes,
+ *     u32 n_families, u32 total_nnz; u32 shape_ptr[n_shapes+1]; total_nnz x
+ *     {u16 a, u16 d, u16 count, u16 pad}; u32 bucket_ptr[n_shapes+1] (families
+ *     of shape s are ids bucket_ptr[s]..bucket_ptr[s+1]-1, in tie-break order);
+ *     u16 fam_inst[n_families][N] ascending instance ids.
+ * Rejected with VP_E_BAD_CATALOG: a shape whose row or column sums differ from
+ * g (Eq. 3); a family that does not select exactly M_ad instances per group
+ * pair, repeats an instance beyond mult, or uses a directed resource twice
+ * (Eq. 4).  A catalog that leaves a group pair uncovered loads (info.covered
+ * = 0); demand on that pair ends with VP_ST_UNCOVERED.
+ * device: CUDA device ordinal that will hold the image.  *out receives the
+ * handle, to be released with vp_free_catalog.  Synchronous.
+ */
+int vp_load_catalog(const void* topology, size_t topology_bytes,
+                    const void* channels, size_t channels_bytes,
+                    int device, vp_catalog** out);
+void vp_free_catalog(vp_catalog* catalog);
+int vp_catalog_info(const vp_catalog* catalog, vp_info* out);
+
+/* Bytes of device scratch vp_schedule_batch needs for a batch of B (multiple of 256). */
+size_t vp_schedule_workspace_bytes(const vp_catalog* catalog, int B, const vp_sched_params* params);
+
+/*
+ * vp_schedule_batch - Algorithm 2 for B independent demand matrices.
+ *
+ * Per matrix: tau from K_target unless given; D_rem <- D; repeat { group sums
+ * (Eq. 5); first shape of maximal score (Eq. 6); for every family of its bucket
+ * MultiStartAA endpoint binding (Eq. 7, 8) and Evaluate (Eq. 9, 10); emit the
+ * first family of maximal utility; D_rem -= X(E) } until D_rem = 0; then
+ * exclusive prefix sums of the per-rank send / receive bytes over the steps.
+ *
+ * All array arguments are device pointers, row-major, caller-owned:
+ *   demand      [B][N][N] int64 bytes from rank i to rank j, zero diagonal
+ *   tau_ns_in   [B] or NULL; entries > 0 override the derived time quantum
+ *   n_steps     [B]            activations emitted
+ *   chan_id     [B][k_max]     global family index of step k, -1 beyond n_steps
+ *   lane_dst    [B][k_max][N]  destination of source rank i in step k, -1 = idle
+ *   lane_inst   [B][k_max][N]  path-instance id of that lane, 0xFFFF = idle
+ *   lane_bytes  [B][k_max][N]  bytes for the pair (i, lane_dst), 0 = idle
+ *   send_off    [B][k_max+1][N] bytes rank i has sent before step k
+ *   recv_off    [B][k_max+1][N] bytes rank j has received before step k; may be NULL
+ *   tau_ns_out  [B] quantum used; may be NULL
+ *   status      [B] VP_ST_* bits
+ * Every element of every output array is written (rows beyond n_steps hold the
+ * idle values; offset rows beyond n_steps repeat the totals).
+ * workspace: device, 256-byte aligned, >= vp_schedule_workspace_bytes; contents
+ * are scratch.  Calls sharing a workspace must be stream-ordered.
+ */
+int vp_schedule_batch(const vp_catalog* catalog, const vp_sched_params* params,
+                      const int64_t* demand, const int64_t* tau_ns_in, int B,
+                      int32_t* n_steps, int32_t* chan_id, int16_t* lane_dst, uint16_t* lane_inst,
+                      int64_t* lane_bytes, int64_t* send_off, int64_t* recv_off,
+                      int64_t* tau_ns_out, int32_t* status,
+                      void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Bytes of device scratch vp_pack needs (multiple of 256). */
+size_t vp_pack_workspace_bytes(int N, int T, int topk, int k_max);
+
+/*
+ * vp_pack - stage one rank's routed token rows in activation x destination
+ * order (Section 5: "groups elements by destination rank and packs each peer's
+ * ... payload contiguously into the ... send buffer").
+ *
+ * Copies (t, slot) with expert_idx >= 0 whose destination rank
+ * j = expert_idx / experts_per_rank differs from `rank` form stream_j in
+ * ascending (t, slot).  Step k of the plan sends lane_bytes[k][rank] bytes to
+ * j = lane_dst[k][rank]: the next lane_bytes/row_bytes rows of stream_j, stored
+ * at staged row send_off[k][rank]/row_bytes onwards.  One row per (token, slot);
+ * copies to the rank itself are not staged (D_ii = 0).
+ *
+ * n_steps_b, lane_dst_b, lane_bytes_b, send_off_b: device pointers to ONE
+ *   matrix's plan as written by vp_schedule_batch (row stride N).
+ * expert_idx [T][topk] int32 device; < 0 = dropped copy.
+ * rows       [T][row_bytes] device.  staged: device, staged_capacity_bytes long.
+ *   When rows, staged and row_bytes are multiples of 16 the copy uses bulk
+ *   asynchronous (TMA) transfers; otherwise a plain-load path.
+ * src_map    [staged_capacity_bytes/row_bytes] int32 device or NULL: receives
+ *   t*topk+slot for each staged row; rows not written keep their content.
+ * status     device int32[1]: VP_ST_PACK_MISMATCH if the routed copies per
+ *   destination differ from the plan (copies beyond the plan are not staged),
+ *   VP_ST_PACK_CAPACITY if send_off[n_steps][rank] > capacity (nothing copied).
+ * workspace: device, 256-byte aligned, >= vp_pack_workspace_bytes.
+ */
+int vp_pack(const int32_t* n_steps_b, const int16_t* lane_dst_b, const int64_t* lane_bytes_b,
+            const int64_t* send_off_b, int N, int rank, int k_max,
+            const int32_t* expert_idx, int T, int topk, int experts_per_rank,
+            const void* rows, int64_t row_bytes,
+            void* staged, int64_t staged_capacity_bytes, int32_t* src_map,
+            int32_t* status, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Host-buffer variants: the same operations with every array in HOST memory
+ * (pinned memory makes the copies asynchronous).  The calls copy inputs to
+ * device scratch, run the kernels above, copy the results back and return
+ * after synchronising the stream.  device_scratch must hold
+ * vp_schedule_host_scratch_bytes / vp_pack_host_scratch_bytes bytes.
+ */
+size_t vp_schedule_host_scratch_bytes(const vp_catalog* catalog, int B, const vp_sched_params* params);
+int vp_schedule_batch_host(const vp_catalog* catalog, const vp_sched_params* params,
+                           const int64_t* demand, const int64_t* tau_ns_in, int B,
+                           int32_t* n_steps, int32_t* chan_id, int16_t* lane_dst, uint16_t* lane_inst,
+                           int64_t* lane_bytes, int64_t* send_off, int64_t* recv_off,
+                           int64_t* tau_ns_out, int32_t* status,
+                           void* device_scratch, size_t device_scratch_bytes, void* cuda_stream);
+size_t vp_pack_host_scratch_bytes(int N, int T, int topk, int k_max, int64_t row_bytes,
+                                  int64_t staged_capacity_bytes);
+int vp_pack_host(const int32_t* n_steps_b, const int16_t* lane_dst_b, const int64_t* lane_bytes_b,
+                 const int64_t* send_off_b, int N, int rank, int k_max,
+                 const int32_t* expert_idx, int T, int topk, int experts_per_rank,
+                 const void* rows, int64_t row_bytes,
+                 void* staged, int64_t staged_capacity_bytes, int32_t* src_map,
+                 int32_t* status, void* device_scratch, size_t device_scratch_bytes, void* cuda_stream);
+
+/* Number of kernels the library has launched in this process (for launch accounting). */
+int64_t vp_kernel_launch_count(void);
+
+/* Static description of a VP_E_* code. */
+const char* vp_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* VARIOPATH_H */

@@ -1,0 +1,282 @@
+"""ctypes binding of ``libvariopath.so``; names follow the C ABI (``vp_*`` without the prefix).
+
+PyTorch is used for device memory and streams only.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+from typing import Optional
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_PKG, "libvariopath.so")
+
+E_BAD_ARG, E_BAD_CATALOG, E_NOMEM, E_CUDA, E_WORKSPACE, E_UNSUPPORTED = -1, -2, -3, -4, -5, -6
+ST_NEGATIVE, ST_OVERFLOW_RISK, ST_DIAG_NONZERO, ST_NOT_GRANULE = 1, 2, 4, 8
+ST_BAD_TAU, ST_UNCOVERED, ST_NO_PROGRESS, ST_STEP_LIMIT = 16, 32, 64, 128
+ST_PACK_MISMATCH, ST_PACK_CAPACITY = 256, 512
+
+
+class VpError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        self.code = code
+        super().__init__(f"{what}: {_strerror(code)} ({code})")
+
+
+class _Info(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("N", "G", "g", "groups_per_node", "n_resources", "n_instances",
+                                          "n_shapes", "n_families", "max_nnz", "max_bucket", "covered",
+                                          "node_symmetric")] + [("rate_lcm", C.c_int64)]
+
+
+class _Params(C.Structure):
+    _fields_ = [("lambda_ns", C.c_int64), ("granule_bytes", C.c_int64), ("k_target", C.c_int32),
+                ("n_start", C.c_int32), ("i_aa", C.c_int32), ("k_max", C.c_int32)]
+
+
+@dataclass
+class SchedParams:
+    """Scheduler parameters (``vp_sched_params``); 0 selects the documented default."""
+    lambda_ns: int = 8000
+    granule_bytes: int = 1
+    k_target: int = 0
+    n_start: int = 0
+    i_aa: int = 0
+    k_max: int = 0
+
+    def _c(self, N: int) -> _Params:
+        return _Params(int(self.lambda_ns), int(self.granule_bytes), int(self.k_target), int(self.n_start),
+                       int(self.i_aa), int(self.k_max) or 8 * N)
+
+
+_lib = None
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def _load():
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise RuntimeError(f"{_LIB_PATH} is missing: build it with `python -m paper_2609_34340_b200.build` "
+                           "(there is no CPU fallback)")
+    lib = C.CDLL(_LIB_PATH)
+    vp, i32, i64, sz, P = C.c_void_p, C.c_int, C.c_int64, C.c_size_t, C.c_void_p
+    lib.vp_load_catalog.argtypes = [P, sz, P, sz, i32, C.POINTER(vp)]
+    lib.vp_free_catalog.argtypes = [vp]
+    lib.vp_free_catalog.restype = None
+    lib.vp_catalog_info.argtypes = [vp, C.POINTER(_Info)]
+    lib.vp_schedule_workspace_bytes.argtypes = [vp, i32, C.POINTER(_Params)]
+    lib.vp_schedule_workspace_bytes.restype = sz
+    sched_args = [vp, C.POINTER(_Params), P, P, i32] + [P] * 9
+    lib.vp_schedule_batch.argtypes = sched_args + [P, sz, P]
+    lib.vp_schedule_host_scratch_bytes.argtypes = [vp, i32, C.POINTER(_Params)]
+    lib.vp_schedule_host_scratch_bytes.restype = sz
+    lib.vp_schedule_batch_host.argtypes = sched_args + [P, sz, P]
+    lib.vp_pack_workspace_bytes.argtypes = [i32, i32, i32, i32]
+    lib.vp_pack_workspace_bytes.restype = sz
+    pack_args = [P, P, P, P, i32, i32, i32, P, i32, i32, i32, P, i64, P, i64, P, P]
+    lib.vp_pack.argtypes = pack_args + [P, sz, P]
+    lib.vp_pack_host_scratch_bytes.argtypes = [i32, i32, i32, i32, i64, i64]
+    lib.vp_pack_host_scratch_bytes.restype = sz
+    lib.vp_pack_host.argtypes = pack_args + [P, sz, P]
+    lib.vp_kernel_launch_count.restype = i64
+    lib.vp_strerror.argtypes = [i32]
+    lib.vp_strerror.restype = C.c_char_p
+    _lib = lib
+    return lib
+
+
+def _strerror(code: int) -> str:
+    return _load().vp_strerror(int(code)).decode()
+
+
+def _check(rc: int, what: str) -> None:
+    if rc != 0:
+        raise VpError(rc, what)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream(stream) -> C.c_void_p:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return C.c_void_p(s.cuda_stream)
+
+
+def kernel_launch_count() -> int:
+    return int(_load().vp_kernel_launch_count())
+
+
+class Catalog:
+    """Handle of a catalog loaded on one device (``vp_catalog``)."""
+
+    def __init__(self, handle: int, device: int):
+        self._h = C.c_void_p(handle)
+        self.device = device
+        info = _Info()
+        _check(_load().vp_catalog_info(self._h, C.byref(info)), "vp_catalog_info")
+        for name, _ in _Info._fields_:
+            setattr(self, name, int(getattr(info, name)))
+
+    def free(self) -> None:
+        if self._h:
+            _load().vp_free_catalog(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.free()
+        except Exception:
+            pass
+
+
+def load_catalog(topology: bytes, channels: bytes, device: int = 0) -> Catalog:
+    """``vp_load_catalog``: validate the blobs (Eq. 3, Eq. 4) and upload the device image."""
+    h = C.c_void_p()
+    topology, channels = bytes(topology), bytes(channels)
+    _check(_load().vp_load_catalog(topology, len(topology), channels, len(channels), int(device), C.byref(h)),
+           "vp_load_catalog")
+    return Catalog(h.value, int(device))
+
+
+def schedule_workspace_bytes(catalog: Catalog, B: int, params: SchedParams) -> int:
+    p = params._c(catalog.N)
+    return int(_load().vp_schedule_workspace_bytes(catalog._h, int(B), C.byref(p)))
+
+
+@dataclass
+class Plan:
+    """Output arrays of ``vp_schedule_batch`` (device or host tensors, layouts as in the header)."""
+    n_steps: torch.Tensor
+    chan_id: torch.Tensor
+    lane_dst: torch.Tensor
+    lane_inst: torch.Tensor
+    lane_bytes: torch.Tensor
+    send_off: torch.Tensor
+    recv_off: torch.Tensor
+    tau_ns: torch.Tensor
+    status: torch.Tensor
+    k_max: int
+
+    @staticmethod
+    def empty(B: int, N: int, k_max: int, device, pin: bool = False) -> "Plan":
+        kw = dict(device=device, pin_memory=pin) if pin else dict(device=device)
+        return Plan(
+            n_steps=torch.empty(B, dtype=torch.int32, **kw),
+            chan_id=torch.empty((B, k_max), dtype=torch.int32, **kw),
+            lane_dst=torch.empty((B, k_max, N), dtype=torch.int16, **kw),
+            lane_inst=torch.empty((B, k_max, N), dtype=torch.uint16, **kw),
+            lane_bytes=torch.empty((B, k_max, N), dtype=torch.int64, **kw),
+            send_off=torch.empty((B, k_max + 1, N), dtype=torch.int64, **kw),
+            recv_off=torch.empty((B, k_max + 1, N), dtype=torch.int64, **kw),
+            tau_ns=torch.empty(B, dtype=torch.int64, **kw),
+            status=torch.empty(B, dtype=torch.int32, **kw),
+            k_max=k_max)
+
+    def cpu(self) -> dict:
+        """Numpy copies keyed like the oracle's output."""
+        out = {k: getattr(self, k).cpu().numpy() for k in ("n_steps", "chan_id", "lane_dst", "lane_bytes",
+                                                             "send_off", "recv_off", "tau_ns", "status")}
+        out["lane_inst"] = self.lane_inst.cpu().view(torch.int16).numpy().view("uint16")
+        out["k_max"] = self.k_max
+        return out
+
+
+def _sched_call(fn, catalog, p, demand, tau_ns_in, B, plan, scratch, stream):
+    return fn(catalog._h, C.byref(p), _ptr(demand), _ptr(tau_ns_in), int(B), _ptr(plan.n_steps),
+              _ptr(plan.chan_id), _ptr(plan.lane_dst), _ptr(plan.lane_inst), _ptr(plan.lane_bytes),
+              _ptr(plan.send_off), _ptr(plan.recv_off), _ptr(plan.tau_ns), _ptr(plan.status),
+              _ptr(scratch), scratch.numel(), _stream(stream))
+
+
+def schedule_batch(catalog: Catalog, params: SchedParams, demand: torch.Tensor,
+                   tau_ns_in: Optional[torch.Tensor] = None, plan: Optional[Plan] = None,
+                   workspace: Optional[torch.Tensor] = None, stream=None) -> Plan:
+    """``vp_schedule_batch`` on device tensors: ``demand`` is ``[B,N,N]`` int64 on the catalog's device."""
+    assert demand.is_cuda and demand.dtype == torch.int64 and demand.is_contiguous()
+    B, N = demand.shape[0], catalog.N
+    assert demand.shape == (B, N, N)
+    p = params._c(N)
+    if plan is None:
+        plan = Plan.empty(B, N, p.k_max, demand.device)
+    if workspace is None:
+        workspace = torch.empty(schedule_workspace_bytes(catalog, B, params), dtype=torch.uint8, device=demand.device)
+    _check(_sched_call(_load().vp_schedule_batch, catalog, p, demand, tau_ns_in, B, plan, workspace, stream),
+           "vp_schedule_batch")
+    return plan
+
+
+def schedule_batch_host(catalog: Catalog, params: SchedParams, demand: torch.Tensor,
+                        tau_ns_in: Optional[torch.Tensor] = None, plan: Optional[Plan] = None,
+                        scratch: Optional[torch.Tensor] = None, stream=None) -> Plan:
+    """``vp_schedule_batch_host``: host tensors in and out (pinned memory recommended)."""
+    assert not demand.is_cuda and demand.dtype == torch.int64 and demand.is_contiguous()
+    B, N = demand.shape[0], catalog.N
+    p = params._c(N)
+    if plan is None:
+        plan = Plan.empty(B, N, p.k_max, "cpu", pin=True)
+    if scratch is None:
+        need = int(_load().vp_schedule_host_scratch_bytes(catalog._h, B, C.byref(p)))
+        scratch = torch.empty(need, dtype=torch.uint8, device=f"cuda:{catalog.device}")
+    _check(_sched_call(_load().vp_schedule_batch_host, catalog, p, demand, tau_ns_in, B, plan, scratch, stream),
+           "vp_schedule_batch_host")
+    return plan
+
+
+def pack_workspace_bytes(N: int, T: int, topk: int, k_max: int) -> int:
+    return int(_load().vp_pack_workspace_bytes(int(N), int(T), int(topk), int(k_max)))
+
+
+def _pack_call(fn, plan, b, N, rank, expert_idx, experts_per_rank, rows, row_bytes, staged, src_map, status,
+               scratch, stream):
+    T, topk = expert_idx.shape
+    return fn(_ptr(plan.n_steps[b:b + 1]), _ptr(plan.lane_dst[b]), _ptr(plan.lane_bytes[b]), _ptr(plan.send_off[b]),
+              int(N), int(rank), int(plan.k_max), _ptr(expert_idx), int(T), int(topk), int(experts_per_rank),
+              _ptr(rows), int(row_bytes), _ptr(staged), staged.numel() * staged.element_size(), _ptr(src_map),
+              _ptr(status), _ptr(scratch), scratch.numel(), _stream(stream))
+
+
+def pack(plan: Plan, b: int, rank: int, expert_idx: torch.Tensor, experts_per_rank: int, rows: torch.Tensor,
+         staged: torch.Tensor, src_map: Optional[torch.Tensor] = None, status: Optional[torch.Tensor] = None,
+         workspace: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """``vp_pack`` for matrix ``b`` of a device plan.  ``rows`` is ``[T, H]`` (any dtype), ``staged`` a
+    pre-allocated device buffer; returns the device status tensor (int32[1])."""
+    N = plan.lane_dst.shape[2]
+    assert expert_idx.is_cuda and expert_idx.dtype == torch.int32 and expert_idx.is_contiguous()
+    assert rows.is_cuda and rows.is_contiguous() and staged.is_cuda and staged.is_contiguous()
+    T, topk = expert_idx.shape
+    row_bytes = rows.shape[1] * rows.element_size()
+    if status is None:
+        status = torch.empty(1, dtype=torch.int32, device=rows.device)
+    if workspace is None:
+        workspace = torch.empty(pack_workspace_bytes(N, T, topk, plan.k_max), dtype=torch.uint8, device=rows.device)
+    _check(_pack_call(_load().vp_pack, plan, b, N, rank, expert_idx, experts_per_rank, rows, row_bytes, staged,
+                      src_map, status, workspace, stream), "vp_pack")
+    return status
+
+
+def pack_host(plan: Plan, b: int, rank: int, expert_idx: torch.Tensor, experts_per_rank: int, rows: torch.Tensor,
+              staged: torch.Tensor, src_map: Optional[torch.Tensor] = None, status: Optional[torch.Tensor] = None,
+              scratch: Optional[torch.Tensor] = None, device: int = 0, stream=None) -> torch.Tensor:
+    """``vp_pack_host``: every array (plan included) in host memory."""
+    N = plan.lane_dst.shape[2]
+    assert not rows.is_cuda and not staged.is_cuda and not plan.lane_dst.is_cuda
+    T, topk = expert_idx.shape
+    row_bytes = rows.shape[1] * rows.element_size()
+    if status is None:
+        status = torch.zeros(1, dtype=torch.int32)
+    if scratch is None:
+        need = int(_load().vp_pack_host_scratch_bytes(N, T, topk, plan.k_max, row_bytes,
+                                                      staged.numel() * staged.element_size()))
+        scratch = torch.empty(need, dtype=torch.uint8, device=f"cuda:{device}")
+    _check(_pack_call(_load().vp_pack_host, plan, b, N, rank, expert_idx, experts_per_rank, rows, row_bytes, staged,
+                      src_map, status, scratch, stream), "vp_pack_host")
+    return status

@@ -1,0 +1,297 @@
+// Catalog loader: parses the topology / channel blobs, validates them against
+// Eq. (3) and Eq. (4) of Section 4.1 and builds the device image the kernels read.
+#include <algorithm>
+#include <cstring>
+#include <new>
+
+#include "vp_internal.h"
+
+long long g_vp_launches = 0;
+
+namespace {
+
+struct Reader {
+    const uint8_t* p;
+    size_t n;
+    bool ok = true;
+    uint32_t u32(size_t off) {
+        if (off + 4 > n) { ok = false; return 0; }
+        return (uint32_t)p[off] | ((uint32_t)p[off + 1] << 8) | ((uint32_t)p[off + 2] << 16) | ((uint32_t)p[off + 3] << 24);
+    }
+    uint16_t u16(size_t off) {
+        if (off + 2 > n) { ok = false; return 0; }
+        return (uint16_t)(p[off] | (p[off + 1] << 8));
+    }
+    uint8_t u8(size_t off) {
+        if (off + 1 > n) { ok = false; return 0; }
+        return p[off];
+    }
+};
+
+struct HostInst {
+    int a, d, kind, mult, n_res, cls;
+    int64_t bw;
+    int res[4];
+};
+
+int64_t gcd_i64(int64_t a, int64_t b) {
+    while (b) { int64_t t = a % b; a = b; b = t; }
+    return a;
+}
+
+template <typename T>
+int upload(vp_catalog* c, const std::vector<T>& v, const T** out) {
+    void* d = nullptr;
+    size_t bytes = std::max<size_t>(v.size(), 1) * sizeof(T);
+    if (cudaMalloc(&d, bytes) != cudaSuccess) return VP_E_NOMEM;
+    c->allocs.push_back(d);
+    if (!v.empty() && cudaMemcpy(d, v.data(), v.size() * sizeof(T), cudaMemcpyHostToDevice) != cudaSuccess) return VP_E_CUDA;
+    *out = (const T*)d;
+    return VP_OK;
+}
+
+}  // namespace
+
+extern "C" void vp_free_catalog(vp_catalog* c) {
+    if (!c) return;
+    int prev = -1;
+    cudaGetDevice(&prev);
+    if (cudaSetDevice(c->device) == cudaSuccess)
+        for (void* p : c->allocs) cudaFree(p);
+    if (prev >= 0) cudaSetDevice(prev);
+    delete c;
+}
+
+extern "C" int vp_catalog_info(const vp_catalog* c, vp_info* out) {
+    if (!c || !out) return VP_E_BAD_ARG;
+    *out = c->info;
+    return VP_OK;
+}
+
+extern "C" int vp_load_catalog(const void* topology, size_t topo_bytes, const void* channels, size_t chan_bytes,
+                               int device, vp_catalog** out) {
+    if (!topology || !channels || !out || device < 0) return VP_E_BAD_ARG;
+    *out = nullptr;
+    Reader t{(const uint8_t*)topology, topo_bytes}, h{(const uint8_t*)channels, chan_bytes};
+    if (t.u32(0) != 0x50545056u || t.u32(4) != 1 || !t.ok) return VP_E_BAD_CATALOG;
+    if (h.u32(0) != 0x48435056u || h.u32(4) != 1 || !h.ok) return VP_E_BAD_CATALOG;
+    const int N = (int)t.u32(8), G = (int)t.u32(12), g = (int)t.u32(16), S = (int)t.u32(20);
+    const int n_res = (int)t.u32(24), n_inst = (int)t.u32(28);
+    if (!t.ok || N <= 0 || G <= 0 || g <= 0 || (long long)G * g != N || n_inst <= 0 || n_res < 0) return VP_E_BAD_CATALOG;
+    if (N > VP_MAX_N || g > VP_MAX_GROUP || n_inst > 0xFFFE || n_res > 0xFFFF) return VP_E_UNSUPPORTED;
+    if (topo_bytes < 32 + (size_t)n_inst * 20) return VP_E_BAD_CATALOG;
+
+    // ---- path instances (Section 4.1), rate classes, lcm of rates
+    std::vector<HostInst> inst(n_inst);
+    std::vector<int64_t> rates;
+    int64_t W = 1, bw_max = 0;
+    for (int r = 0; r < n_inst; r++) {
+        size_t o = 32 + (size_t)r * 20;
+        HostInst& q = inst[r];
+        q.a = t.u16(o); q.d = t.u16(o + 2); q.kind = t.u8(o + 4); q.n_res = t.u8(o + 5);
+        q.mult = t.u16(o + 6); q.bw = t.u32(o + 8);
+        if (q.a >= G || q.d >= G || q.n_res > 4 || q.bw <= 0 || q.mult < 1) return VP_E_BAD_CATALOG;
+        for (int k = 0; k < q.n_res; k++) {
+            q.res[k] = t.u16(o + 12 + 2 * k);
+            if (q.res[k] >= n_res) return VP_E_BAD_CATALOG;
+        }
+        if (r > 0 && (inst[r - 1].a > q.a || (inst[r - 1].a == q.a && inst[r - 1].d > q.d))) return VP_E_BAD_CATALOG;
+        auto it = std::find(rates.begin(), rates.end(), q.bw);
+        if (it == rates.end()) { rates.push_back(q.bw); q.cls = (int)rates.size() - 1; }
+        else q.cls = (int)(it - rates.begin());
+        if (rates.size() > VP_MAX_CLASSES) return VP_E_UNSUPPORTED;
+        W = W / gcd_i64(W, q.bw) * q.bw;
+        if (W >= ((int64_t)1 << 20)) return VP_E_UNSUPPORTED;
+        bw_max = std::max(bw_max, q.bw);
+    }
+
+    // ---- shapes and families
+    if ((int)h.u32(8) != N) return VP_E_BAD_CATALOG;
+    const int n_shapes = (int)h.u32(12), n_fam = (int)h.u32(16), total_nnz = (int)h.u32(20);
+    if (!h.ok || n_shapes <= 0 || n_fam <= 0 || total_nnz <= 0) return VP_E_BAD_CATALOG;
+    const size_t off_sptr = 24, off_nnz = off_sptr + 4 * ((size_t)n_shapes + 1);
+    const size_t off_bptr = off_nnz + 8 * (size_t)total_nnz, off_fam = off_bptr + 4 * ((size_t)n_shapes + 1);
+    if (chan_bytes < off_fam + 2 * (size_t)n_fam * N) return VP_E_BAD_CATALOG;
+    std::vector<uint32_t> shape_ptr(n_shapes + 1), bucket_ptr(n_shapes + 1);
+    for (int s = 0; s <= n_shapes; s++) {
+        shape_ptr[s] = h.u32(off_sptr + 4 * (size_t)s);
+        bucket_ptr[s] = h.u32(off_bptr + 4 * (size_t)s);
+    }
+    if (shape_ptr[0] != 0 || (int)shape_ptr[n_shapes] != total_nnz || bucket_ptr[0] != 0 || (int)bucket_ptr[n_shapes] != n_fam)
+        return VP_E_BAD_CATALOG;
+
+    std::vector<int> M((size_t)G * G, 0), cnt((size_t)G * G, 0), used(n_res + 1, 0), times(n_inst, 0);
+    std::vector<int> rowsum(G), colsum(G);
+    std::vector<char> seen((size_t)G * G, 0);
+    std::vector<uint32_t> fam_slot((size_t)n_fam * N);
+    std::vector<uint8_t> fam_inslot((size_t)n_fam * N);
+    int max_nnz = 0, max_bucket = 0;
+    for (int s = 0; s < n_shapes; s++) {
+        if (shape_ptr[s + 1] <= shape_ptr[s] || bucket_ptr[s + 1] < bucket_ptr[s]) return VP_E_BAD_CATALOG;
+        max_nnz = std::max(max_nnz, (int)(shape_ptr[s + 1] - shape_ptr[s]));
+        max_bucket = std::max(max_bucket, (int)(bucket_ptr[s + 1] - bucket_ptr[s]));
+        std::fill(rowsum.begin(), rowsum.end(), 0);
+        std::fill(colsum.begin(), colsum.end(), 0);
+        for (uint32_t e = shape_ptr[s]; e < shape_ptr[s + 1]; e++) {
+            int a = h.u16(off_nnz + 8 * (size_t)e), d = h.u16(off_nnz + 8 * (size_t)e + 2), m = h.u16(off_nnz + 8 * (size_t)e + 4);
+            if (a >= G || d >= G || m == 0 || M[(size_t)a * G + d] != 0) return VP_E_BAD_CATALOG;
+            M[(size_t)a * G + d] = m;
+            rowsum[a] += m; colsum[d] += m;
+            seen[(size_t)a * G + d] = 1;
+        }
+        for (int a = 0; a < G; a++)
+            if (rowsum[a] != g || colsum[a] != g) return VP_E_BAD_CATALOG;                  // Eq. (3)
+        for (uint32_t f = bucket_ptr[s]; f < bucket_ptr[s + 1]; f++) {                      // Eq. (4)
+            int fill[VP_MAX_N] = {0};
+            int prev = -1;
+            for (int r = 0; r < N; r++) {
+                int id = h.u16(off_fam + 2 * ((size_t)f * N + r));
+                if (id >= n_inst || id < prev) return VP_E_BAD_CATALOG;
+                prev = id;
+                const HostInst& q = inst[id];
+                if (q.a != r / g) return VP_E_BAD_CATALOG;
+                if (++cnt[(size_t)q.a * G + q.d] > M[(size_t)q.a * G + q.d]) return VP_E_BAD_CATALOG;
+                if (++times[id] > q.mult) return VP_E_BAD_CATALOG;
+                for (int k = 0; k < q.n_res; k++)
+                    if (used[q.res[k]]++) return VP_E_BAD_CATALOG;
+                if (fill[q.d] >= g) return VP_E_BAD_CATALOG;
+                fam_slot[(size_t)f * N + r] = (uint32_t)id | ((uint32_t)q.d << 16) | ((uint32_t)q.cls << 24);
+                fam_inslot[(size_t)f * N + q.d * g + fill[q.d]++] = (uint8_t)r;
+            }
+            for (int r = 0; r < N; r++) {   // N lanes with every count <= M_ad and sum M = N  =>  counts equal M
+                const HostInst& q = inst[h.u16(off_fam + 2 * ((size_t)f * N + r))];
+                cnt[(size_t)q.a * G + q.d] = 0;
+                times[h.u16(off_fam + 2 * ((size_t)f * N + r))] = 0;
+                for (int k = 0; k < q.n_res; k++) used[q.res[k]] = 0;
+            }
+        }
+        for (uint32_t e = shape_ptr[s]; e < shape_ptr[s + 1]; e++)
+            M[(size_t)h.u16(off_nnz + 8 * (size_t)e) * G + h.u16(off_nnz + 8 * (size_t)e + 2)] = 0;
+    }
+    if (!h.ok) return VP_E_BAD_CATALOG;
+    int covered = 1;
+    for (int a = 0; a < G; a++)
+        for (int d = 0; d < G; d++)
+            if ((a != d || g >= 2) && !seen[(size_t)a * G + d]) covered = 0;
+
+    // ---- is every shape invariant under a shift of the node index?
+    int sym = 0, P = 1;
+    if (S >= 1 && G % S == 0 && G / S >= 2) {
+        P = G / S;
+        sym = 1;
+        std::vector<int> Mfull((size_t)G * G, 0);
+        for (int s = 0; s < n_shapes && sym; s++) {
+            for (uint32_t e = shape_ptr[s]; e < shape_ptr[s + 1]; e++)
+                Mfull[(size_t)h.u16(off_nnz + 8 * (size_t)e) * G + h.u16(off_nnz + 8 * (size_t)e + 2)] = h.u16(off_nnz + 8 * (size_t)e + 4);
+            for (uint32_t e = shape_ptr[s]; e < shape_ptr[s + 1] && sym; e++) {
+                int a = h.u16(off_nnz + 8 * (size_t)e), d = h.u16(off_nnz + 8 * (size_t)e + 2);
+                int a2 = (a + S) % G, d2 = (d + S) % G;
+                if (Mfull[(size_t)a2 * G + d2] != Mfull[(size_t)a * G + d]) sym = 0;
+            }
+            for (uint32_t e = shape_ptr[s]; e < shape_ptr[s + 1]; e++)
+                Mfull[(size_t)h.u16(off_nnz + 8 * (size_t)e) * G + h.u16(off_nnz + 8 * (size_t)e + 2)] = 0;
+        }
+        if (!sym) P = 1;
+    }
+
+    // ---- Eq. (6) terms: (table index, lane count)
+    std::vector<uint32_t> term_ptr(n_shapes + 1, 0), term;
+    for (int s = 0; s < n_shapes; s++) {
+        for (uint32_t e = shape_ptr[s]; e < shape_ptr[s + 1]; e++) {
+            int a = h.u16(off_nnz + 8 * (size_t)e), d = h.u16(off_nnz + 8 * (size_t)e + 2), m = h.u16(off_nnz + 8 * (size_t)e + 4);
+            if (sym) {
+                if (a / S != 0) continue;                      // node 0 represents every node
+                int delta = d / S, q = a % S, q2 = d % S;
+                term.push_back((uint32_t)((delta * S + q) * S + q2) | ((uint32_t)m << 16));
+            } else {
+                term.push_back((uint32_t)(a * G + d) | ((uint32_t)m << 16));
+            }
+        }
+        term_ptr[s + 1] = (uint32_t)term.size();
+    }
+
+    // ---- quantum rule: resources every path of a group pair crosses
+    std::vector<std::vector<uint16_t>> forced_cells(n_res);
+    std::vector<uint32_t> forced_bw(std::max(n_res, 1), 0);
+    {
+        std::vector<int> common(n_res + 1);
+        int r0 = 0;
+        while (r0 < n_inst) {
+            int r1 = r0;
+            while (r1 < n_inst && inst[r1].a == inst[r0].a && inst[r1].d == inst[r0].d) r1++;
+            std::fill(common.begin(), common.end(), 0);
+            int64_t best = 0;
+            for (int r = r0; r < r1; r++) {
+                best = std::max(best, inst[r].bw);
+                for (int k = 0; k < inst[r].n_res; k++) common[inst[r].res[k]]++;
+            }
+            for (int l = 0; l < n_res; l++)
+                if (common[l] == r1 - r0) {
+                    forced_cells[l].push_back((uint16_t)(inst[r0].a * G + inst[r0].d));
+                    forced_bw[l] = (uint32_t)std::max<int64_t>(forced_bw[l], best);
+                }
+            r0 = r1;
+        }
+    }
+    std::vector<uint32_t> forced_ptr(n_res + 1, 0);
+    std::vector<uint16_t> forced_cell;
+    for (int l = 0; l < n_res; l++) {
+        forced_cell.insert(forced_cell.end(), forced_cells[l].begin(), forced_cells[l].end());
+        forced_ptr[l + 1] = (uint32_t)forced_cell.size();
+    }
+
+    // ---- device image
+    vp_catalog* c = new (std::nothrow) vp_catalog();
+    if (!c) return VP_E_NOMEM;
+    c->device = device;
+    int prev = -1;
+    cudaGetDevice(&prev);
+    if (cudaSetDevice(device) != cudaSuccess) { delete c; return VP_E_CUDA; }
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete c; return VP_E_CUDA; }
+    c->sm_count = prop.multiProcessorCount;
+    c->max_smem_optin = (int)prop.sharedMemPerBlockOptin;
+    DevCat& dc = c->dc;
+    memset(&dc, 0, sizeof(dc));
+    dc.N = N; dc.G = G; dc.g = g; dc.S = S; dc.P = P;
+    dc.n_inst = n_inst; dc.n_shapes = n_shapes; dc.n_families = n_fam; dc.n_res = n_res;
+    dc.n_classes = (int)rates.size(); dc.sym = sym; dc.tbl_size = sym ? P * S * S : G * G;
+    dc.max_bucket = max_bucket; dc.bw_max = bw_max; dc.W = W;
+    for (size_t k = 0; k < rates.size(); k++) { dc.class_bw[k] = rates[k]; dc.class_wdiv[k] = W / rates[k]; }
+    int rc = VP_OK;
+    if (!rc) rc = upload(c, term_ptr, &dc.shape_ptr);
+    if (!rc) rc = upload(c, term, &dc.term);
+    if (!rc) rc = upload(c, bucket_ptr, &dc.bucket_ptr);
+    if (!rc) rc = upload(c, fam_slot, &dc.fam_slot);
+    if (!rc) rc = upload(c, fam_inslot, &dc.fam_inslot);
+    if (!rc) rc = upload(c, forced_ptr, &dc.forced_ptr);
+    if (!rc) rc = upload(c, forced_cell, &dc.forced_cell);
+    if (!rc) rc = upload(c, forced_bw, &dc.forced_bw);
+    if (rc) {
+        vp_free_catalog(c);
+        if (prev >= 0) cudaSetDevice(prev);
+        return rc;
+    }
+    vp_info& I = c->info;
+    I.N = N; I.G = G; I.g = g; I.groups_per_node = S; I.n_resources = n_res; I.n_instances = n_inst;
+    I.n_shapes = n_shapes; I.n_families = n_fam; I.max_nnz = max_nnz; I.max_bucket = max_bucket;
+    I.covered = covered; I.node_symmetric = sym; I.rate_lcm = W;
+    if (prev >= 0) cudaSetDevice(prev);
+    *out = c;
+    return VP_OK;
+}
+
+extern "C" int64_t vp_kernel_launch_count(void) { return g_vp_launches; }
+
+extern "C" const char* vp_strerror(int code) {
+    switch (code) {
+        case VP_OK: return "ok";
+        case VP_E_BAD_ARG: return "bad argument";
+        case VP_E_BAD_CATALOG: return "catalog blob malformed or violates the shape/family constraints";
+        case VP_E_NOMEM: return "out of memory";
+        case VP_E_CUDA: return "CUDA runtime error";
+        case VP_E_WORKSPACE: return "workspace missing, misaligned or too small";
+        case VP_E_UNSUPPORTED: return "catalog outside the supported limits (g <= 4, N <= 256, <= 8 path rates)";
+        default: return "unknown error";
+    }
+}

@@ -1,0 +1,386 @@
+// vp_pack: stage one rank's routed token rows in activation x destination order
+// (Section 5, "Device-resident buffer layout").
+//
+// Four kernels on the caller's stream:
+//   count : per 256-copy chunk, how many copies go to each destination rank
+//   plan  : exclusive scan of those counts over chunks (per destination) and the
+//           rank's segment table: for every destination, the activations that
+//           send to it, with the stream position they start at and their first
+//           staged row (from the plan's send offsets)
+//   map   : stable position of every copy inside its destination's stream ->
+//           staged row (binary search in the segment table); writes src_map
+//   copy  : token-major: every source row is read ONCE and written to each of
+//           its staged rows.  Rows travel global -> shared -> global as bulk
+//           asynchronous copies (TMA): one warp per CTA drives a ring of
+//           shared-memory stages, an mbarrier per stage signals the load, and
+//           the up to topk stores of a token form one bulk group whose read
+//           completion frees the stage.
+#include <cuda_runtime.h>
+
+#include "vp_internal.h"
+
+namespace {
+
+constexpr int kItems = 8;                  // 32-copy rounds per warp chunk
+constexpr int kChunk = 32 * kItems;        // copies per warp chunk
+constexpr int kWarpsPerBlock = 8;
+constexpr int kPiece = 16384;              // bytes per bulk transfer (rows longer than this are split)
+constexpr int kMinBulkRow = 2048;          // shorter rows use the plain-load kernel
+constexpr unsigned kSpinLimit = 1u << 22;  // bounded mbarrier wait
+constexpr int VP_ST_INTERNAL_TIMEOUT = 1 << 30;
+
+struct PackWs {
+    int32_t* flags;      // [0] abort, [1] n_segments
+    int32_t* hist;       // [n_chunks][N] counts, then exclusive bases
+    int32_t* len;        // [N] routed copies per destination
+    int32_t* planned;    // [N] rows the plan sends to each destination
+    int32_t* seg_ptr;    // [N+1]
+    int32_t* seg_start;  // [k_max] stream position of a segment's first row
+    int32_t* seg_row;    // [k_max] staged row of a segment's first row
+    int32_t* dst_row;    // [T*topk] staged row of each copy, -1 = not staged
+    size_t bytes;
+};
+
+PackWs carve(void* base, int N, int T, int topk, int k_max) {
+    PackWs w;
+    size_t o = 0;
+    auto take = [&](size_t n) { size_t at = o; o += vp_align256(n); return (char*)base + at; };
+    long long E = (long long)T * topk;
+    int n_chunks = (int)((E + kChunk - 1) / kChunk);
+    w.flags = (int32_t*)take(256);
+    w.hist = (int32_t*)take((size_t)n_chunks * N * 4);
+    w.len = (int32_t*)take((size_t)N * 4);
+    w.planned = (int32_t*)take((size_t)N * 4);
+    w.seg_ptr = (int32_t*)take((size_t)(N + 1) * 4);
+    w.seg_start = (int32_t*)take((size_t)k_max * 4);
+    w.seg_row = (int32_t*)take((size_t)k_max * 4);
+    w.dst_row = (int32_t*)take((size_t)E * 4);
+    w.bytes = o;
+    return w;
+}
+
+__device__ __forceinline__ int dest_of(int x, int experts_per_rank, int N, int rank) {
+    // destination rank of a routed copy, or -1 if it is not staged (dropped, local, out of range)
+    if (x < 0) return -1;
+    int j = x / experts_per_rank;
+    return (j >= N || j == rank) ? -1 : j;
+}
+
+__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+pack_count_kernel(const int32_t* __restrict__ idx, long long E, int N, int rank, int experts_per_rank,
+                  int32_t* __restrict__ hist, int32_t* __restrict__ status) {
+    __shared__ int wh[kWarpsPerBlock][VP_MAX_N];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const long long chunk = (long long)blockIdx.x * kWarpsPerBlock + warp;
+    const long long e0 = chunk * kChunk;
+    if (e0 >= E) return;
+    for (int j = lane; j < N; j += 32) wh[warp][j] = 0;
+    __syncwarp();
+    bool bad = false;
+    for (int it = 0; it < kItems; it++) {
+        long long e = e0 + it * 32 + lane;
+        if (e < E) {
+            int x = idx[e];
+            int j = dest_of(x, experts_per_rank, N, rank);
+            if (x >= 0 && x / experts_per_rank >= N) bad = true;
+            if (j >= 0) atomicAdd(&wh[warp][j], 1);
+        }
+    }
+    __syncwarp();
+    for (int j = lane; j < N; j += 32) hist[chunk * N + j] = wh[warp][j];
+    if (bad) atomicOr(status, VP_ST_PACK_MISMATCH);
+}
+
+__global__ void __launch_bounds__(VP_MAX_N)
+pack_plan_kernel(const int32_t* __restrict__ n_steps_p, const int16_t* __restrict__ lane_dst,
+                 const int64_t* __restrict__ lane_bytes, const int64_t* __restrict__ send_off, int N, int rank,
+                 int k_max, int n_chunks, int64_t row_bytes, int64_t capacity_bytes, PackWs w,
+                 int32_t* __restrict__ status) {
+    __shared__ int s_cnt[VP_MAX_N + 1];
+    const int j = threadIdx.x;
+    int K = *n_steps_p;
+    if (K > k_max) K = k_max;
+    if (K < 0) K = 0;
+    if (j < N) {
+        int run = 0;                                       // exclusive scan over chunks
+        for (int c = 0; c < n_chunks; c++) {
+            int v = w.hist[(size_t)c * N + j];
+            w.hist[(size_t)c * N + j] = run;
+            run += v;
+        }
+        w.len[j] = run;
+        int cnt = 0;
+        for (int k = 0; k < K; k++) cnt += (lane_dst[(size_t)k * N + rank] == j);
+        s_cnt[j] = cnt;
+    }
+    __syncthreads();
+    if (j == 0) {
+        int run = 0;
+        for (int d = 0; d < N; d++) { int v = s_cnt[d]; s_cnt[d] = run; run += v; }
+        s_cnt[N] = run;
+        int st = 0;
+        if (send_off[(size_t)K * N + rank] > capacity_bytes) { st |= VP_ST_PACK_CAPACITY; w.flags[0] = 1; }
+        if (st) atomicOr(status, st);
+    }
+    __syncthreads();
+    if (j == 0) w.seg_ptr[N] = s_cnt[N];
+    if (j < N) {
+        w.seg_ptr[j] = s_cnt[j];
+        int p = s_cnt[j];
+        long long cum = 0;
+        bool bad = false;
+        for (int k = 0; k < K; k++) {
+            if (lane_dst[(size_t)k * N + rank] != j) continue;
+            int64_t bytes = lane_bytes[(size_t)k * N + rank];
+            if (bytes % row_bytes) bad = true;
+            w.seg_start[p] = (int32_t)cum;
+            w.seg_row[p] = (int32_t)(send_off[(size_t)k * N + rank] / row_bytes);
+            cum += bytes / row_bytes;
+            p++;
+        }
+        w.planned[j] = (int32_t)cum;
+        if (j == rank) { if (cum != 0) bad = true; }
+        else if (cum != w.len[j]) bad = true;
+        if (bad) atomicOr(status, VP_ST_PACK_MISMATCH);
+    }
+}
+
+__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+pack_map_kernel(const int32_t* __restrict__ idx, long long E, int N, int rank, int experts_per_rank, PackWs w,
+                int32_t* __restrict__ src_map) {
+    __shared__ int base[kWarpsPerBlock][VP_MAX_N];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const long long chunk = (long long)blockIdx.x * kWarpsPerBlock + warp;
+    const long long e0 = chunk * kChunk;
+    if (e0 >= E) return;
+    const bool aborted = w.flags[0] != 0;
+    for (int j = lane; j < N; j += 32) base[warp][j] = w.hist[chunk * N + j];
+    __syncwarp();
+    for (int it = 0; it < kItems; it++) {
+        long long e = e0 + it * 32 + lane;
+        int j = -1;
+        if (e < E) j = dest_of(idx[e], experts_per_rank, N, rank);
+        const unsigned peers = __match_any_sync(0xffffffffu, j >= 0 ? j : -1 - lane);
+        int row = -1;
+        if (j >= 0) {
+            const int p = base[warp][j] + __popc(peers & ((1u << lane) - 1));   // position in stream_j
+            if (!aborted && p < w.planned[j]) {
+                int lo = w.seg_ptr[j], hi = w.seg_ptr[j + 1] - 1;              // last segment starting at or before p
+                while (lo < hi) {
+                    int mid = (lo + hi + 1) >> 1;
+                    if (w.seg_start[mid] <= p) lo = mid; else hi = mid - 1;
+                }
+                row = w.seg_row[lo] + (p - w.seg_start[lo]);
+            }
+        }
+        __syncwarp();
+        if (j >= 0 && (peers & ((1u << lane) - 1)) == 0) base[warp][j] += __popc(peers);
+        __syncwarp();
+        if (e < E) {
+            w.dst_row[e] = row;
+            if (row >= 0 && src_map) src_map[row] = (int32_t)e;
+        }
+    }
+}
+
+// ---- bulk-copy (TMA) primitives -------------------------------------------------------------
+
+__device__ __forceinline__ unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(unsigned bar, unsigned count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(unsigned bar, unsigned bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity) {
+    unsigned ok;
+    asm volatile(
+        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ void bulk_load(unsigned dst_smem, const void* src, unsigned bytes, unsigned bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst_smem), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void bulk_store(void* dst, unsigned src_smem, unsigned bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src_smem), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N_PENDING>
+__device__ __forceinline__ void bulk_wait_read() {
+    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N_PENDING) : "memory");
+}
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
+// One warp per CTA.  A "unit" is one piece (<= kPiece bytes) of one token's row.  Units are
+// dealt to CTAs round robin.  Unit u is loaded into stage u % S, kLook units ahead of its stores.
+template <int S>
+__global__ void __launch_bounds__(32)
+pack_copy_bulk_kernel(const char* __restrict__ rows, char* __restrict__ staged, const int32_t* __restrict__ dst_row,
+                      const int32_t* __restrict__ flags, int T, int topk, long long row_bytes, int pieces,
+                      int32_t* __restrict__ status) {
+    constexpr int kLook = S / 2;
+    extern __shared__ __align__(128) unsigned char ring[];
+    __shared__ __align__(8) unsigned long long bars[S];
+    const int lane = threadIdx.x;
+    if (flags[0]) return;
+    if (lane == 0) {
+        for (int s = 0; s < S; s++) mbar_init(smem_u32(&bars[s]), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    const long long units = (long long)T * pieces;
+    const long long count = units > blockIdx.x ? (units - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+    const int rounds = (topk + 31) / 32;            // destinations are handled 32 slots at a time
+    unsigned phase = 0;                              // parity per stage (bit s)
+    unsigned loaded = 0;                             // stage holds a load that was issued (bit s)
+    bool failed = false;
+    for (long long it = 0; it < count + kLook && !failed; it++) {
+        if (it < count) {                            // ---- issue the load of unit `it`
+            const long long u = blockIdx.x + it * gridDim.x;
+            const long long t = u / pieces;
+            const int s = (int)(it % S);
+            bool any = false;
+            for (int r = 0; r < rounds; r++) {
+                const int slot = r * 32 + lane;
+                any |= slot < topk && dst_row[t * topk + slot] >= 0;
+            }
+            any = __any_sync(0xffffffffu, any);
+            bulk_wait_read<S - kLook - 1>();         // every lane: its stores that last read this stage are done
+            __syncwarp();
+            if (lane == 0) {
+                if (any) {
+                    const int p = (int)(u % pieces);
+                    const unsigned bytes = (unsigned)min((long long)kPiece, row_bytes - (long long)p * kPiece);
+                    const unsigned bar = smem_u32(&bars[s]);
+                    mbar_expect_tx(bar, bytes);
+                    bulk_load(smem_u32(ring + (size_t)s * kPiece), rows + t * row_bytes + (long long)p * kPiece, bytes, bar);
+                }
+            }
+            loaded = any ? (loaded | (1u << s)) : (loaded & ~(1u << s));
+        }
+        const long long m = it - kLook;
+        if (m >= 0) {                                // ---- unit m: wait for its load, issue its stores
+            const long long u = blockIdx.x + m * gridDim.x;
+            const long long t = u / pieces;
+            const int p = (int)(u % pieces);
+            const int s = (int)(m % S);
+            if (loaded & (1u << s)) {
+                const unsigned bar = smem_u32(&bars[s]);
+                unsigned spins = 0;
+                while (!mbar_try_wait(bar, (phase >> s) & 1u)) {
+                    if (++spins > kSpinLimit) { failed = true; break; }
+                }
+                failed = __any_sync(0xffffffffu, failed);
+                phase ^= 1u << s;
+                if (!failed) {
+                    const unsigned bytes = (unsigned)min((long long)kPiece, row_bytes - (long long)p * kPiece);
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    for (int r = 0; r < rounds; r++) {
+                        const int slot = r * 32 + lane;
+                        const int row = slot < topk ? dst_row[t * topk + slot] : -1;
+                        if (row >= 0)
+                            bulk_store(staged + (long long)row * row_bytes + (long long)p * kPiece,
+                                       smem_u32(ring + (size_t)s * kPiece), bytes);
+                    }
+                }
+            }
+            bulk_commit();                           // one group per unit from every lane, empty or not
+        }
+    }
+    bulk_wait_all();                                 // stores must finish before shared memory is released
+    if (failed && lane == 0) atomicOr(status, VP_ST_INTERNAL_TIMEOUT);
+}
+
+// Plain-load path (short or unaligned rows): one warp per token, V-byte vectors.
+template <typename V>
+__global__ void __launch_bounds__(256)
+pack_copy_plain_kernel(const char* __restrict__ rows, char* __restrict__ staged, const int32_t* __restrict__ dst_row,
+                       const int32_t* __restrict__ flags, int T, int topk, long long row_bytes) {
+    if (flags[0]) return;
+    const int lane = threadIdx.x & 31;
+    const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const long long n_warps = ((long long)gridDim.x * blockDim.x) >> 5;
+    const long long vecs = row_bytes / (long long)sizeof(V);
+    for (long long t = warp; t < T; t += n_warps) {
+        const V* src = (const V*)(rows + t * row_bytes);
+        for (int s0 = 0; s0 < topk; s0 += 8) {
+            int row[8];
+            bool any = false;
+#pragma unroll
+            for (int s = 0; s < 8; s++) {
+                row[s] = (s0 + s < topk) ? dst_row[t * topk + s0 + s] : -1;
+                any |= row[s] >= 0;
+            }
+            if (!any) continue;
+            for (long long v = lane; v < vecs; v += 32) {
+                const V x = src[v];
+#pragma unroll
+                for (int s = 0; s < 8; s++)
+                    if (row[s] >= 0) ((V*)(staged + (long long)row[s] * row_bytes))[v] = x;
+            }
+        }
+    }
+}
+
+}  // namespace
+
+extern "C" size_t vp_pack_workspace_bytes(int N, int T, int topk, int k_max) {
+    if (N <= 0 || N > VP_MAX_N || T <= 0 || topk <= 0 || k_max <= 0) return 0;
+    return carve(nullptr, N, T, topk, k_max).bytes;
+}
+
+extern "C" int vp_pack(const int32_t* n_steps_b, const int16_t* lane_dst_b, const int64_t* lane_bytes_b,
+                       const int64_t* send_off_b, int N, int rank, int k_max, const int32_t* expert_idx, int T,
+                       int topk, int experts_per_rank, const void* rows, int64_t row_bytes, void* staged,
+                       int64_t staged_capacity_bytes, int32_t* src_map, int32_t* status, void* workspace,
+                       size_t workspace_bytes, void* cuda_stream) {
+    if (!n_steps_b || !lane_dst_b || !lane_bytes_b || !send_off_b || !expert_idx || !rows || !staged || !status)
+        return VP_E_BAD_ARG;
+    if (N <= 0 || N > VP_MAX_N || rank < 0 || rank >= N || k_max <= 0 || T <= 0 || topk <= 0 || experts_per_rank <= 0 ||
+        row_bytes <= 0 || staged_capacity_bytes < 0)
+        return VP_E_BAD_ARG;
+    if (staged_capacity_bytes / row_bytes >= ((int64_t)1 << 31) || (long long)T * topk >= ((long long)1 << 31))
+        return VP_E_UNSUPPORTED;
+    if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < vp_pack_workspace_bytes(N, T, topk, k_max))
+        return VP_E_WORKSPACE;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    PackWs w = carve(workspace, N, T, topk, k_max);
+    const long long E = (long long)T * topk;
+    const int n_chunks = (int)((E + kChunk - 1) / kChunk);
+    const int blocks = (n_chunks + kWarpsPerBlock - 1) / kWarpsPerBlock;
+    if (cudaMemsetAsync(w.flags, 0, 256, stream) != cudaSuccess) return VP_E_CUDA;
+    if (cudaMemsetAsync(status, 0, sizeof(int32_t), stream) != cudaSuccess) return VP_E_CUDA;
+    pack_count_kernel<<<blocks, kWarpsPerBlock * 32, 0, stream>>>(expert_idx, E, N, rank, experts_per_rank, w.hist, status);
+    pack_plan_kernel<<<1, VP_MAX_N, 0, stream>>>(n_steps_b, lane_dst_b, lane_bytes_b, send_off_b, N, rank, k_max, n_chunks,
+                                                 row_bytes, staged_capacity_bytes, w, status);
+    pack_map_kernel<<<blocks, kWarpsPerBlock * 32, 0, stream>>>(expert_idx, E, N, rank, experts_per_rank, w, src_map);
+    g_vp_launches += 3;
+
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+        return VP_E_CUDA;
+    const bool aligned16 = row_bytes % 16 == 0 && ((uintptr_t)rows & 15) == 0 && ((uintptr_t)staged & 15) == 0;
+    if (aligned16 && row_bytes >= kMinBulkRow) {
+        constexpr int S = 6;
+        const int pieces = (int)((row_bytes + kPiece - 1) / kPiece);
+        const size_t smem = (size_t)S * kPiece;
+        if (cudaFuncSetAttribute(pack_copy_bulk_kernel<S>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+            return VP_E_CUDA;
+        pack_copy_bulk_kernel<S><<<sms * 2, 32, smem, stream>>>((const char*)rows, (char*)staged, w.dst_row, w.flags, T, topk,
+                                                                row_bytes, pieces, status);
+    } else {
+        const int grid = sms * 8;
+        const uintptr_t mix = (uintptr_t)rows | (uintptr_t)staged | (uintptr_t)row_bytes;
+        if (mix % 16 == 0)
+            pack_copy_plain_kernel<uint4><<<grid, 256, 0, stream>>>((const char*)rows, (char*)staged, w.dst_row, w.flags, T, topk, row_bytes);
+        else if (mix % 4 == 0)
+            pack_copy_plain_kernel<uint32_t><<<grid, 256, 0, stream>>>((const char*)rows, (char*)staged, w.dst_row, w.flags, T, topk, row_bytes);
+        else
+            pack_copy_plain_kernel<uint8_t><<<grid, 256, 0, stream>>>((const char*)rows, (char*)staged, w.dst_row, w.flags, T, topk, row_bytes);
+    }
+    g_vp_launches++;
+    return cudaGetLastError() == cudaSuccess ? VP_OK : VP_E_CUDA;
+}

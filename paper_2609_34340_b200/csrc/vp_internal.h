@@ -1,0 +1,49 @@
+// Internal declarations shared by the library's translation units.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <vector>
+
+#include "variopath.h"
+
+#define VP_MAX_CLASSES 8          // distinct path rates in one catalog
+#define VP_MAX_GROUP 4            // ranks per group handled by the permutation search
+#define VP_MAX_N 256
+#define VP_ENTRY_LIMIT ((int64_t)1 << 40)
+
+// Device-side view of a catalog; every pointer is device memory owned by vp_catalog.
+struct DevCat {
+    int N, G, g, S, P;            // ranks, groups, group size, groups per node, nodes
+    int n_inst, n_shapes, n_families, n_res, n_classes;
+    int sym;                      // 1: shape terms index per-node-offset sums, 0: D-hat cells
+    int tbl_size;                 // entries of the score table (G*G or P*S*S)
+    int max_bucket;
+    // Eq. (6): shape s has terms term[shape_ptr[s] .. shape_ptr[s+1]) = table index | count << 16
+    const uint32_t* shape_ptr;
+    const uint32_t* term;
+    const uint32_t* bucket_ptr;
+    // family f, slot r: instance id | destination group << 16 | rate class << 24
+    const uint32_t* fam_slot;
+    // family f, in-slot d*g+q: slot index (N <= 256)
+    const uint8_t* fam_inslot;
+    // quantum rule: resource l is forced for the D-hat cells forced_cell[forced_ptr[l] .. forced_ptr[l+1])
+    const uint32_t* forced_ptr;
+    const uint16_t* forced_cell;
+    const uint32_t* forced_bw;
+    int64_t class_bw[VP_MAX_CLASSES];
+    int64_t class_wdiv[VP_MAX_CLASSES];   // rate_lcm / bw
+    int64_t bw_max, W;
+};
+
+struct vp_catalog {
+    int device;
+    vp_info info;
+    DevCat dc;
+    std::vector<void*> allocs;
+    int sm_count;
+    int max_smem_optin;
+};
+
+extern long long g_vp_launches;
+
+static inline size_t vp_align256(size_t x) { return (x + 255) & ~(size_t)255; }

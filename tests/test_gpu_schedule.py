@@ -1,0 +1,229 @@
+"""GPU parity: vp_schedule_batch (through the C ABI) against the CPU oracle, bit for bit."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from workloads import (SchedParams as WParams, complete_catalog, crossbar_catalog, crossbar_topology,
+                       node_template_catalog, tree_topology, uniform_demand)
+from workloads.configs import build_config
+from workloads.topology import Catalog
+
+pytestmark = pytest.mark.gpu
+
+KEYS = ("status", "n_steps", "tau_ns", "chan_id", "lane_dst", "lane_inst", "lane_bytes", "send_off", "recv_off")
+
+
+@pytest.fixture(scope="module")
+def vp():
+    import paper_2609_34340_b200 as vp
+    assert torch.cuda.is_available(), "these tests need a GPU"
+    assert os.path.exists(vp.library_path()), "libvariopath.so has not been built"
+    return vp
+
+
+def _params(vp, w: WParams):
+    return vp.SchedParams(lambda_ns=w.lambda_ns, granule_bytes=w.granule_bytes, k_target=w.k_target,
+                          n_start=w.n_start, i_aa=w.i_aa, k_max=w.k_max)
+
+
+def _both(vp, oracle_lib, cat, demand, wparams, tau=None, threads=8):
+    oc = oracle_lib.OracleCatalog(cat.topology.blob(), cat.blob())
+    dc = vp.load_catalog(cat.topology.blob(), cat.blob())
+    D = torch.as_tensor(demand, dtype=torch.int64)
+    tau_t = None if tau is None else torch.as_tensor(tau, dtype=torch.int64).cuda()
+    plan = vp.schedule_batch(dc, _params(vp, wparams), D.cuda().contiguous(), tau_t)
+    torch.cuda.synchronize()
+    got = plan.cpu()
+    want = oc.schedule_batch(D.numpy(), wparams, tau_in=None if tau is None else np.asarray(tau), threads=threads)
+    return got, want, oc, dc
+
+
+def _assert_same(got, want, which=None):
+    for k in KEYS:
+        g, w = got[k], want[k]
+        if which is not None:
+            g, w = g[which], w[which]
+        if not np.array_equal(g, w):
+            bad = np.argwhere(np.asarray(g) != np.asarray(w))
+            raise AssertionError(f"{k} differs at {bad[:5].tolist()} ({len(bad)} entries); "
+                                 f"got {np.asarray(g)[tuple(bad[0])]} want {np.asarray(w)[tuple(bad[0])]}")
+
+
+def _random_batch(rng, B, N, u, hi, density):
+    D = rng.integers(0, hi + 1, size=(B, N, N)) * (rng.random((B, N, N)) < density) * u
+    for b in range(B):
+        np.fill_diagonal(D[b], 0)
+    return D.astype(np.int64)
+
+
+TOPOS = {
+    "node8": lambda: complete_catalog(tree_topology(1)),
+    "node8_64_50": lambda: complete_catalog(tree_topology(1, pcie_bw=64, nic_bw=50)),
+    "fig1_g3": lambda: complete_catalog(tree_topology(1, g=3, pcie_bw=64, nic_bw=50)),
+    "g2_two_nodes": lambda: complete_catalog(tree_topology(2, g=2)),
+    "g1_two_nodes": lambda: complete_catalog(tree_topology(2, g=1)),
+    "two_nodes": lambda: complete_catalog(tree_topology(2)),
+    "two_nodes_64_50": lambda: complete_catalog(tree_topology(2, pcie_bw=64, nic_bw=50)),
+    "template_4_nodes": lambda: node_template_catalog(tree_topology(4)),
+    "template_3_nodes_g3": lambda: node_template_catalog(tree_topology(3, g=3, nic_bw=50)),
+    "crossbar4": lambda: crossbar_catalog(crossbar_topology(4)),
+}
+
+
+@pytest.mark.parametrize("name", sorted(TOPOS))
+def test_random_demands_match_oracle(vp, oracle_lib, name):
+    cat = TOPOS[name]()
+    N = cat.topology.N
+    rng = np.random.default_rng(sum(map(ord, name)))
+    for u, hi, density, lam in [(256, 3, 1.0, 8000), (1, 100000, 0.5, 0), (4096, 50, 0.15, 123), (64, 1, 0.05, 8000)]:
+        D = _random_batch(rng, 37, N, u, hi, density)
+        D[5] = 0                                     # an empty matrix inside the batch
+        w = WParams(lambda_ns=lam, granule_bytes=u, n_start=0).resolved(N)
+        got, want, oc, _ = _both(vp, oracle_lib, cat, D, w)
+        assert (want["status"] == 0).all()
+        _assert_same(got, want)
+
+
+def test_parameters_and_tau_override(vp, oracle_lib):
+    cat = complete_catalog(tree_topology(2))
+    rng = np.random.default_rng(3)
+    D = _random_batch(rng, 16, 16, 512, 200, 0.7)
+    for w in [WParams(granule_bytes=512, n_start=1, i_aa=1, k_target=16, k_max=200),
+              WParams(granule_bytes=512, n_start=2, i_aa=5, k_target=48, k_max=300),
+              WParams(granule_bytes=512, n_start=7, i_aa=2, k_target=5, k_max=64, lambda_ns=0)]:
+        tau = rng.integers(0, 3, size=16) * rng.integers(1, 5000, size=16)   # 0 = derive
+        got, want, *_ = _both(vp, oracle_lib, cat, D, w.resolved(16), tau=tau)
+        _assert_same(got, want)
+
+
+def test_status_codes_and_partial_plans(vp, oracle_lib):
+    cat = complete_catalog(tree_topology(1))
+    good = uniform_demand(8, 6400).numpy()
+    D = np.stack([good] * 8)
+    D[1, 2, 2] = 64                 # diagonal
+    D[2, 1, 3] = -64                # negative
+    D[3, 1, 3] = 65                 # not a granule multiple
+    D[4, 1, 3] = 1 << 40            # overflow risk
+    D[5, 0, 0] = -1; D[5, 4, 5] = 3  # several flags at once
+    tau = np.zeros(8, np.int64); tau[6] = (1 << 40) + 1
+    w = WParams(granule_bytes=64).resolved(8)
+    got, want, *_ = _both(vp, oracle_lib, cat, D, w, tau=tau)
+    _assert_same(got, want)
+    assert got["status"].tolist() == [0, vp.ST_DIAG_NONZERO, vp.ST_NEGATIVE, vp.ST_NOT_GRANULE, vp.ST_OVERFLOW_RISK,
+                                      vp.ST_NEGATIVE | vp.ST_NOT_GRANULE, vp.ST_BAD_TAU, 0]
+    # step limit
+    w = WParams(granule_bytes=64, k_max=5).resolved(8)
+    got, want, *_ = _both(vp, oracle_lib, cat, D[:1], w)
+    _assert_same(got, want)
+    assert got["status"][0] == vp.ST_STEP_LIMIT and got["n_steps"][0] == 5
+    # uncovered: a catalog with the all-PIX shape only
+    only_pix = Catalog(cat.topology, [cat.shapes[-1]], [cat.buckets[-1]])
+    got, want, _, dc = _both(vp, oracle_lib, only_pix, D[:1], WParams(granule_bytes=64).resolved(8))
+    _assert_same(got, want)
+    assert got["status"][0] == vp.ST_UNCOVERED and dc.covered == 0
+
+
+def test_library_rejects_bad_arguments(vp):
+    cat = complete_catalog(tree_topology(1))
+    dc = vp.load_catalog(cat.topology.blob(), cat.blob())
+    D = uniform_demand(8, 64).unsqueeze(0).cuda()
+    with pytest.raises(vp.VpError) as e:
+        vp.schedule_batch(dc, vp.SchedParams(granule_bytes=0), D)
+    assert e.value.code == vp.E_BAD_ARG
+    with pytest.raises(vp.VpError) as e:
+        vp.schedule_batch(dc, vp.SchedParams(), D, workspace=torch.empty(16, dtype=torch.uint8, device="cuda"))
+    assert e.value.code == vp.E_WORKSPACE
+    with pytest.raises(vp.VpError) as e:
+        vp.load_catalog(cat.topology.blob(), cat.blob()[:-2])
+    assert e.value.code == vp.E_BAD_CATALOG
+    big = crossbar_catalog(crossbar_topology(6))
+    with pytest.raises(vp.VpError) as e:
+        vp.load_catalog(big.topology.blob(), big.blob())
+    assert e.value.code == vp.E_UNSUPPORTED
+    info = dc
+    assert (info.N, info.G, info.g, info.n_shapes, info.n_families, info.covered) == (8, 2, 4, 3, 6, 1)
+
+
+def test_deterministic_and_batch_independent(vp, oracle_lib):
+    c = build_config(2, device="cuda", batch=24)
+    cat = c["catalog"]
+    dc = vp.load_catalog(cat.topology.blob(), cat.blob())
+    p = _params(vp, c["params"])
+    D = c["demand"].cuda()
+    a = vp.schedule_batch(dc, p, D).cpu()
+    b = vp.schedule_batch(dc, p, D).cpu()
+    one = [vp.schedule_batch(dc, p, D[i:i + 1].contiguous()).cpu() for i in (0, 7, 23)]
+    torch.cuda.synchronize()
+    for k in KEYS:
+        assert np.array_equal(a[k], b[k])
+        for i, o in zip((0, 7, 23), one):
+            assert np.array_equal(a[k][i], o[k][0])
+
+
+def test_host_buffer_variant(vp, oracle_lib):
+    c = build_config(1, device="cuda", batch=8)
+    cat = c["catalog"]
+    oc = oracle_lib.OracleCatalog(cat.topology.blob(), cat.blob())
+    dc = vp.load_catalog(cat.topology.blob(), cat.blob())
+    plan = vp.schedule_batch_host(dc, _params(vp, c["params"]), c["demand"].pin_memory())
+    want = oc.schedule_batch(c["demand"].numpy(), c["params"])
+    _assert_same(plan.cpu(), want)
+
+
+@pytest.mark.parametrize("idx", [1, 2])
+def test_config_full_batch(vp, oracle_lib, idx):
+    c = build_config(idx, device="cuda")
+    got, want, oc, _ = _both(vp, oracle_lib, c["catalog"], c["demand"], c["params"], threads=os.cpu_count())
+    assert (want["status"] == 0).all()
+    _assert_same(got, want)
+
+
+def _validate_all(oc, D, got, granule):
+    for b in range(D.shape[0]):
+        plan = {k: got[k][b] for k in KEYS}
+        assert got["status"][b] == 0
+        assert oc.check_plan(D[b], plan, int(got["tau_ns"][b]), granule) == 0, f"matrix {b} invalid"
+        K = int(got["n_steps"][b])
+        assert (got["send_off"][b][K] == D[b].sum(1)).all() and (got["recv_off"][b][K] == D[b].sum(0)).all()
+
+
+def test_config3_full_batch(vp, oracle_lib):
+    """1024 matrices, N=64: every plan is checked for validity; a sample is compared bit for bit."""
+    c = build_config(3, device="cuda")
+    cat, w = c["catalog"], c["params"]
+    oc = oracle_lib.OracleCatalog(cat.topology.blob(), cat.blob())
+    dc = vp.load_catalog(cat.topology.blob(), cat.blob())
+    assert dc.node_symmetric == 1
+    D = c["demand"]
+    got = vp.schedule_batch(dc, _params(vp, w), D.cuda()).cpu()
+    Dn = D.numpy()
+    _validate_all(oc, Dn, got, w.granule_bytes)
+    sample = np.random.default_rng(0).choice(D.shape[0], size=96, replace=False)
+    want = oc.schedule_batch(Dn[sample], w, threads=os.cpu_count())
+    _assert_same({k: got[k][sample] if k != "k_max" else got[k] for k in got}, want)
+
+
+def test_config4_full_batch(vp, oracle_lib):
+    """4096 matrices, N=256, in sub-batches that reuse the output buffers; validity for all,
+    bit-exact comparison on a sample."""
+    c = build_config(4, device="cuda")
+    cat, w = c["catalog"], c["params"]
+    oc = oracle_lib.OracleCatalog(cat.topology.blob(), cat.blob())
+    dc = vp.load_catalog(cat.topology.blob(), cat.blob())
+    assert dc.node_symmetric == 1 and (dc.n_shapes, dc.n_families) == (4095, 4160)
+    D = c["demand"]
+    p = _params(vp, w)
+    sub = 256
+    plan = vp.Plan.empty(sub, 256, p.k_max or 2048, "cuda")
+    rng = np.random.default_rng(0)
+    for lo in range(0, D.shape[0], sub):
+        part = D[lo:lo + sub]
+        plan = vp.schedule_batch(dc, p, part.cuda().contiguous(), plan=plan)
+        got = plan.cpu()
+        Dn = part.numpy()
+        _validate_all(oc, Dn, got, w.granule_bytes)
+        sample = rng.choice(sub, size=1, replace=False)
+        want = oc.schedule_batch(Dn[sample], w)
+        _assert_same({k: got[k][sample] if k != "k_max" else got[k] for k in got}, want)

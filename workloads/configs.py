@@ -113,7 +113,7 @@ def build_config(idx: int, device: str = "cpu", batch: Optional[int] = None,
 
 
 def build_pack_case(device: str = "cpu", tokens: int = 16384, hidden: int = 7168,
-                    rank: int = 0, nodes: int = 2, experts: int = 256, topk: int = 8,
+                    rank: int = 8, nodes: int = 2, experts: int = 256, topk: int = 8,
                     s: float = 1.2, seed: Optional[int] = None) -> dict:
     """Config 5: all ranks route ``tokens`` tokens (top-k over ``experts``), giving one demand
     matrix; ``rank``'s routing indices and bf16 rows (random bits, every row distinct with
