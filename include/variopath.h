@@ -144,7 +144,8 @@ size_t vp_schedule_workspace_bytes(const vp_catalog* catalog, int B, const vp_sc
  * Every element of every output array is written (rows beyond n_steps hold the
  * idle values; offset rows beyond n_steps repeat the totals).
  * workspace: device, 256-byte aligned, >= vp_schedule_workspace_bytes; contents
- * are scratch.  Calls sharing a workspace must be stream-ordered.
+ * are scratch (see vp_schedule_read_stats for the counters it keeps).  Calls
+ * sharing a workspace must be stream-ordered.
  */
 int vp_schedule_batch(const vp_catalog* catalog, const vp_sched_params* params,
                       const int64_t* demand, const int64_t* tau_ns_in, int B,
@@ -210,6 +211,24 @@ int vp_pack_host(const int32_t* n_steps_b, const int16_t* lane_dst_b, const int6
                  const void* rows, int64_t row_bytes,
                  void* staged, int64_t staged_capacity_bytes, int32_t* src_map,
                  int32_t* status, void* device_scratch, size_t device_scratch_bytes, void* cuda_stream);
+
+/*
+ * Work counters of the last vp_schedule_batch that used `workspace` (device): copies three
+ * uint64 to host `out3` after synchronising the stream: activations emitted, (family, start)
+ * binding tasks run, AA sweeps run over all tasks.  Used to count the algorithmic operations
+ * of Section 4.2 "Planning complexity" for a measured batch.
+ */
+int vp_schedule_read_stats(const void* workspace, void* cuda_stream, uint64_t* out3);
+
+/*
+ * Per-kernel timing for benchmarks (off by default).  While enabled, every call records CUDA
+ * events on the caller's stream around its own launches; vp_profile_read synchronises those
+ * events, returns the summed device time and the number of timed launches of one kind since
+ * the last read (kind 0: schedule kernel, 1: the three pack index kernels as a group, 2: the
+ * pack copy kernel) and discards them.  Creating events allocates driver resources.
+ */
+int vp_profile_enable(int on);
+int vp_profile_read(int kind, double* total_ms, int64_t* launches);
 
 /* Number of kernels the library has launched in this process (for launch accounting). */
 int64_t vp_kernel_launch_count(void);

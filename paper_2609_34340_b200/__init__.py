@@ -18,6 +18,9 @@ from .binding import (  # noqa: F401
     pack,
     pack_host,
     kernel_launch_count,
+    schedule_read_stats,
+    profile_enable,
+    profile_read,
     library_path,
     ST_NEGATIVE, ST_OVERFLOW_RISK, ST_DIAG_NONZERO, ST_NOT_GRANULE, ST_BAD_TAU, ST_UNCOVERED,
     ST_NO_PROGRESS, ST_STEP_LIMIT, ST_PACK_MISMATCH, ST_PACK_CAPACITY,

@@ -87,6 +87,9 @@ def _load():
     lib.vp_pack_host_scratch_bytes.restype = sz
     lib.vp_pack_host.argtypes = pack_args + [P, sz, P]
     lib.vp_kernel_launch_count.restype = i64
+    lib.vp_schedule_read_stats.argtypes = [P, P, P]
+    lib.vp_profile_enable.argtypes = [i32]
+    lib.vp_profile_read.argtypes = [i32, C.POINTER(C.c_double), C.POINTER(i64)]
     lib.vp_strerror.argtypes = [i32]
     lib.vp_strerror.restype = C.c_char_p
     _lib = lib
@@ -113,6 +116,24 @@ def _stream(stream) -> C.c_void_p:
 
 def kernel_launch_count() -> int:
     return int(_load().vp_kernel_launch_count())
+
+
+def schedule_read_stats(workspace: torch.Tensor, stream=None) -> dict:
+    """``vp_schedule_read_stats``: work counters of the last batch scheduled with ``workspace``."""
+    out = (C.c_uint64 * 3)()
+    _check(_load().vp_schedule_read_stats(_ptr(workspace), _stream(stream), out), "vp_schedule_read_stats")
+    return dict(activations=int(out[0]), tasks=int(out[1]), sweeps=int(out[2]))
+
+
+def profile_enable(on: bool) -> None:
+    _check(_load().vp_profile_enable(1 if on else 0), "vp_profile_enable")
+
+
+def profile_read(kind: int):
+    """``vp_profile_read``: (total device ms, launches) of kind 0 schedule / 1 pack index / 2 pack copy."""
+    ms, n = C.c_double(0), C.c_int64(0)
+    _check(_load().vp_profile_read(int(kind), C.byref(ms), C.byref(n)), "vp_profile_read")
+    return float(ms.value), int(n.value)
 
 
 class Catalog:

@@ -353,11 +353,14 @@ extern "C" int vp_pack(const int32_t* n_steps_b, const int16_t* lane_dst_b, cons
     const int blocks = (n_chunks + kWarpsPerBlock - 1) / kWarpsPerBlock;
     if (cudaMemsetAsync(w.flags, 0, 256, stream) != cudaSuccess) return VP_E_CUDA;
     if (cudaMemsetAsync(status, 0, sizeof(int32_t), stream) != cudaSuccess) return VP_E_CUDA;
+    vp_prof_mark(1, 0, stream);
     pack_count_kernel<<<blocks, kWarpsPerBlock * 32, 0, stream>>>(expert_idx, E, N, rank, experts_per_rank, w.hist, status);
     pack_plan_kernel<<<1, VP_MAX_N, 0, stream>>>(n_steps_b, lane_dst_b, lane_bytes_b, send_off_b, N, rank, k_max, n_chunks,
                                                  row_bytes, staged_capacity_bytes, w, status);
     pack_map_kernel<<<blocks, kWarpsPerBlock * 32, 0, stream>>>(expert_idx, E, N, rank, experts_per_rank, w, src_map);
     g_vp_launches += 3;
+    vp_prof_mark(1, 1, stream);
+    vp_prof_mark(2, 0, stream);
 
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
@@ -382,5 +385,6 @@ extern "C" int vp_pack(const int32_t* n_steps_b, const int16_t* lane_dst_b, cons
             pack_copy_plain_kernel<uint8_t><<<grid, 256, 0, stream>>>((const char*)rows, (char*)staged, w.dst_row, w.flags, T, topk, row_bytes);
     }
     g_vp_launches++;
+    vp_prof_mark(2, 1, stream);
     return cudaGetLastError() == cudaSuccess ? VP_OK : VP_E_CUDA;
 }

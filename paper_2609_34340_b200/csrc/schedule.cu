@@ -144,6 +144,7 @@ vp_schedule_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand, co
     uint8_t* bind_src = smem_raw + L.bind_src;
     uint8_t* bind_dst = smem_raw + L.bind_dst;
     __shared__ int s_b, s_flags, s_shape, s_task;
+    unsigned long long n_act = 0, n_tasks_done = 0, n_sweeps = 0;     // work counters (per warp / thread 0)
     __shared__ int64_t s_tau, s_left, s_score;
     __shared__ int64_t s_cap[VP_MAX_CLASSES];
 
@@ -320,6 +321,7 @@ vp_schedule_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand, co
                         }
                         __syncwarp();
                         F_new = warp_sum_i64(part);                      // Eq. (8), in bytes
+                        n_sweeps++;
                         if (F_new <= F_old) break;
                         F_old = F_new;
                     }
@@ -330,6 +332,7 @@ vp_schedule_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand, co
                         tmax = max_i64(tmax, x * dc.class_wdiv[cls]);
                     }
                     tmax = warp_max_i64(tmax);
+                    n_tasks_done++;
                     if (lane == 0) {
                         task_f[task] = F_new;
                         task_den[task] = F_new > 0 ? kp.lambda_ns * dc.W + tmax : 1;
@@ -413,12 +416,16 @@ vp_schedule_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand, co
         }
         for (int kk = k + tid; kk < kp.k_max; kk += NT) chan_id[(size_t)b * kp.k_max + kk] = -1;
         if (tid == 0) {
+            n_act += (unsigned long long)k;
             n_steps[b] = k;
             status[b] = st;
             if (tau_out) tau_out[b] = tau;
         }
         __syncthreads();
     }
+    unsigned long long* stats = (unsigned long long*)(counter + 4);
+    if (tid == 0 && n_act) atomicAdd(&stats[0], n_act);
+    if (lane == 0 && n_tasks_done) { atomicAdd(&stats[1], n_tasks_done); atomicAdd(&stats[2], n_sweeps); }
 }
 
 struct Launch {
@@ -514,6 +521,7 @@ extern "C" int vp_schedule_batch(const vp_catalog* c, const vp_sched_params* p, 
         chan_id, lane_dst, lane_inst, lane_bytes, send_off, recv_off, tau_ns_out, status, ws_drem, counter,     \
         L.drem_in_smem)
         if (!rc) {
+            vp_prof_mark(0, 0, stream);
             switch (c->dc.g) {
                 case 1: VP_LAUNCH(1); break;
                 case 2: VP_LAUNCH(2); break;
@@ -522,9 +530,17 @@ extern "C" int vp_schedule_batch(const vp_catalog* c, const vp_sched_params* p, 
             }
             g_vp_launches++;
             if (cudaGetLastError() != cudaSuccess) rc = VP_E_CUDA;
+            vp_prof_mark(0, 1, stream);
         }
 #undef VP_LAUNCH
     }
     if (prev >= 0) cudaSetDevice(prev);
     return rc;
+}
+
+extern "C" int vp_schedule_read_stats(const void* workspace, void* cuda_stream, uint64_t* out3) {
+    if (!workspace || !out3) return VP_E_BAD_ARG;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    if (cudaMemcpyAsync(out3, (const char*)workspace + 16, 24, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return VP_E_CUDA;
+    return cudaStreamSynchronize(stream) == cudaSuccess ? VP_OK : VP_E_CUDA;
 }

@@ -46,4 +46,8 @@ struct vp_catalog {
 
 extern long long g_vp_launches;
 
+// Profiling hook: when enabled, records a CUDA event on `stream` before (edge 0) / after (edge 1)
+// the kernels of one kind (0 schedule kernel, 1 pack index kernels, 2 pack copy kernel).
+void vp_prof_mark(int kind, int edge, cudaStream_t stream);
+
 static inline size_t vp_align256(size_t x) { return (x + 255) & ~(size_t)255; }

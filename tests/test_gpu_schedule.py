@@ -183,7 +183,7 @@ def test_config_full_batch(vp, oracle_lib, idx):
 def _validate_all(oc, D, got, granule):
     for b in range(D.shape[0]):
         plan = {k: got[k][b] for k in KEYS}
-        assert got["status"][b] == 0
+        assert got["status"][b] == 0, f"matrix {b}: status {got['status'][b]} after {got['n_steps'][b]} steps"
         assert oc.check_plan(D[b], plan, int(got["tau_ns"][b]), granule) == 0, f"matrix {b} invalid"
         K = int(got["n_steps"][b])
         assert (got["send_off"][b][K] == D[b].sum(1)).all() and (got["recv_off"][b][K] == D[b].sum(0)).all()
@@ -215,8 +215,8 @@ def test_config4_full_batch(vp, oracle_lib):
     assert dc.node_symmetric == 1 and (dc.n_shapes, dc.n_families) == (4095, 4160)
     D = c["demand"]
     p = _params(vp, w)
-    sub = 256
-    plan = vp.Plan.empty(sub, 256, p.k_max or 2048, "cuda")
+    sub = 128
+    plan = vp.Plan.empty(sub, 256, p.k_max, "cuda")
     rng = np.random.default_rng(0)
     for lo in range(0, D.shape[0], sub):
         part = D[lo:lo + sub]
@@ -224,6 +224,8 @@ def test_config4_full_batch(vp, oracle_lib):
         got = plan.cpu()
         Dn = part.numpy()
         _validate_all(oc, Dn, got, w.granule_bytes)
-        sample = rng.choice(sub, size=1, replace=False)
+        sample = rng.choice(sub, size=1, replace=False) if lo % 256 == 0 else []
+        if not len(sample):
+            continue
         want = oc.schedule_batch(Dn[sample], w)
         _assert_same({k: got[k][sample] if k != "k_max" else got[k] for k in got}, want)

@@ -108,7 +108,9 @@ def build_config(idx: int, device: str = "cpu", batch: Optional[int] = None,
                                        _matrix_seed(base, b), device=device))
     else:
         raise ValueError("scheduler configs are 1..4; use build_pack_case for config 5")
-    params = SchedParams(granule_bytes=granule).resolved(N)
+    # the one-NIC-per-switch tree needs at least 16*(G-2) rounds for dense cross-node demand, which
+    # at N=256 already exceeds 8N for skewed matrices: config 4 gets room for 16N activations
+    params = SchedParams(granule_bytes=granule, k_max=16 * N if idx == 4 else 0).resolved(N)
     return dict(config=idx, catalog=cat, demand=torch.stack(mats), params=params)
 
 
