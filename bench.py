@@ -190,13 +190,17 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    for _ in range(args.warmup):
+    sampler = ClockSampler(local_rank)     # sampled from warm-up to the end of the timed region
+    sampler.start()
+    t_warm, n_warm = time.perf_counter(), 0
+    while n_warm < args.warmup or (time.perf_counter() - t_warm < args.min_warmup_s and n_warm < 100000):
         step()
+        n_warm += 1
+        if n_warm % 16 == 0:
+            torch.cuda.synchronize()
     barrier()
     assert int(pstatus.item()) == 0 and int(plan.status.max().item()) == 0, "workload did not schedule cleanly"
 
-    sampler = ClockSampler(local_rank)
-    sampler.start()
     vp.profile_enable(True)
     for k in range(3):
         vp.profile_read(k)
@@ -223,7 +227,7 @@ def run_ours(args):
     value = aggregate_value(B, world, ms_per_step / 1e3)
 
     sched_avg = sched_ms / max(n_sched, 1) * (B // sub)
-    if sub < B:
+    if sub < B or args.no_e2e:
         e2e_ms, h2d, d2h, e2e_steps = None, 0, 0, 0
     else:
         e2e_ms, h2d, d2h, e2e_steps = run_e2e(vp, args, world, local_rank, dev, sched, pk, dc, params, pplan, idx, rows,
@@ -317,7 +321,7 @@ def finish(args, world, cat, w, B, N, T, topk, R, prank, row_bytes, pack_bytes, 
                 if e2e_ms else None),
         "gpu_launches": int(launches), "clocks": clocks,
     }
-    line["cpu_baseline"] = cpu_baseline(sched, pk, budget_s=20.0) if world == 1 else None
+    line["cpu_baseline"] = cpu_baseline(sched, pk, budget_s=20.0) if world == 1 and not args.no_cpu_baseline else None
     print(json.dumps(line))
 
 
@@ -416,6 +420,11 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--sched-config", type=int, default=2, choices=[1, 2, 3, 4])
+    ap.add_argument("--min-warmup-s", type=float, default=1.0,
+                    help="keep warming up (beyond --warmup steps) until this many seconds have passed, so that "
+                         "clocks settle and nvidia-smi has samples under load")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the CPU oracle leg (profiling runs)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":

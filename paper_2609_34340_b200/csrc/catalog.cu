@@ -124,7 +124,8 @@ extern "C" int vp_load_catalog(const void* topology, size_t topo_bytes, const vo
     std::vector<int> rowsum(G), colsum(G);
     std::vector<char> seen((size_t)G * G, 0);
     std::vector<uint32_t> fam_slot((size_t)n_fam * N);
-    std::vector<uint8_t> fam_inslot((size_t)n_fam * N);
+    std::vector<uint8_t> fam_cls((size_t)n_fam * N);
+    std::vector<uint16_t> fam_in((size_t)n_fam * N);
     int max_nnz = 0, max_bucket = 0;
     for (int s = 0; s < n_shapes; s++) {
         if (shape_ptr[s + 1] <= shape_ptr[s] || bucket_ptr[s + 1] < bucket_ptr[s]) return VP_E_BAD_CATALOG;
@@ -156,7 +157,8 @@ extern "C" int vp_load_catalog(const void* topology, size_t topo_bytes, const vo
                     if (used[q.res[k]]++) return VP_E_BAD_CATALOG;
                 if (fill[q.d] >= g) return VP_E_BAD_CATALOG;
                 fam_slot[(size_t)f * N + r] = (uint32_t)id | ((uint32_t)q.d << 16) | ((uint32_t)q.cls << 24);
-                fam_inslot[(size_t)f * N + q.d * g + fill[q.d]++] = (uint8_t)r;
+                fam_cls[(size_t)f * N + r] = (uint8_t)q.cls;
+                fam_in[(size_t)f * N + q.d * g + fill[q.d]++] = (uint16_t)(r | (q.cls << 8));
             }
             for (int r = 0; r < N; r++) {   // N lanes with every count <= M_ad and sum M = N  =>  counts equal M
                 const HostInst& q = inst[h.u16(off_fam + 2 * ((size_t)f * N + r))];
@@ -259,11 +261,19 @@ extern "C" int vp_load_catalog(const void* topology, size_t topo_bytes, const vo
     dc.max_bucket = max_bucket; dc.bw_max = bw_max; dc.W = W;
     for (size_t k = 0; k < rates.size(); k++) { dc.class_bw[k] = rates[k]; dc.class_wdiv[k] = W / rates[k]; }
     int rc = VP_OK;
-    if (!rc) rc = upload(c, term_ptr, &dc.shape_ptr);
-    if (!rc) rc = upload(c, term, &dc.term);
+    // fixed-stride copy of the terms (max_terms per shape, zero-count padding) so the scoring loop unrolls
+    int max_terms = 0;
+    for (int s = 0; s < n_shapes; s++) max_terms = std::max(max_terms, (int)(term_ptr[s + 1] - term_ptr[s]));
+    std::vector<uint32_t> term_pad((size_t)n_shapes * max_terms, 0);
+    for (int s = 0; s < n_shapes; s++)
+        for (uint32_t e = term_ptr[s]; e < term_ptr[s + 1]; e++) term_pad[(size_t)s * max_terms + (e - term_ptr[s])] = term[e];
+    dc.max_terms = max_terms;
+    if (!rc) rc = upload(c, term_pad, &dc.term);
     if (!rc) rc = upload(c, bucket_ptr, &dc.bucket_ptr);
     if (!rc) rc = upload(c, fam_slot, &dc.fam_slot);
-    if (!rc) rc = upload(c, fam_inslot, &dc.fam_inslot);
+    if (!rc) rc = upload(c, fam_cls, &dc.fam_cls);
+    if (!rc) rc = upload(c, fam_in, &dc.fam_in);
+    dc.n_terms = (int)term.size();      // real (unpadded) multiply-adds of one scoring pass
     if (!rc) rc = upload(c, forced_ptr, &dc.forced_ptr);
     if (!rc) rc = upload(c, forced_cell, &dc.forced_cell);
     if (!rc) rc = upload(c, forced_bw, &dc.forced_bw);

@@ -4,15 +4,30 @@
 // from a counter).  The residual demand D_rem lives in shared memory when
 // N <= 64 and in an L2-resident workspace slot otherwise; the group sums D-hat
 // are kept in shared memory and updated incrementally after every activation.
-// Per iteration: (A) every thread scores shapes (Eq. 6) and a block-wide
-// (value, lowest index) arg-max picks M*; (B) every (family, start) pair of
-// the bucket is one warp-level task that runs the Alternating Algorithm, one
-// lane per rank group, each lane solving its g x g assignment by enumerating
-// the g! permutations in lexicographic order (Eq. 7, 8) and then evaluating
-// Eq. (9), (10); (C) warp 0 picks the best start per family and the family of
-// largest utility by exact 128-bit cross-multiplication; (D) all threads emit
-// the activation, subtract it from D_rem / D-hat and advance the running
-// send / receive offsets.
+// The catalog (shape terms, per-family slot tables) is staged in shared memory
+// once per CTA when it fits.
+//
+// Value type.  Every demand entry and every lane capacity is a multiple of the
+// granule, so a matrix whose capacities are below 2^25 granules is decomposed
+// in 32-bit granule units (credits, sums of four credits and a 5-bit
+// permutation tag then fit one 32-bit key); other matrices run the same code
+// on 64-bit byte values.  Both give the same plan.
+//
+// Per iteration, three block barriers:
+//  (A) every thread scores shapes (Eq. 6) on fixed-stride term lists; a
+//      (value, lowest index) arg-max by warp shuffles, then across warps through
+//      shared memory, picks M*;
+//  (B) every (family, start) pair of the bucket is one warp-level task that runs
+//      the Alternating Algorithm (Eq. 7, 8).  For groups of four ranks a team
+//      of 8 / 4 / 2 lanes shares one rank group: the 16 credits go to shared
+//      memory, each lane evaluates its 3 / 6 / 12 of the 24 permutations, and a
+//      shuffle reduction keeps the first maximum in lexicographic order.  With
+//      more than 16 groups (or other group sizes) one lane owns a group and
+//      enumerates all g! permutations in registers.  Then Evaluate (Eq. 9, 10);
+//  (C) every warp redundantly picks the best start per family and the family of
+//      largest utility (exact 128-bit cross-multiplication), no barrier;
+//  (D) all threads emit the activation, subtract it from D_rem / D-hat and write
+//      the next row of the running send / receive offsets.
 #include <cuda_runtime.h>
 
 #include <utility>
@@ -24,32 +39,42 @@ namespace {
 struct KParams {
     int64_t lambda_ns, granule;
     int k_target, n_start, i_aa, k_max;
-    int max_tasks;
+    int max_tasks, stage_terms, stage_fam, stage_bucket, drem_in_smem;
 };
 
 struct Smem {                 // offsets (bytes) into dynamic shared memory
-    int drem, dhat, tbl, send_acc, recv_acc, red, task_f, task_den, bind_src, bind_dst, total;
+    int drem, dhat, tbl, send_acc, recv_acc, red, task_f, task_den, bind_src, bind_dst, cred, slotw;
+    int term, fam_in, fam_cls, bucket, total;
 };
 
-__host__ __device__ inline Smem smem_layout(const DevCat& dc, int max_tasks, bool drem_in_smem) {
+__host__ __device__ inline int align16(int x) { return (x + 15) & ~15; }
+__host__ __device__ inline int cred_bytes_per_warp(int lpg) { return lpg > 1 ? (32 / lpg) * 17 * 8 : 0; }
+
+__host__ __device__ inline Smem smem_layout(const DevCat& dc, const KParams& kp, int n_warps, int lpg) {
     Smem L;
     int o = 0;
-    L.drem = o;      o += drem_in_smem ? dc.N * dc.N * 8 : 0;
+    L.drem = o;      o += kp.drem_in_smem ? dc.N * dc.N * 8 : 0;
     L.dhat = o;      o += dc.G * dc.G * 8;
     L.tbl = o;       o += dc.sym ? dc.tbl_size * 8 : 0;
     L.send_acc = o;  o += dc.N * 8;
     L.recv_acc = o;  o += dc.N * 8;
     L.red = o;       o += 64 * 8;
-    L.task_f = o;    o += max_tasks * 8;
-    L.task_den = o;  o += max_tasks * 8;
-    L.bind_src = o;  o += (max_tasks * dc.N + 15) & ~15;
-    L.bind_dst = o;  o += (max_tasks * dc.N + 15) & ~15;
+    L.task_f = o;    o += kp.max_tasks * 8;
+    L.task_den = o;  o += kp.max_tasks * 8;
+    L.cred = o;      o += n_warps * cred_bytes_per_warp(lpg);
+    L.slotw = o;     o += dc.max_bucket * dc.N * 4;
+    L.bind_src = o;  o += align16(kp.max_tasks * dc.N);
+    L.bind_dst = o;  o += align16(kp.max_tasks * dc.N);
+    L.term = o;      o += kp.stage_terms ? align16(dc.n_shapes * dc.max_terms * 4) : 0;
+    L.fam_in = o;    o += kp.stage_fam ? align16(dc.n_families * dc.N * 2) : 0;
+    L.fam_cls = o;   o += kp.stage_fam ? align16(dc.n_families * dc.N) : 0;
+    L.bucket = o;    o += kp.stage_bucket ? align16((dc.n_shapes + 1) * 4) : 0;
     L.total = o;
     return L;
 }
 
-__device__ __forceinline__ int64_t min_i64(int64_t a, int64_t b) { return a < b ? a : b; }
-__device__ __forceinline__ int64_t max_i64(int64_t a, int64_t b) { return a > b ? a : b; }
+template <typename T> __device__ __forceinline__ T min_v(T a, T b) { return a < b ? a : b; }
+template <typename T> __device__ __forceinline__ T max_v(T a, T b) { return a > b ? a : b; }
 __device__ __forceinline__ int64_t ceil_div_i64(int64_t a, int64_t b) { return (a + b - 1) / b; }
 
 // q-th element of the p-th lexicographic permutation of g items (factorial number system)
@@ -72,35 +97,41 @@ __host__ __device__ constexpr unsigned perm_packed(int g, int p) {   // 2 bits p
     for (int q = 0; q < g; q++) w |= (unsigned)perm_entry(g, p, q) << (2 * q);
     return w;
 }
+__host__ __device__ constexpr unsigned long long perm4_word(int w) {  // packed permutations 8w .. 8w+7, one per byte
+    unsigned long long x = 0;
+    for (int k = 0; k < 8; k++) x |= (unsigned long long)perm_packed(4, w * 8 + k) << (8 * k);
+    return x;
+}
+__device__ __forceinline__ unsigned perm4_packed_rt(int p) {
+    constexpr unsigned long long W0 = perm4_word(0), W1 = perm4_word(1), W2 = perm4_word(2);
+    const unsigned long long w = p < 8 ? W0 : (p < 16 ? W1 : W2);
+    return (unsigned)(w >> (8 * (p & 7))) & 0xffu;
+}
+
 template <int GS, int P, int Q> struct PermAt { static constexpr int value = perm_entry(GS, P, Q); };
 template <int GS, int P> struct PermPacked { static constexpr unsigned value = perm_packed(GS, P); };
 
-template <int GS, int P, int... Q>
-__device__ __forceinline__ int64_t perm_value(const int64_t (&c)[GS][GS], std::integer_sequence<int, Q...>) {
+template <int GS, typename V, int P, int... Q>
+__device__ __forceinline__ V perm_value(const V (&c)[GS][GS], std::integer_sequence<int, Q...>) {
     return (c[PermAt<GS, P, Q>::value][Q] + ...);
 }
-template <int GS, int P>
-__device__ __forceinline__ void perm_try(const int64_t (&c)[GS][GS], int64_t& best, unsigned& bpk) {
-    const int64_t v = perm_value<GS, P>(c, std::make_integer_sequence<int, GS>{});
-    if (v > best) { best = v; bpk = PermPacked<GS, P>::value; }
-}
-template <int GS, int... P>
-__device__ __forceinline__ int64_t best_assignment_impl(const int64_t (&c)[GS][GS], unsigned& bpk,
-                                                        std::integer_sequence<int, P...>) {
-    int64_t best = -1;
-    bpk = 0;
-    (perm_try<GS, P>(c, best, bpk), ...);
+template <int GS, typename V, int... P>
+__device__ __forceinline__ V best_assignment_impl(const V (&c)[GS][GS], unsigned& bpk, std::integer_sequence<int, P...>) {
+    V best = 0;
+    bpk = PermPacked<GS, 0>::value;
+    bool first = true;
+    (([&] {
+         const V v = perm_value<GS, V, P>(c, std::make_integer_sequence<int, GS>{});
+         if (first || v > best) { best = v; bpk = PermPacked<GS, P>::value; first = false; }
+     }()),
+     ...);
     return best;
 }
-// Exact g x g assignment: maximise sum_q c[phi(q)][q] over all g! permutations, enumerated in
-// lexicographic order of (phi(0), ..., phi(g-1)); the first maximum wins.
-template <int GS>
-__device__ __forceinline__ int64_t best_assignment(const int64_t (&c)[GS][GS], int (&phi)[GS]) {
-    unsigned bpk;
-    const int64_t best = best_assignment_impl<GS>(c, bpk, std::make_integer_sequence<int, factorial(GS)>{});
-#pragma unroll
-    for (int q = 0; q < GS; q++) phi[q] = (int)((bpk >> (2 * q)) & 3u);
-    return best;
+// Exact g x g assignment in registers: maximise sum_q c[phi(q)][q] over all g! permutations, enumerated
+// in lexicographic order of (phi(0), ..., phi(g-1)); the first maximum wins.  Returns phi packed 2 bits each.
+template <int GS, typename V>
+__device__ __forceinline__ V best_assignment(const V (&c)[GS][GS], unsigned& bpk) {
+    return best_assignment_impl<GS, V>(c, bpk, std::make_integer_sequence<int, factorial(GS)>{});
 }
 
 __device__ __forceinline__ int64_t warp_sum_i64(int64_t v) {
@@ -110,7 +141,7 @@ __device__ __forceinline__ int64_t warp_sum_i64(int64_t v) {
 }
 __device__ __forceinline__ int64_t warp_max_i64(int64_t v) {
 #pragma unroll
-    for (int o = 16; o; o >>= 1) v = max_i64(v, __shfl_xor_sync(0xffffffffu, v, o));
+    for (int o = 16; o; o >>= 1) v = max_v(v, __shfl_xor_sync(0xffffffffu, v, o));
     return v;
 }
 
@@ -122,39 +153,485 @@ __device__ __forceinline__ bool util_greater(int64_t f1, int64_t d1, int64_t f2,
     return hi1 > hi2 || (hi1 == hi2 && lo1 > lo2);
 }
 
-template <int GS>
-__global__ void __launch_bounds__(512)
+// ---- team path (groups of four ranks, LPG lanes per group) -----------------------------------------
+//
+// Team lane tl owns the credit elements (i, q) with q in qv[] and i in iv[]:
+//   LPG 8: q = tl & 3, i in {tl >> 2, (tl >> 2) + 2};  LPG 4: q = tl, all i;  LPG 2: q in {tl, tl + 2}, all i
+// and the permutations tl*PPL .. tl*PPL + PPL - 1 (PPL = 24 / LPG).
+template <int LPG> struct TeamCfg {
+    static constexpr int NQ = LPG >= 4 ? 1 : 4 / LPG;
+    static constexpr int NI = LPG == 8 ? 2 : 4;
+    static constexpr int PPL = 24 / LPG;
+    static constexpr int NW = (PPL + 3) / 4;          // 32-bit words holding this lane's packed permutations
+};
+
+// Best permutation of the team's 4 x 4 credit tile (first maximum in lexicographic order); every team
+// lane returns the value and receives the permutation packed 2 bits per position.
+template <int LPG>
+__device__ __forceinline__ int64_t team_best(const int64_t* cred, int tl, const unsigned (&mp)[TeamCfg<LPG>::NW],
+                                             unsigned& bpk) {
+    constexpr int PPL = TeamCfg<LPG>::PPL;
+    int64_t best = -1;
+    int bp = 0;
+    bpk = 0;
+#pragma unroll
+    for (int pp = 0; pp < PPL; pp++) {
+        const unsigned pk = (mp[pp >> 2] >> (8 * (pp & 3))) & 0xffu;
+        const int64_t v = cred[(pk & 3) * 4] + cred[((pk >> 2) & 3) * 4 + 1] + cred[((pk >> 4) & 3) * 4 + 2] +
+                          cred[((pk >> 6) & 3) * 4 + 3];
+        if (v > best) { best = v; bp = tl * PPL + pp; bpk = pk; }
+    }
+#pragma unroll
+    for (int o = LPG / 2; o; o >>= 1) {                // within the team: larger value, then lower permutation index
+        const int64_t ov = __shfl_xor_sync(0xffffffffu, best, o);
+        const int op = __shfl_xor_sync(0xffffffffu, bp, o);
+        const unsigned ok = __shfl_xor_sync(0xffffffffu, bpk, o);
+        if (ov > best || (ov == best && op < bp)) { best = ov; bp = op; bpk = ok; }
+    }
+    return best;
+}
+// 32-bit granule units: value and permutation travel as one key (sum << 5 | 31 - p), so a plain maximum
+// keeps the larger sum and, among equal sums, the lower permutation index.  Sums are below 2^27.
+// pidx[pp][q] is the tile element (row * 4 + q) the lane's pp-th permutation reads at position q; lut maps
+// the 5-bit tag back to the packed permutation.
+template <int LPG>
+__device__ __forceinline__ uint32_t team_best(const uint32_t* cred, int tl, const unsigned (&mp)[TeamCfg<LPG>::NW],
+                                              const uint8_t (&pidx)[TeamCfg<LPG>::PPL][4], const uint8_t* lut,
+                                              unsigned& bpk) {
+    constexpr int PPL = TeamCfg<LPG>::PPL;
+    const uint32_t tag0 = (uint32_t)(31 - tl * PPL);
+    uint32_t key = 0;
+#pragma unroll
+    for (int pp = 0; pp < PPL; pp++) {
+        const uint32_t v = cred[pidx[pp][0]] + cred[pidx[pp][1]] + cred[pidx[pp][2]] + cred[pidx[pp][3]];
+        key = max_v(key, (v << 5) + (tag0 - pp));
+    }
+#pragma unroll
+    for (int o = LPG / 2; o; o >>= 1) key = max_v(key, __shfl_xor_sync(0xffffffffu, key, o));
+    bpk = lut[key & 31u];
+    return key >> 5;
+}
+template <int LPG>
+__device__ __forceinline__ int64_t team_best(const int64_t* cred, int tl, const unsigned (&mp)[TeamCfg<LPG>::NW],
+                                             const uint8_t (&pidx)[TeamCfg<LPG>::PPL][4], const uint8_t* lut,
+                                             unsigned& bpk) {
+    return team_best<LPG>(cred, tl, mp, bpk);
+}
+
+// Per-CTA pointers and constants shared by the two value types.
+struct Ctx {
+    int N, G, tid, NT, lane, warp, n_warps;
+    int64_t *Dhat, *tbl, *send_acc, *recv_acc, *red, *task_f, *task_den;
+    uint8_t *bind_src, *bind_dst;
+    uint32_t* slotw;
+    unsigned char* cred_warp;          // this warp's credit tiles
+    const uint32_t* p_term;
+    const uint16_t* p_fam_in;
+    const uint8_t* p_fam_cls;
+    const uint32_t* p_bucket_ptr;
+    const uint8_t* perm_lut;           // tag (31 - p) -> packed permutation p of four items
+    const int64_t* tscale;             // per rate class: (rate_lcm / bw) x bytes per value unit
+    int32_t* chan_id_b;                // this matrix's outputs
+    int16_t* lane_dst_b;
+    uint16_t* lane_inst_b;
+    int64_t *lane_bytes_b, *send_off_b, *recv_off_b;
+};
+
+struct Counters { unsigned long long tasks, sweeps; long long cyc[6], t_mark; };
+
+#ifdef VP_PHASE_TIMING
+#define VP_TICK(i) do { long long now_ = clock64(); cnt.cyc[i] += now_ - cnt.t_mark; cnt.t_mark = now_; } while (0)
+#else
+#define VP_TICK(i) do { } while (0)
+#endif
+
+// Algorithm 2 main loop for one matrix whose residual demand is held as values of type V
+// (V = int64_t: bytes, unit = 1; V = uint32_t: granules, unit = granule_bytes).
+template <int GS, int LPG, typename V>
+__device__ __forceinline__ void decompose(const DevCat& dc, const KParams& kp, const Ctx& c, V* Drem, const V* cap,
+                                          int64_t unit, int64_t left, int& k, int& st, Counters& cnt) {
+    using TC = TeamCfg<LPG>;
+    const int N = c.N, G = c.G, tid = c.tid, NT = c.NT, lane = c.lane, warp = c.warp, n_warps = c.n_warps;
+    const int team = lane / LPG, tl = lane % LPG;
+    int qv[TC::NQ], iv[TC::NI];
+    unsigned mp[TC::NW];
+    if constexpr (LPG > 1) {
+#pragma unroll
+        for (int kq = 0; kq < TC::NQ; kq++) qv[kq] = (tl & 3) + kq * LPG;
+#pragma unroll
+        for (int m = 0; m < TC::NI; m++) iv[m] = LPG == 8 ? (tl >> 2) + 2 * m : m;
+#pragma unroll
+        for (int w = 0; w < TC::NW; w++) mp[w] = 0;
+#pragma unroll
+        for (int pp = 0; pp < TC::PPL; pp++) mp[pp >> 2] |= perm4_packed_rt(tl * TC::PPL + pp) << (8 * (pp & 3));
+    }
+    uint8_t pidx[TC::PPL][4];
+    if constexpr (LPG > 1) {
+#pragma unroll
+        for (int pp = 0; pp < TC::PPL; pp++) {
+            const unsigned pk = (mp[pp >> 2] >> (8 * (pp & 3))) & 0xffu;
+#pragma unroll
+            for (int q = 0; q < 4; q++) pidx[pp][q] = (uint8_t)(((pk >> (2 * q)) & 3) * 4 + q);
+        }
+    }
+    V* cred = (V*)c.cred_warp + team * 17;
+    const int n_score_warps = min(n_warps, (dc.n_shapes + 31) >> 5);
+
+    for (;;) {
+        if (left == 0) break;
+        if (k == kp.k_max) { st |= VP_ST_STEP_LIMIT; break; }
+        // (A) Eq. (6): shape scores, first maximum
+        if (dc.sym) {
+            const int S = dc.S, P = dc.P;
+            for (int e = tid; e < dc.tbl_size; e += NT) {
+                int q2 = e % S, q = (e / S) % S, delta = e / (S * S);
+                int64_t s = 0;
+                for (int n = 0; n < P; n++) {
+                    int n2 = n + delta; if (n2 >= P) n2 -= P;
+                    s += c.Dhat[(size_t)(n * S + q) * G + n2 * S + q2];
+                }
+                c.tbl[e] = s;
+            }
+            __syncthreads();
+        }
+        if (warp < n_score_warps) {
+            int64_t best = -1;
+            int best_s = 0x7fffffff;
+            for (int s = tid; s < dc.n_shapes; s += NT) {
+                const uint32_t* tp = c.p_term + (size_t)s * dc.max_terms;
+                int64_t score = 0;
+#pragma unroll 4
+                for (int e = 0; e < dc.max_terms; e++) {
+                    const uint32_t w = tp[e];
+                    score += c.tbl[w & 0xffffu] * (int64_t)(w >> 16);
+                }
+                if (score > best) { best = score; best_s = s; }     // ascending s: keeps the first maximum
+            }
+#pragma unroll
+            for (int o = 16; o; o >>= 1) {
+                int64_t ov = __shfl_xor_sync(0xffffffffu, best, o);
+                int oi = __shfl_xor_sync(0xffffffffu, best_s, o);
+                if (ov > best || (ov == best && oi < best_s)) { best = ov; best_s = oi; }
+            }
+            if (lane == 0) { c.red[warp] = best; c.red[32 + warp] = best_s; }
+        }
+        __syncthreads();
+        int64_t best = -1;
+        int best_s = 0x7fffffff;
+        for (int w = 0; w < n_score_warps; w++) {
+            const int64_t v = c.red[w];
+            const int si = (int)c.red[32 + w];
+            if (v > best || (v == best && si < best_s)) { best = v; best_s = si; }
+        }
+        if (best <= 0) { st |= VP_ST_UNCOVERED; break; }
+        const int f0 = (int)c.p_bucket_ptr[best_s], H = (int)c.p_bucket_ptr[best_s + 1] - f0;
+        const int n_tasks = H * kp.n_start;
+        VP_TICK(1);
+
+        // (B) MultiStartAA: one warp per (family, start)
+        for (int task = warp; task < n_tasks; task += n_warps) {
+            const int h = task / kp.n_start, f = f0 + h, t = task % kp.n_start;
+            const uint16_t* fin = c.p_fam_in + (size_t)f * N;
+            const uint8_t* fcls = c.p_fam_cls + (size_t)f * N;
+            uint8_t* srcb = c.bind_src + (size_t)task * N;
+            uint8_t* dstb = c.bind_dst + (size_t)task * N;
+            // the family's slot words (instance ids) are fetched now and parked in shared memory for step (D)
+            uint32_t slot_pre[(VP_MAX_N + 31) / 32];
+            if (t == 0) {
+#pragma unroll
+                for (int rr = 0; rr < (VP_MAX_N + 31) / 32; rr++)
+                    if (rr * 32 + lane < N) slot_pre[rr] = __ldg(&dc.fam_slot[(size_t)f * N + rr * 32 + lane]);
+            }
+            for (int d = lane; d < G; d += 32)
+#pragma unroll
+                for (int q = 0; q < GS; q++) dstb[fin[d * GS + q] & 0xff] = (uint8_t)(d * GS + (q + t) % GS);
+            int64_t F_old = -1, F_new = -1, tmax = 0;
+            if constexpr (LPG > 1) {
+                // team path: one rank group per team of LPG lanes (G <= 32 / LPG)
+                const bool active = team < G;
+                const int a = team;               // the team's group: source group, then destination group
+                V cap_out[TC::NQ], cap_in[TC::NQ];
+                int r_in[TC::NQ], cls_in[TC::NQ];
+#pragma unroll
+                for (int kq = 0; kq < TC::NQ; kq++) {
+                    cap_out[kq] = 0; cap_in[kq] = 0; r_in[kq] = 0; cls_in[kq] = 0;
+                    if (active) {
+                        const unsigned w = fin[a * 4 + qv[kq]];
+                        cap_out[kq] = cap[fcls[a * 4 + qv[kq]]];
+                        cls_in[kq] = (int)(w >> 8);
+                        cap_in[kq] = cap[cls_in[kq]];
+                        r_in[kq] = (int)(w & 0xff);
+                    }
+                }
+                __syncwarp();
+                unsigned bpk = 0;
+                for (int sweep = 0; sweep < kp.i_aa; sweep++) {
+                    if (active) {                              // source half: credits of source group a
+#pragma unroll
+                        for (int kq = 0; kq < TC::NQ; kq++) {
+                            const int dq = dstb[a * 4 + qv[kq]];
+#pragma unroll
+                            for (int m = 0; m < TC::NI; m++)
+                                cred[iv[m] * 4 + qv[kq]] = min_v(Drem[(size_t)(a * 4 + iv[m]) * N + dq], cap_out[kq]);
+                        }
+                    }
+                    __syncwarp();
+                    team_best<LPG>(cred, tl, mp, pidx, c.perm_lut, bpk);
+                    if (active && tl < (LPG < 4 ? LPG : 4)) {
+#pragma unroll
+                        for (int kq = 0; kq < TC::NQ; kq++)
+                            srcb[a * 4 + qv[kq]] = (uint8_t)(a * 4 + ((bpk >> (2 * qv[kq])) & 3));
+                    }
+                    __syncwarp();
+                    if (active) {                              // destination half: credits into group a
+#pragma unroll
+                        for (int kq = 0; kq < TC::NQ; kq++) {
+                            const int sq = srcb[r_in[kq]];
+#pragma unroll
+                            for (int m = 0; m < TC::NI; m++)
+                                cred[iv[m] * 4 + qv[kq]] = min_v(Drem[(size_t)sq * N + a * 4 + iv[m]], cap_in[kq]);
+                        }
+                    }
+                    __syncwarp();
+                    const V v = team_best<LPG>(cred, tl, mp, pidx, c.perm_lut, bpk);
+                    if (active && tl < (LPG < 4 ? LPG : 4)) {
+#pragma unroll
+                        for (int kq = 0; kq < TC::NQ; kq++)
+                            dstb[r_in[kq]] = (uint8_t)(a * 4 + ((bpk >> (2 * qv[kq])) & 3));
+                    }
+                    // Eq. (8): sum over the teams.  Every lane of a team holds the team's value and the
+                    // exchanges connect equal team lanes only, so all 32 lanes end with the same total.
+                    int64_t part = active ? (int64_t)v : 0;
+#pragma unroll
+                    for (int o = 16; o >= LPG; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+                    F_new = part;
+                    cnt.sweeps++;
+                    if (F_new <= F_old) break;
+                    F_old = F_new;
+                    __syncwarp();
+                }
+                // Eq. (9) volumes are the chosen credits of the last destination half; slowest lane of Eq. (10)
+                if (active && tl < (LPG < 4 ? LPG : 4)) {
+#pragma unroll
+                    for (int kq = 0; kq < TC::NQ; kq++) {
+                        const V x = cred[((bpk >> (2 * qv[kq])) & 3) * 4 + qv[kq]];
+                        tmax = max_v(tmax, (int64_t)x * c.tscale[cls_in[kq]]);
+                    }
+                }
+                __syncwarp();
+            } else {
+                // register path: one lane per rank group
+                __syncwarp();
+                for (int sweep = 0; sweep < kp.i_aa; sweep++) {
+                    for (int a = lane; a < G; a += 32) {            // source half
+                        V cr[GS][GS];
+                        unsigned bpk;
+#pragma unroll
+                        for (int q = 0; q < GS; q++) {
+                            const int r = a * GS + q;
+                            const V cp = cap[fcls[r]];
+                            const int dq = dstb[r];
+#pragma unroll
+                            for (int i = 0; i < GS; i++) cr[i][q] = min_v(Drem[(size_t)(a * GS + i) * N + dq], cp);
+                        }
+                        best_assignment<GS, V>(cr, bpk);
+#pragma unroll
+                        for (int q = 0; q < GS; q++) srcb[a * GS + q] = (uint8_t)(a * GS + ((bpk >> (2 * q)) & 3));
+                    }
+                    __syncwarp();
+                    int64_t part = 0;
+                    tmax = 0;
+                    for (int d = lane; d < G; d += 32) {            // destination half
+                        V cr[GS][GS];
+                        int rq[GS], cls[GS];
+                        unsigned bpk;
+#pragma unroll
+                        for (int q = 0; q < GS; q++) {
+                            const unsigned w = fin[d * GS + q];
+                            rq[q] = (int)(w & 0xff);
+                            cls[q] = (int)(w >> 8);
+                            const V cp = cap[cls[q]];
+                            const int sq = srcb[rq[q]];
+#pragma unroll
+                            for (int j = 0; j < GS; j++) cr[j][q] = min_v(Drem[(size_t)sq * N + d * GS + j], cp);
+                        }
+                        part += (int64_t)best_assignment<GS, V>(cr, bpk);
+#pragma unroll
+                        for (int q = 0; q < GS; q++) {
+                            const int j = (int)((bpk >> (2 * q)) & 3);
+                            dstb[rq[q]] = (uint8_t)(d * GS + j);
+                            V x = cr[0][q];                           // the chosen credit = the lane's volume, Eq. (9)
+#pragma unroll
+                            for (int jj = 1; jj < GS; jj++) if (j == jj) x = cr[jj][q];
+                            tmax = max_v(tmax, (int64_t)x * c.tscale[cls[q]]);
+                        }
+                    }
+                    __syncwarp();
+                    F_new = warp_sum_i64(part);                      // Eq. (8)
+                    cnt.sweeps++;
+                    if (F_new <= F_old) break;
+                    F_old = F_new;
+                }
+            }
+            tmax = warp_max_i64(tmax);
+            cnt.tasks++;
+            if (t == 0) {
+#pragma unroll
+                for (int rr = 0; rr < (VP_MAX_N + 31) / 32; rr++)
+                    if (rr * 32 + lane < N) c.slotw[h * N + rr * 32 + lane] = slot_pre[rr];
+            }
+            if (lane == 0) {
+                c.task_f[task] = F_new;
+                c.task_den[task] = F_new > 0 ? kp.lambda_ns * dc.W + tmax : 1;
+            }
+        }
+        __syncthreads();
+        VP_TICK(2);
+
+        // (C) best start per family (largest F, lowest t), then largest utility, lowest family;
+        //     every warp computes it for itself, over the lanes 0 .. H-1 only
+        int64_t bf = -1, bd = 1;
+        int bt = 0x7fffffff;
+        for (int h = lane; h < H; h += 32) {
+            int64_t ff = -1; int tt = 0;
+            for (int t = 0; t < kp.n_start; t++)
+                if (c.task_f[h * kp.n_start + t] > ff) { ff = c.task_f[h * kp.n_start + t]; tt = h * kp.n_start + t; }
+            if (bt == 0x7fffffff || util_greater(ff, c.task_den[tt], bf, bd)) { bf = ff; bd = c.task_den[tt]; bt = tt; }
+        }
+        int width = 1;
+        while (width < H && width < 32) width <<= 1;
+        for (int o = width >> 1; o; o >>= 1) {
+            int64_t of = __shfl_xor_sync(0xffffffffu, bf, o), od = __shfl_xor_sync(0xffffffffu, bd, o);
+            int ot = __shfl_xor_sync(0xffffffffu, bt, o);
+            bool take = false;
+            if (ot != 0x7fffffff) {
+                if (bt == 0x7fffffff) take = true;
+                else if (util_greater(of, od, bf, bd)) take = true;
+                else if (!util_greater(bf, bd, of, od) && ot < bt) take = true;
+            }
+            if (take) { bf = of; bd = od; bt = ot; }
+        }
+        const int wtask = __shfl_sync(0xffffffffu, bt, 0);
+        const int64_t wF = __shfl_sync(0xffffffffu, bf, 0);
+        if (wF <= 0) { st |= VP_ST_NO_PROGRESS; break; }
+        VP_TICK(3);
+
+        // (D) emit activation k, D_rem -= X(E), update D-hat, write offset row k+1
+        {
+            const int h = wtask / kp.n_start;
+            const uint32_t* slot = c.slotw + h * N;
+            const uint8_t* srcb = c.bind_src + (size_t)wtask * N;
+            const uint8_t* dstb = c.bind_dst + (size_t)wtask * N;
+            const size_t row = (size_t)k * N, orow = (size_t)(k + 1) * N;
+            for (int r = tid; r < N; r += NT) {
+                const uint32_t w = slot[r];
+                const int i = srcb[r], j = dstb[r];
+                const V x = min_v(cap[(w >> 24) & 0xf], Drem[(size_t)i * N + j]);
+                int64_t sa = c.send_acc[i], ra = c.recv_acc[j];
+                if (x > 0) {
+                    const int64_t bytes = (int64_t)x * unit;
+                    c.lane_dst_b[row + i] = (int16_t)j;
+                    c.lane_inst_b[row + i] = (uint16_t)(w & 0xffffu);
+                    c.lane_bytes_b[row + i] = bytes;
+                    Drem[(size_t)i * N + j] -= x;
+                    atomicAdd((unsigned long long*)&c.Dhat[(i / GS) * G + (j / GS)], (unsigned long long)(-(int64_t)x));
+                    sa += bytes; ra += bytes;
+                    c.send_acc[i] = sa;
+                    c.recv_acc[j] = ra;
+                } else {
+                    c.lane_dst_b[row + i] = -1;
+                    c.lane_inst_b[row + i] = 0xFFFF;
+                    c.lane_bytes_b[row + i] = 0;
+                }
+                c.send_off_b[orow + i] = sa;              // src and dst are permutations: every rank is written once
+                if (c.recv_off_b) c.recv_off_b[orow + j] = ra;
+            }
+            if (tid == 0) c.chan_id_b[k] = f0 + h;
+            left -= wF;
+        }
+        k++;
+        __syncthreads();
+        VP_TICK(4);
+    }
+}
+
+template <int GS, int LPG>
+__global__ void __launch_bounds__(LPG > 1 ? 256 : 512, LPG > 1 ? 2 : 1)
 vp_schedule_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand, const int64_t* __restrict__ tau_in, int B,
                    int32_t* __restrict__ n_steps, int32_t* __restrict__ chan_id, int16_t* __restrict__ lane_dst,
                    uint16_t* __restrict__ lane_inst, int64_t* __restrict__ lane_bytes, int64_t* __restrict__ send_off,
                    int64_t* __restrict__ recv_off, int64_t* __restrict__ tau_out, int32_t* __restrict__ status,
-                   int64_t* ws_drem, unsigned int* counter, int drem_in_smem) {
+                   int64_t* ws_drem, unsigned int* counter) {
+    static_assert(LPG == 1 || GS == 4, "lane teams are defined for groups of four ranks");
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    const Smem L = smem_layout(dc, kp.max_tasks, drem_in_smem != 0);
     const int N = dc.N, G = dc.G, tid = threadIdx.x, NT = blockDim.x;
     const int lane = tid & 31, warp = tid >> 5, n_warps = NT >> 5;
-    int64_t* Drem = drem_in_smem ? (int64_t*)(smem_raw + L.drem) : ws_drem + (size_t)blockIdx.x * N * N;
-    int64_t* Dhat = (int64_t*)(smem_raw + L.dhat);
-    int64_t* tbl = dc.sym ? (int64_t*)(smem_raw + L.tbl) : Dhat;
-    int64_t* send_acc = (int64_t*)(smem_raw + L.send_acc);
-    int64_t* recv_acc = (int64_t*)(smem_raw + L.recv_acc);
-    int64_t* red = (int64_t*)(smem_raw + L.red);
-    int64_t* task_f = (int64_t*)(smem_raw + L.task_f);
-    int64_t* task_den = (int64_t*)(smem_raw + L.task_den);
-    uint8_t* bind_src = smem_raw + L.bind_src;
-    uint8_t* bind_dst = smem_raw + L.bind_dst;
-    __shared__ int s_b, s_flags, s_shape, s_task;
-    unsigned long long n_act = 0, n_tasks_done = 0, n_sweeps = 0;     // work counters (per warp / thread 0)
-    __shared__ int64_t s_tau, s_left, s_score;
-    __shared__ int64_t s_cap[VP_MAX_CLASSES];
+    const Smem L = smem_layout(dc, kp, n_warps, LPG);
+    int64_t* Drem = kp.drem_in_smem ? (int64_t*)(smem_raw + L.drem) : ws_drem + (size_t)blockIdx.x * N * N;
+    Ctx c;
+    c.N = N; c.G = G; c.tid = tid; c.NT = NT; c.lane = lane; c.warp = warp; c.n_warps = n_warps;
+    c.Dhat = (int64_t*)(smem_raw + L.dhat);
+    c.tbl = dc.sym ? (int64_t*)(smem_raw + L.tbl) : c.Dhat;
+    c.send_acc = (int64_t*)(smem_raw + L.send_acc);
+    c.recv_acc = (int64_t*)(smem_raw + L.recv_acc);
+    c.red = (int64_t*)(smem_raw + L.red);
+    c.task_f = (int64_t*)(smem_raw + L.task_f);
+    c.task_den = (int64_t*)(smem_raw + L.task_den);
+    c.bind_src = smem_raw + L.bind_src;
+    c.bind_dst = smem_raw + L.bind_dst;
+    c.slotw = (uint32_t*)(smem_raw + L.slotw);
+    c.cred_warp = smem_raw + L.cred + warp * cred_bytes_per_warp(LPG);
+    __shared__ int s_b, s_flags, s_units;
+    __shared__ int64_t s_tau, s_left;
+    __shared__ int64_t s_cap[VP_MAX_CLASSES], s_tscale[VP_MAX_CLASSES];
+    __shared__ uint32_t s_cap32[VP_MAX_CLASSES];
+    __shared__ uint8_t s_perm_lut[32];
+    c.tscale = s_tscale;
+    c.perm_lut = s_perm_lut;
+    if (tid < 32) s_perm_lut[tid] = (uint8_t)(31 - tid < 24 ? perm4_packed_rt(31 - tid) : 0);
+    unsigned long long n_act = 0;                          // work counters (thread 0 / lane 0 of each warp)
+    Counters cnt;
+    cnt.tasks = 0; cnt.sweeps = 0; cnt.t_mark = 0;
+    for (int i = 0; i < 6; i++) cnt.cyc[i] = 0;
+
+    // ---- stage the catalog
+    c.p_term = dc.term;
+    c.p_fam_in = dc.fam_in;
+    c.p_fam_cls = dc.fam_cls;
+    if (kp.stage_terms) {
+        uint32_t* st = (uint32_t*)(smem_raw + L.term);
+        for (int e = tid; e < dc.n_shapes * dc.max_terms; e += NT) st[e] = dc.term[e];
+        c.p_term = st;
+    }
+    c.p_bucket_ptr = dc.bucket_ptr;
+    if (kp.stage_bucket) {
+        uint32_t* bp = (uint32_t*)(smem_raw + L.bucket);
+        for (int e = tid; e <= dc.n_shapes; e += NT) bp[e] = dc.bucket_ptr[e];
+        c.p_bucket_ptr = bp;
+    }
+    if (kp.stage_fam) {
+        uint16_t* fi = (uint16_t*)(smem_raw + L.fam_in);
+        uint8_t* fc = smem_raw + L.fam_cls;
+        for (int e = tid; e < dc.n_families * N; e += NT) { fi[e] = dc.fam_in[e]; fc[e] = dc.fam_cls[e]; }
+        c.p_fam_in = fi; c.p_fam_cls = fc;
+    }
 
     for (;;) {
         if (tid == 0) { s_b = (int)atomicAdd(counter, 1u); s_flags = 0; }
         __syncthreads();
         const int b = s_b;
         if (b >= B) break;
+#ifdef VP_PHASE_TIMING
+        cnt.t_mark = clock64();
+#endif
         const int64_t* D = demand + (size_t)b * N * N;
         const size_t lane_base = (size_t)b * kp.k_max * N, off_base = (size_t)b * (kp.k_max + 1) * N;
+        c.chan_id_b = chan_id + (size_t)b * kp.k_max;
+        c.lane_dst_b = lane_dst + lane_base;
+        c.lane_inst_b = lane_inst + lane_base;
+        c.lane_bytes_b = lane_bytes + lane_base;
+        c.send_off_b = send_off + off_base;
+        c.recv_off_b = recv_off ? recv_off + off_base : nullptr;
 
         // ---- validate, copy D into D_rem
         int flags = 0;
@@ -172,9 +649,9 @@ vp_schedule_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand, co
         if (tid == 0 && (tau_given < 0 || tau_given > VP_ENTRY_LIMIT)) flags |= VP_ST_BAD_TAU;
         if (flags) atomicOr(&s_flags, flags);
         for (int i = tid; i < N; i += NT) {
-            send_acc[i] = 0; recv_acc[i] = 0;
-            send_off[off_base + i] = 0;
-            if (recv_off) recv_off[off_base + i] = 0;
+            c.send_acc[i] = 0; c.recv_acc[i] = 0;
+            c.send_off_b[i] = 0;
+            if (c.recv_off_b) c.recv_off_b[i] = 0;
         }
         __syncthreads();
         int st = s_flags;
@@ -191,7 +668,7 @@ vp_schedule_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand, co
                     col += Drem[(size_t)j * N + i];
                 }
                 tot += row;
-                est = max_i64(est, max_i64(ceil_div_i64(row, dc.bw_max), ceil_div_i64(col, dc.bw_max)));
+                est = max_v(est, max_v(ceil_div_i64(row, dc.bw_max), ceil_div_i64(col, dc.bw_max)));
             }
             for (int cell = tid; cell < G * G; cell += NT) {
                 int a = cell / G, d = cell % G;
@@ -200,221 +677,64 @@ vp_schedule_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand, co
                 for (int i = 0; i < GS; i++)
 #pragma unroll
                     for (int j = 0; j < GS; j++) s += Drem[(size_t)(a * GS + i) * N + d * GS + j];
-                Dhat[cell] = s;
+                c.Dhat[cell] = s;
             }
             __syncthreads();
             for (int l = tid; l < dc.n_res; l += NT) {
                 uint32_t bwl = dc.forced_bw[l];
                 if (!bwl) continue;
                 int64_t f = 0;
-                for (uint32_t e = dc.forced_ptr[l]; e < dc.forced_ptr[l + 1]; e++) f += Dhat[dc.forced_cell[e]];
-                est = max_i64(est, ceil_div_i64(f, (int64_t)bwl));
+                for (uint32_t e = dc.forced_ptr[l]; e < dc.forced_ptr[l + 1]; e++) f += c.Dhat[dc.forced_cell[e]];
+                est = max_v(est, ceil_div_i64(f, (int64_t)bwl));
             }
             est = warp_max_i64(est);
             tot = warp_sum_i64(tot);
-            if (lane == 0) { red[warp] = est; red[32 + warp] = tot; }
+            if (lane == 0) { c.red[warp] = est; c.red[32 + warp] = tot; }
             __syncthreads();
             if (tid == 0) {
                 int64_t e = 0, t = 0;
-                for (int w = 0; w < n_warps; w++) { e = max_i64(e, red[w]); t += red[32 + w]; }
-                int64_t tq = tau_given > 0 ? tau_given : max_i64(1, ceil_div_i64(e, (int64_t)kp.k_target));
-                s_tau = tq; s_left = t;
-                for (int c = 0; c < dc.n_classes; c++) {
-                    int64_t cap = (tq * dc.class_bw[c]) / kp.granule * kp.granule;
-                    s_cap[c] = cap < kp.granule ? kp.granule : cap;
+                for (int w = 0; w < n_warps; w++) { e = max_v(e, c.red[w]); t += c.red[32 + w]; }
+                int64_t tq = tau_given > 0 ? tau_given : max_v((int64_t)1, ceil_div_i64(e, (int64_t)kp.k_target));
+                int64_t cap_max = 0;
+                for (int cl = 0; cl < dc.n_classes; cl++) {
+                    int64_t cp = (tq * dc.class_bw[cl]) / kp.granule * kp.granule;
+                    s_cap[cl] = cp < kp.granule ? kp.granule : cp;
+                    cap_max = max_v(cap_max, s_cap[cl]);
                 }
+                // granule units: capacities below 2^25 granules, every entry below 2^32 granules
+                const int units = cap_max / kp.granule < ((int64_t)1 << 25) && kp.granule >= 256;
+                for (int cl = 0; cl < dc.n_classes; cl++) {
+                    s_cap32[cl] = (uint32_t)(units ? s_cap[cl] / kp.granule : 0);
+                    s_tscale[cl] = dc.class_wdiv[cl] * (units ? kp.granule : 1);
+                }
+                s_tau = tq; s_left = t; s_units = units;
             }
             __syncthreads();
             tau = s_tau;
-
-            // ---- Algorithm 2 main loop
-            for (;;) {
-                if (s_left == 0) break;
-                if (k == kp.k_max) { st |= VP_ST_STEP_LIMIT; break; }
-                // (A) Eq. (6): shape scores, first maximum
-                if (dc.sym) {
-                    const int S = dc.S, P = dc.P;
-                    for (int e = tid; e < dc.tbl_size; e += NT) {
-                        int q2 = e % S, q = (e / S) % S, delta = e / (S * S);
-                        int64_t s = 0;
-                        for (int n = 0; n < P; n++) {
-                            int n2 = n + delta; if (n2 >= P) n2 -= P;
-                            s += Dhat[(size_t)(n * S + q) * G + n2 * S + q2];
-                        }
-                        tbl[e] = s;
-                    }
-                    __syncthreads();
-                }
-                int64_t best = -1;
-                int best_s = 0x7fffffff;
-                for (int s = tid; s < dc.n_shapes; s += NT) {
-                    int64_t score = 0;
-                    for (uint32_t e = dc.shape_ptr[s]; e < dc.shape_ptr[s + 1]; e++) {
-                        uint32_t w = __ldg(&dc.term[e]);
-                        score += tbl[w & 0xffffu] * (int64_t)(w >> 16);
-                    }
-                    if (score > best) { best = score; best_s = s; }     // ascending s: keeps the first maximum
-                }
-#pragma unroll
-                for (int o = 16; o; o >>= 1) {
-                    int64_t ov = __shfl_xor_sync(0xffffffffu, best, o);
-                    int oi = __shfl_xor_sync(0xffffffffu, best_s, o);
-                    if (ov > best || (ov == best && oi < best_s)) { best = ov; best_s = oi; }
-                }
-                if (lane == 0) { red[warp] = best; red[32 + warp] = best_s; }
+            const bool units = s_units != 0;
+            VP_TICK(0);
+            if (units) {
+                // the byte copy is no longer needed: overwrite it with the demand in granules
+                uint32_t* Drem32 = (uint32_t*)Drem;
+                for (int e = tid; e < N * N; e += NT) Drem32[e] = (uint32_t)(D[e] / kp.granule);
+                for (int cell = tid; cell < G * G; cell += NT) c.Dhat[cell] /= kp.granule;
                 __syncthreads();
-                if (tid == 0) {
-                    int64_t bv = -1; int bi = 0x7fffffff;
-                    for (int w = 0; w < n_warps; w++)
-                        if (red[w] > bv || (red[w] == bv && (int)red[32 + w] < bi)) { bv = red[w]; bi = (int)red[32 + w]; }
-                    s_score = bv; s_shape = bi;
-                }
-                __syncthreads();
-                if (s_score <= 0) { st |= VP_ST_UNCOVERED; break; }
-                const int f0 = (int)dc.bucket_ptr[s_shape], H = (int)dc.bucket_ptr[s_shape + 1] - f0;
-                const int n_tasks = H * kp.n_start;
-
-                // (B) MultiStartAA: one warp per (family, start), one lane per rank group
-                for (int task = warp; task < n_tasks; task += n_warps) {
-                    const int f = f0 + task / kp.n_start, t = task % kp.n_start;
-                    const uint32_t* slot = dc.fam_slot + (size_t)f * N;
-                    const uint8_t* inslot = dc.fam_inslot + (size_t)f * N;
-                    uint8_t* srcb = bind_src + (size_t)task * N;
-                    uint8_t* dstb = bind_dst + (size_t)task * N;
-                    for (int d = lane; d < G; d += 32)
-#pragma unroll
-                        for (int q = 0; q < GS; q++) dstb[inslot[d * GS + q]] = (uint8_t)(d * GS + (q + t) % GS);
-                    __syncwarp();
-                    int64_t F_old = -1, F_new = -1;
-                    for (int sweep = 0; sweep < kp.i_aa; sweep++) {
-                        for (int a = lane; a < G; a += 32) {            // source half
-                            int64_t c[GS][GS];
-                            int phi[GS];
-#pragma unroll
-                            for (int q = 0; q < GS; q++) {
-                                const int r = a * GS + q;
-                                const int64_t cap = s_cap[(__ldg(&slot[r]) >> 24) & 0xf];
-                                const int dq = dstb[r];
-#pragma unroll
-                                for (int i = 0; i < GS; i++) c[i][q] = min_i64(Drem[(size_t)(a * GS + i) * N + dq], cap);
-                            }
-                            best_assignment<GS>(c, phi);
-#pragma unroll
-                            for (int q = 0; q < GS; q++) srcb[a * GS + q] = (uint8_t)(a * GS + phi[q]);
-                        }
-                        __syncwarp();
-                        int64_t part = 0;
-                        for (int d = lane; d < G; d += 32) {            // destination half
-                            int64_t c[GS][GS];
-                            int phi[GS], rq[GS];
-#pragma unroll
-                            for (int q = 0; q < GS; q++) {
-                                rq[q] = inslot[d * GS + q];
-                                const int64_t cap = s_cap[(__ldg(&slot[rq[q]]) >> 24) & 0xf];
-                                const int sq = srcb[rq[q]];
-#pragma unroll
-                                for (int j = 0; j < GS; j++) c[j][q] = min_i64(Drem[(size_t)sq * N + d * GS + j], cap);
-                            }
-                            part += best_assignment<GS>(c, phi);
-#pragma unroll
-                            for (int q = 0; q < GS; q++) dstb[rq[q]] = (uint8_t)(d * GS + phi[q]);
-                        }
-                        __syncwarp();
-                        F_new = warp_sum_i64(part);                      // Eq. (8), in bytes
-                        n_sweeps++;
-                        if (F_new <= F_old) break;
-                        F_old = F_new;
-                    }
-                    int64_t tmax = 0;                                    // Eq. (9), slowest lane of Eq. (10)
-                    for (int r = lane; r < N; r += 32) {
-                        const int cls = (__ldg(&slot[r]) >> 24) & 0xf;
-                        const int64_t x = min_i64(s_cap[cls], Drem[(size_t)srcb[r] * N + dstb[r]]);
-                        tmax = max_i64(tmax, x * dc.class_wdiv[cls]);
-                    }
-                    tmax = warp_max_i64(tmax);
-                    n_tasks_done++;
-                    if (lane == 0) {
-                        task_f[task] = F_new;
-                        task_den[task] = F_new > 0 ? kp.lambda_ns * dc.W + tmax : 1;
-                    }
-                }
-                __syncthreads();
-
-                // (C) best start per family (largest F, lowest t), then largest utility, lowest family
-                if (warp == 0) {
-                    int64_t bf = -1, bd = 1;
-                    int bt = 0x7fffffff;
-                    for (int h = lane; h < H; h += 32) {
-                        int64_t ff = -1; int tt = 0;
-                        for (int t = 0; t < kp.n_start; t++)
-                            if (task_f[h * kp.n_start + t] > ff) { ff = task_f[h * kp.n_start + t]; tt = h * kp.n_start + t; }
-                        if (bt == 0x7fffffff || util_greater(ff, task_den[tt], bf, bd)) { bf = ff; bd = task_den[tt]; bt = tt; }
-                    }
-#pragma unroll
-                    for (int o = 16; o; o >>= 1) {
-                        int64_t of = __shfl_xor_sync(0xffffffffu, bf, o), od = __shfl_xor_sync(0xffffffffu, bd, o);
-                        int ot = __shfl_xor_sync(0xffffffffu, bt, o);
-                        bool take = false;
-                        if (ot != 0x7fffffff) {
-                            if (bt == 0x7fffffff) take = true;
-                            else if (util_greater(of, od, bf, bd)) take = true;
-                            else if (!util_greater(bf, bd, of, od) && ot < bt) take = true;
-                        }
-                        if (take) { bf = of; bd = od; bt = ot; }
-                    }
-                    if (lane == 0) { s_task = bt; red[0] = bf; }
-                }
-                __syncthreads();
-                const int wtask = s_task;
-                const int64_t wF = red[0];
-                if (wF <= 0) { st |= VP_ST_NO_PROGRESS; break; }
-
-                // (D) emit activation k, D_rem -= X(E), update D-hat and the running offsets
-                {
-                    const int f = f0 + wtask / kp.n_start;
-                    const uint32_t* slot = dc.fam_slot + (size_t)f * N;
-                    const uint8_t* srcb = bind_src + (size_t)wtask * N;
-                    const uint8_t* dstb = bind_dst + (size_t)wtask * N;
-                    const size_t row = lane_base + (size_t)k * N;
-                    for (int r = tid; r < N; r += NT) {
-                        const uint32_t w = __ldg(&slot[r]);
-                        const int i = srcb[r], j = dstb[r];
-                        const int64_t x = min_i64(s_cap[(w >> 24) & 0xf], Drem[(size_t)i * N + j]);
-                        if (x > 0) {
-                            lane_dst[row + i] = (int16_t)j;
-                            lane_inst[row + i] = (uint16_t)(w & 0xffffu);
-                            lane_bytes[row + i] = x;
-                            Drem[(size_t)i * N + j] -= x;
-                            atomicAdd((unsigned long long*)&Dhat[(i / GS) * G + (j / GS)], (unsigned long long)(-x));
-                            send_acc[i] += x;
-                            recv_acc[j] += x;
-                        } else {
-                            lane_dst[row + i] = -1;
-                            lane_inst[row + i] = 0xFFFF;
-                            lane_bytes[row + i] = 0;
-                        }
-                    }
-                    if (tid == 0) { chan_id[(size_t)b * kp.k_max + k] = f; s_left -= wF; }
-                }
-                __syncthreads();
-                k++;
-                for (int i = tid; i < N; i += NT) {
-                    send_off[off_base + (size_t)k * N + i] = send_acc[i];
-                    if (recv_off) recv_off[off_base + (size_t)k * N + i] = recv_acc[i];
-                }
+                decompose<GS, LPG, uint32_t>(dc, kp, c, Drem32, s_cap32, kp.granule, s_left / kp.granule, k, st, cnt);
+            } else {
+                decompose<GS, LPG, int64_t>(dc, kp, c, Drem, s_cap, 1, s_left, k, st, cnt);
             }
         }
         __syncthreads();
         // ---- idle rows beyond n_steps; offset rows repeat the totals
         for (size_t e = (size_t)k * N + tid; e < (size_t)kp.k_max * N; e += NT) {
-            lane_dst[lane_base + e] = -1;
-            lane_inst[lane_base + e] = 0xFFFF;
-            lane_bytes[lane_base + e] = 0;
+            c.lane_dst_b[e] = -1;
+            c.lane_inst_b[e] = 0xFFFF;
+            c.lane_bytes_b[e] = 0;
             const int i = (int)(e % N);
-            send_off[off_base + N + e] = send_acc[i];
-            if (recv_off) recv_off[off_base + N + e] = recv_acc[i];
+            c.send_off_b[N + e] = c.send_acc[i];
+            if (c.recv_off_b) c.recv_off_b[N + e] = c.recv_acc[i];
         }
-        for (int kk = k + tid; kk < kp.k_max; kk += NT) chan_id[(size_t)b * kp.k_max + kk] = -1;
+        for (int kk = k + tid; kk < kp.k_max; kk += NT) c.chan_id_b[kk] = -1;
         if (tid == 0) {
             n_act += (unsigned long long)k;
             n_steps[b] = k;
@@ -422,35 +742,39 @@ vp_schedule_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand, co
             if (tau_out) tau_out[b] = tau;
         }
         __syncthreads();
+        VP_TICK(5);
     }
     unsigned long long* stats = (unsigned long long*)(counter + 4);
     if (tid == 0 && n_act) atomicAdd(&stats[0], n_act);
-    if (lane == 0 && n_tasks_done) { atomicAdd(&stats[1], n_tasks_done); atomicAdd(&stats[2], n_sweeps); }
+    if (lane == 0 && cnt.tasks) { atomicAdd(&stats[1], cnt.tasks); atomicAdd(&stats[2], cnt.sweeps); }
+#ifdef VP_PHASE_TIMING
+    if (tid == 0) for (int i = 0; i < 6; i++) atomicAdd(&stats[3 + i], (unsigned long long)cnt.cyc[i]);
+#endif
 }
 
 struct Launch {
-    int threads, grid, drem_in_smem, max_tasks;
+    int threads, grid, lpg;
     size_t smem;
+    KParams kp;
 };
 
-template <int GS>
-int plan_launch(const vp_catalog* c, int B, const KParams& kp, Launch* out) {
-    const DevCat& dc = c->dc;
-    Launch L;
-    L.max_tasks = kp.max_tasks;
-    L.threads = dc.N <= 16 ? 128 : (dc.N <= 64 ? 256 : 512);
-    L.drem_in_smem = dc.N <= 64;
-    L.smem = (size_t)smem_layout(dc, kp.max_tasks, L.drem_in_smem).total;
-    if (L.smem + 1024 > (size_t)c->max_smem_optin) return VP_E_UNSUPPORTED;
-    if (cudaFuncSetAttribute(vp_schedule_kernel<GS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.smem) != cudaSuccess)
-        return VP_E_CUDA;
-    int per_sm = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, vp_schedule_kernel<GS>, L.threads, L.smem) != cudaSuccess || per_sm < 1)
-        return VP_E_CUDA;
-    long long cap = (long long)per_sm * c->sm_count;
-    L.grid = (int)(B < cap ? B : cap);
-    *out = L;
-    return VP_OK;
+typedef void (*KernelFn)(DevCat, KParams, const int64_t*, const int64_t*, int, int32_t*, int32_t*, int16_t*, uint16_t*,
+                         int64_t*, int64_t*, int64_t*, int64_t*, int32_t*, int64_t*, unsigned int*);
+
+KernelFn pick_kernel(int g, int lpg) {
+    switch (g) {
+        case 1: return vp_schedule_kernel<1, 1>;
+        case 2: return vp_schedule_kernel<2, 1>;
+        case 3: return vp_schedule_kernel<3, 1>;
+        case 4:
+            switch (lpg) {
+                case 8: return vp_schedule_kernel<4, 8>;
+                case 4: return vp_schedule_kernel<4, 4>;
+                case 2: return vp_schedule_kernel<4, 2>;
+                default: return vp_schedule_kernel<4, 1>;
+            }
+    }
+    return nullptr;
 }
 
 int resolve_params(const vp_catalog* c, const vp_sched_params* p, KParams* kp) {
@@ -466,31 +790,46 @@ int resolve_params(const vp_catalog* c, const vp_sched_params* p, KParams* kp) {
     return VP_OK;
 }
 
-int plan_any(const vp_catalog* c, int B, const KParams& kp, Launch* L) {
-    switch (c->dc.g) {
-        case 1: return plan_launch<1>(c, B, kp, L);
-        case 2: return plan_launch<2>(c, B, kp, L);
-        case 3: return plan_launch<3>(c, B, kp, L);
-        case 4: return plan_launch<4>(c, B, kp, L);
-    }
-    return VP_E_UNSUPPORTED;
+int plan_launch(const vp_catalog* c, int B, const vp_sched_params* p, Launch* out) {
+    const DevCat& dc = c->dc;
+    Launch L;
+    int rc = resolve_params(c, p, &L.kp);
+    if (rc) return rc;
+    L.lpg = 1;
+    if (dc.g == 4) L.lpg = dc.G <= 4 ? 8 : (dc.G <= 8 ? 4 : (dc.G <= 16 ? 2 : 1));
+    L.threads = dc.N <= 64 ? 256 : 512;
+    L.kp.drem_in_smem = dc.N <= 64;
+    L.kp.stage_terms = (size_t)dc.n_shapes * dc.max_terms * 4 <= 32 * 1024;
+    L.kp.stage_fam = (size_t)dc.n_families * dc.N * 3 <= 64 * 1024;
+    L.kp.stage_bucket = ((size_t)dc.n_shapes + 1) * 4 <= 32 * 1024;
+    L.smem = (size_t)smem_layout(dc, L.kp, L.threads / 32, L.lpg).total;
+    if (L.smem + 2048 > (size_t)c->max_smem_optin) return VP_E_UNSUPPORTED;
+    KernelFn fn = pick_kernel(dc.g, L.lpg);
+    if (!fn) return VP_E_UNSUPPORTED;
+    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.smem) != cudaSuccess) return VP_E_CUDA;
+    int per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, L.threads, L.smem) != cudaSuccess || per_sm < 1)
+        return VP_E_CUDA;
+    long long cap = (long long)per_sm * c->sm_count;
+    L.grid = (int)(B < cap ? B : cap);
+    *out = L;
+    return VP_OK;
 }
 
 size_t workspace_bytes(const vp_catalog* c, const Launch& L) {
-    size_t drem = L.drem_in_smem ? 0 : (size_t)L.grid * c->dc.N * c->dc.N * 8;
+    size_t drem = L.kp.drem_in_smem ? 0 : (size_t)L.grid * c->dc.N * c->dc.N * 8;
     return vp_align256(256 + drem);
 }
 
 }  // namespace
 
 extern "C" size_t vp_schedule_workspace_bytes(const vp_catalog* c, int B, const vp_sched_params* p) {
-    KParams kp;
     Launch L;
-    if (B <= 0 || resolve_params(c, p, &kp) != VP_OK) return 0;
+    if (B <= 0 || !c || !p) return 0;
     int prev = -1;
     cudaGetDevice(&prev);
     cudaSetDevice(c->device);
-    int rc = plan_any(c, B, kp, &L);
+    int rc = plan_launch(c, B, p, &L);
     if (prev >= 0) cudaSetDevice(prev);
     return rc == VP_OK ? workspace_bytes(c, L) : 0;
 }
@@ -500,39 +839,29 @@ extern "C" int vp_schedule_batch(const vp_catalog* c, const vp_sched_params* p, 
                                  int16_t* lane_dst, uint16_t* lane_inst, int64_t* lane_bytes, int64_t* send_off,
                                  int64_t* recv_off, int64_t* tau_ns_out, int32_t* status, void* workspace,
                                  size_t workspace_bytes_given, void* cuda_stream) {
-    KParams kp;
-    int rc = resolve_params(c, p, &kp);
-    if (rc) return rc;
+    if (!c || !p) return VP_E_BAD_ARG;
     if (B <= 0 || !demand || !n_steps || !chan_id || !lane_dst || !lane_inst || !lane_bytes || !send_off || !status)
         return VP_E_BAD_ARG;
     int prev = -1;
     cudaGetDevice(&prev);
     if (cudaSetDevice(c->device) != cudaSuccess) return VP_E_CUDA;
     Launch L;
-    rc = plan_any(c, B, kp, &L);
+    int rc = plan_launch(c, B, p, &L);
     if (!rc && (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes_given < workspace_bytes(c, L))) rc = VP_E_WORKSPACE;
     if (!rc) {
         cudaStream_t stream = (cudaStream_t)cuda_stream;
         unsigned int* counter = (unsigned int*)workspace;
         int64_t* ws_drem = (int64_t*)((char*)workspace + 256);
         if (cudaMemsetAsync(counter, 0, 256, stream) != cudaSuccess) rc = VP_E_CUDA;
-#define VP_LAUNCH(GS)                                                                                           \
-    vp_schedule_kernel<GS><<<L.grid, L.threads, L.smem, stream>>>(c->dc, kp, demand, tau_ns_in, B, n_steps,     \
-        chan_id, lane_dst, lane_inst, lane_bytes, send_off, recv_off, tau_ns_out, status, ws_drem, counter,     \
-        L.drem_in_smem)
         if (!rc) {
             vp_prof_mark(0, 0, stream);
-            switch (c->dc.g) {
-                case 1: VP_LAUNCH(1); break;
-                case 2: VP_LAUNCH(2); break;
-                case 3: VP_LAUNCH(3); break;
-                case 4: VP_LAUNCH(4); break;
-            }
+            pick_kernel(c->dc.g, L.lpg)<<<L.grid, L.threads, L.smem, stream>>>(
+                c->dc, L.kp, demand, tau_ns_in, B, n_steps, chan_id, lane_dst, lane_inst, lane_bytes, send_off, recv_off,
+                tau_ns_out, status, ws_drem, counter);
             g_vp_launches++;
             if (cudaGetLastError() != cudaSuccess) rc = VP_E_CUDA;
             vp_prof_mark(0, 1, stream);
         }
-#undef VP_LAUNCH
     }
     if (prev >= 0) cudaSetDevice(prev);
     return rc;

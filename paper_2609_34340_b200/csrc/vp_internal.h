@@ -18,14 +18,18 @@ struct DevCat {
     int sym;                      // 1: shape terms index per-node-offset sums, 0: D-hat cells
     int tbl_size;                 // entries of the score table (G*G or P*S*S)
     int max_bucket;
-    // Eq. (6): shape s has terms term[shape_ptr[s] .. shape_ptr[s+1]) = table index | count << 16
-    const uint32_t* shape_ptr;
+    // Eq. (6): shape s has terms term[s*max_terms .. s*max_terms + max_terms) = table index | count << 16
+    // (shapes with fewer terms are padded with zero counts)
     const uint32_t* term;
+    int max_terms;
     const uint32_t* bucket_ptr;
     // family f, slot r: instance id | destination group << 16 | rate class << 24
     const uint32_t* fam_slot;
-    // family f, in-slot d*g+q: slot index (N <= 256)
-    const uint8_t* fam_inslot;
+    // family f, slot r: rate class (the out-slots of group a are slots a*g .. a*g+g-1)
+    const uint8_t* fam_cls;
+    // family f, in-slot d*g+q of destination group d: slot index (N <= 256) | rate class << 8
+    const uint16_t* fam_in;
+    int n_terms;
     // quantum rule: resource l is forced for the D-hat cells forced_cell[forced_ptr[l] .. forced_ptr[l+1])
     const uint32_t* forced_ptr;
     const uint16_t* forced_cell;
