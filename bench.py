@@ -116,10 +116,11 @@ class ClockSampler:
 # workload
 # ------------------------------------------------------------------------------------------
 
-def build_workload(sched_config: int, device: str, rank_seed: int):
+def build_workload(args, device: str):
+    """The timed inputs.  ``--batch / --token-scale / --pack-tokens`` shrink them (CPU tests only)."""
     from workloads.configs import build_config, build_pack_case
-    sched = build_config(sched_config, device=device)
-    pack = build_pack_case(device=device)
+    sched = build_config(args.sched_config, device=device, batch=args.batch, token_scale=args.token_scale)
+    pack = build_pack_case(device=device, tokens=args.pack_tokens)
     return sched, pack
 
 
@@ -151,7 +152,7 @@ def run_ours(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device(dev))
 
-    sched, pk = build_workload(args.sched_config, dev, rank)
+    sched, pk = build_workload(args, dev)
     cat, w = sched["catalog"], sched["params"]
     dc = vp.load_catalog(cat.topology.blob(), cat.blob(), device=local_rank)
     params = vp_params(vp, w)
@@ -380,7 +381,7 @@ def run_reference(args):
     rank, _, world = _dist_env()
     if rank != 0:
         return
-    sched, pk = build_workload(args.sched_config, "cpu" if not _has_cuda() else "cuda", 0)
+    sched, pk = build_workload(args, "cpu" if not _has_cuda() else "cuda")
     sched["demand"] = sched["demand"].cpu()
     cores = os.cpu_count() or 1
     oc, poc, plan_one = _oracle_setup(sched, pk)
@@ -420,6 +421,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--sched-config", type=int, default=2, choices=[1, 2, 3, 4])
+    ap.add_argument("--batch", type=int, default=None, help="truncate the scheduler batch (tests)")
+    ap.add_argument("--token-scale", type=float, default=1.0, help="scale token counts (tests)")
+    ap.add_argument("--pack-tokens", type=int, default=16384, help="tokens of the packed rank (tests)")
     ap.add_argument("--min-warmup-s", type=float, default=1.0,
                     help="keep warming up (beyond --warmup steps) until this many seconds have passed, so that "
                          "clocks settle and nvidia-smi has samples under load")
