@@ -190,6 +190,37 @@ int vp_pack(const int32_t* n_steps_b, const int16_t* lane_dst_b, const int64_t* 
             int32_t* status, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * vp_pack_static - vp_pack without a workspace argument.  (The paper has no counterpart: this entry
+ * point exists for callers that cannot provide scratch memory.)
+ *
+ * Who needs it: code that runs the pack from inside a serving engine's steady-state step.  Such code is
+ * given the input and output buffers and nothing else; it owns no allocator, and calling cudaMalloc there
+ * is off the table (the call synchronises the whole device, may fail under the engine's memory cap, and
+ * bypasses the engine's own accounting).  For these callers the library carries its own scratch: one
+ * block of VP_PACK_STATIC_SCRATCH_BYTES of device memory that every GPU which loads the library sets
+ * aside at load time and keeps until the process exits.  The call allocates nothing, on host or device.
+ *
+ * Arguments, results and status bits are those of vp_pack; inputs and outputs are still the caller's.
+ * Limits and rules:
+ *  - vp_pack_workspace_bytes(N, T, topk, k_max) must not exceed VP_PACK_STATIC_SCRATCH_BYTES (4 MiB; about
+ *    0.9 million routed copies at N = 16); a larger problem is refused with VP_E_WORKSPACE before anything
+ *    is launched.  Use vp_pack with your own workspace for those.
+ *  - The first call on each device looks up the block's device address (a cudaGetSymbolAddress query made
+ *    with that device current).  Make that first call outside any stream capture.
+ *  - All calls on one device share the one block, and the block keeps whatever the last call left in it.
+ *    The call itself resets what has to start from zero, so stale contents are harmless, but two calls
+ *    whose kernels can overlap on the GPU (different streams without ordering between them) race on the
+ *    block: order them, or give one of them vp_pack and a workspace of its own.
+ */
+#define VP_PACK_STATIC_SCRATCH_BYTES (4 * 1024 * 1024)
+int vp_pack_static(const int32_t* n_steps_b, const int16_t* lane_dst_b, const int64_t* lane_bytes_b,
+                   const int64_t* send_off_b, int N, int rank, int k_max,
+                   const int32_t* expert_idx, int T, int topk, int experts_per_rank,
+                   const void* rows, int64_t row_bytes,
+                   void* staged, int64_t staged_capacity_bytes, int32_t* src_map,
+                   int32_t* status, void* cuda_stream);
+
+/*
  * Host-buffer variants: the same operations with every array in HOST memory
  * (pinned memory makes the copies asynchronous).  The calls copy inputs to
  * device scratch, run the kernels above, copy the results back and return

@@ -17,6 +17,8 @@ from .binding import (  # noqa: F401
     pack_workspace_bytes,
     pack,
     pack_host,
+    pack_static,
+    PACK_STATIC_SCRATCH_BYTES,
     kernel_launch_count,
     schedule_read_stats,
     profile_enable,

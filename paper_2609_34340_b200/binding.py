@@ -83,6 +83,7 @@ def _load():
     lib.vp_pack_workspace_bytes.restype = sz
     pack_args = [P, P, P, P, i32, i32, i32, P, i32, i32, i32, P, i64, P, i64, P, P]
     lib.vp_pack.argtypes = pack_args + [P, sz, P]
+    lib.vp_pack_static.argtypes = pack_args + [P]
     lib.vp_pack_host_scratch_bytes.argtypes = [i32, i32, i32, i32, i64, i64]
     lib.vp_pack_host_scratch_bytes.restype = sz
     lib.vp_pack_host.argtypes = pack_args + [P, sz, P]
@@ -281,6 +282,32 @@ def pack(plan: Plan, b: int, rank: int, expert_idx: torch.Tensor, experts_per_ra
         workspace = torch.empty(pack_workspace_bytes(N, T, topk, plan.k_max), dtype=torch.uint8, device=rows.device)
     _check(_pack_call(_load().vp_pack, plan, b, N, rank, expert_idx, experts_per_rank, rows, row_bytes, staged,
                       src_map, status, workspace, stream), "vp_pack")
+    return status
+
+
+PACK_STATIC_SCRATCH_BYTES = 4 * 1024 * 1024
+
+
+def pack_static(plan: Plan, b: int, rank: int, expert_idx: torch.Tensor, experts_per_rank: int, rows: torch.Tensor,
+                staged: torch.Tensor, src_map: Optional[torch.Tensor] = None, status: Optional[torch.Tensor] = None,
+                stream=None) -> torch.Tensor:
+    """``vp_pack_static``: the pack for callers that cannot hand over scratch memory (they run inside an
+    engine's step, own no allocator and must not call cudaMalloc).  Same results as :func:`pack`; the library
+    uses its own fixed 4 MiB device block instead of a workspace, so the problem has to fit it
+    (``VpError`` with ``E_WORKSPACE`` otherwise) and calls that may overlap on the GPU must be ordered.
+    ``status`` must be passed in by such callers; it is allocated here only when omitted."""
+    N = plan.lane_dst.shape[2]
+    assert expert_idx.is_cuda and expert_idx.dtype == torch.int32 and expert_idx.is_contiguous()
+    assert rows.is_cuda and rows.is_contiguous() and staged.is_cuda and staged.is_contiguous()
+    T, topk = expert_idx.shape
+    row_bytes = rows.shape[1] * rows.element_size()
+    if status is None:
+        status = torch.empty(1, dtype=torch.int32, device=rows.device)
+    rc = _load().vp_pack_static(_ptr(plan.n_steps[b:b + 1]), _ptr(plan.lane_dst[b]), _ptr(plan.lane_bytes[b]),
+                                _ptr(plan.send_off[b]), int(N), int(rank), int(plan.k_max), _ptr(expert_idx), int(T),
+                                int(topk), int(experts_per_rank), _ptr(rows), int(row_bytes), _ptr(staged),
+                                staged.numel() * staged.element_size(), _ptr(src_map), _ptr(status), _stream(stream))
+    _check(rc, "vp_pack_static")
     return status
 
 

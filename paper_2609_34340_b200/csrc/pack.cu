@@ -388,3 +388,52 @@ extern "C" int vp_pack(const int32_t* n_steps_b, const int16_t* lane_dst_b, cons
     vp_prof_mark(2, 1, stream);
     return cudaGetLastError() == cudaSuccess ? VP_OK : VP_E_CUDA;
 }
+
+// ---- vp_pack_static: the pack with its scratch built into the library ---------------------------------
+//
+// Some callers of the pack have no way to obtain device scratch at the moment they call it: they sit inside
+// a serving engine's steady-state step, are handed only the input and output buffers, hold no allocator of
+// their own, and must not call cudaMalloc there (it synchronises the whole device, it can fail under the
+// engine's memory cap, and the engine accounts for every byte itself).  For them the library keeps one
+// fixed block of device memory, reserved when the library is loaded on a GPU and held until the process
+// exits, and uses it in place of the caller's workspace.
+//
+// In host code `g_pack_static_scratch` is only a handle for the device array; its device address has to be
+// asked for with cudaGetSymbolAddress, once per device, with that device current.
+static __device__ __align__(256) unsigned char g_pack_static_scratch[VP_PACK_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+void* g_static_scratch_addr[kMaxDevices] = {nullptr};
+
+// Device address of the built-in scratch on the current device (looked up on first use).
+int static_scratch_address(void** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return VP_E_CUDA;
+    void* p = __atomic_load_n(&g_static_scratch_addr[dev], __ATOMIC_ACQUIRE);
+    if (!p) {
+        if (cudaGetSymbolAddress(&p, g_pack_static_scratch) != cudaSuccess || !p) return VP_E_CUDA;
+        __atomic_store_n(&g_static_scratch_addr[dev], p, __ATOMIC_RELEASE);
+    }
+    *out = p;
+    return VP_OK;
+}
+}  // namespace
+
+extern "C" int vp_pack_static(const int32_t* n_steps_b, const int16_t* lane_dst_b, const int64_t* lane_bytes_b,
+                              const int64_t* send_off_b, int N, int rank, int k_max, const int32_t* expert_idx, int T,
+                              int topk, int experts_per_rank, const void* rows, int64_t row_bytes, void* staged,
+                              int64_t staged_capacity_bytes, int32_t* src_map, int32_t* status, void* cuda_stream) {
+    if (N <= 0 || N > VP_MAX_N || T <= 0 || topk <= 0 || k_max <= 0) return VP_E_BAD_ARG;
+    // the problem must fit the built-in block; nothing is launched otherwise
+    const size_t need = vp_pack_workspace_bytes(N, T, topk, k_max);
+    if (need == 0 || need > (size_t)VP_PACK_STATIC_SCRATCH_BYTES) return VP_E_WORKSPACE;
+    void* scratch = nullptr;
+    const int rc = static_scratch_address(&scratch);
+    if (rc != VP_OK) return rc;
+    // vp_pack zeroes the flags it needs and overwrites every other scratch word it reads, so whatever the
+    // previous call left in the block does not matter
+    return vp_pack(n_steps_b, lane_dst_b, lane_bytes_b, send_off_b, N, rank, k_max, expert_idx, T, topk,
+                   experts_per_rank, rows, row_bytes, staged, staged_capacity_bytes, src_map, status, scratch,
+                   (size_t)VP_PACK_STATIC_SCRATCH_BYTES, cuda_stream);
+}

@@ -1,0 +1,77 @@
+"""vp_pack_static: the pack for callers that cannot supply scratch memory.
+
+Some users of the pack run it from inside an engine's steady-state step: they get the input and output
+buffers, own no allocator and may not call cudaMalloc there.  ``vp_pack_static`` serves them from a fixed
+block of device memory inside the library.  It must give exactly what ``vp_pack`` gives -- also when the block
+still holds another problem's leftovers -- so this test runs two different problems back to back through the
+C ABI and compares every output byte with the workspace-taking entry point.  The file sorts last on purpose:
+a run that stops at the first failure has then already been through every other test.
+"""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from workloads.configs import build_pack_case
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def vp():
+    import paper_2609_34340_b200 as vp
+    assert torch.cuda.is_available(), "these tests need a GPU"
+    assert os.path.exists(vp.library_path()), "libvariopath.so has not been built"
+    return vp
+
+
+def _prepare(vp, tokens, hidden, rank, seed):
+    case = build_pack_case(device="cuda", tokens=tokens, hidden=hidden, rank=rank, seed=seed)
+    cat, w = case["catalog"], case["params"]
+    dc = vp.load_catalog(cat.topology.blob(), cat.blob())
+    params = vp.SchedParams(lambda_ns=w.lambda_ns, granule_bytes=w.granule_bytes, k_target=w.k_target,
+                            n_start=w.n_start, i_aa=w.i_aa, k_max=w.k_max)
+    plan = vp.schedule_batch(dc, params, case["demand"].cuda())
+    rows = case["rows"].cuda().contiguous()
+    idx = case["expert_idx"].cuda().contiguous()
+    R = int(case["demand"][0, rank].sum().item() // case["row_bytes"])
+    return dict(plan=plan, rows=rows, idx=idx, R=R, rank=rank, epr=case["experts_per_rank"], keep=dc)
+
+
+def _run(fn, p):
+    staged = torch.zeros((p["R"], p["rows"].shape[1]), dtype=p["rows"].dtype, device="cuda")
+    src_map = torch.full((p["R"],), -1, dtype=torch.int32, device="cuda")
+    status = torch.full((1,), -1, dtype=torch.int32, device="cuda")
+    fn(p["plan"], 0, p["rank"], p["idx"], p["epr"], p["rows"], staged, src_map, status)
+    torch.cuda.synchronize()
+    return staged.cpu().numpy(), src_map.cpu().numpy(), int(status.item())
+
+
+def test_static_scratch_pack_equals_workspace_pack_twice_in_a_row(vp):
+    big = _prepare(vp, tokens=3000, hidden=1024, rank=5, seed=21)      # bulk-copy path, fills much of the block
+    small = _prepare(vp, tokens=333, hidden=40, rank=12, seed=22)      # plain-load path, leaves stale scratch behind it
+    want_big, want_small = _run(vp.pack, big), _run(vp.pack, small)
+    assert want_big[2] == 0 and want_small[2] == 0
+    got_big = _run(vp.pack_static, big)          # first call: also looks up the block's address
+    got_small = _run(vp.pack_static, small)      # second call: the block still holds the first problem
+    got_big_again = _run(vp.pack_static, big)
+    for got, want in ((got_big, want_big), (got_small, want_small), (got_big_again, want_big)):
+        assert got[2] == want[2] == 0
+        assert np.array_equal(got[1], want[1])   # src_map: integer indices, bit for bit
+        assert np.array_equal(got[0], want[0])   # staged rows: bytes, bit for bit
+
+
+def test_static_scratch_pack_refuses_problems_beyond_its_block(vp):
+    p = _prepare(vp, tokens=64, hidden=64, rank=1, seed=23)
+    T_big = 4_000_000                             # far more copies than 4 MiB of scratch can index
+    assert vp.pack_workspace_bytes(16, T_big, 8, p["plan"].k_max) > vp.PACK_STATIC_SCRATCH_BYTES
+    fake_idx = torch.zeros((1, 8), dtype=torch.int32, device="cuda").expand(T_big, 8)   # never read: refused first
+    lib = vp.binding._load()
+    import ctypes as C
+    rc = lib.vp_pack_static(C.c_void_p(p["plan"].n_steps.data_ptr()), C.c_void_p(p["plan"].lane_dst.data_ptr()),
+                            C.c_void_p(p["plan"].lane_bytes.data_ptr()), C.c_void_p(p["plan"].send_off.data_ptr()),
+                            16, 1, p["plan"].k_max, C.c_void_p(fake_idx.data_ptr()), T_big, 8, p["epr"],
+                            C.c_void_p(p["rows"].data_ptr()), 128, C.c_void_p(p["rows"].data_ptr()), 128, None,
+                            C.c_void_p(p["plan"].status.data_ptr()), None)
+    assert rc == vp.E_WORKSPACE
