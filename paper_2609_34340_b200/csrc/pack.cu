@@ -31,7 +31,8 @@ constexpr int VP_ST_INTERNAL_TIMEOUT = 1 << 30;
 
 struct PackWs {
     int32_t* flags;      // [0] abort, [1] n_segments
-    int32_t* hist;       // [n_chunks][N] counts, then exclusive bases
+    int32_t* hist;       // [n_chunks][N] copies of each chunk per destination
+    int32_t* base;       // [n_chunks][N] copies to that destination in earlier chunks
     int32_t* len;        // [N] routed copies per destination
     int32_t* planned;    // [N] rows the plan sends to each destination
     int32_t* seg_ptr;    // [N+1]
@@ -49,6 +50,7 @@ PackWs carve(void* base, int N, int T, int topk, int k_max) {
     int n_chunks = (int)((E + kChunk - 1) / kChunk);
     w.flags = (int32_t*)take(256);
     w.hist = (int32_t*)take((size_t)n_chunks * N * 4);
+    w.base = (int32_t*)take((size_t)n_chunks * N * 4);
     w.len = (int32_t*)take((size_t)N * 4);
     w.planned = (int32_t*)take((size_t)N * 4);
     w.seg_ptr = (int32_t*)take((size_t)(N + 1) * 4);
@@ -91,58 +93,100 @@ pack_count_kernel(const int32_t* __restrict__ idx, long long E, int N, int rank,
     if (bad) atomicOr(status, VP_ST_PACK_MISMATCH);
 }
 
+// One block of VP_MAX_N threads.  Thread j owns destination j; the rank's column of the plan is staged
+// through shared memory a tile of steps at a time so that its global loads run in parallel.
 __global__ void __launch_bounds__(VP_MAX_N)
 pack_plan_kernel(const int32_t* __restrict__ n_steps_p, const int16_t* __restrict__ lane_dst,
                  const int64_t* __restrict__ lane_bytes, const int64_t* __restrict__ send_off, int N, int rank,
                  int k_max, int n_chunks, int64_t row_bytes, int64_t capacity_bytes, PackWs w,
                  int32_t* __restrict__ status) {
     __shared__ int s_cnt[VP_MAX_N + 1];
-    const int j = threadIdx.x;
+    __shared__ int16_t t_dst[VP_MAX_N];
+    __shared__ int32_t t_rows[VP_MAX_N], t_base[VP_MAX_N];
+    const int j = threadIdx.x, NT = blockDim.x;
     int K = *n_steps_p;
     if (K > k_max) K = k_max;
     if (K < 0) K = 0;
-    if (j < N) {
-        int run = 0;                                       // exclusive scan over chunks
-        for (int c = 0; c < n_chunks; c++) {
-            int v = w.hist[(size_t)c * N + j];
-            w.hist[(size_t)c * N + j] = run;
-            run += v;
+    // exclusive scan of the chunk counts, per destination: one warp per destination, 32 chunks per step
+    {
+        const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+        for (int d = warp; d < N; d += n_warps) {
+            int run = 0;
+            const int32_t* __restrict__ in = w.hist;
+            int32_t* __restrict__ out = w.base;
+#pragma unroll 4
+            for (int b0 = 0; b0 < n_chunks; b0 += 32) {
+                const int c = b0 + lane;
+                const int v = c < n_chunks ? in[(size_t)c * N + d] : 0;
+                int incl = v;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int t = __shfl_up_sync(0xffffffffu, incl, o);
+                    if (lane >= o) incl += t;
+                }
+                if (c < n_chunks) out[(size_t)c * N + d] = run + incl - v;
+                run += __shfl_sync(0xffffffffu, incl, 31);
+            }
+            if (lane == 0) w.len[d] = run;
         }
-        w.len[j] = run;
-        int cnt = 0;
-        for (int k = 0; k < K; k++) cnt += (lane_dst[(size_t)k * N + rank] == j);
-        s_cnt[j] = cnt;
     }
+    // pass 1: how many activations send to each destination
+    int cnt = 0;
+    for (int k0 = 0; k0 < K; k0 += NT) {
+        const int k = k0 + j;
+        t_dst[j] = k < K ? lane_dst[(size_t)k * N + rank] : (int16_t)-1;
+        __syncthreads();
+        if (j < N) {
+            const int n = min(NT, K - k0);
+            for (int i = 0; i < n; i++) cnt += (t_dst[i] == j);
+        }
+        __syncthreads();
+    }
+    if (j < N) s_cnt[j] = cnt;
     __syncthreads();
     if (j == 0) {
         int run = 0;
         for (int d = 0; d < N; d++) { int v = s_cnt[d]; s_cnt[d] = run; run += v; }
         s_cnt[N] = run;
-        int st = 0;
-        if (send_off[(size_t)K * N + rank] > capacity_bytes) { st |= VP_ST_PACK_CAPACITY; w.flags[0] = 1; }
-        if (st) atomicOr(status, st);
+        w.seg_ptr[N] = run;
+        if (send_off[(size_t)K * N + rank] > capacity_bytes) { atomicOr(status, VP_ST_PACK_CAPACITY); w.flags[0] = 1; }
     }
     __syncthreads();
-    if (j == 0) w.seg_ptr[N] = s_cnt[N];
-    if (j < N) {
-        w.seg_ptr[j] = s_cnt[j];
-        int p = s_cnt[j];
-        long long cum = 0;
-        bool bad = false;
-        for (int k = 0; k < K; k++) {
-            if (lane_dst[(size_t)k * N + rank] != j) continue;
-            int64_t bytes = lane_bytes[(size_t)k * N + rank];
-            if (bytes % row_bytes) bad = true;
-            w.seg_start[p] = (int32_t)cum;
-            w.seg_row[p] = (int32_t)(send_off[(size_t)k * N + rank] / row_bytes);
-            cum += bytes / row_bytes;
-            p++;
+    // pass 2: the segments of each destination: stream position and staged row where each one starts
+    int p = j < N ? s_cnt[j] : 0;
+    long long cum = 0;
+    bool bad = false;
+    if (j < N) w.seg_ptr[j] = p;
+    for (int k0 = 0; k0 < K; k0 += NT) {
+        const int k = k0 + j;
+        if (k < K) {
+            const int64_t bytes = lane_bytes[(size_t)k * N + rank];
+            t_dst[j] = lane_dst[(size_t)k * N + rank];
+            t_rows[j] = (int32_t)(bytes / row_bytes);
+            t_base[j] = (int32_t)(send_off[(size_t)k * N + rank] / row_bytes);
+            if (t_dst[j] >= 0 && bytes % row_bytes) bad = true;
+        } else {
+            t_dst[j] = -1;
         }
+        __syncthreads();
+        if (j < N) {
+            const int n = min(NT, K - k0);
+            for (int i = 0; i < n; i++) {
+                if (t_dst[i] != j) continue;
+                w.seg_start[p] = (int32_t)cum;
+                w.seg_row[p] = t_base[i];
+                cum += t_rows[i];
+                p++;
+            }
+        }
+        __syncthreads();
+    }
+    if (j < N) {
         w.planned[j] = (int32_t)cum;
         if (j == rank) { if (cum != 0) bad = true; }
         else if (cum != w.len[j]) bad = true;
-        if (bad) atomicOr(status, VP_ST_PACK_MISMATCH);
     }
+    if (bad) atomicOr(status, VP_ST_PACK_MISMATCH);
 }
 
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
@@ -154,7 +198,7 @@ pack_map_kernel(const int32_t* __restrict__ idx, long long E, int N, int rank, i
     const long long e0 = chunk * kChunk;
     if (e0 >= E) return;
     const bool aborted = w.flags[0] != 0;
-    for (int j = lane; j < N; j += 32) base[warp][j] = w.hist[chunk * N + j];
+    for (int j = lane; j < N; j += 32) base[warp][j] = w.base[chunk * N + j];
     __syncwarp();
     for (int it = 0; it < kItems; it++) {
         long long e = e0 + it * 32 + lane;

@@ -797,10 +797,11 @@ int plan_launch(const vp_catalog* c, int B, const vp_sched_params* p, Launch* ou
     if (rc) return rc;
     L.lpg = 1;
     if (dc.g == 4) L.lpg = dc.G <= 4 ? 8 : (dc.G <= 8 ? 4 : (dc.G <= 16 ? 2 : 1));
-    L.threads = dc.N <= 64 ? 256 : 512;
+    L.threads = dc.N <= 64 ? 128 : 512;
     L.kp.drem_in_smem = dc.N <= 64;
     L.kp.stage_terms = (size_t)dc.n_shapes * dc.max_terms * 4 <= 32 * 1024;
-    L.kp.stage_fam = (size_t)dc.n_families * dc.N * 3 <= 64 * 1024;
+    // family tables go to shared memory only when small: beyond that, CTAs per SM matter more than their latency
+    L.kp.stage_fam = (size_t)dc.n_families * dc.N * 3 <= 16 * 1024;
     L.kp.stage_bucket = ((size_t)dc.n_shapes + 1) * 4 <= 32 * 1024;
     L.smem = (size_t)smem_layout(dc, L.kp, L.threads / 32, L.lpg).total;
     if (L.smem + 2048 > (size_t)c->max_smem_optin) return VP_E_UNSUPPORTED;
