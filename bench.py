@@ -32,6 +32,8 @@ METRIC = "matrices_scheduled_per_sec"
 UNIT = "matrices/s"
 INT64_OPS_PER_LANE_CLK = 0.5    # one 64-bit add/min/compare needs two 32-bit ALU issues
 SM_COUNT, LANES_PER_SM = 148, 128
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch on the default workload (ncu, see profiles/)
+NCU_DRAM_BYTES_PER_LAUNCH = {"pack_copy_bulk_kernel": 235_827_968 + 1_792_440_000, "vp_schedule_kernel": 633_856 + 512}
 
 
 def _dist_env():
@@ -291,12 +293,16 @@ def finish(args, world, cat, w, B, N, T, topk, R, prank, row_bytes, pack_bytes, 
     alu_peak_max = SM_COUNT * LANES_PER_SM * INT64_OPS_PER_LANE_CLK * peaks["sm_max_mhz"] * 1e6 / 1e12
     alu_peak_now = SM_COUNT * LANES_PER_SM * INT64_OPS_PER_LANE_CLK * sm_mhz * 1e6 / 1e12
     sched_tops = ops / (sched_avg * 1e-3) / 1e12
+    # DRAM bytes per launch from the ncu captures summarised under profiles/ (default workload only)
+    default_workload = args.sched_config == 2 and args.batch is None and args.pack_tokens == 16384
+    traffic_copy = NCU_DRAM_BYTES_PER_LAUNCH["pack_copy_bulk_kernel"] if default_workload else None
+    traffic_sched = NCU_DRAM_BYTES_PER_LAUNCH["vp_schedule_kernel"] if default_workload else None
     roof_pack = dict(kernel="pack_copy_bulk_kernel", bound="hbm", achieved=round(pack_gbs, 1), peak=peaks["hbm_gbs"],
-                     unit="GB/s", frac=round(pack_gbs / peaks["hbm_gbs"], 4), traffic=None,
+                     unit="GB/s", frac=round(pack_gbs / peaks["hbm_gbs"], 4), traffic=traffic_copy,
                      peak_source=peaks["source"], ms_per_launch=round(copy_avg, 4),
                      algorithmic_bytes_per_launch=copy_bytes)
     roof_sched = dict(kernel="vp_schedule_kernel", bound="alu", achieved=round(sched_tops, 4), peak=round(alu_peak_max, 2),
-                      unit="Tops/s (64-bit integer)", frac=round(sched_tops / alu_peak_max, 5), traffic=None,
+                      unit="Tops/s (64-bit integer)", frac=round(sched_tops / alu_peak_max, 5), traffic=traffic_sched,
                       peak_source="derived: 148 SMs x 128 lanes x 0.5 64-bit ops/clk x max SM clock",
                       frac_at_sampled_clock=round(sched_tops / alu_peak_now, 5), ms_per_launch=round(sched_avg, 4),
                       algorithmic_ops_per_launch=int(ops))
