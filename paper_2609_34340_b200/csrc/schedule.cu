@@ -799,7 +799,8 @@ int plan_launch(const vp_catalog* c, int B, const vp_sched_params* p, Launch* ou
     if (dc.g == 4) L.lpg = dc.G <= 4 ? 8 : (dc.G <= 8 ? 4 : (dc.G <= 16 ? 2 : 1));
     L.threads = dc.N <= 64 ? 128 : 512;
     L.kp.drem_in_smem = dc.N <= 64;
-    L.kp.stage_terms = (size_t)dc.n_shapes * dc.max_terms * 4 <= 32 * 1024;
+    // terms go to shared memory when small, or when the CTA is alone on its SM anyway (512 threads)
+    L.kp.stage_terms = (size_t)dc.n_shapes * dc.max_terms * 4 <= (L.threads >= 512 ? 128 * 1024 : 32 * 1024);
     // family tables go to shared memory only when small: beyond that, CTAs per SM matter more than their latency
     L.kp.stage_fam = (size_t)dc.n_families * dc.N * 3 <= 16 * 1024;
     L.kp.stage_bucket = ((size_t)dc.n_shapes + 1) * 4 <= 32 * 1024;
