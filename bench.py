@@ -235,10 +235,50 @@ def run_ours(args):
     else:
         e2e_ms, h2d, d2h, e2e_steps = run_e2e(vp, args, world, local_rank, dev, sched, pk, dc, params, pplan, idx, rows,
                                               R, barrier)
+    tools = run_tools(vp, dev, load_peaks()) if args.tools and rank == 0 else None
     if rank != 0:
         return
+    sched["_tools"] = tools
     finish(args, world, cat, w, B, N, T, topk, R, prank, row_bytes, pack_bytes, copy_bytes, stats, clocks, launches,
            sched_avg, index_ms, copy_ms, n_copy, ms_per_step, value, e2e_ms, h2d, d2h, e2e_steps, sched, pk)
+
+
+def run_tools(vp, dev, peaks):
+    """The two kernels around the scheduler (`--tools`): Eq. (2) plan time over the config-3 plans and the
+    demand rows of 16 ranks from config-5-sized routing.  Device-resident, CUDA-event timed."""
+    import torch
+    from workloads.configs import build_config
+    from workloads.demand import moe_routing
+    c = build_config(3, device=dev)
+    cat, w = c["catalog"], c["params"]
+    dc = vp.load_catalog(cat.topology.blob(), cat.blob(), device=torch.device(dev).index or 0)
+    plan = vp.schedule_batch(dc, vp_params(vp, w), c["demand"].to(dev).contiguous())
+    out = torch.empty(plan.n_steps.shape[0], dtype=torch.int64, device=dev)
+    steps = int(plan.n_steps.sum().item())
+
+    def timed(fn, reps=20):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps
+
+    ms_t = timed(lambda: vp.plan_time(dc, plan, w.lambda_ns, out=out))
+    bytes_t = steps * cat.topology.N * 10                       # lane_bytes (8) + lane_inst (2) of every emitted step
+    idx = moe_routing(16 * 16384, 256, 8, 1.2, seed=5, device=dev).reshape(16, 16384, 8).contiguous()
+    rows = torch.empty((16, 16), dtype=torch.int64, device=dev)
+    st = torch.empty(1, dtype=torch.int32, device=dev)
+    ms_d = timed(lambda: vp.demand_from_routing(idx, 16, 16, 14336, out=rows, status=st))
+    bytes_d = idx.numel() * 4
+    return {"plan_time": {"workload": f"config 3 plans: 1024 matrices, {steps} activations x 64 lanes", "ms": round(ms_t, 4),
+                          "gb_per_s": round(bytes_t / ms_t / 1e6, 1), "frac_of_hbm_peak": round(bytes_t / ms_t / 1e6 / peaks["hbm_gbs"], 4)},
+            "demand_from_routing": {"workload": "16 ranks x 16384 tokens x top-8 (8.4 MB of indices, L2-resident)",
+                                    "ms": round(ms_d, 4), "gb_per_s": round(bytes_d / ms_d / 1e6, 1)}}
 
 
 def run_e2e(vp, args, world, local_rank, dev, sched, pk, dc, params, pplan, idx, rows, R, barrier):
@@ -328,6 +368,8 @@ def finish(args, world, cat, w, B, N, T, topk, R, prank, row_bytes, pack_bytes, 
                 if e2e_ms else None),
         "gpu_launches": int(launches), "clocks": clocks,
     }
+    if sched.get("_tools"):
+        line["next_rows"] = sched["_tools"]
     line["cpu_baseline"] = cpu_baseline(sched, pk, budget_s=20.0) if world == 1 and not args.no_cpu_baseline else None
     print(json.dumps(line))
 
@@ -433,6 +475,7 @@ def main():
     ap.add_argument("--min-warmup-s", type=float, default=1.0,
                     help="keep warming up (beyond --warmup steps) until this many seconds have passed, so that "
                          "clocks settle and nvidia-smi has samples under load")
+    ap.add_argument("--tools", action="store_true", help="also time vp_plan_time and vp_demand_from_routing")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the CPU oracle leg (profiling runs)")
     args = ap.parse_args()

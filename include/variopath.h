@@ -244,6 +244,27 @@ int vp_pack_host(const int32_t* n_steps_b, const int16_t* lane_dst_b, const int6
                  int32_t* status, void* device_scratch, size_t device_scratch_bytes, void* cuda_stream);
 
 /*
+ * vp_plan_time - modeled completion time of each plan of a batch, Eq. (2) of Section 3:
+ *   T(S) = sum_k ( lambda + max_i x_ki / bw(p_ki) ).
+ * To stay in integers the result is scaled by rate_lcm (vp_info): time_xw[b] = rate_lcm * T(S_b) in
+ * nanoseconds.  Inputs are the device arrays vp_schedule_batch wrote (same B, k_max); time_xw is device
+ * int64[B].  Only steps below n_steps[b] count.
+ */
+int vp_plan_time(const vp_catalog* catalog, int B, int k_max, const int32_t* n_steps, const uint16_t* lane_inst,
+                 const int64_t* lane_bytes, int64_t lambda_ns, int64_t* time_xw, void* cuda_stream);
+
+/*
+ * vp_demand_from_routing - the demand rows of n_src source ranks from their top-k routing indices
+ * (Section 6 "Workloads": demand matrices derived from top-k MoE routing; Section 3: D_ii = 0).
+ *   expert_idx  device int32 [n_src][T][topk]; < 0 = dropped copy; expert e lives on rank e / experts_per_rank
+ *   demand_rows device int64 [n_src][N]: row s is D[src0 + s][.] = row_bytes x copies to each destination,
+ *               the entry for the source rank itself is 0.  Point it at &D[src0][0] of an N x N matrix.
+ *   status      device int32[1]: 1 if some index addresses a rank >= N (that copy is ignored), else 0.
+ */
+int vp_demand_from_routing(const int32_t* expert_idx, int n_src, int T, int topk, int experts_per_rank, int N,
+                           int src0, int64_t row_bytes, int64_t* demand_rows, int32_t* status, void* cuda_stream);
+
+/*
  * Work counters of the last vp_schedule_batch that used `workspace` (device): copies three
  * uint64 to host `out3` after synchronising the stream: activations emitted, (family, start)
  * binding tasks run, AA sweeps run over all tasks.  Used to count the algorithmic operations

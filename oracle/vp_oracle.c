@@ -710,3 +710,28 @@ int vpo_pack(const int32_t *n_steps, const int16_t *lane_dst, const int64_t *lan
     free(stream); free(fill); free(cursor); free(len);
     return st;
 }
+
+/* ------------------------------------------------- demand from routing */
+
+/*
+ * Demand rows from top-k routing (Section 6, "Workloads": demand matrices derived from top-k MoE
+ * routing).  Source rank src0+s routes T tokens; copy (t, slot) goes to expert idx[s][t][slot], which lives
+ * on rank idx / experts_per_rank; D[src][dst] = row_bytes x number of such copies, D[src][src] = 0
+ * (Section 3).  Negative indices are dropped copies.  Returns 1 if an index addresses a rank >= N.
+ */
+int vpo_demand_from_routing(const int32_t *idx, int n_src, int T, int topk, int experts_per_rank, int N, int src0,
+                            int64_t row_bytes, int64_t *rows)
+{
+    int bad = 0;
+    memset(rows, 0, sizeof(int64_t) * (size_t)n_src * N);
+    for (int s = 0; s < n_src; s++)
+        for (int t = 0; t < T; t++)
+            for (int k = 0; k < topk; k++) {
+                int x = idx[((size_t)s * T + t) * topk + k];
+                if (x < 0) continue;
+                int j = x / experts_per_rank;
+                if (j >= N) { bad = 1; continue; }
+                if (j != src0 + s) rows[(size_t)s * N + j] += row_bytes;
+            }
+    return bad;
+}

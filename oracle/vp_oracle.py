@@ -53,6 +53,8 @@ def _load():
                                        C.c_int64, C.c_int] + [C.c_void_p] * 9 + [C.c_void_p, C.c_int, C.c_void_p])
         _lib.vpo_schedule_batch.argtypes = ([C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int64,
                                              C.c_int, C.c_int, C.c_int, C.c_int64, C.c_int] + [C.c_void_p] * 9)
+        _lib.vpo_demand_from_routing.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
+                                                 C.c_int64, C.c_void_p]
         _lib.vpo_pack.argtypes = ([C.c_void_p] * 4 + [C.c_int] * 3 + [C.c_void_p, C.c_int, C.c_int, C.c_int,
                                   C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p])
     return _lib
@@ -66,6 +68,17 @@ def _param(params, name, default=0):
     if isinstance(params, dict):
         return int(params.get(name, default))
     return int(getattr(params, name, default))
+
+
+def demand_from_routing(expert_idx, experts_per_rank: int, N: int, row_bytes: int, src0: int = 0):
+    """Demand rows ``[n_src, N]`` of the sources ``src0..`` from ``[n_src, T, topk]`` routing indices; also the
+    out-of-range flag."""
+    idx = np.ascontiguousarray(expert_idx, dtype=np.int32)
+    n_src, T, topk = idx.shape
+    rows = np.zeros((n_src, N), np.int64)
+    bad = _load().vpo_demand_from_routing(_p(idx), n_src, T, topk, int(experts_per_rank), int(N), int(src0),
+                                          int(row_bytes), _p(rows))
+    return rows, int(bad)
 
 
 class OracleCatalog:
@@ -188,6 +201,10 @@ class OracleCatalog:
                                         _p(np.ascontiguousarray(plan["lane_inst"])),
                                         _p(np.ascontiguousarray(plan["lane_bytes"])), int(lambda_ns))
         return Fraction(int(v), self.W)
+
+    def modeled_time_xw(self, plan: dict, lambda_ns: int) -> int:
+        """Eq. (2) scaled by the lcm of the path rates (an integer, nanoseconds x W)."""
+        return int(self.modeled_time(plan, lambda_ns) * self.W)
 
     def check_plan(self, D, plan: dict, tau: int = 0, granule: int = 1) -> int:
         D = np.ascontiguousarray(D, dtype=np.int64)

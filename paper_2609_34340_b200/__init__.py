@@ -20,6 +20,8 @@ from .binding import (  # noqa: F401
     pack_static,
     PACK_STATIC_SCRATCH_BYTES,
     kernel_launch_count,
+    plan_time,
+    demand_from_routing,
     schedule_read_stats,
     profile_enable,
     profile_read,

@@ -88,6 +88,8 @@ def _load():
     lib.vp_pack_host_scratch_bytes.restype = sz
     lib.vp_pack_host.argtypes = pack_args + [P, sz, P]
     lib.vp_kernel_launch_count.restype = i64
+    lib.vp_plan_time.argtypes = [vp, i32, i32, P, P, P, i64, P, P]
+    lib.vp_demand_from_routing.argtypes = [P, i32, i32, i32, i32, i32, i32, i64, P, P, P]
     lib.vp_schedule_read_stats.argtypes = [P, P, P]
     lib.vp_profile_enable.argtypes = [i32]
     lib.vp_profile_read.argtypes = [i32, C.POINTER(C.c_double), C.POINTER(i64)]
@@ -251,6 +253,32 @@ def schedule_batch_host(catalog: Catalog, params: SchedParams, demand: torch.Ten
     _check(_sched_call(_load().vp_schedule_batch_host, catalog, p, demand, tau_ns_in, B, plan, scratch, stream),
            "vp_schedule_batch_host")
     return plan
+
+
+def plan_time(catalog: Catalog, plan: Plan, lambda_ns: int, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """``vp_plan_time``: ``rate_lcm x`` modeled completion time (Eq. 2) of every plan, int64 ``[B]`` on device."""
+    B = plan.n_steps.shape[0]
+    if out is None:
+        out = torch.empty(B, dtype=torch.int64, device=plan.n_steps.device)
+    _check(_load().vp_plan_time(catalog._h, int(B), int(plan.k_max), _ptr(plan.n_steps), _ptr(plan.lane_inst),
+                                _ptr(plan.lane_bytes), int(lambda_ns), _ptr(out), _stream(stream)), "vp_plan_time")
+    return out
+
+
+def demand_from_routing(expert_idx: torch.Tensor, experts_per_rank: int, N: int, row_bytes: int, src0: int = 0,
+                        out: Optional[torch.Tensor] = None, status: Optional[torch.Tensor] = None, stream=None):
+    """``vp_demand_from_routing``: ``expert_idx`` is ``[n_src, T, topk]`` int32 on device; returns
+    (``[n_src, N]`` int64 demand rows, status int32[1])."""
+    assert expert_idx.is_cuda and expert_idx.dtype == torch.int32 and expert_idx.is_contiguous() and expert_idx.dim() == 3
+    n_src, T, topk = expert_idx.shape
+    if out is None:
+        out = torch.empty((n_src, N), dtype=torch.int64, device=expert_idx.device)
+    if status is None:
+        status = torch.empty(1, dtype=torch.int32, device=expert_idx.device)
+    _check(_load().vp_demand_from_routing(_ptr(expert_idx), int(n_src), int(T), int(topk), int(experts_per_rank), int(N),
+                                          int(src0), int(row_bytes), _ptr(out), _ptr(status), _stream(stream)),
+           "vp_demand_from_routing")
+    return out, status
 
 
 def pack_workspace_bytes(N: int, T: int, topk: int, k_max: int) -> int:

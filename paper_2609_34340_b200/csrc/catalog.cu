@@ -277,6 +277,9 @@ extern "C" int vp_load_catalog(const void* topology, size_t topo_bytes, const vo
     if (!rc) rc = upload(c, forced_ptr, &dc.forced_ptr);
     if (!rc) rc = upload(c, forced_cell, &dc.forced_cell);
     if (!rc) rc = upload(c, forced_bw, &dc.forced_bw);
+    std::vector<uint32_t> inst_wdiv(n_inst);
+    for (int r = 0; r < n_inst; r++) inst_wdiv[r] = (uint32_t)(W / inst[r].bw);
+    if (!rc) rc = upload(c, inst_wdiv, &dc.inst_wdiv);
     if (rc) {
         vp_free_catalog(c);
         if (prev >= 0) cudaSetDevice(prev);

@@ -34,6 +34,8 @@ struct DevCat {
     const uint32_t* forced_ptr;
     const uint16_t* forced_cell;
     const uint32_t* forced_bw;
+    // per path instance: rate_lcm / bw (Eq. 2 lane times are bytes x this, in 1/rate_lcm ns)
+    const uint32_t* inst_wdiv;
     int64_t class_bw[VP_MAX_CLASSES];
     int64_t class_wdiv[VP_MAX_CLASSES];   // rate_lcm / bw
     int64_t bw_max, W;

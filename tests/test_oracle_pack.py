@@ -84,3 +84,20 @@ def test_pack_error_statuses(oracle_lib):
     other[0, 0] = (other[0, 0] + epr) % 32                    # routing no longer matches the plan
     assert oc.pack(plan, 1, other, epr, rows, R)[2] & oracle.ST_PACK_MISMATCH
     assert oc.pack(plan, 1, idx, epr, rows, R)[2] == 0
+
+
+def test_demand_from_routing_equals_a_library_histogram(oracle_lib):
+    """The demand rows are a 2-D histogram of (source, destination rank) pairs: numpy's bincount is the pin."""
+    rng = np.random.default_rng(4)
+    n_src, T, topk, epr, N, rb = 5, 300, 6, 4, 8, 1024
+    idx = rng.integers(-1, N * epr, size=(n_src, T, topk)).astype(np.int32)      # -1 = dropped copy
+    rows, bad = oracle_lib.demand_from_routing(idx, epr, N, rb, src0=2)
+    assert bad == 0
+    want = np.zeros((n_src, N), np.int64)
+    for s in range(n_src):
+        d = idx[s][idx[s] >= 0] // epr
+        want[s] = np.bincount(d, minlength=N) * rb
+        want[s, 2 + s] = 0
+    assert np.array_equal(rows, want)
+    idx[0, 0, 0] = N * epr                                                         # a rank that does not exist
+    assert oracle_lib.demand_from_routing(idx, epr, N, rb, src0=2)[1] == 1
