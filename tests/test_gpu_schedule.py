@@ -229,3 +229,30 @@ def test_config4_full_batch(vp, oracle_lib):
             continue
         want = oc.schedule_batch(Dn[sample], w)
         _assert_same({k: got[k][sample] if k != "k_max" else got[k] for k in got}, want)
+
+
+def test_extreme_values_stay_exact(vp, oracle_lib):
+    """Entries just below 2^40, lambda just below 2^40, tau at its limit, mixed rates (rate lcm 1600):
+    the 128-bit utility compare and the 64-bit byte path must agree with the oracle's __int128."""
+    cat = complete_catalog(tree_topology(2, pcie_bw=64, nic_bw=50))
+    rng = np.random.default_rng(17)
+    big = (1 << 40) - 1
+    D = np.zeros((6, 16, 16), np.int64)
+    D[0] = rng.integers(big - 1000, big + 1, size=(16, 16))
+    D[1] = rng.integers(0, 2, size=(16, 16)) * big
+    D[2] = rng.integers(0, big + 1, size=(16, 16))
+    D[3, 0, 9] = big
+    D[4] = rng.integers(0, 3, size=(16, 16))
+    D[5] = rng.integers(big // 2, big, size=(16, 16)) * (rng.random((16, 16)) < 0.2)
+    for b in range(6):
+        np.fill_diagonal(D[b], 0)
+    tau = np.array([0, 0, 1 << 40, 1, 0, 12345], np.int64)
+    w = WParams(lambda_ns=(1 << 40) - 1, granule_bytes=1, k_target=7, k_max=400).resolved(16)
+    got, want, *_ = _both(vp, oracle_lib, cat, D, w, tau=tau)
+    _assert_same(got, want)
+    assert (got["status"] & ~vp.ST_STEP_LIMIT == 0).all()
+    # the same matrices scaled to a 4096-byte granule take the 32-bit unit path where capacities allow
+    D2 = (D // 4096) * 4096
+    w2 = WParams(lambda_ns=0, granule_bytes=4096, k_target=48, k_max=400).resolved(16)
+    got, want, *_ = _both(vp, oracle_lib, cat, D2, w2)
+    _assert_same(got, want)
