@@ -117,6 +117,26 @@ int vp_load_catalog(const void* topology, size_t topology_bytes,
 void vp_free_catalog(vp_catalog* catalog);
 int vp_catalog_info(const vp_catalog* catalog, vp_info* out);
 
+/*
+ * vp_build_catalog - offline catalog construction, Algorithm 1 of Section 4.1 (host code, no GPU work).
+ *
+ * Enumerates, by the pruned binary depth-first search of Algorithm 1 (CanAdd: resource disjointness and the
+ * per-group degree limit g; SuffixOK; Complete), every multiset of the topology's path instances that gives
+ * each group exactly g outgoing and g incoming lanes without using a directed resource twice, groups the
+ * families by shape, applies PruneFamilies (duplicates; same footprints with no lower and somewhere higher
+ * rates) and serialises the result as a channels blob (layout under vp_load_catalog; shapes ordered by their
+ * sorted (a, d, count) lists, families by instance-id list).  The search is exponential in the number of
+ * instances (Section 4.1): it is meant for one or two nodes; more than 2^22 families gives VP_E_UNSUPPORTED.
+ *
+ * topology: host blob (layout under vp_load_catalog; apply PrunePaths before serialising it).
+ * channels_out: host buffer of capacity_bytes, or NULL to query the size.  *bytes_needed always receives the
+ * blob size; n_shapes_out / n_families_out (may be NULL) the catalog size (the columns of Table 3).
+ * Returns VP_E_WORKSPACE if the buffer is too small, VP_E_BAD_CATALOG for a malformed topology or one that
+ * admits no family at all.
+ */
+int vp_build_catalog(const void* topology, size_t topology_bytes, void* channels_out, size_t capacity_bytes,
+                     size_t* bytes_needed, int32_t* n_shapes_out, int32_t* n_families_out);
+
 /* Bytes of device scratch vp_schedule_batch needs for a batch of B (multiple of 256). */
 size_t vp_schedule_workspace_bytes(const vp_catalog* catalog, int B, const vp_sched_params* params);
 

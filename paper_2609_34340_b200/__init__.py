@@ -11,6 +11,7 @@ from .binding import (  # noqa: F401
     Plan,
     SchedParams,
     load_catalog,
+    build_catalog,
     schedule_workspace_bytes,
     schedule_batch,
     schedule_batch_host,

@@ -88,6 +88,7 @@ def _load():
     lib.vp_pack_host_scratch_bytes.restype = sz
     lib.vp_pack_host.argtypes = pack_args + [P, sz, P]
     lib.vp_kernel_launch_count.restype = i64
+    lib.vp_build_catalog.argtypes = [P, sz, P, sz, C.POINTER(sz), C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
     lib.vp_plan_time.argtypes = [vp, i32, i32, P, P, P, i64, P, P]
     lib.vp_demand_from_routing.argtypes = [P, i32, i32, i32, i32, i32, i32, i64, P, P, P]
     lib.vp_schedule_read_stats.argtypes = [P, P, P]
@@ -169,6 +170,18 @@ def load_catalog(topology: bytes, channels: bytes, device: int = 0) -> Catalog:
     _check(_load().vp_load_catalog(topology, len(topology), channels, len(channels), int(device), C.byref(h)),
            "vp_load_catalog")
     return Catalog(h.value, int(device))
+
+
+def build_catalog(topology: bytes):
+    """``vp_build_catalog`` (Algorithm 1, host code): returns (channels blob, n_shapes, n_families)."""
+    topology = bytes(topology)
+    need, ns, nf = C.c_size_t(0), C.c_int32(0), C.c_int32(0)
+    _check(_load().vp_build_catalog(topology, len(topology), None, 0, C.byref(need), C.byref(ns), C.byref(nf)),
+           "vp_build_catalog")
+    buf = C.create_string_buffer(need.value)
+    _check(_load().vp_build_catalog(topology, len(topology), buf, need.value, C.byref(need), C.byref(ns), C.byref(nf)),
+           "vp_build_catalog")
+    return buf.raw[:need.value], int(ns.value), int(nf.value)
 
 
 def schedule_workspace_bytes(catalog: Catalog, B: int, params: SchedParams) -> int:

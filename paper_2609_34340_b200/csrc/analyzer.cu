@@ -1,0 +1,195 @@
+// vp_build_catalog: offline catalog construction, Algorithm 1 of Section 4.1 (host code).
+//
+// Pruned binary DFS over the path instances in id order.  A state is (next instance t, chosen multiset B);
+// the include branch is taken when CanAdd holds (resource disjointness and the per-group degree limits g),
+// SuffixOK cuts states whose remaining instances cannot fill every group's g outgoing and g incoming slots,
+// Complete states are recorded under their shape M.  An instance of lane multiplicity m (PIX) is decided in
+// one level as "0..m lanes".  PruneFamilies then drops, inside each bucket, exact duplicates and families
+// that another family matches footprint by footprint with no lower and somewhere higher rates.
+// Output order (what the scheduler's tie-breaks refer to): shapes by their sorted (a, d, count) list,
+// families inside a bucket by their instance-id list.
+#include <algorithm>
+#include <cstring>
+#include <map>
+#include <vector>
+
+#include "vp_internal.h"
+
+namespace {
+
+struct AInst {
+    int a, d, mult, n_res;
+    long long bw;
+    int res[4];
+};
+
+struct Analyzer {
+    int N, G, g, n_res;
+    std::vector<AInst> inst;
+    std::vector<std::vector<int>> out_suffix, in_suffix;   // lanes still available from instance t on, per group
+    std::vector<int> out_deg, in_deg, chosen;
+    std::vector<unsigned char> used;                        // directed resources taken by the partial family
+    std::vector<std::vector<uint16_t>> found;
+    size_t limit;
+    bool overflow = false;
+
+    bool complete() const {
+        for (int a = 0; a < G; a++)
+            if (out_deg[a] != g || in_deg[a] != g) return false;
+        return true;
+    }
+    bool suffix_ok(int t) const {
+        for (int a = 0; a < G; a++)
+            if (out_deg[a] + out_suffix[t][a] < g || in_deg[a] + in_suffix[t][a] < g) return false;
+        return true;
+    }
+    void explore(int t) {
+        if (overflow) return;
+        if (complete()) {
+            if (found.size() >= limit) { overflow = true; return; }
+            found.emplace_back(chosen.begin(), chosen.end());
+            return;
+        }
+        if (t >= (int)inst.size() || !suffix_ok(t)) return;
+        explore(t + 1);                                     // exclude r_t
+        const AInst& r = inst[t];
+        for (int k = 0; k < r.n_res; k++)                  // CanAdd: resource disjointness
+            if (used[r.res[k]]) return;
+        for (int k = 0; k < r.n_res; k++) used[r.res[k]] = 1;
+        int added = 0;
+        for (int c = 1; c <= r.mult; c++) {                 // CanAdd: degree limits, one more lane each round
+            if (out_deg[r.a] + 1 > g || in_deg[r.d] + 1 > g) break;
+            out_deg[r.a]++; in_deg[r.d]++;
+            chosen.push_back(t);
+            added++;
+            explore(t + 1);
+        }
+        for (int k = 0; k < added; k++) { out_deg[r.a]--; in_deg[r.d]--; chosen.pop_back(); }
+        for (int k = 0; k < r.n_res; k++) used[r.res[k]] = 0;
+    }
+};
+
+typedef std::vector<std::pair<std::pair<int, int>, int>> Shape;   // sorted ((a, d), count)
+
+uint32_t rd32(const uint8_t* p) { return (uint32_t)p[0] | ((uint32_t)p[1] << 8) | ((uint32_t)p[2] << 16) | ((uint32_t)p[3] << 24); }
+uint16_t rd16(const uint8_t* p) { return (uint16_t)(p[0] | (p[1] << 8)); }
+void wr32(std::vector<uint8_t>& o, uint32_t v) { for (int k = 0; k < 4; k++) o.push_back((uint8_t)(v >> (8 * k))); }
+void wr16(std::vector<uint8_t>& o, uint16_t v) { o.push_back((uint8_t)v); o.push_back((uint8_t)(v >> 8)); }
+
+// per group pair: the (sorted footprint, rate) of every lane, sorted; used by the dominance test
+typedef std::map<std::pair<int, int>, std::vector<std::pair<std::vector<int>, long long>>> Signature;
+
+Signature signature(const Analyzer& A, const std::vector<uint16_t>& fam) {
+    Signature s;
+    for (uint16_t id : fam) {
+        const AInst& r = A.inst[id];
+        std::vector<int> fp(r.res, r.res + r.n_res);
+        std::sort(fp.begin(), fp.end());
+        s[{r.a, r.d}].push_back({fp, r.bw});
+    }
+    for (auto& kv : s) std::sort(kv.second.begin(), kv.second.end());
+    return s;
+}
+
+// x is dominated by y: same footprints lane by lane, y nowhere slower, somewhere faster
+bool dominated(const Signature& x, const Signature& y) {
+    bool strict = false;
+    for (const auto& kv : x) {
+        auto it = y.find(kv.first);
+        if (it == y.end() || it->second.size() != kv.second.size()) return false;
+        for (size_t k = 0; k < kv.second.size(); k++) {
+            if (kv.second[k].first != it->second[k].first) return false;
+            if (it->second[k].second < kv.second[k].second) return false;
+            if (it->second[k].second > kv.second[k].second) strict = true;
+        }
+    }
+    return strict;
+}
+
+}  // namespace
+
+extern "C" int vp_build_catalog(const void* topology, size_t topo_bytes, void* channels_out, size_t capacity_bytes,
+                                size_t* bytes_needed, int32_t* n_shapes_out, int32_t* n_families_out) {
+    if (!topology || !bytes_needed) return VP_E_BAD_ARG;
+    const uint8_t* t = (const uint8_t*)topology;
+    if (topo_bytes < 32 || rd32(t) != 0x50545056u || rd32(t + 4) != 1) return VP_E_BAD_CATALOG;
+    Analyzer A;
+    A.N = (int)rd32(t + 8); A.G = (int)rd32(t + 12); A.g = (int)rd32(t + 16); A.n_res = (int)rd32(t + 24);
+    const int n_inst = (int)rd32(t + 28);
+    if (A.N <= 0 || A.G <= 0 || A.g <= 0 || (long long)A.G * A.g != A.N || n_inst <= 0 || n_inst > 0xFFFE || A.n_res < 0 ||
+        A.N > 0xFFFF || topo_bytes < 32 + (size_t)n_inst * 20)
+        return VP_E_BAD_CATALOG;
+    A.inst.resize(n_inst);
+    for (int r = 0; r < n_inst; r++) {
+        const uint8_t* p = t + 32 + (size_t)r * 20;
+        AInst& q = A.inst[r];
+        q.a = rd16(p); q.d = rd16(p + 2); q.n_res = p[5]; q.mult = rd16(p + 6); q.bw = rd32(p + 8);
+        if (q.a >= A.G || q.d >= A.G || q.n_res > 4 || q.mult < 1 || q.bw <= 0) return VP_E_BAD_CATALOG;
+        for (int k = 0; k < q.n_res; k++) {
+            q.res[k] = rd16(p + 12 + 2 * k);
+            if (q.res[k] >= A.n_res) return VP_E_BAD_CATALOG;
+        }
+        if (r > 0 && (A.inst[r - 1].a > q.a || (A.inst[r - 1].a == q.a && A.inst[r - 1].d > q.d))) return VP_E_BAD_CATALOG;
+    }
+    A.out_suffix.assign(n_inst + 1, std::vector<int>(A.G, 0));
+    A.in_suffix.assign(n_inst + 1, std::vector<int>(A.G, 0));
+    for (int r = n_inst - 1; r >= 0; r--) {
+        A.out_suffix[r] = A.out_suffix[r + 1];
+        A.in_suffix[r] = A.in_suffix[r + 1];
+        A.out_suffix[r][A.inst[r].a] += A.inst[r].mult;
+        A.in_suffix[r][A.inst[r].d] += A.inst[r].mult;
+    }
+    A.out_deg.assign(A.G, 0);
+    A.in_deg.assign(A.G, 0);
+    A.used.assign(A.n_res + 1, 0);
+    A.limit = (size_t)1 << 22;                              // more families than this is not a usable catalog
+    A.explore(0);
+    if (A.overflow) return VP_E_UNSUPPORTED;
+    if (A.found.empty()) return VP_E_BAD_CATALOG;
+
+    // buckets by shape, pruned, in canonical order
+    std::map<Shape, std::vector<std::vector<uint16_t>>> buckets;
+    for (auto& fam : A.found) {
+        std::map<std::pair<int, int>, int> cnt;
+        for (uint16_t id : fam) cnt[{A.inst[id].a, A.inst[id].d}]++;
+        buckets[Shape(cnt.begin(), cnt.end())].push_back(fam);
+    }
+    size_t n_fam = 0, total_nnz = 0;
+    for (auto& kv : buckets) {
+        auto& fams = kv.second;
+        std::sort(fams.begin(), fams.end());
+        fams.erase(std::unique(fams.begin(), fams.end()), fams.end());
+        std::vector<Signature> sig;
+        for (auto& f : fams) sig.push_back(signature(A, f));
+        std::vector<std::vector<uint16_t>> keep;
+        for (size_t x = 0; x < fams.size(); x++) {
+            bool dom = false;
+            for (size_t y = 0; y < fams.size() && !dom; y++)
+                if (y != x && dominated(sig[x], sig[y])) dom = true;
+            if (!dom) keep.push_back(fams[x]);
+        }
+        fams.swap(keep);
+        n_fam += fams.size();
+        total_nnz += kv.first.size();
+    }
+    std::vector<uint8_t> o;
+    wr32(o, 0x48435056u); wr32(o, 1); wr32(o, (uint32_t)A.N); wr32(o, (uint32_t)buckets.size());
+    wr32(o, (uint32_t)n_fam); wr32(o, (uint32_t)total_nnz);
+    uint32_t run = 0;
+    for (auto& kv : buckets) { wr32(o, run); run += (uint32_t)kv.first.size(); }
+    wr32(o, run);
+    for (auto& kv : buckets)
+        for (auto& e : kv.first) { wr16(o, (uint16_t)e.first.first); wr16(o, (uint16_t)e.first.second); wr16(o, (uint16_t)e.second); wr16(o, 0); }
+    run = 0;
+    for (auto& kv : buckets) { wr32(o, run); run += (uint32_t)kv.second.size(); }
+    wr32(o, run);
+    for (auto& kv : buckets)
+        for (auto& f : kv.second)
+            for (uint16_t id : f) wr16(o, id);
+    *bytes_needed = o.size();
+    if (n_shapes_out) *n_shapes_out = (int32_t)buckets.size();
+    if (n_families_out) *n_families_out = (int32_t)n_fam;
+    if (!channels_out || capacity_bytes < o.size()) return channels_out ? VP_E_WORKSPACE : VP_OK;
+    memcpy(channels_out, o.data(), o.size());
+    return VP_OK;
+}

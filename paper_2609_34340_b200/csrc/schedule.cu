@@ -567,7 +567,11 @@ vp_schedule_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand, co
     const int N = dc.N, G = dc.G, tid = threadIdx.x, NT = blockDim.x;
     const int lane = tid & 31, warp = tid >> 5, n_warps = NT >> 5;
     const Smem L = smem_layout(dc, kp, n_warps, LPG);
-    int64_t* Drem = kp.drem_in_smem ? (int64_t*)(smem_raw + L.drem) : ws_drem + (size_t)blockIdx.x * N * N;
+    // lane teams are only used up to 16 groups (N <= 64), where D_rem is always in shared memory: saying so at
+    // compile time lets every access to it be a shared-memory instruction with 32-bit addressing
+    int64_t* Drem;
+    if constexpr (LPG > 1) Drem = (int64_t*)(smem_raw + L.drem);
+    else Drem = kp.drem_in_smem ? (int64_t*)(smem_raw + L.drem) : ws_drem + (size_t)blockIdx.x * N * N;
     Ctx c;
     c.N = N; c.G = G; c.tid = tid; c.NT = NT; c.lane = lane; c.warp = warp; c.n_warps = n_warps;
     c.Dhat = (int64_t*)(smem_raw + L.dhat);
