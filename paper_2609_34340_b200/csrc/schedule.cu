@@ -346,6 +346,7 @@ __device__ __forceinline__ void decompose(const DevCat& dc, const KParams& kp, c
 #pragma unroll
                 for (int q = 0; q < GS; q++) dstb[fin[d * GS + q] & 0xff] = (uint8_t)(d * GS + (q + t) % GS);
             int64_t F_old = -1, F_new = -1, tmax = 0;
+            bool tmax_done = false;
             if constexpr (LPG > 1) {
                 // team path: one rank group per team of LPG lanes (G <= 32 / LPG)
                 const bool active = team < G;
@@ -401,21 +402,34 @@ __device__ __forceinline__ void decompose(const DevCat& dc, const KParams& kp, c
                     }
                     // Eq. (8): sum over the teams.  Every lane of a team holds the team's value and the
                     // exchanges connect equal team lanes only, so all 32 lanes end with the same total.
-                    int64_t part = active ? (int64_t)v : 0;
+                    if constexpr (sizeof(V) == 4) {
+                        // at most 64 lanes of less than 2^25 granules each: the total fits 32 bits, one warp-reduce
+                        F_new = (int64_t)__reduce_add_sync(0xffffffffu, (active && tl == 0) ? (uint32_t)v : 0u);
+                    } else {
+                        int64_t part = active ? (int64_t)v : 0;
 #pragma unroll
-                    for (int o = 16; o >= LPG; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
-                    F_new = part;
+                        for (int o = 16; o >= LPG; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+                        F_new = part;
+                    }
                     cnt.sweeps++;
                     if (F_new <= F_old) break;
                     F_old = F_new;
                     __syncwarp();
                 }
                 // Eq. (9) volumes are the chosen credits of the last destination half; slowest lane of Eq. (10)
+                V xmax = 0;
                 if (active && tl < (LPG < 4 ? LPG : 4)) {
 #pragma unroll
                     for (int kq = 0; kq < TC::NQ; kq++) {
                         const V x = cred[((bpk >> (2 * qv[kq])) & 3) * 4 + qv[kq]];
+                        xmax = max_v(xmax, x);
                         tmax = max_v(tmax, (int64_t)x * c.tscale[cls_in[kq]]);
+                    }
+                }
+                if constexpr (sizeof(V) == 4) {
+                    if (dc.n_classes == 1) {          // one path rate: the slowest lane carries the largest volume
+                        tmax = (int64_t)__reduce_max_sync(0xffffffffu, (uint32_t)xmax) * c.tscale[0];
+                        tmax_done = true;
                     }
                 }
                 __syncwarp();
@@ -473,7 +487,7 @@ __device__ __forceinline__ void decompose(const DevCat& dc, const KParams& kp, c
                     F_old = F_new;
                 }
             }
-            tmax = warp_max_i64(tmax);
+            if (!tmax_done) tmax = warp_max_i64(tmax);
             cnt.tasks++;
             if (t == 0) {
 #pragma unroll
