@@ -284,6 +284,41 @@ int vp_plan_time(const vp_catalog* catalog, int B, int k_max, const int32_t* n_s
 int vp_demand_from_routing(const int32_t* expert_idx, int n_src, int T, int topk, int experts_per_rank, int N,
                            int src0, int64_t row_bytes, int64_t* demand_rows, int32_t* status, void* cuda_stream);
 
+/* Bytes of device scratch vp_unpack needs (multiple of 256); 0 if the sizes are not supported. */
+size_t vp_unpack_workspace_bytes(int N, int64_t capacity_rows, int experts_per_rank, int k_max);
+
+/*
+ * vp_unpack - the receive side of the buffer layout (Section 5: "the receive kernel unpacks them
+ * directly into the output layout").
+ *
+ * In step k of the plan rank j receives, from its one sender i of that step (lane_dst[k][i] == j), the
+ * rows stored at receive-buffer byte offset recv_off[k][j] onwards.  The output is expert-major: the rows
+ * for local expert 0, then 1, ...; inside an expert by source rank; inside a source in arrival order
+ * (which, with vp_pack on the sending side, is the sender's ascending (token, slot) order).
+ *
+ * n_steps_b, lane_dst_b, recv_off_b: device pointers to ONE matrix's plan (row stride N).
+ * recv        [capacity_rows][row_bytes] device: the receive buffer; rows beyond
+ *             recv_off[n_steps][rank] / row_bytes are ignored.
+ * recv_expert [capacity_rows] int32 device: local expert id (0 .. experts_per_rank-1) of each received
+ *             row (the metadata that travels beside the payload).
+ * out         [capacity_rows][row_bytes] device; rows beyond the received count keep their content.
+ * expert_off  [experts_per_rank + 1] int32 device: first output row of each local expert, then the total.
+ * out_src, out_map [capacity_rows] int32 device or NULL: source rank and receive-buffer row of each
+ *             output row.
+ * status      device int32[1]: VP_ST_PACK_CAPACITY if more rows were received than capacity_rows
+ *             (nothing is copied); VP_ST_PACK_MISMATCH if an offset is not a multiple of row_bytes, a
+ *             received segment has no sender in the plan, or an expert id is out of range (that row is
+ *             left out).
+ * Limits: N * experts_per_rank <= 1024 and capacity_rows < 2^31, else VP_E_UNSUPPORTED.
+ * workspace: device, 256-byte aligned, >= vp_unpack_workspace_bytes.
+ */
+int vp_unpack(const int32_t* n_steps_b, const int16_t* lane_dst_b, const int64_t* recv_off_b,
+              int N, int rank, int k_max,
+              const void* recv, int64_t row_bytes, int64_t capacity_rows,
+              const int32_t* recv_expert, int experts_per_rank,
+              void* out, int32_t* expert_off, int32_t* out_src, int32_t* out_map,
+              int32_t* status, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /*
  * Work counters of the last vp_schedule_batch that used `workspace` (device): copies three
  * uint64 to host `out3` after synchronising the stream: activations emitted, (family, start)
@@ -297,7 +332,7 @@ int vp_schedule_read_stats(const void* workspace, void* cuda_stream, uint64_t* o
  * events on the caller's stream around its own launches; vp_profile_read synchronises those
  * events, returns the summed device time and the number of timed launches of one kind since
  * the last read (kind 0: schedule kernel, 1: the three pack index kernels as a group, 2: the
- * pack copy kernel) and discards them.  Creating events allocates driver resources.
+ * pack copy kernel, 3: the unpack copy kernel) and discards them.  Creating events allocates driver resources.
  */
 int vp_profile_enable(int on);
 int vp_profile_read(int kind, double* total_ms, int64_t* launches);

@@ -735,3 +735,54 @@ int vpo_demand_from_routing(const int32_t *idx, int n_src, int T, int topk, int 
             }
     return bad;
 }
+
+/* ------------------------------------------------------------ unpack */
+
+/*
+ * Receive side of the buffer layout (Section 5: "the receive kernel unpacks them directly into the
+ * output layout").  Rank `rank` has received, for every step k in which some source i sends to it
+ * (lane_dst[k][i] == rank; at most one such i), that step's rows at byte offset recv_off[k][rank] of the
+ * receive buffer; recv_expert[r] is the local expert (0 .. experts_per_rank-1) of received row r.  The
+ * output is expert-major: all rows of local expert 0, then 1, ...; inside an expert by source rank, inside a
+ * source in arrival order (which is the source's (token, slot) order).  expert_off[e] is the first output row of
+ * expert e (expert_off[experts_per_rank] = total), out_src / out_map (optional) give each output row's source
+ * rank and the received row it came from.  Returns status bits.
+ */
+int vpo_unpack(const int32_t *n_steps, const int16_t *lane_dst, const int64_t *recv_off, int N, int rank, int k_max,
+               const void *recv, int64_t row_bytes, int64_t capacity_rows, const int32_t *recv_expert,
+               int experts_per_rank, void *out, int32_t *expert_off, int32_t *out_src, int32_t *out_map)
+{
+    (void)k_max;
+    int K = *n_steps, st = 0;
+    int64_t total = recv_off[(size_t)K * N + rank];
+    for (int e = 0; e <= experts_per_rank; e++) expert_off[e] = 0;
+    if (total % row_bytes) st |= VPO_ST_PACK_MISMATCH;
+    int64_t R = total / row_bytes;
+    if (R > capacity_rows) return st | VPO_ST_PACK_CAPACITY;
+    int *src_of = (int *)malloc(sizeof(int) * (size_t)(R + 1));
+    for (int64_t r = 0; r < R; r++) src_of[r] = -1;
+    for (int k = 0; k < K; k++) {
+        int64_t lo = recv_off[(size_t)k * N + rank], hi = recv_off[(size_t)(k + 1) * N + rank];
+        if (hi == lo) continue;
+        if (lo % row_bytes || hi % row_bytes) { st |= VPO_ST_PACK_MISMATCH; continue; }
+        int src = -1;
+        for (int i = 0; i < N; i++) if (lane_dst[(size_t)k * N + i] == rank) src = i;
+        for (int64_t r = lo / row_bytes; r < hi / row_bytes; r++) src_of[r] = src;
+    }
+    int64_t o = 0;
+    for (int e = 0; e < experts_per_rank; e++) {
+        expert_off[e] = (int32_t)o;
+        for (int i = 0; i < N; i++)
+            for (int64_t r = 0; r < R; r++) {
+                if (src_of[r] != i || recv_expert[r] != e) continue;
+                memcpy((char *)out + (size_t)o * row_bytes, (const char *)recv + (size_t)r * row_bytes, (size_t)row_bytes);
+                if (out_src) out_src[o] = i;
+                if (out_map) out_map[o] = (int32_t)r;
+                o++;
+            }
+    }
+    expert_off[experts_per_rank] = (int32_t)o;
+    if (o != R) st |= VPO_ST_PACK_MISMATCH;      /* a row with an expert id out of range or without a source */
+    free(src_of);
+    return st;
+}

@@ -55,6 +55,8 @@ def _load():
                                              C.c_int, C.c_int, C.c_int, C.c_int64, C.c_int] + [C.c_void_p] * 9)
         _lib.vpo_demand_from_routing.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
                                                  C.c_int64, C.c_void_p]
+        _lib.vpo_unpack.argtypes = ([C.c_void_p] * 3 + [C.c_int] * 3 + [C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_int]
+                                    + [C.c_void_p] * 4)
         _lib.vpo_pack.argtypes = ([C.c_void_p] * 4 + [C.c_int] * 3 + [C.c_void_p, C.c_int, C.c_int, C.c_int,
                                   C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p])
     return _lib
@@ -274,3 +276,23 @@ class OracleCatalog:
                               _p(idx), T, topk, int(experts_per_rank), _p(rows_b), row_bytes, _p(staged),
                               capacity_rows * row_bytes, _p(src_map))
         return staged, src_map, int(st)
+
+    # ---- unpack ---------------------------------------------------------
+    def unpack(self, plan: dict, rank: int, recv, recv_expert, experts_per_rank: int):
+        """Expert-major unpack of ``rank``'s receive buffer ``recv`` ([R, row_bytes] bytes view) for a one-matrix
+        plan.  Returns (out rows, expert_off, out_src, out_map, status)."""
+        recv_b = np.ascontiguousarray(recv).view(np.uint8)
+        R = recv_b.shape[0]
+        recv_b = recv_b.reshape(R, -1)
+        row_bytes = recv_b.shape[1]
+        exp = np.ascontiguousarray(recv_expert, dtype=np.int32)
+        out = np.zeros_like(recv_b)
+        expert_off = np.zeros(experts_per_rank + 1, np.int32)
+        out_src = np.full(R, -1, np.int32)
+        out_map = np.full(R, -1, np.int32)
+        n_steps = np.asarray([plan["n_steps"]], dtype=np.int32)
+        st = _load().vpo_unpack(_p(n_steps), _p(np.ascontiguousarray(plan["lane_dst"])),
+                                _p(np.ascontiguousarray(plan["recv_off"])), self.N, int(rank), int(plan["k_max"]),
+                                _p(recv_b), row_bytes, R, _p(exp), int(experts_per_rank), _p(out), _p(expert_off),
+                                _p(out_src), _p(out_map))
+        return out, expert_off, out_src, out_map, int(st)

@@ -20,6 +20,8 @@ from .binding import (  # noqa: F401
     pack_host,
     pack_static,
     PACK_STATIC_SCRATCH_BYTES,
+    unpack_workspace_bytes,
+    unpack,
     kernel_launch_count,
     plan_time,
     demand_from_routing,

@@ -87,6 +87,9 @@ def _load():
     lib.vp_pack_host_scratch_bytes.argtypes = [i32, i32, i32, i32, i64, i64]
     lib.vp_pack_host_scratch_bytes.restype = sz
     lib.vp_pack_host.argtypes = pack_args + [P, sz, P]
+    lib.vp_unpack_workspace_bytes.argtypes = [i32, i64, i32, i32]
+    lib.vp_unpack_workspace_bytes.restype = sz
+    lib.vp_unpack.argtypes = [P, P, P, i32, i32, i32, P, i64, i64, P, i32, P, P, P, P, P, P, sz, P]
     lib.vp_kernel_launch_count.restype = i64
     lib.vp_build_catalog.argtypes = [P, sz, P, sz, C.POINTER(sz), C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
     lib.vp_plan_time.argtypes = [vp, i32, i32, P, P, P, i64, P, P]
@@ -369,3 +372,37 @@ def pack_host(plan: Plan, b: int, rank: int, expert_idx: torch.Tensor, experts_p
     _check(_pack_call(_load().vp_pack_host, plan, b, N, rank, expert_idx, experts_per_rank, rows, row_bytes, staged,
                       src_map, status, scratch, stream), "vp_pack_host")
     return status
+
+
+def unpack_workspace_bytes(N: int, capacity_rows: int, experts_per_rank: int, k_max: int) -> int:
+    return int(_load().vp_unpack_workspace_bytes(int(N), int(capacity_rows), int(experts_per_rank), int(k_max)))
+
+
+def unpack(plan: Plan, b: int, rank: int, recv: torch.Tensor, recv_expert: torch.Tensor, experts_per_rank: int,
+           out: torch.Tensor, expert_off: Optional[torch.Tensor] = None, out_src: Optional[torch.Tensor] = None,
+           out_map: Optional[torch.Tensor] = None, status: Optional[torch.Tensor] = None,
+           workspace: Optional[torch.Tensor] = None, stream=None):
+    """``vp_unpack`` for matrix ``b`` of a device plan: ``recv`` ``[capacity_rows, H]`` is rank ``rank``'s
+    receive buffer, ``recv_expert`` the local expert of each received row, ``out`` ``[capacity_rows, H]`` the
+    expert-major output.  Returns ``(expert_off, status)`` (device int32 ``[experts_per_rank + 1]`` and ``[1]``)."""
+    N = plan.lane_dst.shape[2]
+    assert recv.is_cuda and recv.is_contiguous() and recv.dim() == 2 and out.is_cuda and out.is_contiguous()
+    assert recv_expert.is_cuda and recv_expert.dtype == torch.int32 and recv_expert.is_contiguous()
+    cap = recv.shape[0]
+    assert recv_expert.numel() >= cap and out.numel() * out.element_size() >= recv.numel() * recv.element_size()
+    row_bytes = recv.shape[1] * recv.element_size()
+    if expert_off is None:
+        expert_off = torch.empty(experts_per_rank + 1, dtype=torch.int32, device=recv.device)
+    if status is None:
+        status = torch.empty(1, dtype=torch.int32, device=recv.device)
+    if workspace is None:
+        need = unpack_workspace_bytes(N, cap, experts_per_rank, plan.k_max)
+        if need == 0:
+            raise VpError(E_UNSUPPORTED, "vp_unpack_workspace_bytes")
+        workspace = torch.empty(need, dtype=torch.uint8, device=recv.device)
+    rc = _load().vp_unpack(_ptr(plan.n_steps[b:b + 1]), _ptr(plan.lane_dst[b]), _ptr(plan.recv_off[b]), int(N), int(rank),
+                           int(plan.k_max), _ptr(recv), int(row_bytes), int(cap), _ptr(recv_expert), int(experts_per_rank),
+                           _ptr(out), _ptr(expert_off), _ptr(out_src), _ptr(out_map), _ptr(status), _ptr(workspace),
+                           workspace.numel(), _stream(stream))
+    _check(rc, "vp_unpack")
+    return expert_off, status

@@ -7,7 +7,7 @@
 #include "vp_internal.h"
 
 namespace {
-constexpr int kKinds = 3;
+constexpr int kKinds = 4;
 bool g_on = false;
 std::vector<cudaEvent_t> g_begin[kKinds], g_end[kKinds];
 }  // namespace

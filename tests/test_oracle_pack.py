@@ -101,3 +101,47 @@ def test_demand_from_routing_equals_a_library_histogram(oracle_lib):
     assert np.array_equal(rows, want)
     idx[0, 0, 0] = N * epr                                                         # a rank that does not exist
     assert oracle_lib.demand_from_routing(idx, epr, N, rb, src0=2)[1] == 1
+
+
+def test_pack_exchange_unpack_round_trip(oracle_lib):
+    """End to end on one node: every rank packs, the chunks travel as the plan says, rank j unpacks.  The result
+    must be what the routing says directly: for each local expert, the rows of all (source, token, slot) copies
+    routed to it, in (source, token, slot) order -- a definition that involves neither plan nor offsets."""
+    from tests.exchange import deliver
+    from workloads import complete_catalog, tree_topology, SchedParams
+    from workloads.demand import demand_from_routing, moe_routing
+    import torch
+    cat = complete_catalog(tree_topology(1))
+    oc = oracle_lib.OracleCatalog(cat.topology.blob(), cat.blob())
+    N, T, topk, E, hidden = 8, 60, 4, 32, 8
+    epr, rb = E // N, hidden * 2
+    idx = moe_routing(N * T, E, topk, 1.0, seed=77).reshape(N, T, topk).numpy()
+    D = demand_from_routing(torch.from_numpy(idx.reshape(N * T, topk)), torch.repeat_interleave(torch.arange(N), T), N, E, rb).numpy()
+    plan = oc.schedule(D, SchedParams(granule_bytes=rb).resolved(N))
+    assert plan["status"] == 0
+    rng = np.random.default_rng(1)
+    rows = rng.integers(0, 65536, size=(N, T, hidden), dtype=np.uint16)
+    staged, meta = {}, {}
+    for i in range(N):
+        R = int(D[i].sum() // rb)
+        s, m, st = oc.pack(plan, i, idx[i], epr, rows[i], R)
+        assert st == 0
+        staged[i], meta[i] = s, idx[i].reshape(-1)[m] % epr          # local expert id travels with each row
+    for j in (0, 5):
+        recv, recv_expert = deliver(plan, j, staged, rb, meta)
+        out, expert_off, out_src, out_map, st = oc.unpack(plan, j, recv, recv_expert, epr)
+        assert st == 0
+        want_rows, want_src, want_off = [], [], [0]
+        for e in range(epr):
+            for i in range(N):
+                if i == j:
+                    continue
+                for t in range(T):
+                    for s in range(topk):
+                        if idx[i, t, s] == j * epr + e:
+                            want_rows.append(rows[i, t]); want_src.append(i)
+            want_off.append(len(want_rows))
+        assert expert_off.tolist() == want_off
+        assert out_src.tolist() == want_src
+        assert np.array_equal(out.view(np.uint16), np.array(want_rows, dtype=np.uint16))
+        assert sorted(out_map.tolist()) == list(range(len(want_rows)))
