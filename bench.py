@@ -275,7 +275,36 @@ def run_tools(vp, dev, peaks):
     st = torch.empty(1, dtype=torch.int32, device=dev)
     ms_d = timed(lambda: vp.demand_from_routing(idx, 16, 16, 14336, out=rows, status=st))
     bytes_d = idx.numel() * 4
-    return {"plan_time": {"workload": f"config 3 plans: 1024 matrices, {steps} activations x 64 lanes", "ms": round(ms_t, 4),
+    # receive side of the packed-buffer configuration: rank 8's receive buffer (random rows, skewed local experts)
+    from workloads.configs import build_pack_case
+    pk = build_pack_case(device=dev)
+    pcat, pw, prank, epr = pk["catalog"], pk["params"], pk["rank"], pk["experts_per_rank"]
+    pdc = vp.load_catalog(pcat.topology.blob(), pcat.blob(), device=torch.device(dev).index or 0)
+    pplan = vp.schedule_batch(pdc, vp_params(vp, pw), pk["demand"].to(dev).contiguous())
+    R = int(pk["demand"][0, :, prank].sum().item() // pk["row_bytes"])
+    gen = torch.Generator(device=dev).manual_seed(9)
+    recv = torch.randint(-32768, 32768, (R, pk["row_bytes"] // 2), dtype=torch.int16, device=dev, generator=gen)
+    prob = torch.rand(epr, device=dev, generator=gen) ** 3
+    rexp = torch.multinomial(prob / prob.sum(), R, replacement=True, generator=gen).to(torch.int32)
+    uout = torch.empty_like(recv)
+    uoff = torch.empty(epr + 1, dtype=torch.int32, device=dev)
+    ust = torch.empty(1, dtype=torch.int32, device=dev)
+    usrc, umap = torch.empty(R, dtype=torch.int32, device=dev), torch.empty(R, dtype=torch.int32, device=dev)
+    uws = torch.empty(vp.unpack_workspace_bytes(16, R, epr, pw.k_max), dtype=torch.uint8, device=dev)
+    un = lambda: vp.unpack(pplan, 0, prank, recv, rexp, epr, uout, uoff, usrc, umap, ust, uws)
+    vp.profile_enable(True)
+    vp.profile_read(3)
+    ms_u = timed(un)
+    ms_copy, n_copy = vp.profile_read(3)
+    vp.profile_enable(False)
+    assert int(ust.item()) == 0 and int(uoff[-1].item()) == R
+    bytes_u = 2 * R * pk["row_bytes"]
+    return {"unpack": {"workload": f"config 5 receive side: rank {prank}, {R} rows x {pk['row_bytes']} B, {epr} local experts",
+                       "ms": round(ms_u, 4), "copy_kernel_ms": round(ms_copy / max(n_copy, 1), 4),
+                       "gb_per_s": round(bytes_u / ms_u / 1e6, 1),
+                       "copy_kernel_gb_per_s": round(bytes_u / (ms_copy / max(n_copy, 1)) / 1e6, 1),
+                       "copy_kernel_frac_of_hbm_peak": round(bytes_u / (ms_copy / max(n_copy, 1)) / 1e6 / peaks["hbm_gbs"], 4)},
+            "plan_time": {"workload": f"config 3 plans: 1024 matrices, {steps} activations x 64 lanes", "ms": round(ms_t, 4),
                           "gb_per_s": round(bytes_t / ms_t / 1e6, 1), "frac_of_hbm_peak": round(bytes_t / ms_t / 1e6 / peaks["hbm_gbs"], 4)},
             "demand_from_routing": {"workload": "16 ranks x 16384 tokens x top-8 (8.4 MB of indices, L2-resident)",
                                     "ms": round(ms_d, 4), "gb_per_s": round(bytes_d / ms_d / 1e6, 1)}}
