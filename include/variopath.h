@@ -320,6 +320,14 @@ int vp_unpack(const int32_t* n_steps_b, const int16_t* lane_dst_b, const int64_t
               int32_t* status, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * How vp_schedule_batch would launch for a batch of B matrices (for benchmarks and tests): out4 (host) receives
+ * {kernel, CTAs, threads per CTA, dynamic shared memory bytes}.  kernel 0 = one CTA per matrix; kernel 1 = one
+ * warp per matrix, chosen for topologies of at most four groups of four ranks once B exceeds the number of CTAs
+ * that fit the GPU at once.  Both kernels produce identical plans.
+ */
+int vp_schedule_launch_info(const vp_catalog* catalog, int B, const vp_sched_params* params, int32_t* out4);
+
+/*
  * Work counters of the last vp_schedule_batch that used `workspace` (device): copies three
  * uint64 to host `out3` after synchronising the stream: activations emitted, (family, start)
  * binding tasks run, AA sweeps run over all tasks.  Used to count the algorithmic operations

@@ -26,6 +26,7 @@ from .binding import (  # noqa: F401
     plan_time,
     demand_from_routing,
     schedule_read_stats,
+    schedule_launch_info,
     profile_enable,
     profile_read,
     library_path,

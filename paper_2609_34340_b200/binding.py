@@ -95,6 +95,7 @@ def _load():
     lib.vp_plan_time.argtypes = [vp, i32, i32, P, P, P, i64, P, P]
     lib.vp_demand_from_routing.argtypes = [P, i32, i32, i32, i32, i32, i32, i64, P, P, P]
     lib.vp_schedule_read_stats.argtypes = [P, P, P]
+    lib.vp_schedule_launch_info.argtypes = [vp, i32, C.POINTER(_Params), P]
     lib.vp_profile_enable.argtypes = [i32]
     lib.vp_profile_read.argtypes = [i32, C.POINTER(C.c_double), C.POINTER(i64)]
     lib.vp_strerror.argtypes = [i32]
@@ -123,6 +124,14 @@ def _stream(stream) -> C.c_void_p:
 
 def kernel_launch_count() -> int:
     return int(_load().vp_kernel_launch_count())
+
+
+def schedule_launch_info(catalog: "Catalog", B: int, params: "SchedParams") -> dict:
+    """``vp_schedule_launch_info``: which kernel and launch shape a batch of ``B`` matrices gets."""
+    out = (C.c_int32 * 4)()
+    p = params._c(catalog.N)
+    _check(_load().vp_schedule_launch_info(catalog._h, int(B), C.byref(p), out), "vp_schedule_launch_info")
+    return dict(kernel="warp per matrix" if out[0] else "CTA per matrix", ctas=int(out[1]), threads=int(out[2]), smem=int(out[3]))
 
 
 def schedule_read_stats(workspace: torch.Tensor, stream=None) -> dict:

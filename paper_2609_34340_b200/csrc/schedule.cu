@@ -770,8 +770,15 @@ vp_schedule_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand, co
 #endif
 }
 
+}  // namespace
+
+#include "schedule_warp.cuh"
+
+namespace {
+
 struct Launch {
     int threads, grid, lpg;
+    int warp_kernel;          // 1: one warp per matrix (vp_schedule_warp_kernel), 0: one CTA per matrix
     size_t smem;
     KParams kp;
 };
@@ -813,6 +820,7 @@ int plan_launch(const vp_catalog* c, int B, const vp_sched_params* p, Launch* ou
     Launch L;
     int rc = resolve_params(c, p, &L.kp);
     if (rc) return rc;
+    L.warp_kernel = 0;
     L.lpg = 1;
     if (dc.g == 4) L.lpg = dc.G <= 4 ? 8 : (dc.G <= 8 ? 4 : (dc.G <= 16 ? 2 : 1));
     L.threads = dc.N <= 64 ? 128 : 512;
@@ -832,6 +840,26 @@ int plan_launch(const vp_catalog* c, int B, const vp_sched_params* p, Launch* ou
         return VP_E_CUDA;
     long long cap = (long long)per_sm * c->sm_count;
     L.grid = (int)(B < cap ? B : cap);
+#ifndef VP_NO_WARP_KERNEL
+    // Small topologies (groups of four, at most four groups, plain D-hat scores) and more matrices than the
+    // CTAs of one wave: one warp per matrix gives up latency per matrix for three to four times as many
+    // matrices in flight, which is what counts once the batch no longer fits the GPU at once.
+    if (dc.g == 4 && dc.G <= 4 && !dc.sym && B > cap) {
+        const int warps = 4;
+        const size_t smem = (size_t)warp_smem_layout(dc, L.kp, warps).total;
+        if (smem + 2048 <= (size_t)c->max_smem_optin) {
+            if (cudaFuncSetAttribute(vp_schedule_warp_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+                return VP_E_CUDA;
+            int wper_sm = 0;
+            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&wper_sm, vp_schedule_warp_kernel, warps * 32, smem) != cudaSuccess || wper_sm < 1)
+                return VP_E_CUDA;
+            const long long wcap = (long long)wper_sm * c->sm_count, want = ((long long)B + warps - 1) / warps;
+            L.warp_kernel = 1; L.lpg = 8; L.threads = warps * 32; L.smem = smem;
+            L.kp.drem_in_smem = 1; L.kp.stage_terms = L.kp.stage_fam = L.kp.stage_bucket = 1;
+            L.grid = (int)(want < wcap ? want : wcap);
+        }
+    }
+#endif
     *out = L;
     return VP_OK;
 }
@@ -875,9 +903,14 @@ extern "C" int vp_schedule_batch(const vp_catalog* c, const vp_sched_params* p, 
         if (cudaMemsetAsync(counter, 0, 256, stream) != cudaSuccess) rc = VP_E_CUDA;
         if (!rc) {
             vp_prof_mark(0, 0, stream);
-            pick_kernel(c->dc.g, L.lpg)<<<L.grid, L.threads, L.smem, stream>>>(
-                c->dc, L.kp, demand, tau_ns_in, B, n_steps, chan_id, lane_dst, lane_inst, lane_bytes, send_off, recv_off,
-                tau_ns_out, status, ws_drem, counter);
+            if (L.warp_kernel)
+                vp_schedule_warp_kernel<<<L.grid, L.threads, L.smem, stream>>>(
+                    c->dc, L.kp, demand, tau_ns_in, B, n_steps, chan_id, lane_dst, lane_inst, lane_bytes, send_off, recv_off,
+                    tau_ns_out, status, counter);
+            else
+                pick_kernel(c->dc.g, L.lpg)<<<L.grid, L.threads, L.smem, stream>>>(
+                    c->dc, L.kp, demand, tau_ns_in, B, n_steps, chan_id, lane_dst, lane_inst, lane_bytes, send_off, recv_off,
+                    tau_ns_out, status, ws_drem, counter);
             g_vp_launches++;
             if (cudaGetLastError() != cudaSuccess) rc = VP_E_CUDA;
             vp_prof_mark(0, 1, stream);
@@ -885,6 +918,19 @@ extern "C" int vp_schedule_batch(const vp_catalog* c, const vp_sched_params* p, 
     }
     if (prev >= 0) cudaSetDevice(prev);
     return rc;
+}
+
+extern "C" int vp_schedule_launch_info(const vp_catalog* c, int B, const vp_sched_params* p, int32_t* out4) {
+    if (B <= 0 || !c || !p || !out4) return VP_E_BAD_ARG;
+    Launch L;
+    int prev = -1;
+    cudaGetDevice(&prev);
+    if (cudaSetDevice(c->device) != cudaSuccess) return VP_E_CUDA;
+    const int rc = plan_launch(c, B, p, &L);
+    if (prev >= 0) cudaSetDevice(prev);
+    if (rc) return rc;
+    out4[0] = L.warp_kernel; out4[1] = L.grid; out4[2] = L.threads; out4[3] = (int32_t)L.smem;
+    return VP_OK;
 }
 
 extern "C" int vp_schedule_read_stats(const void* workspace, void* cuda_stream, uint64_t* out3) {

@@ -256,3 +256,86 @@ def test_extreme_values_stay_exact(vp, oracle_lib):
     w2 = WParams(lambda_ns=0, granule_bytes=4096, k_target=48, k_max=400).resolved(16)
     got, want, *_ = _both(vp, oracle_lib, cat, D2, w2)
     _assert_same(got, want)
+
+
+def _tiled_case(vp, oracle_lib, cat, base, wparams, reps, tau=None):
+    """Schedules ``reps`` copies of the base batch in one call (so that the batch exceeds one wave of CTAs and the
+    warp-per-matrix kernel runs) and compares every copy with the oracle's plan of the base matrix."""
+    oc = oracle_lib.OracleCatalog(cat.topology.blob(), cat.blob())
+    dc = vp.load_catalog(cat.topology.blob(), cat.blob())
+    D = torch.as_tensor(base, dtype=torch.int64)
+    nb = D.shape[0]
+    big = D.repeat(reps, 1, 1).contiguous()
+    tau_t = None if tau is None else torch.as_tensor(np.tile(tau, reps), dtype=torch.int64).cuda()
+    p = _params(vp, wparams)
+    info = vp.schedule_launch_info(dc, big.shape[0], p)
+    assert info["kernel"] == "warp per matrix", info
+    got = vp.schedule_batch(dc, p, big.cuda(), tau_t).cpu()
+    want = oc.schedule_batch(D.numpy(), wparams, tau_in=None if tau is None else np.asarray(tau), threads=8)
+    for r in range(reps):
+        for key in KEYS:
+            g = got[key][r * nb:(r + 1) * nb]
+            if not np.array_equal(g, want[key]):
+                bad = np.argwhere(np.asarray(g) != np.asarray(want[key]))
+                raise AssertionError(f"copy {r}: {key} differs at {bad[:5].tolist()} ({len(bad)} entries)")
+    return got, want
+
+
+@pytest.mark.parametrize("name", ["node8", "node8_64_50", "two_nodes", "two_nodes_64_50"])
+def test_warp_kernel_random_demands(vp, oracle_lib, name):
+    """Batches beyond one wave take the one-warp-per-matrix kernel: same plans, bit for bit (32-bit granule units
+    and 64-bit byte values, uniform and mixed rates, empty matrices, several parameter sets)."""
+    cat = TOPOS[name]()
+    N = cat.topology.N
+    rng = np.random.default_rng(sum(map(ord, name)) + 1)
+    for u, hi, density, lam, extra in [(256, 3, 1.0, 8000, {}), (1, 100000, 0.5, 0, {}), (4096, 50, 0.15, 123, {"n_start": 1, "i_aa": 1}),
+                                       (64, 1, 0.05, 8000, {"n_start": 7, "i_aa": 2, "k_target": 5}),
+                                       (512, 300, 0.8, 8000, {"n_start": 2, "i_aa": 5, "k_target": 48})]:
+        D = _random_batch(rng, 100, N, u, hi, density)
+        D[5] = 0
+        w = WParams(lambda_ns=lam, granule_bytes=u, **extra).resolved(N)
+        tau = rng.integers(0, 3, size=100) * rng.integers(1, 5000, size=100) if extra else None
+        _tiled_case(vp, oracle_lib, cat, D, w, reps=26, tau=tau)
+
+
+def test_warp_kernel_status_codes_and_extremes(vp, oracle_lib):
+    cat = complete_catalog(tree_topology(1))
+    good = uniform_demand(8, 6400).numpy()
+    D = np.stack([good] * 8)
+    D[1, 2, 2] = 64
+    D[2, 1, 3] = -64
+    D[3, 1, 3] = 65
+    D[4, 1, 3] = 1 << 40
+    D[5, 0, 0] = -1; D[5, 4, 5] = 3
+    tau = np.zeros(8, np.int64); tau[6] = (1 << 40) + 1
+    got, want = _tiled_case(vp, oracle_lib, cat, D, WParams(granule_bytes=64).resolved(8), reps=330, tau=tau)
+    assert got["status"][:8].tolist() == [0, vp.ST_DIAG_NONZERO, vp.ST_NEGATIVE, vp.ST_NOT_GRANULE, vp.ST_OVERFLOW_RISK,
+                                          vp.ST_NEGATIVE | vp.ST_NOT_GRANULE, vp.ST_BAD_TAU, 0]
+    got, want = _tiled_case(vp, oracle_lib, cat, D[:1], WParams(granule_bytes=64, k_max=5).resolved(8), reps=2600)
+    assert got["status"][0] == vp.ST_STEP_LIMIT and got["n_steps"][-1] == 5
+    only_pix = Catalog(cat.topology, [cat.shapes[-1]], [cat.buckets[-1]])
+    got, want = _tiled_case(vp, oracle_lib, only_pix, D[:1], WParams(granule_bytes=64).resolved(8), reps=2600)
+    assert got["status"][-1] == vp.ST_UNCOVERED
+    # entries, lambda and tau at their limits with mixed rates: the 64-bit path and the 128-bit utility compare
+    cat2 = complete_catalog(tree_topology(2, pcie_bw=64, nic_bw=50))
+    rng = np.random.default_rng(17)
+    big = (1 << 40) - 1
+    E = np.zeros((6, 16, 16), np.int64)
+    E[0] = rng.integers(big - 1000, big + 1, size=(16, 16))
+    E[1] = rng.integers(0, 2, size=(16, 16)) * big
+    E[2] = rng.integers(0, big + 1, size=(16, 16))
+    E[3, 0, 9] = big
+    E[4] = rng.integers(0, 3, size=(16, 16))
+    E[5] = rng.integers(big // 2, big, size=(16, 16)) * (rng.random((16, 16)) < 0.2)
+    for b in range(6):
+        np.fill_diagonal(E[b], 0)
+    tau = np.array([0, 0, 1 << 40, 1, 0, 12345], np.int64)
+    w = WParams(lambda_ns=(1 << 40) - 1, granule_bytes=1, k_target=7, k_max=400).resolved(16)
+    _tiled_case(vp, oracle_lib, cat2, E, w, reps=420, tau=tau)
+    E2 = (E // 4096) * 4096
+    _tiled_case(vp, oracle_lib, cat2, E2, WParams(lambda_ns=0, granule_bytes=4096, k_target=48, k_max=400).resolved(16), reps=420)
+
+
+def test_warp_kernel_config2_tiled(vp, oracle_lib):
+    c = build_config(2)
+    _tiled_case(vp, oracle_lib, c["catalog"], c["demand"].numpy(), c["params"], reps=4)
