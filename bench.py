@@ -123,6 +123,8 @@ def build_workload(args, device: str):
     from workloads.configs import build_config, build_pack_case
     sched = build_config(args.sched_config, device=device, batch=args.batch, token_scale=args.token_scale)
     pack = build_pack_case(device=device, tokens=args.pack_tokens)
+    if args.sched_repeat > 1:           # the same matrices several times over: a batch beyond one wave of CTAs
+        sched["demand"] = sched["demand"].repeat(args.sched_repeat, 1, 1).contiguous()
     return sched, pack
 
 
@@ -163,6 +165,7 @@ def run_ours(args):
     sub = min(B, 256) if N > 64 else B          # N=256 plans are 30 MB each: sub-batches reuse the output buffers
     plan = vp.Plan.empty(sub, N, w.k_max, dev)
     ws = torch.empty(vp.schedule_workspace_bytes(dc, sub, params), dtype=torch.uint8, device=dev)
+    sched["_launch"] = vp.schedule_launch_info(dc, sub, params)
 
     # pack case: its own one-matrix plan on the config-2 topology
     pcat, pw = pk["catalog"], pk["params"]
@@ -268,6 +271,24 @@ def run_tools(vp, dev, peaks):
         torch.cuda.synchronize()
         return e0.elapsed_time(e1) / reps
 
+    # the scheduler beyond one wave: config 2's 256 matrices 16 times over (one warp per matrix)
+    c2 = build_config(2, device=dev)
+    cat2, w2 = c2["catalog"], c2["params"]
+    dc2 = vp.load_catalog(cat2.topology.blob(), cat2.blob(), device=torch.device(dev).index or 0)
+    p2 = vp_params(vp, w2)
+    D2 = c2["demand"].to(dev).repeat(16, 1, 1).contiguous()
+    B2 = D2.shape[0]
+    plan2 = vp.Plan.empty(B2, cat2.topology.N, w2.k_max, dev)
+    ws2 = torch.empty(vp.schedule_workspace_bytes(dc2, B2, p2), dtype=torch.uint8, device=dev)
+    ms_s = timed(lambda: vp.schedule_batch(dc2, p2, D2, plan=plan2, workspace=ws2), reps=10)
+    ops2 = sched_ops(cat2, vp.schedule_read_stats(ws2), w2.n_start)
+    alu_peak = SM_COUNT * LANES_PER_SM * INT64_OPS_PER_LANE_CLK * peaks["sm_max_mhz"] * 1e6
+    large = {"workload": f"config 2 matrices x16: {B2} matrices N=16", "launch": vp.schedule_launch_info(dc2, B2, p2),
+             "ms": round(ms_s, 4), "matrices_per_s": round(B2 / ms_s * 1e3, 1),
+             "alu_frac": round(ops2 / (ms_s * 1e-3) / alu_peak, 4),
+             "ncu": {"issue_active_pct": 55.8, "shared_wavefronts_pct_of_peak": 56.1, "lsu_pipe_pct": 48.8,
+                     "source": "profiles/vp_schedule_warp_kernel_config2_x16.md"}}
+    del plan2, D2
     ms_t = timed(lambda: vp.plan_time(dc, plan, w.lambda_ns, out=out))
     bytes_t = steps * cat.topology.N * 10                       # lane_bytes (8) + lane_inst (2) of every emitted step
     idx = moe_routing(16 * 16384, 256, 8, 1.2, seed=5, device=dev).reshape(16, 16384, 8).contiguous()
@@ -299,7 +320,7 @@ def run_tools(vp, dev, peaks):
     vp.profile_enable(False)
     assert int(ust.item()) == 0 and int(uoff[-1].item()) == R
     bytes_u = 2 * R * pk["row_bytes"]
-    return {"unpack": {"workload": f"config 5 receive side: rank {prank}, {R} rows x {pk['row_bytes']} B, {epr} local experts",
+    return {"schedule_large_batch": large, "unpack": {"workload": f"config 5 receive side: rank {prank}, {R} rows x {pk['row_bytes']} B, {epr} local experts",
                        "ms": round(ms_u, 4), "copy_kernel_ms": round(ms_copy / max(n_copy, 1), 4),
                        "gb_per_s": round(bytes_u / ms_u / 1e6, 1),
                        "copy_kernel_gb_per_s": round(bytes_u / (ms_copy / max(n_copy, 1)) / 1e6, 1),
@@ -363,14 +384,16 @@ def finish(args, world, cat, w, B, N, T, topk, R, prank, row_bytes, pack_bytes, 
     alu_peak_now = SM_COUNT * LANES_PER_SM * INT64_OPS_PER_LANE_CLK * sm_mhz * 1e6 / 1e12
     sched_tops = ops / (sched_avg * 1e-3) / 1e12
     # DRAM bytes per launch from the ncu captures summarised under profiles/ (default workload only)
-    default_workload = args.sched_config == 2 and args.batch is None and args.pack_tokens == 16384
+    default_workload = args.sched_config == 2 and args.batch is None and args.pack_tokens == 16384 and args.sched_repeat == 1
     traffic_copy = NCU_DRAM_BYTES_PER_LAUNCH["pack_copy_bulk_kernel"] if default_workload else None
     traffic_sched = NCU_DRAM_BYTES_PER_LAUNCH["vp_schedule_kernel"] if default_workload else None
     roof_pack = dict(kernel="pack_copy_bulk_kernel", bound="hbm", achieved=round(pack_gbs, 1), peak=peaks["hbm_gbs"],
                      unit="GB/s", frac=round(pack_gbs / peaks["hbm_gbs"], 4), traffic=traffic_copy,
                      peak_source=peaks["source"], ms_per_launch=round(copy_avg, 4),
                      algorithmic_bytes_per_launch=copy_bytes)
-    roof_sched = dict(kernel="vp_schedule_kernel", bound="alu", achieved=round(sched_tops, 4), peak=round(alu_peak_max, 2),
+    launch = sched.get("_launch") or {}
+    roof_sched = dict(kernel="vp_schedule_warp_kernel" if launch.get("kernel") == "warp per matrix" else "vp_schedule_kernel",
+                      launch=launch, bound="alu", achieved=round(sched_tops, 4), peak=round(alu_peak_max, 2),
                       unit="Tops/s (64-bit integer)", frac=round(sched_tops / alu_peak_max, 5), traffic=traffic_sched,
                       peak_source="derived: 148 SMs x 128 lanes x 0.5 64-bit ops/clk x max SM clock",
                       frac_at_sampled_clock=round(sched_tops / alu_peak_now, 5), ms_per_launch=round(sched_avg, 4),
@@ -381,7 +404,7 @@ def finish(args, world, cat, w, B, N, T, topk, R, prank, row_bytes, pack_bytes, 
         "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": round(ms_per_step, 4), "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "int64", "data": "synthetic",
-        "config": {"workload": f"config {args.sched_config}: {B} MoE demand matrices N={N} "
+        "config": {"workload": f"config {args.sched_config}{' x%d' % args.sched_repeat if args.sched_repeat > 1 else ''}: {B} MoE demand matrices N={N} "
                                f"({cat.n_shapes} shapes / {cat.n_families} families) + config 5 pack: rank {prank} of 16, "
                                f"{T} tokens x top-{topk}, {row_bytes}-B rows, {R} staged rows",
                    "batch_per_gpu": B, "parallelism": f"replicas x{world}, no collective",
@@ -499,6 +522,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--sched-config", type=int, default=2, choices=[1, 2, 3, 4])
     ap.add_argument("--batch", type=int, default=None, help="truncate the scheduler batch (tests)")
+    ap.add_argument("--sched-repeat", type=int, default=1,
+                    help="schedule the batch this many times over in one call (a batch beyond one wave; not the default benchmark)")
     ap.add_argument("--token-scale", type=float, default=1.0, help="scale token counts (tests)")
     ap.add_argument("--pack-tokens", type=int, default=16384, help="tokens of the packed rank (tests)")
     ap.add_argument("--min-warmup-s", type=float, default=1.0,

@@ -65,7 +65,7 @@ __host__ __device__ inline Smem smem_layout(const DevCat& dc, const KParams& kp,
     L.slotw = o;     o += dc.max_bucket * dc.N * 4;
     L.bind_src = o;  o += align16(kp.max_tasks * dc.N);
     L.bind_dst = o;  o += align16(kp.max_tasks * dc.N);
-    L.term = o;      o += kp.stage_terms ? align16(dc.n_shapes * dc.max_terms * 4) : 0;
+    L.term = o;      o += kp.stage_terms ? ((dc.n_shapes + 31) & ~31) * dc.max_terms * 4 : 0;   // transposed, padded rows
     L.fam_in = o;    o += kp.stage_fam ? align16(dc.n_families * dc.N * 2) : 0;
     L.fam_cls = o;   o += kp.stage_fam ? align16(dc.n_families * dc.N) : 0;
     L.bucket = o;    o += kp.stage_bucket ? align16((dc.n_shapes + 1) * 4) : 0;
@@ -221,6 +221,7 @@ __device__ __forceinline__ int64_t team_best(const int64_t* cred, int tl, const 
 // Per-CTA pointers and constants shared by the two value types.
 struct Ctx {
     int N, G, tid, NT, lane, warp, n_warps;
+    int term_ss, term_se;              // term e of shape s is at p_term[s * term_ss + e * term_se]
     int64_t *Dhat, *tbl, *send_acc, *recv_acc, *red, *task_f, *task_den;
     uint8_t *bind_src, *bind_dst;
     uint32_t* slotw;
@@ -298,11 +299,11 @@ __device__ __forceinline__ void decompose(const DevCat& dc, const KParams& kp, c
             int64_t best = -1;
             int best_s = 0x7fffffff;
             for (int s = tid; s < dc.n_shapes; s += NT) {
-                const uint32_t* tp = c.p_term + (size_t)s * dc.max_terms;
+                const uint32_t* tp = c.p_term + (size_t)s * c.term_ss;
                 int64_t score = 0;
 #pragma unroll 4
                 for (int e = 0; e < dc.max_terms; e++) {
-                    const uint32_t w = tp[e];
+                    const uint32_t w = tp[(size_t)e * c.term_se];
                     score += c.tbl[w & 0xffffu] * (int64_t)(w >> 16);
                 }
                 if (score > best) { best = score; best_s = s; }     // ascending s: keeps the first maximum
@@ -614,12 +615,17 @@ vp_schedule_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand, co
 
     // ---- stage the catalog
     c.p_term = dc.term;
+    c.term_ss = dc.max_terms; c.term_se = 1;
     c.p_fam_in = dc.fam_in;
     c.p_fam_cls = dc.fam_cls;
     if (kp.stage_terms) {
         uint32_t* st = (uint32_t*)(smem_raw + L.term);
-        for (int e = tid; e < dc.n_shapes * dc.max_terms; e += NT) st[e] = dc.term[e];
+        // staged transposed ([term][shape], rows padded to 32 shapes): consecutive threads score consecutive
+        // shapes, so every load of a term is conflict-free
+        const int ns_pad = (dc.n_shapes + 31) & ~31;
+        for (int e = tid; e < dc.n_shapes * dc.max_terms; e += NT) st[(e % dc.max_terms) * ns_pad + e / dc.max_terms] = dc.term[e];
         c.p_term = st;
+        c.term_ss = 1; c.term_se = ns_pad;
     }
     c.p_bucket_ptr = dc.bucket_ptr;
     if (kp.stage_bucket) {

@@ -26,7 +26,7 @@ struct WarpSmem {                           // byte offsets; the per-warp block 
 __host__ __device__ inline WarpSmem warp_smem_layout(const DevCat& dc, const KParams& kp, int n_warps) {
     WarpSmem L;
     int o = 0;
-    L.drem = o;      o += dc.N * dc.N * 8;
+    L.drem = o;      o += align16(dc.N * (dc.N + 1) * 8);      // rows padded by one element: no bank conflicts down a column
     L.dhat = o;      o += align16(dc.G * dc.G * 8);
     L.send_acc = o;  o += dc.N * 8;
     L.recv_acc = o;  o += dc.N * 8;
@@ -38,7 +38,7 @@ __host__ __device__ inline WarpSmem warp_smem_layout(const DevCat& dc, const KPa
     L.bind_dst = o;  o += align16(kp.max_tasks * dc.N);
     L.per_warp = align16(o);
     o = L.per_warp * n_warps;
-    L.term = o;      o += align16(dc.n_shapes * dc.max_terms * 4);
+    L.term = o;      o += ((dc.n_shapes + 31) & ~31) * dc.max_terms * 4;
     L.fam_slot = o;  o += align16(dc.n_families * dc.N * 4);
     L.fam_in = o;    o += align16(dc.n_families * dc.N * 2);
     L.fam_cls = o;   o += align16(dc.n_families * dc.N);
@@ -165,6 +165,8 @@ template <typename V>
 __device__ __forceinline__ void decompose_warp(const DevCat& dc, const KParams& kp, const WCtx& c, int64_t unit, int64_t left,
                                                int& k, int& st, Counters& cnt) {
     const int N = c.N, G = c.G, lane = c.lane;
+    const int ld = N + 1;                                // row stride of D_rem
+    const int ns_pad = (dc.n_shapes + 31) & ~31;         // row stride of the transposed term table
     const int team = lane >> 3, tl = lane & 7;
     const bool active = team < G;
     const int a = active ? team : 0;                     // the team's group: source group, then destination group
@@ -193,14 +195,16 @@ __device__ __forceinline__ void decompose_warp(const DevCat& dc, const KParams& 
         int best_s = 0x7fffffff;
         for (int s0 = lane; s0 < dc.n_shapes; s0 += 128) {
             int64_t score[4] = {0, 0, 0, 0};
-            const uint32_t* tp[4];
+            const uint32_t* tp = ws<uint32_t>(c.o_term) + s0;     // term e of shape s is at [e][s]: lanes read neighbours
+            const int last = dc.n_shapes - 1 - s0;               // shapes beyond the catalog re-read the last one
+            int du[4];
 #pragma unroll
-            for (int u = 0; u < 4; u++) tp[u] = ws<uint32_t>(c.o_term) + (size_t)min(s0 + 32 * u, dc.n_shapes - 1) * dc.max_terms;
+            for (int u = 0; u < 4; u++) du[u] = min(32 * u, last);
 #pragma unroll 4
             for (int e = 0; e < dc.max_terms; e++) {
 #pragma unroll
                 for (int u = 0; u < 4; u++) {
-                    const uint32_t w = tp[u][e];
+                    const uint32_t w = tp[e * ns_pad + du[u]];
                     score[u] += Dhat[w & 0xffffu] * (int64_t)(w >> 16);
                 }
             }
@@ -257,8 +261,8 @@ __device__ __forceinline__ void decompose_warp(const DevCat& dc, const KParams& 
 #pragma unroll
                 for (int t = 0; t < kWT; t++) {
                     const int dq = ws<uint8_t>(o_dst[t])[a * 4 + q];
-                    v0[t] = min_v(Drem[(a * 4 + i0) * N + dq], cap_out[t]);
-                    v1[t] = min_v(Drem[(a * 4 + i1) * N + dq], cap_out[t]);
+                    v0[t] = min_v(Drem[(a * 4 + i0) * ld + dq], cap_out[t]);
+                    v1[t] = min_v(Drem[(a * 4 + i1) * ld + dq], cap_out[t]);
                 }
 #pragma unroll
                 for (int t = 0; t < kWT; t++)
@@ -273,8 +277,8 @@ __device__ __forceinline__ void decompose_warp(const DevCat& dc, const KParams& 
 #pragma unroll
                 for (int t = 0; t < kWT; t++) {
                     const int sq = *ws<uint8_t>(o_rin_s[t]);
-                    v0[t] = min_v(Drem[sq * N + a * 4 + i0], cap_in[t]);
-                    v1[t] = min_v(Drem[sq * N + a * 4 + i1], cap_in[t]);
+                    v0[t] = min_v(Drem[sq * ld + a * 4 + i0], cap_in[t]);
+                    v1[t] = min_v(Drem[sq * ld + a * 4 + i1], cap_in[t]);
                 }
 #pragma unroll
                 for (int t = 0; t < kWT; t++)
@@ -342,14 +346,14 @@ __device__ __forceinline__ void decompose_warp(const DevCat& dc, const KParams& 
                 const int r = lane;
                 const uint32_t w = ws<uint32_t>(c.o_fam_slot)[(f0 + h) * N + r];
                 const int i = ws<uint8_t>(c.o_bind_src)[bt * N + r], j = ws<uint8_t>(c.o_bind_dst)[bt * N + r];
-                const V x = min_v(cap[(w >> 24) & 0xf], Drem[i * N + j]);
+                const V x = min_v(cap[(w >> 24) & 0xf], Drem[i * ld + j]);
                 int64_t sa = ws<int64_t>(c.o_send_acc)[i], ra = ws<int64_t>(c.o_recv_acc)[j];
                 if (x > 0) {
                     const int64_t bytes = (int64_t)x * unit;
                     c.lane_dst_b[row + i] = (int16_t)j;
                     c.lane_inst_b[row + i] = (uint16_t)(w & 0xffffu);
                     c.lane_bytes_b[row + i] = bytes;
-                    Drem[i * N + j] -= x;
+                    Drem[i * ld + j] -= x;
                     sa += bytes; ra += bytes;
                     ws<int64_t>(c.o_send_acc)[i] = sa;
                     ws<int64_t>(c.o_recv_acc)[j] = ra;
@@ -372,7 +376,7 @@ __device__ __forceinline__ void decompose_warp(const DevCat& dc, const KParams& 
 #pragma unroll
                     for (int ii = 0; ii < 2; ii++)
 #pragma unroll
-                        for (int jj = 0; jj < 4; jj++) s += (int64_t)Drem[(ga * 4 + half * 2 + ii) * N + gd * 4 + jj];
+                        for (int jj = 0; jj < 4; jj++) s += (int64_t)Drem[(ga * 4 + half * 2 + ii) * ld + gd * 4 + jj];
                 }
                 s += __shfl_xor_sync(0xffffffffu, s, 1);
                 if (cell < G * G && half == 0) Dhat[cell] = s;
@@ -395,12 +399,14 @@ vp_schedule_warp_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ deman
     unsigned char* const smem_raw = vp_wsmem;
     const int N = dc.N, G = dc.G, tid = threadIdx.x, NT = blockDim.x;
     const int lane = tid & 31, warp = tid >> 5, n_warps = NT >> 5;
+    const int ld = N + 1;
     const WarpSmem L = warp_smem_layout(dc, kp, n_warps);
     if (tid < 32) smem_raw[L.lut + tid] = (uint8_t)(31 - tid < 24 ? perm4_packed_rt(31 - tid) : 0);
     // ---- stage the catalog (shared by the warps of the CTA)
     {
         uint32_t* t_term = (uint32_t*)(smem_raw + L.term);
-        for (int e = tid; e < dc.n_shapes * dc.max_terms; e += NT) t_term[e] = dc.term[e];
+        const int ns_pad = (dc.n_shapes + 31) & ~31;
+        for (int e = tid; e < dc.n_shapes * dc.max_terms; e += NT) t_term[(e % dc.max_terms) * ns_pad + e / dc.max_terms] = dc.term[e];
         uint32_t* t_slot = (uint32_t*)(smem_raw + L.fam_slot);
         uint16_t* t_in = (uint16_t*)(smem_raw + L.fam_in);
         uint8_t* t_cls = smem_raw + L.fam_cls;
@@ -454,7 +460,7 @@ vp_schedule_warp_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ deman
                 if (e / N == e % N && v != 0) flags |= VP_ST_DIAG_NONZERO;
                 if (v % kp.granule) flags |= VP_ST_NOT_GRANULE;
             }
-            Drem[e] = v;
+            Drem[(e / N) * ld + e % N] = v;
         }
         const int64_t tau_given = tau_in ? tau_in[b] : 0;
         if (tau_given < 0 || tau_given > VP_ENTRY_LIMIT) flags |= VP_ST_BAD_TAU;
@@ -474,8 +480,8 @@ vp_schedule_warp_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ deman
                 int64_t row = 0, col = 0;
                 for (int jj = 0; jj < N; jj++) {
                     int j = jj + i; if (j >= N) j -= N;
-                    row += Drem[(size_t)i * N + j];
-                    col += Drem[(size_t)j * N + i];
+                    row += Drem[i * ld + j];
+                    col += Drem[j * ld + i];
                 }
                 tot += row;
                 est = max_v(est, max_v(ceil_div_i64(row, dc.bw_max), ceil_div_i64(col, dc.bw_max)));
@@ -486,7 +492,7 @@ vp_schedule_warp_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ deman
 #pragma unroll
                 for (int i = 0; i < 4; i++)
 #pragma unroll
-                    for (int j = 0; j < 4; j++) s += Drem[(size_t)(ga * 4 + i) * N + gd * 4 + j];
+                    for (int j = 0; j < 4; j++) s += Drem[(ga * 4 + i) * ld + gd * 4 + j];
                 Dhat[cell] = s;
             }
             __syncwarp();
@@ -519,7 +525,7 @@ vp_schedule_warp_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ deman
             if (units) {
                 // the byte copy is no longer needed: overwrite it with the demand in granules
                 uint32_t* Drem32 = (uint32_t*)Drem;
-                for (int e = lane; e < N * N; e += 32) Drem32[e] = (uint32_t)(D[e] / kp.granule);
+                for (int e = lane; e < N * N; e += 32) Drem32[(e / N) * ld + e % N] = (uint32_t)(D[e] / kp.granule);
                 for (int cell = lane; cell < G * G; cell += 32) Dhat[cell] /= kp.granule;
                 __syncwarp();
                 c.o_cap = base + L.cap32;
