@@ -320,7 +320,28 @@ def run_tools(vp, dev, peaks):
     vp.profile_enable(False)
     assert int(ust.item()) == 0 and int(uoff[-1].item()) == R
     bytes_u = 2 * R * pk["row_bytes"]
-    return {"schedule_large_batch": large, "unpack": {"workload": f"config 5 receive side: rank {prank}, {R} rows x {pk['row_bytes']} B, {epr} local experts",
+    # return direction at the source: what rank 8 sent comes back (plan of D^T) and is put into the token layout
+    bplan = vp.schedule_batch(pdc, vp_params(vp, pw), pk["demand"].to(dev).transpose(1, 2).contiguous())
+    Rb = int(pk["demand"][0, prank, :].sum().item() // pk["row_bytes"])
+    ridx = pk["expert_idx"].to(dev).contiguous()
+    Tt, tk = ridx.shape
+    rrecv = torch.randint(-32768, 32768, (Rb, pk["row_bytes"] // 2), dtype=torch.int16, device=dev, generator=gen)
+    tout = torch.empty((Tt * tk, pk["row_bytes"] // 2), dtype=torch.int16, device=dev)
+    tst = torch.empty(1, dtype=torch.int32, device=dev)
+    tws = torch.empty(int(vp.binding._load().vp_unpack_tokens_workspace_bytes(16, Tt, tk, epr, Rb, pw.k_max)), dtype=torch.uint8, device=dev)
+    vp.profile_enable(True)
+    vp.profile_read(3)
+    ms_r = timed(lambda: vp.unpack_tokens(bplan, 0, prank, ridx, epr, rrecv, tout, None, tst, tws))
+    ms_rcopy, n_rcopy = vp.profile_read(3)
+    vp.profile_enable(False)
+    assert int(tst.item()) == 0
+    bytes_r = 2 * Rb * pk["row_bytes"]
+    ret = {"workload": f"config 5 return side: rank {prank}, {Rb} rows x {pk['row_bytes']} B back into {Tt} x top-{tk} slots",
+           "ms": round(ms_r, 4), "copy_kernel_ms": round(ms_rcopy / max(n_rcopy, 1), 4), "gb_per_s": round(bytes_r / ms_r / 1e6, 1),
+           "copy_kernel_gb_per_s": round(bytes_r / (ms_rcopy / max(n_rcopy, 1)) / 1e6, 1),
+           "copy_kernel_frac_of_hbm_peak": round(bytes_r / (ms_rcopy / max(n_rcopy, 1)) / 1e6 / peaks["hbm_gbs"], 4)}
+    del rrecv, tout
+    return {"schedule_large_batch": large, "unpack_tokens": ret, "unpack": {"workload": f"config 5 receive side: rank {prank}, {R} rows x {pk['row_bytes']} B, {epr} local experts",
                        "ms": round(ms_u, 4), "copy_kernel_ms": round(ms_copy / max(n_copy, 1), 4),
                        "gb_per_s": round(bytes_u / ms_u / 1e6, 1),
                        "copy_kernel_gb_per_s": round(bytes_u / (ms_copy / max(n_copy, 1)) / 1e6, 1),

@@ -319,6 +319,40 @@ int vp_unpack(const int32_t* n_steps_b, const int16_t* lane_dst_b, const int64_t
               void* out, int32_t* expert_off, int32_t* out_src, int32_t* out_map,
               int32_t* status, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* Bytes of device scratch vp_unpack_tokens needs (multiple of 256); 0 if the sizes are not supported. */
+size_t vp_unpack_tokens_workspace_bytes(int N, int T, int topk, int experts_per_rank, int64_t capacity_rows, int k_max);
+
+/*
+ * vp_unpack_tokens - receive side of the RETURN AlltoAllv (Section 1: expert parallelism "dispatches
+ * activations to experts and returns their outputs"; Section 5: "the receive kernel unpacks them directly
+ * into the output layout").
+ *
+ * The return call carries the transposed demand and has a plan of its own (vp_schedule_batch on D^T); the
+ * plan arguments below are that plan's.  On the sending side each expert rank j stages its expert-major
+ * rows (the output order of vp_unpack) with vp_pack, using topk = 1, experts_per_rank = 1 and the row's
+ * source rank as its "expert index": the stream for destination i is then ordered by expert id, then by
+ * i's own (token, slot).  Here rank i maps that stream back: in step k the one sender j with
+ * lane_dst[k][j] == rank delivers the next lane_bytes[k][j] / row_bytes rows of its stream at byte offset
+ * recv_off[k][rank]; the n-th row of j's stream belongs to the n-th of this rank's copies routed to j in
+ * (expert id, token, slot) order, and is written to out row token*topk + slot.
+ *
+ * expert_idx  [T][topk] int32 device: this rank's routing (the one vp_pack dispatched with).
+ * recv        [capacity_rows][row_bytes] device: the return receive buffer.
+ * out         [T*topk][row_bytes] device: rows of copies that do not travel (dropped, or routed to this
+ *             rank itself) keep their content.
+ * out_map     [T*topk] int32 device or NULL: receive-buffer row of each copy, -1 if it does not travel.
+ * status      device int32[1]: VP_ST_PACK_CAPACITY if recv_off[n_steps][rank] exceeds the buffer (nothing is
+ *             unpacked); VP_ST_PACK_MISMATCH if a sender's rows differ in number from the copies routed to it
+ *             or an offset is not a multiple of row_bytes.
+ * Limits: N * experts_per_rank <= 1024, T*topk and capacity_rows < 2^31, else VP_E_UNSUPPORTED.
+ */
+int vp_unpack_tokens(const int32_t* n_steps_b, const int16_t* lane_dst_b, const int64_t* lane_bytes_b,
+                     const int64_t* recv_off_b, int N, int rank, int k_max,
+                     const int32_t* expert_idx, int T, int topk, int experts_per_rank,
+                     const void* recv, int64_t row_bytes, int64_t capacity_rows,
+                     void* out, int32_t* out_map,
+                     int32_t* status, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /*
  * How vp_schedule_batch would launch for a batch of B matrices (for benchmarks and tests): out4 (host) receives
  * {kernel, CTAs, threads per CTA, dynamic shared memory bytes}.  kernel 0 = one CTA per matrix; kernel 1 = one

@@ -786,3 +786,52 @@ int vpo_unpack(const int32_t *n_steps, const int16_t *lane_dst, const int64_t *r
     free(src_of);
     return st;
 }
+
+/* ------------------------------------------------------------ return direction */
+
+/*
+ * Receive side of the RETURN AlltoAllv (Section 1: expert parallelism "dispatches activations to experts and
+ * returns their outputs"; Section 5: "the receive kernel unpacks them directly into the output layout").
+ * The return call carries demand D^T and has a plan of its own (n_steps, lane_dst, lane_bytes, recv_off below
+ * are that plan's).  Rank `rank` routed copies (t, slot) to experts expert_idx[t][slot]; the rank j that hosts
+ * an expert sends the outputs back in its expert-major order, i.e. for source `rank`: by expert id, then by
+ * (t, slot).  In step k of the return plan the one sender j with lane_dst[k][j] == rank delivers the next
+ * lane_bytes[k][j] / row_bytes rows of that stream at byte offset recv_off[k][rank] of the receive buffer.
+ * The output layout is the token layout: out row t*topk+slot receives the output of copy (t, slot); rows of
+ * local or dropped copies are left alone.  out_map (optional, [T*topk]) receives the receive-buffer row of each
+ * copy, -1 for copies that do not travel.  Returns status bits.
+ */
+int vpo_unpack_tokens(const int32_t *n_steps, const int16_t *lane_dst, const int64_t *lane_bytes, const int64_t *recv_off,
+                      int N, int rank, int k_max, const int32_t *expert_idx, int T, int topk, int experts_per_rank,
+                      const void *recv, int64_t row_bytes, int64_t capacity_rows, void *out, int32_t *out_map)
+{
+    (void)k_max;
+    int K = *n_steps, st = 0;
+    int64_t copies = (int64_t)T * topk;
+    if (out_map) for (int64_t c = 0; c < copies; c++) out_map[c] = -1;
+    if (recv_off[(size_t)K * N + rank] > capacity_rows * row_bytes) return VPO_ST_PACK_CAPACITY;
+    int64_t *order = (int64_t *)malloc(sizeof(int64_t) * (size_t)(copies + 1));
+    for (int j = 0; j < N; j++) {
+        if (j == rank) continue;
+        /* stream of sender j: this rank's copies to j by (expert id, t, slot) */
+        int64_t n = 0;
+        for (int e = j * experts_per_rank; e < (j + 1) * experts_per_rank; e++)
+            for (int64_t c = 0; c < copies; c++)
+                if (expert_idx[c] == e) order[n++] = c;
+        int64_t pos = 0;
+        for (int k = 0; k < K; k++) {
+            if (lane_dst[(size_t)k * N + j] != rank) continue;
+            int64_t bytes = lane_bytes[(size_t)k * N + j], at = recv_off[(size_t)k * N + rank];
+            if (bytes % row_bytes || at % row_bytes) { st |= VPO_ST_PACK_MISMATCH; continue; }
+            for (int64_t r = 0; r < bytes / row_bytes; r++, pos++) {
+                if (pos >= n) { st |= VPO_ST_PACK_MISMATCH; continue; }
+                int64_t row = at / row_bytes + r;
+                memcpy((char *)out + (size_t)order[pos] * row_bytes, (const char *)recv + (size_t)row * row_bytes, (size_t)row_bytes);
+                if (out_map) out_map[order[pos]] = (int32_t)row;
+            }
+        }
+        if (pos != n) st |= VPO_ST_PACK_MISMATCH;
+    }
+    free(order);
+    return st;
+}

@@ -57,6 +57,8 @@ def _load():
                                                  C.c_int64, C.c_void_p]
         _lib.vpo_unpack.argtypes = ([C.c_void_p] * 3 + [C.c_int] * 3 + [C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_int]
                                     + [C.c_void_p] * 4)
+        _lib.vpo_unpack_tokens.argtypes = ([C.c_void_p] * 4 + [C.c_int] * 3 + [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p,
+                                            C.c_int64, C.c_int64, C.c_void_p, C.c_void_p])
         _lib.vpo_pack.argtypes = ([C.c_void_p] * 4 + [C.c_int] * 3 + [C.c_void_p, C.c_int, C.c_int, C.c_int,
                                   C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p])
     return _lib
@@ -278,6 +280,26 @@ class OracleCatalog:
         return staged, src_map, int(st)
 
     # ---- unpack ---------------------------------------------------------
+    def unpack_tokens(self, plan: dict, rank: int, expert_idx, experts_per_rank: int, recv, out=None):
+        """Receive side of the return direction: ``plan`` is the one-matrix plan of the return call, ``expert_idx``
+        ``[T, topk]`` this rank's routing, ``recv`` its return receive buffer ([R, row_bytes] bytes view).  Returns
+        (out rows [T*topk, row_bytes], out_map, status); rows of copies that do not travel keep ``out``'s content."""
+        recv_b = np.ascontiguousarray(recv).view(np.uint8)
+        R = recv_b.shape[0]
+        recv_b = recv_b.reshape(R, -1)
+        row_bytes = recv_b.shape[1]
+        idx = np.ascontiguousarray(expert_idx, dtype=np.int32)
+        T, topk = idx.shape
+        if out is None:
+            out = np.zeros((T * topk, row_bytes), np.uint8)
+        out_map = np.full(T * topk, -1, np.int32)
+        n_steps = np.asarray([plan["n_steps"]], dtype=np.int32)
+        st = _load().vpo_unpack_tokens(_p(n_steps), _p(np.ascontiguousarray(plan["lane_dst"])),
+                                       _p(np.ascontiguousarray(plan["lane_bytes"])), _p(np.ascontiguousarray(plan["recv_off"])),
+                                       self.N, int(rank), int(plan["k_max"]), _p(idx), T, topk, int(experts_per_rank),
+                                       _p(recv_b), row_bytes, R, _p(out), _p(out_map))
+        return out, out_map, int(st)
+
     def unpack(self, plan: dict, rank: int, recv, recv_expert, experts_per_rank: int):
         """Expert-major unpack of ``rank``'s receive buffer ``recv`` ([R, row_bytes] bytes view) for a one-matrix
         plan.  Returns (out rows, expert_off, out_src, out_map, status)."""

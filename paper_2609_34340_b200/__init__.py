@@ -22,6 +22,7 @@ from .binding import (  # noqa: F401
     PACK_STATIC_SCRATCH_BYTES,
     unpack_workspace_bytes,
     unpack,
+    unpack_tokens,
     kernel_launch_count,
     plan_time,
     demand_from_routing,

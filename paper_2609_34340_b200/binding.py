@@ -90,6 +90,9 @@ def _load():
     lib.vp_unpack_workspace_bytes.argtypes = [i32, i64, i32, i32]
     lib.vp_unpack_workspace_bytes.restype = sz
     lib.vp_unpack.argtypes = [P, P, P, i32, i32, i32, P, i64, i64, P, i32, P, P, P, P, P, P, sz, P]
+    lib.vp_unpack_tokens_workspace_bytes.argtypes = [i32, i32, i32, i32, i64, i32]
+    lib.vp_unpack_tokens_workspace_bytes.restype = sz
+    lib.vp_unpack_tokens.argtypes = [P, P, P, P, i32, i32, i32, P, i32, i32, i32, P, i64, i64, P, P, P, P, sz, P]
     lib.vp_kernel_launch_count.restype = i64
     lib.vp_build_catalog.argtypes = [P, sz, P, sz, C.POINTER(sz), C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
     lib.vp_plan_time.argtypes = [vp, i32, i32, P, P, P, i64, P, P]
@@ -415,3 +418,31 @@ def unpack(plan: Plan, b: int, rank: int, recv: torch.Tensor, recv_expert: torch
                            workspace.numel(), _stream(stream))
     _check(rc, "vp_unpack")
     return expert_off, status
+
+
+def unpack_tokens(plan: Plan, b: int, rank: int, expert_idx: torch.Tensor, experts_per_rank: int, recv: torch.Tensor,
+                  out: torch.Tensor, out_map: Optional[torch.Tensor] = None, status: Optional[torch.Tensor] = None,
+                  workspace: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """``vp_unpack_tokens`` for matrix ``b`` of the RETURN call's device plan: ``recv`` ``[capacity_rows, H]`` is rank
+    ``rank``'s return receive buffer, ``expert_idx`` ``[T, topk]`` its routing, ``out`` ``[T*topk, H]`` the token
+    layout.  Returns the device status tensor (int32[1])."""
+    N = plan.lane_dst.shape[2]
+    assert expert_idx.is_cuda and expert_idx.dtype == torch.int32 and expert_idx.is_contiguous() and expert_idx.dim() == 2
+    assert recv.is_cuda and recv.is_contiguous() and recv.dim() == 2 and out.is_cuda and out.is_contiguous()
+    T, topk = expert_idx.shape
+    cap = recv.shape[0]
+    row_bytes = recv.shape[1] * recv.element_size()
+    assert out.numel() * out.element_size() >= T * topk * row_bytes
+    if status is None:
+        status = torch.empty(1, dtype=torch.int32, device=recv.device)
+    if workspace is None:
+        need = int(_load().vp_unpack_tokens_workspace_bytes(int(N), int(T), int(topk), int(experts_per_rank), int(cap), int(plan.k_max)))
+        if need == 0:
+            raise VpError(E_UNSUPPORTED, "vp_unpack_tokens_workspace_bytes")
+        workspace = torch.empty(need, dtype=torch.uint8, device=recv.device)
+    rc = _load().vp_unpack_tokens(_ptr(plan.n_steps[b:b + 1]), _ptr(plan.lane_dst[b]), _ptr(plan.lane_bytes[b]), _ptr(plan.recv_off[b]),
+                                  int(N), int(rank), int(plan.k_max), _ptr(expert_idx), int(T), int(topk), int(experts_per_rank),
+                                  _ptr(recv), int(row_bytes), int(cap), _ptr(out), _ptr(out_map), _ptr(status), _ptr(workspace),
+                                  workspace.numel(), _stream(stream))
+    _check(rc, "vp_unpack_tokens")
+    return status

@@ -180,3 +180,101 @@ def test_unpack_config5_size(vp, oracle_lib):
     got, want, cap = _run(vp, oc, plan, one, 8, recv, expert, epr)
     assert got[4] == 0 and int(got[1][-1]) == R
     _assert_unpack(got, want, cap)
+
+
+# ---- return direction ---------------------------------------------------------------------------------
+
+def _return_case(vp, oracle_lib, case, rank, seed, extra_rows=0):
+    """The return call of a packed-buffer case: plan of D^T, rank's routing, a synthetic return receive buffer."""
+    Dt = case["demand"].transpose(1, 2).contiguous()
+    oc, plan, one = _plans(vp, oracle_lib, case["catalog"], Dt, case["params"])
+    rb = case["row_bytes"]
+    R = int(Dt[0, :, rank].sum().item() // rb)             # what rank receives back = what it sent
+    rng = np.random.default_rng(seed)
+    recv = torch.from_numpy(rng.integers(0, 256, size=(R + extra_rows, rb), dtype=np.uint8)).view(torch.int16)
+    return oc, plan, one, R, recv
+
+
+def _run_tokens(vp, oc, plan, one, rank, idx, epr, recv):
+    T, topk = idx.shape
+    out = torch.full((T * topk + GUARD, recv.shape[1]), 0x1111, dtype=recv.dtype, device="cuda")
+    out_map = torch.full((T * topk + GUARD,), -7, dtype=torch.int32, device="cuda")
+    st = vp.unpack_tokens(plan, 0, rank, idx.cuda().contiguous(), epr, recv.cuda().contiguous(), out[:T * topk], out_map)
+    torch.cuda.synchronize()
+    base = np.full((T * topk, recv.shape[1]), 0x1111, dtype=np.int16).view(np.uint8)
+    w_out, w_map, w_st = oc.unpack_tokens(one, rank, idx.numpy(), epr, recv.numpy(), base)
+    got_out, got_map = out.cpu().numpy(), out_map.cpu().numpy()
+    assert int(st.item()) == w_st
+    assert np.array_equal(got_map[:T * topk], w_map)
+    assert np.array_equal(got_out[:T * topk].view(np.uint8), w_out)
+    assert (got_map[T * topk:] == -7).all() and (got_out[T * topk:] == 0x1111).all()
+    return w_st, w_map
+
+
+@pytest.mark.parametrize("tokens,hidden,rank,extra", [(300, 1024, 0, 0), (1000, 7168, 3, 5), (257, 8200, 15, 0), (500, 64, 2, 0)])
+def test_unpack_tokens_matches_oracle(vp, oracle_lib, tokens, hidden, rank, extra):
+    case = build_pack_case(device="cpu", tokens=tokens, hidden=hidden, rank=rank, seed=31)
+    oc, plan, one, R, recv = _return_case(vp, oracle_lib, case, rank, seed=rank, extra_rows=extra)
+    st, w_map = _run_tokens(vp, oc, plan, one, rank, case["expert_idx"], case["experts_per_rank"], recv)
+    assert st == 0 and int((w_map >= 0).sum()) == R
+
+
+def test_unpack_tokens_statuses(vp, oracle_lib):
+    case = build_pack_case(device="cpu", tokens=200, hidden=1024, rank=4, seed=33)
+    epr = case["experts_per_rank"]
+    oc, plan, one, R, recv = _return_case(vp, oracle_lib, case, 4, seed=2)
+    idx = case["expert_idx"].clone()
+    idx[7, 2] = -1                                           # the routing lost a copy the plan still delivers
+    st, _ = _run_tokens(vp, oc, plan, one, 4, idx, epr, recv)
+    assert st == vp.ST_PACK_MISMATCH
+    st, w_map = _run_tokens(vp, oc, plan, one, 4, case["expert_idx"], epr, recv[:R - 1])
+    assert st == vp.ST_PACK_CAPACITY and (w_map == -1).all()
+
+
+def test_dispatch_and_return_round_trip_on_gpu(vp, oracle_lib):
+    """The oracle-level round trip with every pack / unpack on the GPU: dispatch pack -> exchange -> vp_unpack ->
+    experts tag their rows -> return vp_pack (topk = 1, destination = source rank) -> exchange -> vp_unpack_tokens."""
+    from tests.exchange import deliver
+    from workloads.demand import demand_from_routing, moe_routing
+    cat = complete_catalog(tree_topology(1))
+    N, T, topk, E, hidden = 8, 300, 4, 32, 1024
+    epr, rb = E // N, hidden * 2
+    idx = moe_routing(N * T, E, topk, 0.9, seed=92).reshape(N, T, topk).to(torch.int32)
+    D = demand_from_routing(idx.reshape(N * T, topk), torch.repeat_interleave(torch.arange(N), T), N, E, rb)
+    w = WParams(granule_bytes=rb).resolved(N)
+    oc, plan, one = _plans(vp, oracle_lib, cat, D.unsqueeze(0), w)
+    _, back, back_one = _plans(vp, oracle_lib, cat, D.t().contiguous().unsqueeze(0), w)
+    rows = torch.randint(0, 32768, (N, T, hidden), dtype=torch.int16, generator=torch.Generator().manual_seed(5))
+    staged, meta = {}, {}
+    for i in range(N):
+        R = int(D[i].sum().item() // rb)
+        s = torch.zeros((R, hidden), dtype=torch.int16, device="cuda")
+        m = torch.full((R,), -1, dtype=torch.int32, device="cuda")
+        assert int(vp.pack(plan, 0, i, idx[i].cuda().contiguous(), epr, rows[i].cuda().contiguous(), s, m).item()) == 0
+        staged[i] = s.cpu().numpy().view(np.uint8).reshape(R, rb)
+        meta[i] = idx[i].reshape(-1).numpy()[m.cpu().numpy()] % epr
+    ret_staged = {}
+    for j in range(N):
+        recv, recv_expert = deliver(one, j, staged, rb, meta)
+        R = recv.shape[0]
+        out = torch.zeros((R, hidden), dtype=torch.int16, device="cuda")
+        out_src = torch.full((R,), -1, dtype=torch.int32, device="cuda")
+        off, st = vp.unpack(plan, 0, j, torch.from_numpy(recv).view(torch.int16).cuda(), torch.from_numpy(recv_expert.astype(np.int32)).cuda(),
+                            epr, out, out_src=out_src)
+        assert int(st.item()) == 0
+        off = off.cpu().tolist()
+        for e in range(epr):
+            out[off[e]:off[e + 1]] ^= (j * epr + e + 1)
+        s = torch.zeros((R, hidden), dtype=torch.int16, device="cuda")
+        assert int(vp.pack(back, 0, j, out_src.reshape(R, 1).contiguous(), 1, out, s).item()) == 0
+        ret_staged[j] = s.cpu().numpy().view(np.uint8).reshape(R, rb)
+    for i in range(N):
+        ret_recv, _ = deliver(back_one, i, ret_staged, rb)
+        out = torch.zeros((T * topk, hidden), dtype=torch.int16, device="cuda")
+        st = vp.unpack_tokens(back, 0, i, idx[i].cuda().contiguous(), epr, torch.from_numpy(ret_recv).view(torch.int16).cuda(), out)
+        assert int(st.item()) == 0
+        got = out.cpu().reshape(T, topk, hidden)
+        e = idx[i].to(torch.int16)
+        remote = (idx[i] // epr != i)
+        want = (rows[i].unsqueeze(1) ^ (e + 1).unsqueeze(2)) * remote.unsqueeze(2)
+        assert torch.equal(got, want.to(torch.int16))

@@ -145,3 +145,55 @@ def test_pack_exchange_unpack_round_trip(oracle_lib):
         assert out_src.tolist() == want_src
         assert np.array_equal(out.view(np.uint16), np.array(want_rows, dtype=np.uint16))
         assert sorted(out_map.tolist()) == list(range(len(want_rows)))
+
+
+def test_dispatch_and_return_round_trip(oracle_lib):
+    """Dispatch and return on one node, every stage by the oracle: pack -> exchange -> unpack (expert-major) -> each
+    expert tags its rows -> return pack (plan of D^T, destination = the row's source) -> exchange -> unpack into the
+    token layout.  Every remote copy (t, slot) of every rank must come back as its own token row tagged by the
+    expert it was routed to: a statement about routing only."""
+    from tests.exchange import deliver
+    from workloads import complete_catalog, tree_topology, SchedParams
+    from workloads.demand import demand_from_routing, moe_routing
+    import torch
+    cat = complete_catalog(tree_topology(1))
+    oc = oracle_lib.OracleCatalog(cat.topology.blob(), cat.blob())
+    N, T, topk, E, hidden = 8, 40, 3, 24, 8
+    epr, rb = E // N, hidden * 2
+    idx = moe_routing(N * T, E, topk, 0.8, seed=91).reshape(N, T, topk).numpy().astype(np.int32)
+    src_of = torch.repeat_interleave(torch.arange(N), T)
+    D = demand_from_routing(torch.from_numpy(idx.reshape(N * T, topk)), src_of, N, E, rb).numpy()
+    w = SchedParams(granule_bytes=rb).resolved(N)
+    plan = oc.schedule(D, w)
+    back = oc.schedule(np.ascontiguousarray(D.T), w)                       # the return call has its own plan
+    assert plan["status"] == 0 and back["status"] == 0
+    rows = np.random.default_rng(4).integers(0, 65536, size=(N, T, hidden), dtype=np.uint16)
+    staged, meta = {}, {}
+    for i in range(N):
+        s, m, st = oc.pack(plan, i, idx[i], epr, rows[i], int(D[i].sum() // rb))
+        assert st == 0
+        staged[i], meta[i] = s, idx[i].reshape(-1)[m] % epr
+    ret_staged = {}
+    for j in range(N):
+        recv, recv_expert = deliver(plan, j, staged, rb, meta)
+        out, expert_off, out_src, out_map, st = oc.unpack(plan, j, recv, recv_expert, epr)
+        assert st == 0
+        y = out.view(np.uint16).copy()
+        for e in range(epr):                                               # expert e of rank j tags what it processed
+            y[expert_off[e]:expert_off[e + 1]] ^= np.uint16(j * epr + e + 1)
+        s, m, st = oc.pack(back, j, out_src.reshape(-1, 1), 1, y, int(D[:, j].sum() // rb))
+        assert st == 0
+        ret_staged[j] = s
+    for i in range(N):
+        ret_recv, _ = deliver(back, i, ret_staged, rb)
+        out = np.zeros((T * topk, rb), np.uint8)
+        out, out_map, st = oc.unpack_tokens(back, i, idx[i], epr, ret_recv, out)
+        assert st == 0
+        got = out.view(np.uint16).reshape(T, topk, hidden)
+        for t in range(T):
+            for s in range(topk):
+                e = idx[i, t, s]
+                if e < 0 or e // epr == i:
+                    assert out_map[t * topk + s] == -1 and not got[t, s].any()
+                else:
+                    assert np.array_equal(got[t, s], rows[i, t] ^ np.uint16(e + 1)), (i, t, s)
