@@ -47,14 +47,17 @@ __device__ __forceinline__ void bulk_wait_read() {
 }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
-// One warp per CTA.  A "unit" is one piece (<= kPiece bytes) of one token's row.  Units are
-// dealt to CTAs round robin.  Unit u is loaded into stage u % S, kLook units ahead of its stores.
+// One warp per CTA.  A "unit" is one piece (<= kPiece bytes) of one source row.  Units are dealt to CTAs round
+// robin.  Unit u is loaded into stage u % S, kLook units ahead of its stores.  The destination rows of a unit
+// (lane = slot, up to 32 slots per round) are fetched one unit ahead of the load that needs them and kept in
+// registers until the unit's stores, so no global-memory latency sits between two bulk copies.
 template <int S>
 __global__ void __launch_bounds__(32)
 pack_copy_bulk_kernel(const char* __restrict__ rows, char* __restrict__ staged, const int32_t* __restrict__ dst_row,
                       const int32_t* __restrict__ flags, int T, int topk, long long row_bytes, int pieces,
                       int32_t* __restrict__ status) {
     constexpr int kLook = S / 2;
+    static_assert(kLook == 3, "the destination-row registers below form a ring of three");
     extern __shared__ __align__(128) unsigned char ring[];
     __shared__ __align__(8) unsigned long long bars[S];
     const int lane = threadIdx.x;
@@ -67,18 +70,32 @@ pack_copy_bulk_kernel(const char* __restrict__ rows, char* __restrict__ staged, 
     const long long units = (long long)T * pieces;
     const long long count = units > blockIdx.x ? (units - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
     const int rounds = (topk + 31) / 32;            // destinations are handled 32 slots at a time
+    const bool one_round = rounds == 1;
     unsigned phase = 0;                              // parity per stage (bit s)
     unsigned loaded = 0;                             // stage holds a load that was issued (bit s)
     bool failed = false;
+    // destination row of this lane's slot: for the unit whose load is issued next (fetched), and for the three
+    // units in flight (r2 newest .. r0 oldest); used when all slots fit one round
+    int fetched = -1, r0 = -1, r1 = -1, r2 = -1;
+    if (one_round && count > 0 && lane < topk) fetched = dst_row[(long long)(blockIdx.x / pieces) * topk + lane];
     for (long long it = 0; it < count + kLook && !failed; it++) {
+        int rows_m = r0;                             // unit it - kLook
+        r0 = r1; r1 = r2; r2 = -1;
         if (it < count) {                            // ---- issue the load of unit `it`
             const long long u = blockIdx.x + it * gridDim.x;
             const long long t = u / pieces;
             const int s = (int)(it % S);
             bool any = false;
-            for (int r = 0; r < rounds; r++) {
-                const int slot = r * 32 + lane;
-                any |= slot < topk && dst_row[t * topk + slot] >= 0;
+            if (one_round) {
+                r2 = fetched;
+                any = fetched >= 0;
+                fetched = -1;
+                if (it + 1 < count && lane < topk) fetched = dst_row[((u + gridDim.x) / pieces) * topk + lane];
+            } else {
+                for (int r = 0; r < rounds; r++) {
+                    const int slot = r * 32 + lane;
+                    any |= slot < topk && dst_row[t * topk + slot] >= 0;
+                }
             }
             any = __any_sync(0xffffffffu, any);
             bulk_wait_read<S - kLook - 1>();         // every lane: its stores that last read this stage are done
@@ -111,12 +128,18 @@ pack_copy_bulk_kernel(const char* __restrict__ rows, char* __restrict__ staged, 
                 if (!failed) {
                     const unsigned bytes = (unsigned)min((long long)kPiece, row_bytes - (long long)p * kPiece);
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                    for (int r = 0; r < rounds; r++) {
-                        const int slot = r * 32 + lane;
-                        const int row = slot < topk ? dst_row[t * topk + slot] : -1;
-                        if (row >= 0)
-                            bulk_store(staged + (long long)row * row_bytes + (long long)p * kPiece,
+                    if (one_round) {
+                        if (rows_m >= 0)
+                            bulk_store(staged + (long long)rows_m * row_bytes + (long long)p * kPiece,
                                        smem_u32(ring + (size_t)s * kPiece), bytes);
+                    } else {
+                        for (int r = 0; r < rounds; r++) {
+                            const int slot = r * 32 + lane;
+                            const int row = slot < topk ? dst_row[t * topk + slot] : -1;
+                            if (row >= 0)
+                                bulk_store(staged + (long long)row * row_bytes + (long long)p * kPiece,
+                                           smem_u32(ring + (size_t)s * kPiece), bytes);
+                        }
                     }
                 }
             }
