@@ -153,6 +153,82 @@ __device__ __forceinline__ bool util_greater(int64_t f1, int64_t d1, int64_t f2,
     return hi1 > hi2 || (hi1 == hi2 && lo1 > lo2);
 }
 
+// Two lanes per group, 32-bit granule units: each lane copies the team's 4 x 4 credit tile into registers once
+// (16 loads at fixed offsets instead of 48 indexed ones) and evaluates twelve permutations on pair sums
+// (c[p0][0] + c[p1][1]) + (c[p2][2] + c[p3][3]), which the compiler shares between permutations: 30 additions
+// instead of 36.  Both lanes run the same code on the permutations that start with row 0 or 1; lane 1 sees the
+// rows rotated by two, so it covers the permutations that start with row 2 or 3, and tags each value with the
+// lexicographic index of the real permutation so that the first maximum still wins.
+__host__ __device__ constexpr int perm_rank4(int a, int b, int c2, int d) {      // lexicographic index of (a, b, c2, d)
+    int r = 0;
+    const int v[4] = {a, b, c2, d};
+    for (int i = 0; i < 4; i++) {
+        int smaller = 0;
+        for (int j = i + 1; j < 4; j++) smaller += v[j] < v[i];
+        int f = 1;
+        for (int k = 2; k <= 3 - i; k++) f *= k;
+        r += smaller * f;
+    }
+    return r;
+}
+template <int P> struct RotRank {         // index of the permutation P with every row rotated by two
+    static constexpr int value = perm_rank4((perm_entry(4, P, 0) + 2) & 3, (perm_entry(4, P, 1) + 2) & 3,
+                                            (perm_entry(4, P, 2) + 2) & 3, (perm_entry(4, P, 3) + 2) & 3);
+};
+template <int... P>
+__device__ __forceinline__ uint32_t reg2_best_impl(const uint32_t (&c)[4][4], int tl, std::integer_sequence<int, P...>) {
+    uint32_t key = 0;
+    ((key = max_v(key, (((c[PermAt<4, P, 0>::value][0] + c[PermAt<4, P, 1>::value][1]) +
+                         (c[PermAt<4, P, 2>::value][2] + c[PermAt<4, P, 3>::value][3])) << 5) +
+                           (uint32_t)(tl ? 31 - RotRank<P>::value : 31 - P))),
+     ...);
+    return key;
+}
+__device__ __forceinline__ uint32_t team_best_reg2(const uint32_t* cred, int tl, const uint8_t* lut, unsigned& bpk) {
+    uint32_t c[4][4];
+#pragma unroll
+    for (int r = 0; r < 4; r++) {
+        const uint32_t* row = cred + ((r + 2 * tl) & 3) * 4;
+#pragma unroll
+        for (int q = 0; q < 4; q++) c[r][q] = row[q];
+    }
+    uint32_t key = reg2_best_impl(c, tl, std::make_integer_sequence<int, 12>{});
+    key = max_v(key, __shfl_xor_sync(0xffffffffu, key, 1));
+    bpk = lut[key & 31u];
+    return key >> 5;
+}
+
+// Eight lanes per group, 32-bit granule units.  Team lane tl evaluates the three permutations 3 tl .. 3 tl + 2.
+// Seen through a relabelling of the rows that depends on the lane only -- row 0 -> tl / 2, the other three
+// ascending for even lanes and descending for odd lanes -- these are always the permutations (0,1,2,3), (0,1,3,2)
+// and (0,2,1,3): every lane runs the same straight-line code on eight credits at fixed offsets from four row
+// pointers (instead of twelve indexed loads), shares the pair sums, and tags value P with the lexicographic
+// index of the real permutation, 6 (tl / 2) + P for even and 6 (tl / 2) + 5 - P for odd lanes.
+struct Reg8Lane {
+    unsigned row[4];      // offset of relabelled row r in the tile, in credits
+    uint32_t tag[3];      // 31 - real permutation index of P = 0, 1, 2
+};
+__device__ __forceinline__ Reg8Lane reg8_lane(int tl) {
+    Reg8Lane L;
+    const int a = tl >> 1, odd = tl & 1;
+    const int rest0 = a == 0 ? 1 : 0, rest1 = a <= 1 ? 2 : 1, rest2 = a == 3 ? 2 : 3;    // the other rows, ascending
+    L.row[0] = (unsigned)a * 4;
+    L.row[1] = (unsigned)(odd ? rest2 : rest0) * 4;
+    L.row[2] = (unsigned)rest1 * 4;
+    L.row[3] = (unsigned)(odd ? rest0 : rest2) * 4;
+#pragma unroll
+    for (int P = 0; P < 3; P++) L.tag[P] = (uint32_t)(31 - (6 * a + (odd ? 5 - P : P)));
+    return L;
+}
+// key = max over the lane's three permutations of (sum << 5 | tag); cred points at the team's tile
+__device__ __forceinline__ uint32_t reg8_key(const uint32_t* cred, const Reg8Lane& L) {
+    const uint32_t *r0 = cred + L.row[0], *r1 = cred + L.row[1], *r2 = cred + L.row[2], *r3 = cred + L.row[3];
+    const uint32_t c00 = r0[0], c11 = r1[1], c21 = r2[1], c12 = r1[2], c22 = r2[2], c32 = r3[2], c23 = r2[3], c33 = r3[3];
+    const uint32_t a01 = c00 + c11;
+    const uint32_t v0 = a01 + (c22 + c33), v1 = a01 + (c32 + c23), v2 = (c00 + c21) + (c12 + c33);
+    return max_v(max_v((v0 << 5) + L.tag[0], (v1 << 5) + L.tag[1]), (v2 << 5) + L.tag[2]);
+}
+
 // ---- team path (groups of four ranks, LPG lanes per group) -----------------------------------------
 //
 // Team lane tl owns the credit elements (i, q) with q in qv[] and i in iv[]:
@@ -199,6 +275,14 @@ __device__ __forceinline__ uint32_t team_best(const uint32_t* cred, int tl, cons
                                               const uint8_t (&pidx)[TeamCfg<LPG>::PPL][4], const uint8_t* lut,
                                               unsigned& bpk) {
     constexpr int PPL = TeamCfg<LPG>::PPL;
+    if constexpr (LPG == 2) return team_best_reg2(cred, tl, lut, bpk);
+    if constexpr (LPG == 8) {
+        uint32_t key = reg8_key(cred, reg8_lane(tl));
+#pragma unroll
+        for (int o = 4; o; o >>= 1) key = max_v(key, __shfl_xor_sync(0xffffffffu, key, o));
+        bpk = lut[key & 31u];
+        return key >> 5;
+    }
     const uint32_t tag0 = (uint32_t)(31 - tl * PPL);
     uint32_t key = 0;
 #pragma unroll

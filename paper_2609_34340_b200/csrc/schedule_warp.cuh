@@ -83,18 +83,10 @@ __device__ __forceinline__ void warp_argmax_first(int64_t& best, int& best_s) {
 // issued back to back (shuffles are not reordered by the compiler).
 __device__ __forceinline__ void team_best_x(const unsigned (&tile)[kWT], int tl, const uint8_t (&pidx)[3][4], unsigned o_lut,
                                             unsigned (&bpk)[kWT], uint32_t (&val)[kWT]) {
-    const uint32_t tag0 = (uint32_t)(31 - tl * 3);
+    const Reg8Lane L = reg8_lane(tl);
     uint32_t key[kWT];
 #pragma unroll
-    for (int t = 0; t < kWT; t++) {
-        const uint32_t* cred = ws<uint32_t>(tile[t]);
-        key[t] = 0;
-#pragma unroll
-        for (int pp = 0; pp < 3; pp++) {
-            const uint32_t v = cred[pidx[pp][0]] + cred[pidx[pp][1]] + cred[pidx[pp][2]] + cred[pidx[pp][3]];
-            key[t] = max_v(key[t], (v << 5) + (tag0 - pp));
-        }
-    }
+    for (int t = 0; t < kWT; t++) key[t] = reg8_key(ws<uint32_t>(tile[t]), L);
 #pragma unroll
     for (int o = 4; o; o >>= 1) {
         uint32_t other[kWT];
