@@ -196,7 +196,7 @@ extern "C" int vp_load_catalog(const void* topology, size_t topo_bytes, const vo
         if (!sym) P = 1;
     }
 
-    // ---- Eq. (6) terms: (table index, lane count)
+    // ---- Eq. (6) terms: (byte offset of the 64-bit table entry, lane count)
     std::vector<uint32_t> term_ptr(n_shapes + 1, 0), term;
     for (int s = 0; s < n_shapes; s++) {
         for (uint32_t e = shape_ptr[s]; e < shape_ptr[s + 1]; e++) {
@@ -204,9 +204,9 @@ extern "C" int vp_load_catalog(const void* topology, size_t topo_bytes, const vo
             if (sym) {
                 if (a / S != 0) continue;                      // node 0 represents every node
                 int delta = d / S, q = a % S, q2 = d % S;
-                term.push_back((uint32_t)((delta * S + q) * S + q2) | ((uint32_t)m << 16));
+                term.push_back((uint32_t)(((delta * S + q) * S + q2) * 8) | ((uint32_t)m << 16));
             } else {
-                term.push_back((uint32_t)(a * G + d) | ((uint32_t)m << 16));
+                term.push_back((uint32_t)((a * G + d) * 8) | ((uint32_t)m << 16));
             }
         }
         term_ptr[s + 1] = (uint32_t)term.size();
@@ -261,6 +261,7 @@ extern "C" int vp_load_catalog(const void* topology, size_t topo_bytes, const vo
     dc.max_bucket = max_bucket; dc.bw_max = bw_max; dc.W = W;
     for (size_t k = 0; k < rates.size(); k++) { dc.class_bw[k] = rates[k]; dc.class_wdiv[k] = W / rates[k]; }
     int rc = VP_OK;
+    if ((long long)dc.tbl_size * 8 > 65536) rc = VP_E_UNSUPPORTED;      // term words carry 16-bit byte offsets into the score table
     // fixed-stride copy of the terms (max_terms per shape, zero-count padding) so the scoring loop unrolls
     int max_terms = 0;
     for (int s = 0; s < n_shapes; s++) max_terms = std::max(max_terms, (int)(term_ptr[s + 1] - term_ptr[s]));

@@ -43,7 +43,7 @@ struct KParams {
 };
 
 struct Smem {                 // offsets (bytes) into dynamic shared memory
-    int drem, dhat, tbl, send_acc, recv_acc, red, task_f, task_den, bind_src, bind_dst, cred, slotw;
+    int drem, dhat, tbl, send_acc, recv_acc, red, task_f, task_den, bind_src, bind_dst, cred, slotw, pair;
     int term, fam_in, fam_cls, bucket, total;
 };
 
@@ -59,6 +59,7 @@ __host__ __device__ inline Smem smem_layout(const DevCat& dc, const KParams& kp,
     L.send_acc = o;  o += dc.N * 8;
     L.recv_acc = o;  o += dc.N * 8;
     L.red = o;       o += 64 * 8;
+    L.pair = o;      o += 16 * 6 * 8;      // per warp pair: partial F (two sweeps in flight) and slowest-lane times
     L.task_f = o;    o += kp.max_tasks * 8;
     L.task_den = o;  o += kp.max_tasks * 8;
     L.cred = o;      o += n_warps * cred_bytes_per_warp(lpg);
@@ -306,7 +307,7 @@ __device__ __forceinline__ int64_t team_best(const int64_t* cred, int tl, const 
 struct Ctx {
     int N, G, tid, NT, lane, warp, n_warps;
     int term_ss, term_se;              // term e of shape s is at p_term[s * term_ss + e * term_se]
-    int64_t *Dhat, *tbl, *send_acc, *recv_acc, *red, *task_f, *task_den;
+    int64_t *Dhat, *tbl, *send_acc, *recv_acc, *red, *task_f, *task_den, *pair;
     uint8_t *bind_src, *bind_dst;
     uint32_t* slotw;
     unsigned char* cred_warp;          // this warp's credit tiles
@@ -367,28 +368,52 @@ __device__ __forceinline__ void decompose(const DevCat& dc, const KParams& kp, c
         if (k == kp.k_max) { st |= VP_ST_STEP_LIMIT; break; }
         // (A) Eq. (6): shape scores, first maximum
         if (dc.sym) {
+            // per-node-offset sums of D-hat; four threads share an entry when the CTA has that many
             const int S = dc.S, P = dc.P;
-            for (int e = tid; e < dc.tbl_size; e += NT) {
-                int q2 = e % S, q = (e / S) % S, delta = e / (S * S);
+            const int parts = dc.tbl_size * 4 <= NT ? 4 : 1;
+            const int total = dc.tbl_size * parts;
+            for (int e0 = warp * 32; e0 < total; e0 += NT) {     // whole warps enter: the shuffles below need every lane
+                const int e4 = e0 + lane;
+                const bool live = e4 < total;
+                const int e = e4 / parts, part = e4 % parts;
+                const int q2 = e % S, q = (e / S) % S, delta = e / (S * S);
                 int64_t s = 0;
-                for (int n = 0; n < P; n++) {
-                    int n2 = n + delta; if (n2 >= P) n2 -= P;
-                    s += c.Dhat[(size_t)(n * S + q) * G + n2 * S + q2];
+                if (live)
+                    for (int n = part; n < P; n += parts) {
+                        int n2 = n + delta; if (n2 >= P) n2 -= P;
+                        s += c.Dhat[(size_t)(n * S + q) * G + n2 * S + q2];
+                    }
+                if (parts == 4) {                       // the four threads of an entry are neighbours in a warp
+                    s += __shfl_xor_sync(0xffffffffu, s, 1);
+                    s += __shfl_xor_sync(0xffffffffu, s, 2);
                 }
-                c.tbl[e] = s;
+                if (live && part == 0) c.tbl[e] = s;
             }
             __syncthreads();
         }
         if (warp < n_score_warps) {
             int64_t best = -1;
             int best_s = 0x7fffffff;
+            const char* tb = (const char*)c.tbl;
+            // a score is at most g x (what is left): when that fits 32 bits the low words of the table suffice
+            const bool narrow = left * GS < ((int64_t)1 << 31);
             for (int s = tid; s < dc.n_shapes; s += NT) {
                 const uint32_t* tp = c.p_term + (size_t)s * c.term_ss;
                 int64_t score = 0;
+                if (narrow) {
+                    uint32_t score32 = 0;
 #pragma unroll 4
-                for (int e = 0; e < dc.max_terms; e++) {
-                    const uint32_t w = tp[(size_t)e * c.term_se];
-                    score += c.tbl[w & 0xffffu] * (int64_t)(w >> 16);
+                    for (int e = 0; e < dc.max_terms; e++) {
+                        const uint32_t w = tp[(size_t)e * c.term_se];
+                        score32 += *(const uint32_t*)(tb + (w & 0xffffu)) * (w >> 16);
+                    }
+                    score = (int64_t)score32;
+                } else {
+#pragma unroll 4
+                    for (int e = 0; e < dc.max_terms; e++) {
+                        const uint32_t w = tp[(size_t)e * c.term_se];
+                        score += *(const int64_t*)(tb + (w & 0xffffu)) * (int64_t)(w >> 16);
+                    }
                 }
                 if (score > best) { best = score; best_s = s; }     // ascending s: keeps the first maximum
             }
@@ -414,7 +439,17 @@ __device__ __forceinline__ void decompose(const DevCat& dc, const KParams& kp, c
         VP_TICK(1);
 
         // (B) MultiStartAA: one warp per (family, start)
-        for (int task = warp; task < n_tasks; task += n_warps) {
+        // With more than 32 groups and one lane per group, two warps share a task (each lane one group) and
+        // meet at a named barrier of 64 threads where a single warp would use __syncwarp.
+        const int W = (GS == 4 && LPG == 1 && G > 32 && n_warps >= 8) ? 2 : 1;
+        const int sub = W == 2 ? (warp & 1) : 0, wgroup = W == 2 ? (warp >> 1) : warp;
+        auto task_sync = [&]() {
+            if constexpr (GS == 4 && LPG == 1) {
+                if (W == 2) { asm volatile("bar.sync %0, 64;" ::"r"(1 + wgroup) : "memory"); return; }
+            }
+            __syncwarp();
+        };
+        for (int task = wgroup; task < n_tasks; task += n_warps / W) {
             const int h = task / kp.n_start, f = f0 + h, t = task % kp.n_start;
             const uint16_t* fin = c.p_fam_in + (size_t)f * N;
             const uint8_t* fcls = c.p_fam_cls + (size_t)f * N;
@@ -422,12 +457,12 @@ __device__ __forceinline__ void decompose(const DevCat& dc, const KParams& kp, c
             uint8_t* dstb = c.bind_dst + (size_t)task * N;
             // the family's slot words (instance ids) are fetched now and parked in shared memory for step (D)
             uint32_t slot_pre[(VP_MAX_N + 31) / 32];
-            if (t == 0) {
+            if (t == 0 && sub == 0) {
 #pragma unroll
                 for (int rr = 0; rr < (VP_MAX_N + 31) / 32; rr++)
                     if (rr * 32 + lane < N) slot_pre[rr] = __ldg(&dc.fam_slot[(size_t)f * N + rr * 32 + lane]);
             }
-            for (int d = lane; d < G; d += 32)
+            for (int d = sub * 32 + lane; d < G; d += 32 * W)
 #pragma unroll
                 for (int q = 0; q < GS; q++) dstb[fin[d * GS + q] & 0xff] = (uint8_t)(d * GS + (q + t) % GS);
             int64_t F_old = -1, F_new = -1, tmax = 0;
@@ -520,9 +555,10 @@ __device__ __forceinline__ void decompose(const DevCat& dc, const KParams& kp, c
                 __syncwarp();
             } else {
                 // register path: one lane per rank group
-                __syncwarp();
+                task_sync();
+                int64_t* pair = c.pair + wgroup * 6;
                 for (int sweep = 0; sweep < kp.i_aa; sweep++) {
-                    for (int a = lane; a < G; a += 32) {            // source half
+                    for (int a = sub * 32 + lane; a < G; a += 32 * W) {            // source half
                         V cr[GS][GS];
                         unsigned bpk;
 #pragma unroll
@@ -537,10 +573,10 @@ __device__ __forceinline__ void decompose(const DevCat& dc, const KParams& kp, c
 #pragma unroll
                         for (int q = 0; q < GS; q++) srcb[a * GS + q] = (uint8_t)(a * GS + ((bpk >> (2 * q)) & 3));
                     }
-                    __syncwarp();
+                    task_sync();
                     int64_t part = 0;
                     tmax = 0;
-                    for (int d = lane; d < G; d += 32) {            // destination half
+                    for (int d = sub * 32 + lane; d < G; d += 32 * W) {            // destination half
                         V cr[GS][GS];
                         int rq[GS], cls[GS];
                         unsigned bpk;
@@ -565,21 +601,34 @@ __device__ __forceinline__ void decompose(const DevCat& dc, const KParams& kp, c
                             tmax = max_v(tmax, (int64_t)x * c.tscale[cls[q]]);
                         }
                     }
-                    __syncwarp();
                     F_new = warp_sum_i64(part);                      // Eq. (8)
-                    cnt.sweeps++;
+                    if (W == 2) {                                    // add the partner warp's half (slots alternate by sweep)
+                        if (lane == 0) pair[(sweep & 1) * 2 + sub] = F_new;
+                        task_sync();
+                        F_new = pair[(sweep & 1) * 2] + pair[(sweep & 1) * 2 + 1];
+                    } else {
+                        __syncwarp();
+                    }
+                    if (sub == 0) cnt.sweeps++;
                     if (F_new <= F_old) break;
                     F_old = F_new;
                 }
+                tmax = warp_max_i64(tmax);
+                if (W == 2) {
+                    if (lane == 0) pair[4 + sub] = tmax;
+                    task_sync();
+                    tmax = max_v(pair[4], pair[5]);
+                }
+                tmax_done = true;
             }
             if (!tmax_done) tmax = warp_max_i64(tmax);
-            cnt.tasks++;
-            if (t == 0) {
+            if (sub == 0) cnt.tasks++;
+            if (t == 0 && sub == 0) {
 #pragma unroll
                 for (int rr = 0; rr < (VP_MAX_N + 31) / 32; rr++)
                     if (rr * 32 + lane < N) c.slotw[h * N + rr * 32 + lane] = slot_pre[rr];
             }
-            if (lane == 0) {
+            if (lane == 0 && sub == 0) {
                 c.task_f[task] = F_new;
                 c.task_den[task] = F_new > 0 ? kp.lambda_ns * dc.W + tmax : 1;
             }
@@ -678,6 +727,7 @@ vp_schedule_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand, co
     c.send_acc = (int64_t*)(smem_raw + L.send_acc);
     c.recv_acc = (int64_t*)(smem_raw + L.recv_acc);
     c.red = (int64_t*)(smem_raw + L.red);
+    c.pair = (int64_t*)(smem_raw + L.pair);
     c.task_f = (int64_t*)(smem_raw + L.task_f);
     c.task_den = (int64_t*)(smem_raw + L.task_den);
     c.bind_src = smem_raw + L.bind_src;

@@ -197,7 +197,7 @@ __device__ __forceinline__ void decompose_warp(const DevCat& dc, const KParams& 
 #pragma unroll
                 for (int u = 0; u < 4; u++) {
                     const uint32_t w = tp[e * ns_pad + du[u]];
-                    score[u] += Dhat[w & 0xffffu] * (int64_t)(w >> 16);
+                    score[u] += *(const int64_t*)((const char*)Dhat + (w & 0xffffu)) * (int64_t)(w >> 16);
                 }
             }
 #pragma unroll

@@ -18,7 +18,7 @@ struct DevCat {
     int sym;                      // 1: shape terms index per-node-offset sums, 0: D-hat cells
     int tbl_size;                 // entries of the score table (G*G or P*S*S)
     int max_bucket;
-    // Eq. (6): shape s has terms term[s*max_terms .. s*max_terms + max_terms) = table index | count << 16
+    // Eq. (6): shape s has terms term[s*max_terms .. s*max_terms + max_terms) = 8 * table index | count << 16
     // (shapes with fewer terms are padded with zero counts)
     const uint32_t* term;
     int max_terms;
