@@ -33,7 +33,7 @@ UNIT = "matrices/s"
 INT64_OPS_PER_LANE_CLK = 0.5    # one 64-bit add/min/compare needs two 32-bit ALU issues
 SM_COUNT, LANES_PER_SM = 148, 128
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch on the default workload (ncu, see profiles/)
-NCU_DRAM_BYTES_PER_LAUNCH = {"pack_copy_bulk_kernel": 235_827_968 + 1_792_440_000, "vp_schedule_kernel": 633_856 + 512}
+NCU_DRAM_BYTES_PER_LAUNCH = {"pack_copy_bulk_kernel": 235_565_824 + 1_791_358_000, "vp_schedule_kernel": 633_344 + 0}
 
 
 def _dist_env():
