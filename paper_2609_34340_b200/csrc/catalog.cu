@@ -275,6 +275,17 @@ extern "C" int vp_load_catalog(const void* topology, size_t topo_bytes, const vo
     if (!rc) rc = upload(c, fam_cls, &dc.fam_cls);
     if (!rc) rc = upload(c, fam_in, &dc.fam_in);
     dc.n_terms = (int)term.size();      // real (unpadded) multiply-adds of one scoring pass
+    if (n_shapes < 65536) {             // inverted terms: entry -> (shape, count)
+        std::vector<uint32_t> inv_ptr(dc.tbl_size + 1, 0), inv(term.size());
+        for (uint32_t w : term) inv_ptr[(w & 0xffffu) / 8 + 1]++;
+        for (int e = 0; e < dc.tbl_size; e++) inv_ptr[e + 1] += inv_ptr[e];
+        std::vector<uint32_t> fill(inv_ptr.begin(), inv_ptr.end() - 1);
+        for (int s = 0; s < n_shapes; s++)
+            for (uint32_t e = term_ptr[s]; e < term_ptr[s + 1]; e++)
+                inv[fill[(term[e] & 0xffffu) / 8]++] = (uint32_t)s | (term[e] & 0xffff0000u);
+        if (!rc) rc = upload(c, inv_ptr, &dc.inv_ptr);
+        if (!rc) rc = upload(c, inv, &dc.inv);
+    }
     if (!rc) rc = upload(c, forced_ptr, &dc.forced_ptr);
     if (!rc) rc = upload(c, forced_cell, &dc.forced_cell);
     if (!rc) rc = upload(c, forced_bw, &dc.forced_bw);

@@ -40,11 +40,12 @@ struct KParams {
     int64_t lambda_ns, granule;
     int k_target, n_start, i_aa, k_max;
     int max_tasks, stage_terms, stage_fam, stage_bucket, drem_in_smem;
+    int incremental;          // keep the shape scores in shared memory and update them after every activation
 };
 
 struct Smem {                 // offsets (bytes) into dynamic shared memory
     int drem, dhat, tbl, send_acc, recv_acc, red, task_f, task_den, bind_src, bind_dst, cred, slotw, pair;
-    int term, fam_in, fam_cls, bucket, total;
+    int term, fam_in, fam_cls, bucket, score, inv, inv_ptr, delta, total;
 };
 
 __host__ __device__ inline int align16(int x) { return (x + 15) & ~15; }
@@ -70,6 +71,10 @@ __host__ __device__ inline Smem smem_layout(const DevCat& dc, const KParams& kp,
     L.fam_in = o;    o += kp.stage_fam ? align16(dc.n_families * dc.N * 2) : 0;
     L.fam_cls = o;   o += kp.stage_fam ? align16(dc.n_families * dc.N) : 0;
     L.bucket = o;    o += kp.stage_bucket ? align16((dc.n_shapes + 1) * 4) : 0;
+    L.score = o;     o += kp.incremental ? dc.n_shapes * 8 : 0;
+    L.inv = o;       o += kp.incremental ? align16(dc.n_terms * 4) : 0;
+    L.inv_ptr = o;   o += kp.incremental ? align16((dc.tbl_size + 1) * 4) : 0;
+    L.delta = o;     o += kp.incremental ? 32 * 8 + 32 * 4 : 0;
     L.total = o;
     return L;
 }
@@ -308,6 +313,9 @@ struct Ctx {
     int N, G, tid, NT, lane, warp, n_warps;
     int term_ss, term_se;              // term e of shape s is at p_term[s * term_ss + e * term_se]
     int64_t *Dhat, *tbl, *send_acc, *recv_acc, *red, *task_f, *task_den, *pair;
+    int64_t *score, *delta;            // incremental scoring: score of every shape; change of the chosen shape's table entries
+    int32_t* dent;                     // ... and which entries those are (-1 = none)
+    const uint32_t *p_inv, *p_inv_ptr;
     uint8_t *bind_src, *bind_dst;
     uint32_t* slotw;
     unsigned char* cred_warp;          // this warp's credit tiles
@@ -363,11 +371,11 @@ __device__ __forceinline__ void decompose(const DevCat& dc, const KParams& kp, c
     V* cred = (V*)c.cred_warp + team * 17;
     const int n_score_warps = min(n_warps, (dc.n_shapes + 31) >> 5);
 
-    for (;;) {
-        if (left == 0) break;
-        if (k == kp.k_max) { st |= VP_ST_STEP_LIMIT; break; }
-        // (A) Eq. (6): shape scores, first maximum
-        if (dc.sym) {
+    const bool inc = kp.incremental != 0;
+    // a score is at most g x (what is left) and only shrinks: when that fits 32 bits the scores are kept as 32-bit
+    // words, which shared memory can add to natively (64-bit adds are compare-and-swap loops)
+    const bool s32 = inc && left * GS < ((int64_t)1 << 31);
+    auto build_table = [&]() {
             // per-node-offset sums of D-hat; four threads share an entry when the CTA has that many
             const int S = dc.S, P = dc.P;
             const int parts = dc.tbl_size * 4 <= NT ? 4 : 1;
@@ -390,7 +398,28 @@ __device__ __forceinline__ void decompose(const DevCat& dc, const KParams& kp, c
                 if (live && part == 0) c.tbl[e] = s;
             }
             __syncthreads();
+    };
+    if (inc) {
+        // incremental scoring: all scores once, then only what an activation changes (see the end of the loop)
+        build_table();
+        const char* tb = (const char*)c.tbl;
+        for (int s = tid; s < dc.n_shapes; s += NT) {
+            const uint32_t* tp = dc.term + (size_t)s * dc.max_terms;
+            int64_t score = 0;
+            for (int e = 0; e < dc.max_terms; e++) {
+                const uint32_t w = __ldg(&tp[e]);
+                score += *(const int64_t*)(tb + (w & 0xffffu)) * (int64_t)(w >> 16);
+            }
+            if (s32) ((uint32_t*)c.score)[s] = (uint32_t)score; else c.score[s] = score;
         }
+        __syncthreads();
+    }
+
+    for (;;) {
+        if (left == 0) break;
+        if (k == kp.k_max) { st |= VP_ST_STEP_LIMIT; break; }
+        // (A) Eq. (6): shape scores, first maximum
+        if (dc.sym && !inc) build_table();
         if (warp < n_score_warps) {
             int64_t best = -1;
             int best_s = 0x7fffffff;
@@ -400,7 +429,9 @@ __device__ __forceinline__ void decompose(const DevCat& dc, const KParams& kp, c
             for (int s = tid; s < dc.n_shapes; s += NT) {
                 const uint32_t* tp = c.p_term + (size_t)s * c.term_ss;
                 int64_t score = 0;
-                if (narrow) {
+                if (inc) {
+                    score = s32 ? (int64_t)((const uint32_t*)c.score)[s] : c.score[s];
+                } else if (narrow) {
                     uint32_t score32 = 0;
 #pragma unroll 4
                     for (int e = 0; e < dc.max_terms; e++) {
@@ -436,6 +467,8 @@ __device__ __forceinline__ void decompose(const DevCat& dc, const KParams& kp, c
         if (best <= 0) { st |= VP_ST_UNCOVERED; break; }
         const int f0 = (int)c.p_bucket_ptr[best_s], H = (int)c.p_bucket_ptr[best_s + 1] - f0;
         const int n_tasks = H * kp.n_start;
+        uint32_t my_term = 0;                              // incremental scoring: this warp's term of the chosen shape
+        if (inc && warp < dc.max_terms) my_term = __ldg(&dc.term[(size_t)best_s * dc.max_terms + warp]);
         VP_TICK(1);
 
         // (B) MultiStartAA: one warp per (family, start)
@@ -699,6 +732,42 @@ __device__ __forceinline__ void decompose(const DevCat& dc, const KParams& kp, c
         }
         k++;
         __syncthreads();
+        if (inc) {
+            // The activation changed D-hat only on the cells of the chosen shape, i.e. only the table entries of its
+            // terms: one warp re-sums an entry, then every shape that uses a changed entry gets count x change.
+            const int S = dc.S, P = dc.P;
+            for (int kk = warp; kk < dc.max_terms; kk += n_warps) {
+                const uint32_t w = kk == warp ? my_term : __ldg(&dc.term[(size_t)best_s * dc.max_terms + kk]);
+                int64_t dlt = 0;
+                int e = -1;
+                if (w >> 16) {                             // the same word in every lane of the warp
+                    e = (int)(w & 0xffffu) >> 3;
+                    const int q2 = e % S, q = (e / S) % S, delta = e / (S * S);
+                    int64_t sum = 0;
+                    for (int n = lane; n < P; n += 32) {
+                        int n2 = n + delta; if (n2 >= P) n2 -= P;
+                        sum += c.Dhat[(size_t)(n * S + q) * G + n2 * S + q2];
+                    }
+                    sum = warp_sum_i64(sum);
+                    dlt = sum - c.tbl[e];
+                    __syncwarp();
+                    if (lane == 0) c.tbl[e] = sum;
+                }
+                if (lane == 0) { c.delta[kk] = dlt; c.dent[kk] = e; }
+            }
+            __syncthreads();
+            for (int kk = 0; kk < dc.max_terms; kk++) {
+                const int e = c.dent[kk];
+                const int64_t dlt = c.delta[kk];
+                if (e < 0 || dlt == 0) continue;
+                for (uint32_t idx = c.p_inv_ptr[e] + tid; idx < c.p_inv_ptr[e + 1]; idx += NT) {
+                    const uint32_t w = c.p_inv[idx];
+                    if (s32) atomicAdd((uint32_t*)c.score + (w & 0xffffu), (uint32_t)(w >> 16) * (uint32_t)dlt);
+                    else atomicAdd((unsigned long long*)&c.score[w & 0xffffu], (unsigned long long)((int64_t)(w >> 16) * dlt));
+                }
+            }
+            __syncthreads();
+        }
         VP_TICK(4);
     }
 }
@@ -728,6 +797,10 @@ vp_schedule_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand, co
     c.recv_acc = (int64_t*)(smem_raw + L.recv_acc);
     c.red = (int64_t*)(smem_raw + L.red);
     c.pair = (int64_t*)(smem_raw + L.pair);
+    c.score = (int64_t*)(smem_raw + L.score);
+    c.delta = (int64_t*)(smem_raw + L.delta);
+    c.dent = (int32_t*)(smem_raw + L.delta + 32 * 8);
+    c.p_inv = dc.inv; c.p_inv_ptr = dc.inv_ptr;
     c.task_f = (int64_t*)(smem_raw + L.task_f);
     c.task_den = (int64_t*)(smem_raw + L.task_den);
     c.bind_src = smem_raw + L.bind_src;
@@ -766,6 +839,13 @@ vp_schedule_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand, co
         uint32_t* bp = (uint32_t*)(smem_raw + L.bucket);
         for (int e = tid; e <= dc.n_shapes; e += NT) bp[e] = dc.bucket_ptr[e];
         c.p_bucket_ptr = bp;
+    }
+    if (kp.incremental) {
+        uint32_t* iv = (uint32_t*)(smem_raw + L.inv);
+        uint32_t* ip = (uint32_t*)(smem_raw + L.inv_ptr);
+        for (int e = tid; e < dc.n_terms; e += NT) iv[e] = dc.inv[e];
+        for (int e = tid; e <= dc.tbl_size; e += NT) ip[e] = dc.inv_ptr[e];
+        c.p_inv = iv; c.p_inv_ptr = ip;
     }
     if (kp.stage_fam) {
         uint16_t* fi = (uint16_t*)(smem_raw + L.fam_in);
@@ -970,6 +1050,17 @@ int plan_launch(const vp_catalog* c, int B, const vp_sched_params* p, Launch* ou
     // family tables go to shared memory only when small: beyond that, CTAs per SM matter more than their latency
     L.kp.stage_fam = (size_t)dc.n_families * dc.N * 3 <= 16 * 1024;
     L.kp.stage_bucket = ((size_t)dc.n_shapes + 1) * 4 <= 32 * 1024;
+    // many shapes over a small node-symmetric score table: keep the scores and update them (the inverted terms
+    // take the place of the staged terms in shared memory)
+    L.kp.incremental = dc.sym && dc.inv && dc.n_shapes >= 512 && dc.max_terms <= 32 && dc.max_terms <= L.threads / 32;
+    if (L.kp.incremental) {
+        const int staged = L.kp.stage_terms;
+        L.kp.stage_terms = 0;
+        if ((size_t)smem_layout(dc, L.kp, L.threads / 32, L.lpg).total + 2048 > (size_t)c->max_smem_optin) {
+            L.kp.incremental = 0;
+            L.kp.stage_terms = staged;
+        }
+    }
     L.smem = (size_t)smem_layout(dc, L.kp, L.threads / 32, L.lpg).total;
     if (L.smem + 2048 > (size_t)c->max_smem_optin) return VP_E_UNSUPPORTED;
     KernelFn fn = pick_kernel(dc.g, L.lpg);

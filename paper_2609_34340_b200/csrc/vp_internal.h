@@ -30,6 +30,10 @@ struct DevCat {
     // family f, in-slot d*g+q of destination group d: slot index (N <= 256) | rate class << 8
     const uint16_t* fam_in;
     int n_terms;
+    // inverted terms, for keeping the scores up to date instead of recomputing them: the shapes that use table
+    // entry e are inv[inv_ptr[e] .. inv_ptr[e+1]) = shape | count << 16 (built when n_shapes < 65536)
+    const uint32_t* inv_ptr;
+    const uint32_t* inv;
     // quantum rule: resource l is forced for the D-hat cells forced_cell[forced_ptr[l] .. forced_ptr[l+1])
     const uint32_t* forced_ptr;
     const uint16_t* forced_cell;
