@@ -339,3 +339,39 @@ def test_warp_kernel_status_codes_and_extremes(vp, oracle_lib):
 def test_warp_kernel_config2_tiled(vp, oracle_lib):
     c = build_config(2)
     _tiled_case(vp, oracle_lib, c["catalog"], c["demand"].numpy(), c["params"], reps=4)
+
+
+@pytest.mark.parametrize("nodes", [12, 16, 24])
+def test_mid_size_template_catalogs(vp, oracle_lib, nodes):
+    """N = 96, 128, 192 with node-template catalogs of 575 .. 2,303 shapes: incremental scores with one warp per task
+    (G <= 32) and with two warps per task (G > 32), 32-bit granule units and 64-bit byte values, mixed rates."""
+    cat = node_template_catalog(tree_topology(nodes, pcie_bw=64, nic_bw=50 if nodes == 16 else 64))
+    N = cat.topology.N
+    rng = np.random.default_rng(nodes)
+    for u, hi, density, extra in [(4096, 40, 0.3, {}), (1, 3_000_000, 0.05, {"n_start": 2, "i_aa": 2}), (256, 2, 1.0, {"k_target": 40})]:
+        D = _random_batch(rng, 5, N, u, hi, density)
+        D[3] = 0
+        w = WParams(granule_bytes=u, k_max=16 * N, **extra).resolved(N)
+        got, want, *_ = _both(vp, oracle_lib, cat, D, w)
+        _assert_same(got, want)
+
+
+def test_batches_around_one_wave(vp, oracle_lib):
+    """Batch sizes just below and above the number of resident CTAs: the kernel changes, the plans do not."""
+    c = build_config(2)
+    cat, w = c["catalog"], c["params"]
+    oc = oracle_lib.OracleCatalog(cat.topology.blob(), cat.blob())
+    dc = vp.load_catalog(cat.topology.blob(), cat.blob())
+    base = c["demand"][:37]
+    want = oc.schedule_batch(base.numpy(), w, threads=8)
+    p = _params(vp, w)
+    kernels = set()
+    for B in (591, 592, 593, 1187):
+        D = base.repeat((B + 36) // 37, 1, 1)[:B].contiguous()
+        kernels.add(vp.schedule_launch_info(dc, B, p)["kernel"])
+        got = vp.schedule_batch(dc, p, D.cuda()).cpu()
+        for key in KEYS:
+            for r0 in range(0, B, 37):
+                n = min(37, B - r0)
+                assert np.array_equal(got[key][r0:r0 + n], want[key][:n]), (B, key, r0)
+    assert kernels == {"CTA per matrix", "warp per matrix"}
