@@ -235,6 +235,38 @@ __device__ __forceinline__ uint32_t reg8_key(const uint32_t* cred, const Reg8Lan
     return max_v(max_v((v0 << 5) + L.tag[0], (v1 << 5) + L.tag[1]), (v2 << 5) + L.tag[2]);
 }
 
+// Four lanes per group, 32-bit granule units.  Team lane tl evaluates the six permutations that start with row tl.
+// With the rows rotated by tl these are the six permutations that start with row 0: every lane runs the same code on
+// ten credits at fixed offsets and six pair sums, and tags value P with the index of the real permutation.
+struct Reg4Lane {
+    unsigned row[4];      // offset of rotated row r in the tile, in credits
+    uint32_t tag[6];      // 31 - real permutation index of P = 0 .. 5
+};
+template <int... P>
+__device__ __forceinline__ void reg4_tags(Reg4Lane& L, int tl, std::integer_sequence<int, P...>) {
+    ((L.tag[P] = (uint32_t)(31 - perm_rank4(tl, (perm_entry(4, P, 1) + tl) & 3, (perm_entry(4, P, 2) + tl) & 3,
+                                            (perm_entry(4, P, 3) + tl) & 3))),
+     ...);
+}
+__device__ __forceinline__ Reg4Lane reg4_lane(int tl) {
+    Reg4Lane L;
+#pragma unroll
+    for (int r = 0; r < 4; r++) L.row[r] = (unsigned)((r + tl) & 3) * 4;
+    reg4_tags(L, tl, std::make_integer_sequence<int, 6>{});
+    return L;
+}
+__device__ __forceinline__ uint32_t reg4_key(const uint32_t* cred, const Reg4Lane& L) {
+    const uint32_t *r0 = cred + L.row[0], *r1 = cred + L.row[1], *r2 = cred + L.row[2], *r3 = cred + L.row[3];
+    const uint32_t c00 = r0[0];
+    const uint32_t a1 = c00 + r1[1], a2 = c00 + r2[1], a3 = c00 + r3[1];
+    const uint32_t c12 = r1[2], c22 = r2[2], c32 = r3[2], c13 = r1[3], c23 = r2[3], c33 = r3[3];
+    const uint32_t v0 = a1 + (c22 + c33), v1 = a1 + (c32 + c23), v2 = a2 + (c12 + c33), v3 = a2 + (c32 + c13),
+                   v4 = a3 + (c12 + c23), v5 = a3 + (c22 + c13);
+    uint32_t key = max_v((v0 << 5) + L.tag[0], (v1 << 5) + L.tag[1]);
+    key = max_v(key, max_v((v2 << 5) + L.tag[2], (v3 << 5) + L.tag[3]));
+    return max_v(key, max_v((v4 << 5) + L.tag[4], (v5 << 5) + L.tag[5]));
+}
+
 // ---- team path (groups of four ranks, LPG lanes per group) -----------------------------------------
 //
 // Team lane tl owns the credit elements (i, q) with q in qv[] and i in iv[]:
@@ -282,6 +314,13 @@ __device__ __forceinline__ uint32_t team_best(const uint32_t* cred, int tl, cons
                                               unsigned& bpk) {
     constexpr int PPL = TeamCfg<LPG>::PPL;
     if constexpr (LPG == 2) return team_best_reg2(cred, tl, lut, bpk);
+    if constexpr (LPG == 4) {
+        uint32_t key = reg4_key(cred, reg4_lane(tl));
+        key = max_v(key, __shfl_xor_sync(0xffffffffu, key, 2));
+        key = max_v(key, __shfl_xor_sync(0xffffffffu, key, 1));
+        bpk = lut[key & 31u];
+        return key >> 5;
+    }
     if constexpr (LPG == 8) {
         uint32_t key = reg8_key(cred, reg8_lane(tl));
 #pragma unroll

@@ -68,6 +68,7 @@ TOPOS = {
     "two_nodes_64_50": lambda: complete_catalog(tree_topology(2, pcie_bw=64, nic_bw=50)),
     "template_4_nodes": lambda: node_template_catalog(tree_topology(4)),
     "template_3_nodes_g3": lambda: node_template_catalog(tree_topology(3, g=3, nic_bw=50)),
+    "template_3_nodes_64_50": lambda: node_template_catalog(tree_topology(3, pcie_bw=64, nic_bw=50)),
     "crossbar4": lambda: crossbar_catalog(crossbar_topology(4)),
 }
 
