@@ -407,7 +407,10 @@ __device__ __forceinline__ void decompose(const DevCat& dc, const KParams& kp, c
             for (int q = 0; q < 4; q++) pidx[pp][q] = (uint8_t)(((pk >> (2 * q)) & 3) * 4 + q);
         }
     }
-    V* cred = (V*)c.cred_warp + team * 17;
+    // Tile placement.  Two lanes per group: lane 1 reads the tile's rows rotated by two, i.e. eight credits away from lane 0,
+    // so the sixteen tiles start in banks 0..7 and 16..23 (tile k at 33 (k mod 8) + 16 (k / 8)): every load of the warp then
+    // touches 32 different banks.  Otherwise tiles are 17 credits apart.
+    V* cred = (V*)c.cred_warp + (LPG == 2 && sizeof(V) == 4 ? 33 * (team & 7) + 16 * (team >> 3) : team * 17);
     const int n_score_warps = min(n_warps, (dc.n_shapes + 31) >> 5);
 
     const bool inc = kp.incremental != 0;
