@@ -2,11 +2,11 @@
 // (Section 5, "Device-resident buffer layout").
 //
 // Four kernels on the caller's stream:
-//   count : per 256-copy chunk, how many copies go to each destination rank
-//   plan  : exclusive scan of those counts over chunks (per destination) and the
-//           rank's segment table: for every destination, the activations that
-//           send to it, with the stream position they start at and their first
-//           staged row (from the plan's send offsets)
+//   count + plan : per 256-copy chunk, how many copies go to each destination rank; one more
+//           block builds, meanwhile, the rank's segment table: for every destination, the
+//           activations that send to it, with the stream position they start at and their
+//           first staged row (from the plan's send offsets)
+//   scan  : exclusive scan of the chunk counts over chunks, one warp per destination
 //   map   : stable position of every copy inside its destination's stream ->
 //           staged row (binary search in the segment table); writes src_map
 //   copy  : token-major: every source row is read ONCE and written to each of
@@ -65,9 +65,8 @@ __device__ __forceinline__ int dest_of(int x, int experts_per_rank, int N, int r
     return (j >= N || j == rank) ? -1 : j;
 }
 
-__global__ void __launch_bounds__(kWarpsPerBlock * 32)
-pack_count_kernel(const int32_t* __restrict__ idx, long long E, int N, int rank, int experts_per_rank,
-                  int32_t* __restrict__ hist, int32_t* __restrict__ status) {
+__device__ __forceinline__ void count_block(const int32_t* __restrict__ idx, long long E, int N, int rank, int experts_per_rank,
+                                            int32_t* __restrict__ hist, int32_t* __restrict__ status) {
     __shared__ int wh[kWarpsPerBlock][VP_MAX_N];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const long long chunk = (long long)blockIdx.x * kWarpsPerBlock + warp;
@@ -92,11 +91,10 @@ pack_count_kernel(const int32_t* __restrict__ idx, long long E, int N, int rank,
 
 // One block of VP_MAX_N threads.  Thread j owns destination j; the rank's column of the plan is staged
 // through shared memory a tile of steps at a time so that its global loads run in parallel.
-__global__ void __launch_bounds__(VP_MAX_N)
-pack_plan_kernel(const int32_t* __restrict__ n_steps_p, const int16_t* __restrict__ lane_dst,
-                 const int64_t* __restrict__ lane_bytes, const int64_t* __restrict__ send_off, int N, int rank,
-                 int k_max, int n_chunks, int64_t row_bytes, int64_t capacity_bytes, PackWs w,
-                 int32_t* __restrict__ status) {
+__device__ __forceinline__ void segments_block(const int32_t* __restrict__ n_steps_p, const int16_t* __restrict__ lane_dst,
+                                               const int64_t* __restrict__ lane_bytes, const int64_t* __restrict__ send_off, int N,
+                                               int rank, int k_max, int64_t row_bytes, int64_t capacity_bytes, PackWs w,
+                                               int32_t* __restrict__ status) {
     __shared__ int s_cnt[VP_MAX_N + 1];
     __shared__ int16_t t_dst[VP_MAX_N];
     __shared__ int32_t t_rows[VP_MAX_N], t_base[VP_MAX_N];
@@ -104,29 +102,6 @@ pack_plan_kernel(const int32_t* __restrict__ n_steps_p, const int16_t* __restric
     int K = *n_steps_p;
     if (K > k_max) K = k_max;
     if (K < 0) K = 0;
-    // exclusive scan of the chunk counts, per destination: one warp per destination, 32 chunks per step
-    {
-        const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
-        for (int d = warp; d < N; d += n_warps) {
-            int run = 0;
-            const int32_t* __restrict__ in = w.hist;
-            int32_t* __restrict__ out = w.base;
-#pragma unroll 4
-            for (int b0 = 0; b0 < n_chunks; b0 += 32) {
-                const int c = b0 + lane;
-                const int v = c < n_chunks ? in[(size_t)c * N + d] : 0;
-                int incl = v;
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const int t = __shfl_up_sync(0xffffffffu, incl, o);
-                    if (lane >= o) incl += t;
-                }
-                if (c < n_chunks) out[(size_t)c * N + d] = run + incl - v;
-                run += __shfl_sync(0xffffffffu, incl, 31);
-            }
-            if (lane == 0) w.len[d] = run;
-        }
-    }
     // pass 1: how many activations send to each destination
     int cnt = 0;
     for (int k0 = 0; k0 < K; k0 += NT) {
@@ -180,10 +155,48 @@ pack_plan_kernel(const int32_t* __restrict__ n_steps_p, const int16_t* __restric
     }
     if (j < N) {
         w.planned[j] = (int32_t)cum;
-        if (j == rank) { if (cum != 0) bad = true; }
-        else if (cum != w.len[j]) bad = true;
+        if (j == rank && cum != 0) bad = true;
     }
     if (bad) atomicOr(status, VP_ST_PACK_MISMATCH);
+}
+
+// The count blocks and, as the last block of the grid, the segment table: the two need nothing from each other.
+__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+pack_count_plan_kernel(const int32_t* __restrict__ idx, long long E, int N, int rank, int experts_per_rank,
+                       const int32_t* __restrict__ n_steps_p, const int16_t* __restrict__ lane_dst,
+                       const int64_t* __restrict__ lane_bytes, const int64_t* __restrict__ send_off, int k_max,
+                       int64_t row_bytes, int64_t capacity_bytes, PackWs w, int32_t* __restrict__ status) {
+    static_assert(kWarpsPerBlock * 32 == VP_MAX_N, "the segment block has one thread per destination");
+    if (blockIdx.x == gridDim.x - 1) segments_block(n_steps_p, lane_dst, lane_bytes, send_off, N, rank, k_max, row_bytes, capacity_bytes, w, status);
+    else count_block(idx, E, N, rank, experts_per_rank, w.hist, status);
+}
+
+// Exclusive scan of the chunk counts, per destination: one warp per destination, 32 chunks per step; then the
+// routed copies of a destination must be as many as the plan sends there.
+__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+pack_scan_kernel(int N, int rank, int n_chunks, PackWs w, int32_t* __restrict__ status) {
+    const int lane = threadIdx.x & 31, d = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+    if (d >= N) return;
+    int run = 0;
+    const int32_t* __restrict__ in = w.hist;
+    int32_t* __restrict__ out = w.base;
+#pragma unroll 4
+    for (int b0 = 0; b0 < n_chunks; b0 += 32) {
+        const int c = b0 + lane;
+        const int v = c < n_chunks ? in[(size_t)c * N + d] : 0;
+        int incl = v;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += t;
+        }
+        if (c < n_chunks) out[(size_t)c * N + d] = run + incl - v;
+        run += __shfl_sync(0xffffffffu, incl, 31);
+    }
+    if (lane == 0) {
+        w.len[d] = run;
+        if (d != rank && run != w.planned[d]) atomicOr(status, VP_ST_PACK_MISMATCH);
+    }
 }
 
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
@@ -253,9 +266,10 @@ extern "C" int vp_pack(const int32_t* n_steps_b, const int16_t* lane_dst_b, cons
     if (cudaMemsetAsync(w.flags, 0, 256, stream) != cudaSuccess) return VP_E_CUDA;
     if (cudaMemsetAsync(status, 0, sizeof(int32_t), stream) != cudaSuccess) return VP_E_CUDA;
     vp_prof_mark(1, 0, stream);
-    pack_count_kernel<<<blocks, kWarpsPerBlock * 32, 0, stream>>>(expert_idx, E, N, rank, experts_per_rank, w.hist, status);
-    pack_plan_kernel<<<1, VP_MAX_N, 0, stream>>>(n_steps_b, lane_dst_b, lane_bytes_b, send_off_b, N, rank, k_max, n_chunks,
-                                                 row_bytes, staged_capacity_bytes, w, status);
+    pack_count_plan_kernel<<<blocks + 1, kWarpsPerBlock * 32, 0, stream>>>(expert_idx, E, N, rank, experts_per_rank, n_steps_b,
+                                                                         lane_dst_b, lane_bytes_b, send_off_b, k_max, row_bytes,
+                                                                         staged_capacity_bytes, w, status);
+    pack_scan_kernel<<<(N + kWarpsPerBlock - 1) / kWarpsPerBlock, kWarpsPerBlock * 32, 0, stream>>>(N, rank, n_chunks, w, status);
     pack_map_kernel<<<blocks, kWarpsPerBlock * 32, 0, stream>>>(expert_idx, E, N, rank, experts_per_rank, w, src_map);
     g_vp_launches += 3;
     vp_prof_mark(1, 1, stream);
