@@ -42,9 +42,11 @@ int64_t gcd_i64(int64_t a, int64_t b) {
 template <typename T>
 int upload(vp_catalog* c, const std::vector<T>& v, const T** out) {
     void* d = nullptr;
-    size_t bytes = std::max<size_t>(v.size(), 1) * sizeof(T);
+    // sizes are rounded up to 16 bytes (zero filled) so that the kernels may stage whole arrays with bulk copies
+    size_t bytes = (std::max<size_t>(v.size(), 1) * sizeof(T) + 15) & ~(size_t)15;
     if (cudaMalloc(&d, bytes) != cudaSuccess) return VP_E_NOMEM;
     c->allocs.push_back(d);
+    if (cudaMemset(d, 0, bytes) != cudaSuccess) return VP_E_CUDA;
     if (!v.empty() && cudaMemcpy(d, v.data(), v.size() * sizeof(T), cudaMemcpyHostToDevice) != cudaSuccess) return VP_E_CUDA;
     *out = (const T*)d;
     return VP_OK;
@@ -270,6 +272,13 @@ extern "C" int vp_load_catalog(const void* topology, size_t topo_bytes, const vo
         for (uint32_t e = term_ptr[s]; e < term_ptr[s + 1]; e++) term_pad[(size_t)s * max_terms + (e - term_ptr[s])] = term[e];
     dc.max_terms = max_terms;
     if (!rc) rc = upload(c, term_pad, &dc.term);
+    {   // the same terms transposed ([term][shape], rows padded to 32 shapes): the layout the kernels keep in shared memory
+        const int ns_pad = (n_shapes + 31) & ~31;
+        std::vector<uint32_t> term_t((size_t)ns_pad * max_terms, 0);
+        for (int s = 0; s < n_shapes; s++)
+            for (int e = 0; e < max_terms; e++) term_t[(size_t)e * ns_pad + s] = term_pad[(size_t)s * max_terms + e];
+        if (!rc) rc = upload(c, term_t, &dc.term_t);
+    }
     if (!rc) rc = upload(c, bucket_ptr, &dc.bucket_ptr);
     if (!rc) rc = upload(c, fam_slot, &dc.fam_slot);
     if (!rc) rc = upload(c, fam_cls, &dc.fam_cls);

@@ -32,6 +32,7 @@
 
 #include <utility>
 
+#include "bulk_copy.cuh"
 #include "vp_internal.h"
 
 namespace {
@@ -67,11 +68,12 @@ __host__ __device__ inline Smem smem_layout(const DevCat& dc, const KParams& kp,
     L.slotw = o;     o += dc.max_bucket * dc.N * 4;
     L.bind_src = o;  o += align16(kp.max_tasks * dc.N);
     L.bind_dst = o;  o += align16(kp.max_tasks * dc.N);
+    o = align16(o);           // the staged arrays are filled by 16-byte bulk copies
     L.term = o;      o += kp.stage_terms ? ((dc.n_shapes + 31) & ~31) * dc.max_terms * 4 : 0;   // transposed, padded rows
     L.fam_in = o;    o += kp.stage_fam ? align16(dc.n_families * dc.N * 2) : 0;
     L.fam_cls = o;   o += kp.stage_fam ? align16(dc.n_families * dc.N) : 0;
     L.bucket = o;    o += kp.stage_bucket ? align16((dc.n_shapes + 1) * 4) : 0;
-    L.score = o;     o += kp.incremental ? dc.n_shapes * 8 : 0;
+    L.score = o;     o += kp.incremental ? align16(dc.n_shapes * 8) : 0;
     L.inv = o;       o += kp.incremental ? align16(dc.n_terms * 4) : 0;
     L.inv_ptr = o;   o += kp.incremental ? align16((dc.tbl_size + 1) * 4) : 0;
     L.delta = o;     o += kp.incremental ? 32 * 8 + 32 * 4 : 0;
@@ -862,38 +864,68 @@ vp_schedule_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand, co
     cnt.tasks = 0; cnt.sweeps = 0; cnt.t_mark = 0;
     for (int i = 0; i < 6; i++) cnt.cyc[i] = 0;
 
-    // ---- stage the catalog
+    // ---- stage the catalog: whole arrays by bulk asynchronous copies (TMA) that complete on one mbarrier; should the
+    // bounded wait give up, the same arrays are copied with plain loads
     c.p_term = dc.term;
     c.term_ss = dc.max_terms; c.term_se = 1;
     c.p_fam_in = dc.fam_in;
     c.p_fam_cls = dc.fam_cls;
-    if (kp.stage_terms) {
-        uint32_t* st = (uint32_t*)(smem_raw + L.term);
-        // staged transposed ([term][shape], rows padded to 32 shapes): consecutive threads score consecutive
-        // shapes, so every load of a term is conflict-free
-        const int ns_pad = (dc.n_shapes + 31) & ~31;
-        for (int e = tid; e < dc.n_shapes * dc.max_terms; e += NT) st[(e % dc.max_terms) * ns_pad + e / dc.max_terms] = dc.term[e];
-        c.p_term = st;
-        c.term_ss = 1; c.term_se = ns_pad;
-    }
     c.p_bucket_ptr = dc.bucket_ptr;
-    if (kp.stage_bucket) {
-        uint32_t* bp = (uint32_t*)(smem_raw + L.bucket);
-        for (int e = tid; e <= dc.n_shapes; e += NT) bp[e] = dc.bucket_ptr[e];
-        c.p_bucket_ptr = bp;
-    }
-    if (kp.incremental) {
-        uint32_t* iv = (uint32_t*)(smem_raw + L.inv);
-        uint32_t* ip = (uint32_t*)(smem_raw + L.inv_ptr);
-        for (int e = tid; e < dc.n_terms; e += NT) iv[e] = dc.inv[e];
-        for (int e = tid; e <= dc.tbl_size; e += NT) ip[e] = dc.inv_ptr[e];
-        c.p_inv = iv; c.p_inv_ptr = ip;
-    }
-    if (kp.stage_fam) {
-        uint16_t* fi = (uint16_t*)(smem_raw + L.fam_in);
-        uint8_t* fc = smem_raw + L.fam_cls;
-        for (int e = tid; e < dc.n_families * N; e += NT) { fi[e] = dc.fam_in[e]; fc[e] = dc.fam_cls[e]; }
-        c.p_fam_in = fi; c.p_fam_cls = fc;
+    {
+        const int ns_pad = (dc.n_shapes + 31) & ~31;
+        const unsigned b_term = kp.stage_terms ? (unsigned)(ns_pad * dc.max_terms * 4) : 0u;
+        const unsigned b_bucket = kp.stage_bucket ? (unsigned)align16((dc.n_shapes + 1) * 4) : 0u;
+        const unsigned b_inv = kp.incremental ? (unsigned)align16(dc.n_terms * 4) : 0u;
+        const unsigned b_invp = kp.incremental ? (unsigned)align16((dc.tbl_size + 1) * 4) : 0u;
+        const unsigned b_fin = kp.stage_fam ? (unsigned)align16(dc.n_families * N * 2) : 0u;
+        const unsigned b_fcls = kp.stage_fam ? (unsigned)align16(dc.n_families * N) : 0u;
+        const unsigned total = b_term + b_bucket + b_inv + b_invp + b_fin + b_fcls;
+        __shared__ __align__(8) unsigned long long s_stage_bar;
+        bool landed = false;
+        if (total > 0 && total < (1u << 20)) {
+            const unsigned bar = smem_u32(&s_stage_bar);
+            if (tid == 0) {
+                mbar_init(bar, 1);
+                asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+                mbar_expect_tx(bar, total);
+                if (b_term) bulk_load(smem_u32(smem_raw + L.term), dc.term_t, b_term, bar);
+                if (b_bucket) bulk_load(smem_u32(smem_raw + L.bucket), dc.bucket_ptr, b_bucket, bar);
+                if (b_inv) bulk_load(smem_u32(smem_raw + L.inv), dc.inv, b_inv, bar);
+                if (b_invp) bulk_load(smem_u32(smem_raw + L.inv_ptr), dc.inv_ptr, b_invp, bar);
+                if (b_fin) bulk_load(smem_u32(smem_raw + L.fam_in), dc.fam_in, b_fin, bar);
+                if (b_fcls) bulk_load(smem_u32(smem_raw + L.fam_cls), dc.fam_cls, b_fcls, bar);
+            }
+            __syncthreads();                                     // the barrier is initialised before anyone polls it
+            landed = __syncthreads_and(mbar_wait_bounded(bar, 0, 1u << 20)) != 0;
+        }
+        if (kp.stage_terms) {
+            uint32_t* st = (uint32_t*)(smem_raw + L.term);
+            // transposed ([term][shape], rows padded to 32 shapes): consecutive threads score consecutive shapes, so
+            // every load of a term is conflict-free
+            if (!landed) for (int e = tid; e < ns_pad * dc.max_terms; e += NT) st[e] = dc.term_t[e];
+            c.p_term = st;
+            c.term_ss = 1; c.term_se = ns_pad;
+        }
+        if (kp.stage_bucket) {
+            uint32_t* bp = (uint32_t*)(smem_raw + L.bucket);
+            if (!landed) for (int e = tid; e <= dc.n_shapes; e += NT) bp[e] = dc.bucket_ptr[e];
+            c.p_bucket_ptr = bp;
+        }
+        if (kp.incremental) {
+            uint32_t* iv = (uint32_t*)(smem_raw + L.inv);
+            uint32_t* ip = (uint32_t*)(smem_raw + L.inv_ptr);
+            if (!landed) {
+                for (int e = tid; e < dc.n_terms; e += NT) iv[e] = dc.inv[e];
+                for (int e = tid; e <= dc.tbl_size; e += NT) ip[e] = dc.inv_ptr[e];
+            }
+            c.p_inv = iv; c.p_inv_ptr = ip;
+        }
+        if (kp.stage_fam) {
+            uint16_t* fi = (uint16_t*)(smem_raw + L.fam_in);
+            uint8_t* fc = smem_raw + L.fam_cls;
+            if (!landed) for (int e = tid; e < dc.n_families * N; e += NT) { fi[e] = dc.fam_in[e]; fc[e] = dc.fam_cls[e]; }
+            c.p_fam_in = fi; c.p_fam_cls = fc;
+        }
     }
 
     for (;;) {

@@ -394,19 +394,43 @@ vp_schedule_warp_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ deman
     const int ld = N + 1;
     const WarpSmem L = warp_smem_layout(dc, kp, n_warps);
     if (tid < 32) smem_raw[L.lut + tid] = (uint8_t)(31 - tid < 24 ? perm4_packed_rt(31 - tid) : 0);
-    // ---- stage the catalog (shared by the warps of the CTA)
+    // ---- stage the catalog (shared by the warps of the CTA): bulk asynchronous copies (TMA) of whole arrays onto one
+    // mbarrier; plain loads if the bounded wait gives up
     {
-        uint32_t* t_term = (uint32_t*)(smem_raw + L.term);
         const int ns_pad = (dc.n_shapes + 31) & ~31;
-        for (int e = tid; e < dc.n_shapes * dc.max_terms; e += NT) t_term[(e % dc.max_terms) * ns_pad + e / dc.max_terms] = dc.term[e];
-        uint32_t* t_slot = (uint32_t*)(smem_raw + L.fam_slot);
-        uint16_t* t_in = (uint16_t*)(smem_raw + L.fam_in);
-        uint8_t* t_cls = smem_raw + L.fam_cls;
-        for (int e = tid; e < dc.n_families * N; e += NT) {
-            t_slot[e] = dc.fam_slot[e]; t_in[e] = dc.fam_in[e]; t_cls[e] = dc.fam_cls[e];
+        const unsigned b_term = (unsigned)(ns_pad * dc.max_terms * 4), b_slot = (unsigned)align16(dc.n_families * N * 4),
+                       b_fin = (unsigned)align16(dc.n_families * N * 2), b_fcls = (unsigned)align16(dc.n_families * N),
+                       b_bucket = (unsigned)align16((dc.n_shapes + 1) * 4);
+        const unsigned total = b_term + b_slot + b_fin + b_fcls + b_bucket;
+        __shared__ __align__(8) unsigned long long s_stage_bar;
+        bool landed = false;
+        if (total < (1u << 20)) {
+            const unsigned bar = smem_u32(&s_stage_bar);
+            if (tid == 0) {
+                mbar_init(bar, 1);
+                asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+                mbar_expect_tx(bar, total);
+                bulk_load(smem_u32(smem_raw + L.term), dc.term_t, b_term, bar);
+                bulk_load(smem_u32(smem_raw + L.fam_slot), dc.fam_slot, b_slot, bar);
+                bulk_load(smem_u32(smem_raw + L.fam_in), dc.fam_in, b_fin, bar);
+                bulk_load(smem_u32(smem_raw + L.fam_cls), dc.fam_cls, b_fcls, bar);
+                bulk_load(smem_u32(smem_raw + L.bucket), dc.bucket_ptr, b_bucket, bar);
+            }
+            __syncthreads();
+            landed = __syncthreads_and(mbar_wait_bounded(bar, 0, 1u << 20)) != 0;
         }
-        uint32_t* t_bp = (uint32_t*)(smem_raw + L.bucket);
-        for (int e = tid; e <= dc.n_shapes; e += NT) t_bp[e] = dc.bucket_ptr[e];
+        if (!landed) {
+            uint32_t* t_term = (uint32_t*)(smem_raw + L.term);
+            for (int e = tid; e < ns_pad * dc.max_terms; e += NT) t_term[e] = dc.term_t[e];
+            uint32_t* t_slot = (uint32_t*)(smem_raw + L.fam_slot);
+            uint16_t* t_in = (uint16_t*)(smem_raw + L.fam_in);
+            uint8_t* t_cls = smem_raw + L.fam_cls;
+            for (int e = tid; e < dc.n_families * N; e += NT) {
+                t_slot[e] = dc.fam_slot[e]; t_in[e] = dc.fam_in[e]; t_cls[e] = dc.fam_cls[e];
+            }
+            uint32_t* t_bp = (uint32_t*)(smem_raw + L.bucket);
+            for (int e = tid; e <= dc.n_shapes; e += NT) t_bp[e] = dc.bucket_ptr[e];
+        }
     }
     __syncthreads();
     WCtx c;

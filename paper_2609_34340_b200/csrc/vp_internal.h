@@ -21,6 +21,7 @@ struct DevCat {
     // Eq. (6): shape s has terms term[s*max_terms .. s*max_terms + max_terms) = 8 * table index | count << 16
     // (shapes with fewer terms are padded with zero counts)
     const uint32_t* term;
+    const uint32_t* term_t;       // the same, transposed: term e of shape s at term_t[e * ((n_shapes + 31) & ~31) + s]
     int max_terms;
     const uint32_t* bucket_ptr;
     // family f, slot r: instance id | destination group << 16 | rate class << 24
