@@ -376,3 +376,43 @@ def test_batches_around_one_wave(vp, oracle_lib):
                 n = min(37, B - r0)
                 assert np.array_equal(got[key][r0:r0 + n], want[key][:n]), (B, key, r0)
     assert kernels == {"CTA per matrix", "warp per matrix"}
+
+
+def test_randomised_topologies_and_parameters(vp, oracle_lib):
+    """A seeded sweep over group sizes 1..4, complete and node-template catalogs, mixed rates, granules, densities,
+    AA parameters, tau overrides and batch sizes on both sides of one wave: every plan equals the oracle's."""
+    rng = np.random.default_rng(2024)
+    cats = {}
+    choices = [("complete", 1, 4), ("complete", 2, 4), ("complete", 1, 3), ("complete", 2, 2), ("complete", 2, 1),
+               ("template", 3, 4), ("template", 4, 4), ("template", 6, 4), ("template", 8, 4), ("template", 3, 3), ("template", 12, 4)]
+    for case in range(120):
+        kind, nodes, g = choices[rng.integers(len(choices))]
+        pb, nb = [(64, 64), (64, 50), (32, 64), (50, 25)][rng.integers(4)]
+        key = (kind, nodes, g, pb, nb)
+        if key not in cats:
+            topo = tree_topology(nodes, g=g, pcie_bw=pb, nic_bw=nb)
+            cats[key] = complete_catalog(topo) if kind == "complete" else node_template_catalog(topo)
+        cat = cats[key]
+        N = cat.topology.N
+        u = int([1, 64, 256, 4096, 14336][rng.integers(5)])
+        hi = int([1, 3, 50, 1000, 100000][rng.integers(5)])
+        density = float([0.03, 0.2, 0.6, 1.0][rng.integers(4)])
+        B = int([1, 7, 40][rng.integers(3)]) if N > 16 else int([1, 33, 700][rng.integers(3)])
+        base = _random_batch(rng, min(B, 40), N, u, hi, density)
+        nb0 = base.shape[0]
+        reps = (B + nb0 - 1) // nb0
+        D = np.tile(base, (reps, 1, 1))[:B]
+        w = WParams(lambda_ns=int([0, 123, 8000][rng.integers(3)]), granule_bytes=u, n_start=int(rng.integers(0, 6)),
+                    i_aa=int(rng.integers(0, 5)), k_target=int([0, 5, 48][rng.integers(3)]), k_max=int(min(16 * N, 2048))).resolved(N)
+        tau = None
+        if rng.random() < 0.3:
+            tau = np.tile((rng.integers(0, 3, size=nb0) * rng.integers(1, 5000, size=nb0)).astype(np.int64), reps)[:B]
+        oc = oracle_lib.OracleCatalog(cat.topology.blob(), cat.blob())
+        dc = vp.load_catalog(cat.topology.blob(), cat.blob())
+        got = vp.schedule_batch(dc, _params(vp, w), torch.from_numpy(D).cuda().contiguous(),
+                                None if tau is None else torch.from_numpy(tau).cuda()).cpu()
+        want = oc.schedule_batch(base, w, tau_in=None if tau is None else tau[:nb0], threads=8)
+        for k in KEYS:
+            for r0 in range(0, B, nb0):
+                m = min(nb0, B - r0)
+                assert np.array_equal(got[k][r0:r0 + m], want[k][:m]), (case, key, u, hi, density, B, k, r0)
