@@ -137,3 +137,12 @@ def test_config5_full_size(vp, oracle_lib):
     assert res[2] == 0
     _assert_pack(res)
     assert res[6] * case["row_bytes"] > 1.7e9
+
+
+@pytest.mark.parametrize("hidden", [1024, 64])
+def test_pack_with_more_than_32_copies_per_token(vp, oracle_lib, hidden):
+    """top-40 routing: the copy handles the destinations of a token 32 slots at a time."""
+    case = build_pack_case(device="cuda", tokens=150, hidden=hidden, rank=5, seed=14, topk=40, experts=256)
+    res = _run_case(vp, oracle_lib, case)
+    assert res[2] == 0
+    _assert_pack(res)
