@@ -28,6 +28,21 @@ __device__ __forceinline__ void bulk_load(unsigned dst_smem, const void* src, un
 __device__ __forceinline__ void bulk_store(void* dst, unsigned src_smem, unsigned bytes) {
     asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src_smem), "r"(bytes) : "memory");
 }
+// Streaming variants: the data is touched once, so it is marked evict-first in L2 and does not push out what
+// neighbouring kernels keep there (catalog, demand, plan arrays).
+__device__ __forceinline__ unsigned long long l2_evict_first_policy() {
+    unsigned long long p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ void bulk_load_stream(unsigned dst_smem, const void* src, unsigned bytes, unsigned bar, unsigned long long policy) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+                 ::"r"(dst_smem), "l"(src), "r"(bytes), "r"(bar), "l"(policy) : "memory");
+}
+__device__ __forceinline__ void bulk_store_stream(void* dst, unsigned src_smem, unsigned bytes, unsigned long long policy) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group.L2::cache_hint [%0], [%1], %2, %3;"
+                 ::"l"(dst), "r"(src_smem), "r"(bytes), "l"(policy) : "memory");
+}
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 template <int N_PENDING>
 __device__ __forceinline__ void bulk_wait_read() {

@@ -32,6 +32,7 @@ pack_copy_bulk_kernel(const char* __restrict__ rows, char* __restrict__ staged, 
     __shared__ __align__(8) unsigned long long bars[S];
     const int lane = threadIdx.x;
     if (flags[0]) return;
+    const unsigned long long stream_policy = l2_evict_first_policy();
     if (lane == 0) {
         for (int s = 0; s < S; s++) mbar_init(smem_u32(&bars[s]), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -76,7 +77,7 @@ pack_copy_bulk_kernel(const char* __restrict__ rows, char* __restrict__ staged, 
                     const unsigned bytes = (unsigned)min((long long)kPiece, row_bytes - (long long)p * kPiece);
                     const unsigned bar = smem_u32(&bars[s]);
                     mbar_expect_tx(bar, bytes);
-                    bulk_load(smem_u32(ring + (size_t)s * kPiece), rows + t * row_bytes + (long long)p * kPiece, bytes, bar);
+                    bulk_load_stream(smem_u32(ring + (size_t)s * kPiece), rows + t * row_bytes + (long long)p * kPiece, bytes, bar, stream_policy);
                 }
             }
             loaded = any ? (loaded | (1u << s)) : (loaded & ~(1u << s));
@@ -100,15 +101,15 @@ pack_copy_bulk_kernel(const char* __restrict__ rows, char* __restrict__ staged, 
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                     if (one_round) {
                         if (rows_m >= 0)
-                            bulk_store(staged + (long long)rows_m * row_bytes + (long long)p * kPiece,
-                                       smem_u32(ring + (size_t)s * kPiece), bytes);
+                            bulk_store_stream(staged + (long long)rows_m * row_bytes + (long long)p * kPiece,
+                                              smem_u32(ring + (size_t)s * kPiece), bytes, stream_policy);
                     } else {
                         for (int r = 0; r < rounds; r++) {
                             const int slot = r * 32 + lane;
                             const int row = slot < topk ? dst_row[t * topk + slot] : -1;
                             if (row >= 0)
-                                bulk_store(staged + (long long)row * row_bytes + (long long)p * kPiece,
-                                           smem_u32(ring + (size_t)s * kPiece), bytes);
+                                bulk_store_stream(staged + (long long)row * row_bytes + (long long)p * kPiece,
+                                                  smem_u32(ring + (size_t)s * kPiece), bytes, stream_policy);
                         }
                     }
                 }
