@@ -118,6 +118,17 @@ void vp_free_catalog(vp_catalog* catalog);
 int vp_catalog_info(const vp_catalog* catalog, vp_info* out);
 
 /*
+ * vp_prune_paths - the path filter that precedes the search, PrunePaths of Section 4.1 ("Pruning and search cost";
+ * host code): a path instance is dropped when another instance of the same group pair uses a subset of its directed
+ * resources at a rate that is not lower, one of the two strictly.  topology: a topology blob (layout under
+ * vp_load_catalog) holding the candidate instances; topology_out receives the same blob with the surviving
+ * instances in their original order.  *bytes_needed is always set; with topology_out == NULL only the size and
+ * *n_kept_out are computed; VP_E_WORKSPACE if capacity_bytes is too small.
+ */
+int vp_prune_paths(const void* topology, size_t topology_bytes, void* topology_out, size_t capacity_bytes,
+                   size_t* bytes_needed, int32_t* n_kept_out);
+
+/*
  * vp_build_catalog - offline catalog construction, Algorithm 1 of Section 4.1 (host code, no GPU work).
  *
  * Enumerates, by the pruned binary depth-first search of Algorithm 1 (CanAdd: resource disjointness and the

@@ -95,6 +95,7 @@ def _load():
     lib.vp_unpack_tokens.argtypes = [P, P, P, P, i32, i32, i32, P, i32, i32, i32, P, i64, i64, P, P, P, P, sz, P]
     lib.vp_kernel_launch_count.restype = i64
     lib.vp_build_catalog.argtypes = [P, sz, P, sz, C.POINTER(sz), C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
+    lib.vp_prune_paths.argtypes = [P, sz, P, sz, C.POINTER(sz), C.POINTER(C.c_int32)]
     lib.vp_plan_time.argtypes = [vp, i32, i32, P, P, P, i64, P, P]
     lib.vp_demand_from_routing.argtypes = [P, i32, i32, i32, i32, i32, i32, i64, P, P, P]
     lib.vp_schedule_read_stats.argtypes = [P, P, P]
@@ -446,3 +447,13 @@ def unpack_tokens(plan: Plan, b: int, rank: int, expert_idx: torch.Tensor, exper
                                   workspace.numel(), _stream(stream))
     _check(rc, "vp_unpack_tokens")
     return status
+
+
+def prune_paths(topology_blob: bytes) -> bytes:
+    """``vp_prune_paths``: the topology blob without its dominated path instances (host code, no GPU)."""
+    need, kept = C.c_size_t(0), C.c_int32(0)
+    lib = _load()
+    _check(lib.vp_prune_paths(topology_blob, len(topology_blob), None, 0, C.byref(need), C.byref(kept)), "vp_prune_paths")
+    out = C.create_string_buffer(need.value)
+    _check(lib.vp_prune_paths(topology_blob, len(topology_blob), out, need.value, C.byref(need), C.byref(kept)), "vp_prune_paths")
+    return out.raw[:need.value]

@@ -193,3 +193,52 @@ extern "C" int vp_build_catalog(const void* topology, size_t topo_bytes, void* c
     memcpy(channels_out, o.data(), o.size());
     return VP_OK;
 }
+
+// PrunePaths of Section 4.1 ("Pruning and search cost"), the filter that runs before the search: a path instance r
+// is dropped when another instance r' of the same group pair has a footprint L(r') that is a subset of L(r) and a
+// rate bw(r') >= bw(r), with at least one of the two strict.  The survivors keep their order.
+extern "C" int vp_prune_paths(const void* topology, size_t topo_bytes, void* topology_out, size_t capacity_bytes,
+                              size_t* bytes_needed, int32_t* n_kept_out) {
+    if (!topology || !bytes_needed) return VP_E_BAD_ARG;
+    const uint8_t* t = (const uint8_t*)topology;
+    if (topo_bytes < 32 || rd32(t) != 0x50545056u || rd32(t + 4) != 1) return VP_E_BAD_CATALOG;
+    const int n_inst = (int)rd32(t + 28);
+    if (n_inst < 0 || n_inst > 0xFFFE || topo_bytes < 32 + (size_t)n_inst * 20) return VP_E_BAD_CATALOG;
+    struct P { int a, d, n_res; long long bw; int res[4]; };
+    std::vector<P> inst(n_inst);
+    for (int r = 0; r < n_inst; r++) {
+        const uint8_t* p = t + 32 + (size_t)r * 20;
+        P& q = inst[r];
+        q.a = rd16(p); q.d = rd16(p + 2); q.n_res = p[5]; q.bw = rd32(p + 8);
+        if (q.n_res > 4) return VP_E_BAD_CATALOG;
+        for (int k = 0; k < q.n_res; k++) q.res[k] = rd16(p + 12 + 2 * k);
+    }
+    auto subset = [](const P& x, const P& y) {               // L(x) is a subset of L(y)
+        for (int i = 0; i < x.n_res; i++) {
+            bool found = false;
+            for (int k = 0; k < y.n_res; k++) found |= x.res[i] == y.res[k];
+            if (!found) return false;
+        }
+        return true;
+    };
+    std::vector<int> keep;
+    for (int r = 0; r < n_inst; r++) {
+        bool dominated = false;
+        for (int o = 0; o < n_inst && !dominated; o++) {
+            if (o == r || inst[o].a != inst[r].a || inst[o].d != inst[r].d) continue;
+            if (!subset(inst[o], inst[r]) || inst[o].bw < inst[r].bw) continue;
+            const bool strict = !subset(inst[r], inst[o]) || inst[o].bw > inst[r].bw;
+            if (strict) dominated = true;
+        }
+        if (!dominated) keep.push_back(r);
+    }
+    *bytes_needed = 32 + keep.size() * 20;
+    if (n_kept_out) *n_kept_out = (int32_t)keep.size();
+    if (!topology_out || capacity_bytes < *bytes_needed) return topology_out ? VP_E_WORKSPACE : VP_OK;
+    uint8_t* o = (uint8_t*)topology_out;
+    memcpy(o, t, 32);
+    const uint32_t n = (uint32_t)keep.size();
+    for (int k = 0; k < 4; k++) o[28 + k] = (uint8_t)(n >> (8 * k));
+    for (size_t i = 0; i < keep.size(); i++) memcpy(o + 32 + i * 20, t + 32 + (size_t)keep[i] * 20, 20);
+    return VP_OK;
+}

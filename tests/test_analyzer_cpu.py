@@ -73,3 +73,34 @@ def test_construction_time_is_small(vp):
     _, ns, nf = vp.build_catalog(topo)
     dt = time.perf_counter() - t0
     assert (ns, nf) == (89, 152) and dt < 2.0
+
+
+def test_prune_paths_matches_the_definition(vp):
+    """vp_prune_paths against the definition written out: r goes when some r' of the same group pair has
+    L(r') within L(r) and bw(r') >= bw(r), one of them strictly (Section 4.1, pruning)."""
+    import random
+    from workloads.topology import prune_paths
+    rng = random.Random(5)
+    base = tree_topology(2, pcie_bw=64, nic_bw=50)
+    cands = list(base.instances)
+    for r in list(base.instances):
+        if not r.res:
+            continue
+        cands.append(Instance(r.src_group, r.dst_group, r.kind, r.bw - 1, 1, r.res))                     # slower twin: dominated
+        cands.append(Instance(r.src_group, r.dst_group, r.kind, r.bw, 1, r.res + (base.n_resources,)))   # extra resource: dominated
+        cands.append(Instance(r.src_group, r.dst_group, r.kind, r.bw + 9, 1, r.res + (base.n_resources + 1,)))  # faster but wider: stays
+        cands.append(Instance(r.src_group, r.dst_group, r.kind, r.bw, 1, r.res))                         # exact twin: both stay
+    rng.shuffle(cands)
+    cands.sort(key=lambda r: (r.src_group, r.dst_group))
+    topo = Topology(base.N, base.G, base.g, base.groups_per_node, base.n_resources + 2, cands)
+    want = Topology(base.N, base.G, base.g, base.groups_per_node, base.n_resources + 2, prune_paths(cands))
+    got = vp.prune_paths(topo.blob())
+    assert got == want.blob()
+    assert len(want.instances) < len(cands)
+    # the instances a generator hands to Algorithm 1 are already a fixed point
+    assert vp.prune_paths(base.blob()) == base.blob()
+    # same-switch NIC loop-back next to the switch-local path: the textbook dominated candidate
+    pix = Instance(0, 0, 0, 64, 4, ())
+    loop = Instance(0, 0, 2, 64, 1, (2, 3))
+    two = Topology(4, 1, 4, 1, 4, [pix, loop])
+    assert vp.prune_paths(two.blob()) == Topology(4, 1, 4, 1, 4, [pix]).blob()
