@@ -118,6 +118,20 @@ void vp_free_catalog(vp_catalog* catalog);
 int vp_catalog_info(const vp_catalog* catalog, vp_info* out);
 
 /*
+ * vp_build_template_catalog - a node-symmetric catalog for many nodes (host code, no GPU work; no counterpart in the
+ * paper, whose Algorithm 1 enumerates every family and grows exponentially with the node count).  One per-node
+ * template is applied to every node: each of the two switch-local groups q of a node gets a network target "none" or
+ * (delta, q2) = group q2 of node (n + delta) mod P (delta = 0 needs q2 != q; the two groups use different q2) and one
+ * flag per direction of the path between the two sibling groups; a group sends as many such lanes as it receives and
+ * switch-local lanes fill the rest of its g slots.  Every family satisfies Eq. (3) / Eq. (4) and is invariant under a
+ * shift of the node index (vp_info.node_symmetric = 1).  Arguments and results as for vp_build_catalog; the topology
+ * must have two groups per node with instance kinds 0 (switch-local), 1 (sibling) and 2 (network), else
+ * VP_E_UNSUPPORTED.  8 nodes: 255 shapes / 272 families; 32 nodes: 4095 / 4160.
+ */
+int vp_build_template_catalog(const void* topology, size_t topology_bytes, void* channels_out, size_t capacity_bytes,
+                              size_t* bytes_needed, int32_t* n_shapes_out, int32_t* n_families_out);
+
+/*
  * vp_prune_paths - the path filter that precedes the search, PrunePaths of Section 4.1 ("Pruning and search cost";
  * host code): a path instance is dropped when another instance of the same group pair uses a subset of its directed
  * resources at a rate that is not lower, one of the two strictly.  topology: a topology blob (layout under

@@ -12,6 +12,7 @@ from .binding import (  # noqa: F401
     SchedParams,
     load_catalog,
     build_catalog,
+    build_template_catalog,
     prune_paths,
     schedule_workspace_bytes,
     schedule_batch,

@@ -95,6 +95,7 @@ def _load():
     lib.vp_unpack_tokens.argtypes = [P, P, P, P, i32, i32, i32, P, i32, i32, i32, P, i64, i64, P, P, P, P, sz, P]
     lib.vp_kernel_launch_count.restype = i64
     lib.vp_build_catalog.argtypes = [P, sz, P, sz, C.POINTER(sz), C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
+    lib.vp_build_template_catalog.argtypes = [P, sz, P, sz, C.POINTER(sz), C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
     lib.vp_prune_paths.argtypes = [P, sz, P, sz, C.POINTER(sz), C.POINTER(C.c_int32)]
     lib.vp_plan_time.argtypes = [vp, i32, i32, P, P, P, i64, P, P]
     lib.vp_demand_from_routing.argtypes = [P, i32, i32, i32, i32, i32, i32, i64, P, P, P]
@@ -457,3 +458,15 @@ def prune_paths(topology_blob: bytes) -> bytes:
     out = C.create_string_buffer(need.value)
     _check(lib.vp_prune_paths(topology_blob, len(topology_blob), out, need.value, C.byref(need), C.byref(kept)), "vp_prune_paths")
     return out.raw[:need.value]
+
+
+def build_template_catalog(topology_blob: bytes):
+    """``vp_build_template_catalog``: (channels blob, shapes, families) of the node-template catalog (host code)."""
+    need, ns, nf = C.c_size_t(0), C.c_int32(0), C.c_int32(0)
+    lib = _load()
+    _check(lib.vp_build_template_catalog(topology_blob, len(topology_blob), None, 0, C.byref(need), C.byref(ns), C.byref(nf)),
+           "vp_build_template_catalog")
+    out = C.create_string_buffer(need.value)
+    _check(lib.vp_build_template_catalog(topology_blob, len(topology_blob), out, need.value, C.byref(need), C.byref(ns), C.byref(nf)),
+           "vp_build_template_catalog")
+    return out.raw[:need.value], int(ns.value), int(nf.value)

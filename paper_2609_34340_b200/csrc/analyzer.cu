@@ -106,24 +106,23 @@ bool dominated(const Signature& x, const Signature& y) {
     return strict;
 }
 
-}  // namespace
-
-extern "C" int vp_build_catalog(const void* topology, size_t topo_bytes, void* channels_out, size_t capacity_bytes,
-                                size_t* bytes_needed, int32_t* n_shapes_out, int32_t* n_families_out) {
-    if (!topology || !bytes_needed) return VP_E_BAD_ARG;
+// Reads a topology blob into an Analyzer (instances, degrees, suffix capacities).  kinds (optional) receives the
+// instances' kind bytes.
+int parse_topology(const void* topology, size_t topo_bytes, Analyzer& A, std::vector<int>* kinds) {
     const uint8_t* t = (const uint8_t*)topology;
     if (topo_bytes < 32 || rd32(t) != 0x50545056u || rd32(t + 4) != 1) return VP_E_BAD_CATALOG;
-    Analyzer A;
     A.N = (int)rd32(t + 8); A.G = (int)rd32(t + 12); A.g = (int)rd32(t + 16); A.n_res = (int)rd32(t + 24);
     const int n_inst = (int)rd32(t + 28);
     if (A.N <= 0 || A.G <= 0 || A.g <= 0 || (long long)A.G * A.g != A.N || n_inst <= 0 || n_inst > 0xFFFE || A.n_res < 0 ||
         A.N > 0xFFFF || topo_bytes < 32 + (size_t)n_inst * 20)
         return VP_E_BAD_CATALOG;
     A.inst.resize(n_inst);
+    if (kinds) kinds->resize(n_inst);
     for (int r = 0; r < n_inst; r++) {
         const uint8_t* p = t + 32 + (size_t)r * 20;
         AInst& q = A.inst[r];
         q.a = rd16(p); q.d = rd16(p + 2); q.n_res = p[5]; q.mult = rd16(p + 6); q.bw = rd32(p + 8);
+        if (kinds) (*kinds)[r] = p[4];
         if (q.a >= A.G || q.d >= A.G || q.n_res > 4 || q.mult < 1 || q.bw <= 0) return VP_E_BAD_CATALOG;
         for (int k = 0; k < q.n_res; k++) {
             q.res[k] = rd16(p + 12 + 2 * k);
@@ -131,23 +130,13 @@ extern "C" int vp_build_catalog(const void* topology, size_t topo_bytes, void* c
         }
         if (r > 0 && (A.inst[r - 1].a > q.a || (A.inst[r - 1].a == q.a && A.inst[r - 1].d > q.d))) return VP_E_BAD_CATALOG;
     }
-    A.out_suffix.assign(n_inst + 1, std::vector<int>(A.G, 0));
-    A.in_suffix.assign(n_inst + 1, std::vector<int>(A.G, 0));
-    for (int r = n_inst - 1; r >= 0; r--) {
-        A.out_suffix[r] = A.out_suffix[r + 1];
-        A.in_suffix[r] = A.in_suffix[r + 1];
-        A.out_suffix[r][A.inst[r].a] += A.inst[r].mult;
-        A.in_suffix[r][A.inst[r].d] += A.inst[r].mult;
-    }
-    A.out_deg.assign(A.G, 0);
-    A.in_deg.assign(A.G, 0);
-    A.used.assign(A.n_res + 1, 0);
-    A.limit = (size_t)1 << 22;                              // more families than this is not a usable catalog
-    A.explore(0);
-    if (A.overflow) return VP_E_UNSUPPORTED;
-    if (A.found.empty()) return VP_E_BAD_CATALOG;
+    return VP_OK;
+}
 
-    // buckets by shape, pruned, in canonical order
+// Buckets the families in A.found by shape, applies PruneFamilies inside each bucket and writes the channels blob in
+// canonical order (shapes by their sorted (a, d, count) list, families by their instance-id list).
+int write_catalog(Analyzer& A, void* channels_out, size_t capacity_bytes, size_t* bytes_needed, int32_t* n_shapes_out,
+                  int32_t* n_families_out) {
     std::map<Shape, std::vector<std::vector<uint16_t>>> buckets;
     for (auto& fam : A.found) {
         std::map<std::pair<int, int>, int> cnt;
@@ -193,6 +182,110 @@ extern "C" int vp_build_catalog(const void* topology, size_t topo_bytes, void* c
     memcpy(channels_out, o.data(), o.size());
     return VP_OK;
 }
+
+}  // namespace
+
+extern "C" int vp_build_catalog(const void* topology, size_t topo_bytes, void* channels_out, size_t capacity_bytes,
+                                size_t* bytes_needed, int32_t* n_shapes_out, int32_t* n_families_out) {
+    if (!topology || !bytes_needed) return VP_E_BAD_ARG;
+    Analyzer A;
+    int rc = parse_topology(topology, topo_bytes, A, nullptr);
+    if (rc) return rc;
+    const int n_inst = (int)A.inst.size();
+    A.out_suffix.assign(n_inst + 1, std::vector<int>(A.G, 0));
+    A.in_suffix.assign(n_inst + 1, std::vector<int>(A.G, 0));
+    for (int r = n_inst - 1; r >= 0; r--) {
+        A.out_suffix[r] = A.out_suffix[r + 1];
+        A.in_suffix[r] = A.in_suffix[r + 1];
+        A.out_suffix[r][A.inst[r].a] += A.inst[r].mult;
+        A.in_suffix[r][A.inst[r].d] += A.inst[r].mult;
+    }
+    A.out_deg.assign(A.G, 0);
+    A.in_deg.assign(A.G, 0);
+    A.used.assign(A.n_res + 1, 0);
+    A.limit = (size_t)1 << 22;                              // more families than this is not a usable catalog
+    A.explore(0);
+    if (A.overflow) return VP_E_UNSUPPORTED;
+    if (A.found.empty()) return VP_E_BAD_CATALOG;
+    return write_catalog(A, channels_out, capacity_bytes, bytes_needed, n_shapes_out, n_families_out);
+}
+
+// A catalog for many nodes without the exponential search: one per-node TEMPLATE applied to every node, so that every
+// family is invariant under a shift of the node index.  (The paper's search, Algorithm 1, grows exponentially with the
+// node count; its Table 3 catalogs for 16 to 32 nodes have a few hundred shapes, which a complete enumeration cannot
+// give.  This construction is this library's reading; it needs two switch-local groups per node, each with one
+// network path to every other group and one path to its sibling group.)  A template gives each of the two groups q of a
+// node a network target "none" or (delta, q2) = group q2 of node (n + delta) mod P -- delta = 0 needs q2 != q, and the two
+// groups must not target the same q2 -- plus one flag per direction of the sibling path; a group must send as many
+// such lanes as it receives, and switch-local lanes fill the rest of its g slots.
+extern "C" int vp_build_template_catalog(const void* topology, size_t topo_bytes, void* channels_out, size_t capacity_bytes,
+                                         size_t* bytes_needed, int32_t* n_shapes_out, int32_t* n_families_out) {
+    if (!topology || !bytes_needed) return VP_E_BAD_ARG;
+    Analyzer A;
+    std::vector<int> kinds;
+    int rc = parse_topology(topology, topo_bytes, A, &kinds);
+    if (rc) return rc;
+    const uint8_t* t = (const uint8_t*)topology;
+    const int S = (int)rd32(t + 20);
+    if (S != 2 || A.G % S) return VP_E_UNSUPPORTED;
+    const int P = A.G / S, g = A.g;
+    std::map<std::pair<std::pair<int, int>, int>, int> by_key;          // (a, d, kind) -> instance id
+    for (int r = 0; r < (int)A.inst.size(); r++) by_key[{{A.inst[r].a, A.inst[r].d}, kinds[r]}] = r;
+    auto find = [&](int a, int d, int kind) {
+        auto it = by_key.find({{a, d}, kind});
+        return it == by_key.end() ? -1 : it->second;
+    };
+    struct Opt { int delta, q2; };                                       // delta < 0: no network lane
+    std::vector<Opt> opts[2];
+    for (int q = 0; q < S; q++) {
+        opts[q].push_back({-1, 0});
+        for (int delta = 0; delta < P; delta++)
+            for (int q2 = 0; q2 < S; q2++)
+                if (!(delta == 0 && q2 == q)) opts[q].push_back({delta, q2});
+    }
+    for (const Opt& n0 : opts[0])
+        for (const Opt& n1 : opts[1])
+            for (int p01 = 0; p01 < 2; p01++)
+                for (int p10 = 0; p10 < 2; p10++) {
+                    if (n0.delta >= 0 && n1.delta >= 0 && n0.q2 == n1.q2) continue;
+                    const Opt nic[2] = {n0, n1};
+                    const int out[2] = {p01 + (n0.delta >= 0), p10 + (n1.delta >= 0)};
+                    const int inn[2] = {p10 + (n0.delta >= 0 && n0.q2 == 0) + (n1.delta >= 0 && n1.q2 == 0),
+                                        p01 + (n0.delta >= 0 && n0.q2 == 1) + (n1.delta >= 0 && n1.q2 == 1)};
+                    if (out[0] != inn[0] || out[1] != inn[1] || std::max(out[0], out[1]) > g) continue;
+                    if (g < 2 && std::min(out[0], out[1]) < g) continue;
+                    std::vector<uint16_t> fam;
+                    bool ok = true;
+                    for (int node = 0; node < P && ok; node++)
+                        for (int q = 0; q < S && ok; q++) {
+                            const int a = node * S + q;
+                            if (g - out[q] > 0) {
+                                const int pix = find(a, a, 0);
+                                if (pix < 0) { ok = false; break; }
+                                for (int k = 0; k < g - out[q]; k++) fam.push_back((uint16_t)pix);
+                            }
+                            if (q == 0 ? p01 : p10) {
+                                const int pxb = find(a, node * S + (1 - q), 1);
+                                if (pxb < 0) { ok = false; break; }
+                                fam.push_back((uint16_t)pxb);
+                            }
+                            if (nic[q].delta >= 0) {
+                                const int d = ((node + nic[q].delta) % P) * S + nic[q].q2;
+                                const int id = find(a, d, 2);
+                                if (id < 0) { ok = false; break; }
+                                fam.push_back((uint16_t)id);
+                            }
+                        }
+                    if (!ok) return VP_E_UNSUPPORTED;             // the topology lacks a path the template needs
+                    std::sort(fam.begin(), fam.end());
+                    A.found.push_back(fam);
+                }
+    if (A.found.empty()) return VP_E_BAD_CATALOG;
+    return write_catalog(A, channels_out, capacity_bytes, bytes_needed, n_shapes_out, n_families_out);
+}
+
+namespace {
+}  // namespace
 
 // PrunePaths of Section 4.1 ("Pruning and search cost"), the filter that runs before the search: a path instance r
 // is dropped when another instance r' of the same group pair has a footprint L(r') that is a subset of L(r) and a

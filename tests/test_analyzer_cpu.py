@@ -104,3 +104,26 @@ def test_prune_paths_matches_the_definition(vp):
     loop = Instance(0, 0, 2, 64, 1, (2, 3))
     two = Topology(4, 1, 4, 1, 4, [pix, loop])
     assert vp.prune_paths(two.blob()) == Topology(4, 1, 4, 1, 4, [pix]).blob()
+
+
+@pytest.mark.parametrize("nodes,g,nic_bw", [(3, 4, 64), (4, 4, 50), (8, 4, 64), (12, 4, 64), (3, 3, 50), (5, 2, 64), (32, 4, 64)])
+def test_template_catalog_same_blob_as_the_python_generator(vp, oracle_lib, nodes, g, nic_bw):
+    from workloads.topology import node_template_catalog
+    topo = tree_topology(nodes, g=g, nic_bw=nic_bw)
+    want = node_template_catalog(topo)
+    blob, ns, nf = vp.build_template_catalog(topo.blob())
+    assert (ns, nf) == (want.n_shapes, want.n_families)
+    assert blob == want.blob()
+    if nodes <= 8:                                   # Eq. (3), Eq. (4) by the oracle's own checker
+        oc = oracle_lib.OracleCatalog(topo.blob(), blob)
+        assert oc.check() == 0 and oc.covers()
+    if nodes == 8:
+        assert (ns, nf) == (255, 272)
+    if nodes == 32:
+        assert (ns, nf) == (4095, 4160)
+
+
+def test_template_catalog_needs_two_groups_per_node(vp):
+    with pytest.raises(vp.VpError) as e:
+        vp.build_template_catalog(crossbar_topology(4).blob())
+    assert e.value.code == vp.E_UNSUPPORTED
