@@ -153,6 +153,20 @@ __device__ __forceinline__ int64_t warp_max_i64(int64_t v) {
     return v;
 }
 
+// First maximum of (value, index) pairs over the warp by warp-reduce instructions: the maximum of the high
+// words, then of the low words among the lanes that hold it, then the lowest index among those.
+__device__ __forceinline__ void warp_argmax_first(int64_t& best, int& best_s) {
+    const uint32_t hi = (uint32_t)((uint64_t)best >> 32), lo = (uint32_t)best;
+    const uint32_t mhi = __reduce_max_sync(0xffffffffu, best < 0 ? 0u : hi);
+    const bool in1 = best >= 0 && hi == mhi;
+    const uint32_t mlo = __reduce_max_sync(0xffffffffu, in1 ? lo : 0u);
+    const bool in2 = in1 && lo == mlo;
+    const unsigned any = __ballot_sync(0xffffffffu, in2);
+    const uint32_t ms = __reduce_min_sync(0xffffffffu, in2 ? (uint32_t)best_s : 0x7fffffffu);
+    best = any ? (int64_t)(((uint64_t)mhi << 32) | mlo) : -1;
+    best_s = (int)ms;
+}
+
 // f1/d1 > f2/d2, exactly, by 128-bit cross-multiplication (all four in [0, 2^63)).
 __device__ __forceinline__ bool util_greater(int64_t f1, int64_t d1, int64_t f2, int64_t d2) {
     unsigned long long a = (unsigned long long)f1, b = (unsigned long long)d2;
@@ -492,12 +506,7 @@ __device__ __forceinline__ void decompose(const DevCat& dc, const KParams& kp, c
                 }
                 if (score > best) { best = score; best_s = s; }     // ascending s: keeps the first maximum
             }
-#pragma unroll
-            for (int o = 16; o; o >>= 1) {
-                int64_t ov = __shfl_xor_sync(0xffffffffu, best, o);
-                int oi = __shfl_xor_sync(0xffffffffu, best_s, o);
-                if (ov > best || (ov == best && oi < best_s)) { best = ov; best_s = oi; }
-            }
+            warp_argmax_first(best, best_s);
             if (lane == 0) { c.red[warp] = best; c.red[32 + warp] = best_s; }
         }
         __syncthreads();

@@ -65,20 +65,6 @@ struct WCtx {
 
 template <typename T> __device__ __forceinline__ T* ws(unsigned off) { return (T*)(vp_wsmem + off); }
 
-// First maximum of (value, index) pairs over the warp by warp-reduce instructions: the maximum of the high
-// words, then of the low words among the lanes that hold it, then the lowest index among those.
-__device__ __forceinline__ void warp_argmax_first(int64_t& best, int& best_s) {
-    const uint32_t hi = (uint32_t)((uint64_t)best >> 32), lo = (uint32_t)best;
-    const uint32_t mhi = __reduce_max_sync(0xffffffffu, best < 0 ? 0u : hi);
-    const bool in1 = best >= 0 && hi == mhi;
-    const uint32_t mlo = __reduce_max_sync(0xffffffffu, in1 ? lo : 0u);
-    const bool in2 = in1 && lo == mlo;
-    const unsigned any = __ballot_sync(0xffffffffu, in2);
-    const uint32_t ms = __reduce_min_sync(0xffffffffu, in2 ? (uint32_t)best_s : 0x7fffffffu);
-    best = any ? (int64_t)(((uint64_t)mhi << 32) | mlo) : -1;
-    best_s = (int)ms;
-}
-
 // team_best for kWT credit tiles at once, written level by level so that the shuffles of the four tasks are
 // issued back to back (shuffles are not reordered by the compiler).
 __device__ __forceinline__ void team_best_x(const unsigned (&tile)[kWT], int tl, const uint8_t (&pidx)[3][4], unsigned o_lut,
