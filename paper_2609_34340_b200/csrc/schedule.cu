@@ -724,29 +724,39 @@ __device__ __forceinline__ void decompose(const DevCat& dc, const KParams& kp, c
 
         // (C) best start per family (largest F, lowest t), then largest utility, lowest family;
         //     every warp computes it for itself, over the lanes 0 .. H-1 only
-        int64_t bf = -1, bd = 1;
-        int bt = 0x7fffffff;
-        for (int h = lane; h < H; h += 32) {
-            int64_t ff = -1; int tt = 0;
-            for (int t = 0; t < kp.n_start; t++)
-                if (c.task_f[h * kp.n_start + t] > ff) { ff = c.task_f[h * kp.n_start + t]; tt = h * kp.n_start + t; }
-            if (bt == 0x7fffffff || util_greater(ff, c.task_den[tt], bf, bd)) { bf = ff; bd = c.task_den[tt]; bt = tt; }
-        }
-        int width = 1;
-        while (width < H && width < 32) width <<= 1;
-        for (int o = width >> 1; o; o >>= 1) {
-            int64_t of = __shfl_xor_sync(0xffffffffu, bf, o), od = __shfl_xor_sync(0xffffffffu, bd, o);
-            int ot = __shfl_xor_sync(0xffffffffu, bt, o);
-            bool take = false;
-            if (ot != 0x7fffffff) {
-                if (bt == 0x7fffffff) take = true;
-                else if (util_greater(of, od, bf, bd)) take = true;
-                else if (!util_greater(bf, bd, of, od) && ot < bt) take = true;
+        int wtask;
+        int64_t wF;
+        if (H == 1 && kp.n_start <= 32) {
+            // one family (the common case): its best start is one arg-max over the lanes, no utilities to compare
+            int64_t ff = lane < kp.n_start ? c.task_f[lane] : -1;
+            int tt = lane;
+            warp_argmax_first(ff, tt);
+            wtask = tt; wF = ff;
+        } else {
+            int64_t bf = -1, bd = 1;
+            int bt = 0x7fffffff;
+            for (int h = lane; h < H; h += 32) {
+                int64_t ff = -1; int tt = 0;
+                for (int t = 0; t < kp.n_start; t++)
+                    if (c.task_f[h * kp.n_start + t] > ff) { ff = c.task_f[h * kp.n_start + t]; tt = h * kp.n_start + t; }
+                if (bt == 0x7fffffff || util_greater(ff, c.task_den[tt], bf, bd)) { bf = ff; bd = c.task_den[tt]; bt = tt; }
             }
-            if (take) { bf = of; bd = od; bt = ot; }
+            int width = 1;
+            while (width < H && width < 32) width <<= 1;
+            for (int o = width >> 1; o; o >>= 1) {
+                int64_t of = __shfl_xor_sync(0xffffffffu, bf, o), od = __shfl_xor_sync(0xffffffffu, bd, o);
+                int ot = __shfl_xor_sync(0xffffffffu, bt, o);
+                bool take = false;
+                if (ot != 0x7fffffff) {
+                    if (bt == 0x7fffffff) take = true;
+                    else if (util_greater(of, od, bf, bd)) take = true;
+                    else if (!util_greater(bf, bd, of, od) && ot < bt) take = true;
+                }
+                if (take) { bf = of; bd = od; bt = ot; }
+            }
+            wtask = __shfl_sync(0xffffffffu, bt, 0);
+            wF = __shfl_sync(0xffffffffu, bf, 0);
         }
-        const int wtask = __shfl_sync(0xffffffffu, bt, 0);
-        const int64_t wF = __shfl_sync(0xffffffffu, bf, 0);
         if (wF <= 0) { st |= VP_ST_NO_PROGRESS; break; }
         VP_TICK(3);
 
