@@ -428,6 +428,7 @@ __device__ __forceinline__ void decompose(const DevCat& dc, const KParams& kp, c
     // touches 32 different banks.  Otherwise tiles are 17 credits apart.
     V* cred = (V*)c.cred_warp + (LPG == 2 && sizeof(V) == 4 ? 33 * (team & 7) + 16 * (team >> 3) : team * 17);
     const int n_score_warps = min(n_warps, (dc.n_shapes + 31) >> 5);
+    const int ns_shift = (kp.n_start & (kp.n_start - 1)) == 0 ? 31 - __clz(kp.n_start) : -1;     // n_start a power of two: shifts for divisions
 
     const bool inc = kp.incremental != 0;
     // a score is at most g x (what is left) and only shrinks: when that fits 32 bits the scores are kept as 32-bit
@@ -536,7 +537,7 @@ __device__ __forceinline__ void decompose(const DevCat& dc, const KParams& kp, c
             __syncwarp();
         };
         for (int task = wgroup; task < n_tasks; task += n_warps / W) {
-            const int h = task / kp.n_start, f = f0 + h, t = task % kp.n_start;
+            const int h = ns_shift >= 0 ? task >> ns_shift : task / kp.n_start, f = f0 + h, t = task - h * kp.n_start;
             const uint16_t* fin = c.p_fam_in + (size_t)f * N;
             const uint8_t* fcls = c.p_fam_cls + (size_t)f * N;
             uint8_t* srcb = c.bind_src + (size_t)task * N;
@@ -548,9 +549,10 @@ __device__ __forceinline__ void decompose(const DevCat& dc, const KParams& kp, c
                 for (int rr = 0; rr < (VP_MAX_N + 31) / 32; rr++)
                     if (rr * 32 + lane < N) slot_pre[rr] = __ldg(&dc.fam_slot[(size_t)f * N + rr * 32 + lane]);
             }
-            for (int d = sub * 32 + lane; d < G; d += 32 * W)
-#pragma unroll
-                for (int q = 0; q < GS; q++) dstb[fin[d * GS + q] & 0xff] = (uint8_t)(d * GS + (q + t) % GS);
+            for (int e = sub * 32 + lane; e < N; e += 32 * W) {      // in-slot e = d * GS + q: start t rotates q by t
+                const int q = e % GS;
+                dstb[fin[e] & 0xff] = (uint8_t)(e - q + (q + t) % GS);
+            }
             int64_t F_old = -1, F_new = -1, tmax = 0;
             bool tmax_done = false;
             if constexpr (LPG > 1) {
@@ -762,7 +764,7 @@ __device__ __forceinline__ void decompose(const DevCat& dc, const KParams& kp, c
 
         // (D) emit activation k, D_rem -= X(E), update D-hat, write offset row k+1
         {
-            const int h = wtask / kp.n_start;
+            const int h = ns_shift >= 0 ? wtask >> ns_shift : wtask / kp.n_start;
             const uint32_t* slot = c.slotw + h * N;
             const uint8_t* srcb = c.bind_src + (size_t)wtask * N;
             const uint8_t* dstb = c.bind_dst + (size_t)wtask * N;
