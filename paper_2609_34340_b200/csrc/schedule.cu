@@ -180,33 +180,27 @@ __device__ __forceinline__ bool util_greater(int64_t f1, int64_t d1, int64_t f2,
 // (c[p0][0] + c[p1][1]) + (c[p2][2] + c[p3][3]), which the compiler shares between permutations: 30 additions
 // instead of 36.  Both lanes run the same code on the permutations that start with row 0 or 1; lane 1 sees the
 // rows rotated by two, so it covers the permutations that start with row 2 or 3, and tags each value with the
-// lexicographic index of the real permutation so that the first maximum still wins.
-__host__ __device__ constexpr int perm_rank4(int a, int b, int c2, int d) {      // lexicographic index of (a, b, c2, d)
-    int r = 0;
-    const int v[4] = {a, b, c2, d};
-    for (int i = 0; i < 4; i++) {
-        int smaller = 0;
-        for (int j = i + 1; j < 4; j++) smaller += v[j] < v[i];
-        int f = 1;
-        for (int k = 2; k <= 3 - i; k++) f *= k;
-        r += smaller * f;
-    }
-    return r;
-}
-template <int P> struct RotRank {         // index of the permutation P with every row rotated by two
-    static constexpr int value = perm_rank4((perm_entry(4, P, 0) + 2) & 3, (perm_entry(4, P, 1) + 2) & 3,
-                                            (perm_entry(4, P, 2) + 2) & 3, (perm_entry(4, P, 3) + 2) & 3);
+// real permutation (as a byte, see below) so that the first maximum still wins.
+// A permutation as one byte with position 0 in the two highest bits: as a number this grows with the lexicographic
+// order, so 255 - byte is a tag that makes "larger key" mean "larger sum, then earlier permutation", and the byte
+// itself says which row goes to which position (no table needed to decode it).
+__host__ __device__ constexpr unsigned perm_byte(int a, int b, int c2, int d) { return (unsigned)(a << 6 | b << 4 | c2 << 2 | d); }
+template <int P, int ROT> struct RotByte {         // the permutation P with every row rotated by ROT
+    static constexpr unsigned value = perm_byte((perm_entry(4, P, 0) + ROT) & 3, (perm_entry(4, P, 1) + ROT) & 3,
+                                                (perm_entry(4, P, 2) + ROT) & 3, (perm_entry(4, P, 3) + ROT) & 3);
 };
+// row placed at position q by a permutation byte
+__device__ __forceinline__ int perm_byte_at(unsigned b, int q) { return (int)((b >> (6 - 2 * q)) & 3u); }
 template <int... P>
 __device__ __forceinline__ uint32_t reg2_best_impl(const uint32_t (&c)[4][4], int tl, std::integer_sequence<int, P...>) {
     uint32_t key = 0;
     ((key = max_v(key, (((c[PermAt<4, P, 0>::value][0] + c[PermAt<4, P, 1>::value][1]) +
-                         (c[PermAt<4, P, 2>::value][2] + c[PermAt<4, P, 3>::value][3])) << 5) +
-                           (uint32_t)(tl ? 31 - RotRank<P>::value : 31 - P))),
+                         (c[PermAt<4, P, 2>::value][2] + c[PermAt<4, P, 3>::value][3])) << 8) +
+                           (uint32_t)(tl ? 255 - RotByte<P, 2>::value : 255 - RotByte<P, 0>::value))),
      ...);
     return key;
 }
-__device__ __forceinline__ uint32_t team_best_reg2(const uint32_t* cred, int tl, const uint8_t* lut, unsigned& bpk) {
+__device__ __forceinline__ uint32_t team_best_reg2(const uint32_t* cred, int tl, unsigned& bpk) {
     uint32_t c[4][4];
 #pragma unroll
     for (int r = 0; r < 4; r++) {
@@ -216,19 +210,19 @@ __device__ __forceinline__ uint32_t team_best_reg2(const uint32_t* cred, int tl,
     }
     uint32_t key = reg2_best_impl(c, tl, std::make_integer_sequence<int, 12>{});
     key = max_v(key, __shfl_xor_sync(0xffffffffu, key, 1));
-    bpk = lut[key & 31u];
-    return key >> 5;
+    bpk = ~key & 255u;
+    return key >> 8;
 }
 
 // Eight lanes per group, 32-bit granule units.  Team lane tl evaluates the three permutations 3 tl .. 3 tl + 2.
 // Seen through a relabelling of the rows that depends on the lane only -- row 0 -> tl / 2, the other three
 // ascending for even lanes and descending for odd lanes -- these are always the permutations (0,1,2,3), (0,1,3,2)
 // and (0,2,1,3): every lane runs the same straight-line code on eight credits at fixed offsets from four row
-// pointers (instead of twelve indexed loads), shares the pair sums, and tags value P with the lexicographic
-// index of the real permutation, 6 (tl / 2) + P for even and 6 (tl / 2) + 5 - P for odd lanes.
+// pointers (instead of twelve indexed loads), shares the pair sums, and tags value P with the real permutation
+// (255 - its byte, see perm_byte).
 struct Reg8Lane {
     unsigned row[4];      // offset of relabelled row r in the tile, in credits
-    uint32_t tag[3];      // 31 - real permutation index of P = 0, 1, 2
+    uint32_t tag[3];      // 255 - byte of the real permutation behind P = 0, 1, 2
 };
 __device__ __forceinline__ Reg8Lane reg8_lane(int tl) {
     Reg8Lane L;
@@ -238,30 +232,31 @@ __device__ __forceinline__ Reg8Lane reg8_lane(int tl) {
     L.row[1] = (unsigned)(odd ? rest2 : rest0) * 4;
     L.row[2] = (unsigned)rest1 * 4;
     L.row[3] = (unsigned)(odd ? rest0 : rest2) * 4;
-#pragma unroll
-    for (int P = 0; P < 3; P++) L.tag[P] = (uint32_t)(31 - (6 * a + (odd ? 5 - P : P)));
+    const int R0 = a, R1 = odd ? rest2 : rest0, R2 = rest1, R3 = odd ? rest0 : rest2;    // real rows behind 0, 1, 2, 3
+    L.tag[0] = 255u - perm_byte(R0, R1, R2, R3);
+    L.tag[1] = 255u - perm_byte(R0, R1, R3, R2);
+    L.tag[2] = 255u - perm_byte(R0, R2, R1, R3);
     return L;
 }
-// key = max over the lane's three permutations of (sum << 5 | tag); cred points at the team's tile
+// key = max over the lane's three permutations of (sum << 8 | tag); cred points at the team's tile
 __device__ __forceinline__ uint32_t reg8_key(const uint32_t* cred, const Reg8Lane& L) {
     const uint32_t *r0 = cred + L.row[0], *r1 = cred + L.row[1], *r2 = cred + L.row[2], *r3 = cred + L.row[3];
     const uint32_t c00 = r0[0], c11 = r1[1], c21 = r2[1], c12 = r1[2], c22 = r2[2], c32 = r3[2], c23 = r2[3], c33 = r3[3];
     const uint32_t a01 = c00 + c11;
     const uint32_t v0 = a01 + (c22 + c33), v1 = a01 + (c32 + c23), v2 = (c00 + c21) + (c12 + c33);
-    return max_v(max_v((v0 << 5) + L.tag[0], (v1 << 5) + L.tag[1]), (v2 << 5) + L.tag[2]);
+    return max_v(max_v((v0 << 8) + L.tag[0], (v1 << 8) + L.tag[1]), (v2 << 8) + L.tag[2]);
 }
 
 // Four lanes per group, 32-bit granule units.  Team lane tl evaluates the six permutations that start with row tl.
 // With the rows rotated by tl these are the six permutations that start with row 0: every lane runs the same code on
-// ten credits at fixed offsets and six pair sums, and tags value P with the index of the real permutation.
+// ten credits at fixed offsets and six pair sums, and tags value P with the real permutation (255 - its byte).
 struct Reg4Lane {
     unsigned row[4];      // offset of rotated row r in the tile, in credits
-    uint32_t tag[6];      // 31 - real permutation index of P = 0 .. 5
+    uint32_t tag[6];      // 255 - byte of the real permutation behind P = 0 .. 5
 };
 template <int... P>
 __device__ __forceinline__ void reg4_tags(Reg4Lane& L, int tl, std::integer_sequence<int, P...>) {
-    ((L.tag[P] = (uint32_t)(31 - perm_rank4(tl, (perm_entry(4, P, 1) + tl) & 3, (perm_entry(4, P, 2) + tl) & 3,
-                                            (perm_entry(4, P, 3) + tl) & 3))),
+    ((L.tag[P] = 255u - perm_byte(tl, (perm_entry(4, P, 1) + tl) & 3, (perm_entry(4, P, 2) + tl) & 3, (perm_entry(4, P, 3) + tl) & 3)),
      ...);
 }
 __device__ __forceinline__ Reg4Lane reg4_lane(int tl) {
@@ -278,9 +273,9 @@ __device__ __forceinline__ uint32_t reg4_key(const uint32_t* cred, const Reg4Lan
     const uint32_t c12 = r1[2], c22 = r2[2], c32 = r3[2], c13 = r1[3], c23 = r2[3], c33 = r3[3];
     const uint32_t v0 = a1 + (c22 + c33), v1 = a1 + (c32 + c23), v2 = a2 + (c12 + c33), v3 = a2 + (c32 + c13),
                    v4 = a3 + (c12 + c23), v5 = a3 + (c22 + c13);
-    uint32_t key = max_v((v0 << 5) + L.tag[0], (v1 << 5) + L.tag[1]);
-    key = max_v(key, max_v((v2 << 5) + L.tag[2], (v3 << 5) + L.tag[3]));
-    return max_v(key, max_v((v4 << 5) + L.tag[4], (v5 << 5) + L.tag[5]));
+    uint32_t key = max_v((v0 << 8) + L.tag[0], (v1 << 8) + L.tag[1]);
+    key = max_v(key, max_v((v2 << 8) + L.tag[2], (v3 << 8) + L.tag[3]));
+    return max_v(key, max_v((v4 << 8) + L.tag[4], (v5 << 8) + L.tag[5]));
 }
 
 // ---- team path (groups of four ranks, LPG lanes per group) -----------------------------------------
@@ -320,47 +315,39 @@ __device__ __forceinline__ int64_t team_best(const int64_t* cred, int tl, const 
     }
     return best;
 }
-// 32-bit granule units: value and permutation travel as one key (sum << 5 | 31 - p), so a plain maximum
-// keeps the larger sum and, among equal sums, the lower permutation index.  Sums are below 2^27.
-// pidx[pp][q] is the tile element (row * 4 + q) the lane's pp-th permutation reads at position q; lut maps
-// the 5-bit tag back to the packed permutation.
+// 32-bit granule units: value and permutation travel as one key (sum << 8 | 255 - permutation byte), so a plain
+// maximum keeps the larger sum and, among equal sums, the earlier permutation.  Sums are below 2^24.  The
+// permutation comes back as its byte (position 0 in the highest two bits, see perm_byte_at).
 template <int LPG>
 __device__ __forceinline__ uint32_t team_best(const uint32_t* cred, int tl, const unsigned (&mp)[TeamCfg<LPG>::NW],
                                               const uint8_t (&pidx)[TeamCfg<LPG>::PPL][4], const uint8_t* lut,
                                               unsigned& bpk) {
-    constexpr int PPL = TeamCfg<LPG>::PPL;
-    if constexpr (LPG == 2) return team_best_reg2(cred, tl, lut, bpk);
+    static_assert(LPG == 2 || LPG == 4 || LPG == 8, "lane teams have two, four or eight lanes");
+    if constexpr (LPG == 2) return team_best_reg2(cred, tl, bpk);
+    uint32_t key;
     if constexpr (LPG == 4) {
-        uint32_t key = reg4_key(cred, reg4_lane(tl));
+        key = reg4_key(cred, reg4_lane(tl));
         key = max_v(key, __shfl_xor_sync(0xffffffffu, key, 2));
         key = max_v(key, __shfl_xor_sync(0xffffffffu, key, 1));
-        bpk = lut[key & 31u];
-        return key >> 5;
-    }
-    if constexpr (LPG == 8) {
-        uint32_t key = reg8_key(cred, reg8_lane(tl));
+    } else {
+        key = reg8_key(cred, reg8_lane(tl));
 #pragma unroll
         for (int o = 4; o; o >>= 1) key = max_v(key, __shfl_xor_sync(0xffffffffu, key, o));
-        bpk = lut[key & 31u];
-        return key >> 5;
     }
-    const uint32_t tag0 = (uint32_t)(31 - tl * PPL);
-    uint32_t key = 0;
-#pragma unroll
-    for (int pp = 0; pp < PPL; pp++) {
-        const uint32_t v = cred[pidx[pp][0]] + cred[pidx[pp][1]] + cred[pidx[pp][2]] + cred[pidx[pp][3]];
-        key = max_v(key, (v << 5) + (tag0 - pp));
-    }
-#pragma unroll
-    for (int o = LPG / 2; o; o >>= 1) key = max_v(key, __shfl_xor_sync(0xffffffffu, key, o));
-    bpk = lut[key & 31u];
-    return key >> 5;
+    bpk = ~key & 255u;
+    return key >> 8;
 }
 template <int LPG>
 __device__ __forceinline__ int64_t team_best(const int64_t* cred, int tl, const unsigned (&mp)[TeamCfg<LPG>::NW],
                                              const uint8_t (&pidx)[TeamCfg<LPG>::PPL][4], const uint8_t* lut,
                                              unsigned& bpk) {
     return team_best<LPG>(cred, tl, mp, bpk);
+}
+
+// Row that the permutation returned by team_best puts at position q: a byte with position 0 on top for 32-bit granule
+// units, two bits per position from the bottom for 64-bit byte values.
+template <typename V> __device__ __forceinline__ int perm_pos(unsigned bpk, int q) {
+    return sizeof(V) == 4 ? perm_byte_at(bpk, q) : (int)((bpk >> (2 * q)) & 3u);
 }
 
 // Per-CTA pointers and constants shared by the two value types.
@@ -589,7 +576,7 @@ __device__ __forceinline__ void decompose(const DevCat& dc, const KParams& kp, c
                     if (active && tl < (LPG < 4 ? LPG : 4)) {
 #pragma unroll
                         for (int kq = 0; kq < TC::NQ; kq++)
-                            srcb[a * 4 + qv[kq]] = (uint8_t)(a * 4 + ((bpk >> (2 * qv[kq])) & 3));
+                            srcb[a * 4 + qv[kq]] = (uint8_t)(a * 4 + perm_pos<V>(bpk, qv[kq]));
                     }
                     __syncwarp();
                     if (active) {                              // destination half: credits into group a
@@ -606,7 +593,7 @@ __device__ __forceinline__ void decompose(const DevCat& dc, const KParams& kp, c
                     if (active && tl < (LPG < 4 ? LPG : 4)) {
 #pragma unroll
                         for (int kq = 0; kq < TC::NQ; kq++)
-                            dstb[r_in[kq]] = (uint8_t)(a * 4 + ((bpk >> (2 * qv[kq])) & 3));
+                            dstb[r_in[kq]] = (uint8_t)(a * 4 + perm_pos<V>(bpk, qv[kq]));
                     }
                     // Eq. (8): sum over the teams.  Every lane of a team holds the team's value and the
                     // exchanges connect equal team lanes only, so all 32 lanes end with the same total.
@@ -629,7 +616,7 @@ __device__ __forceinline__ void decompose(const DevCat& dc, const KParams& kp, c
                 if (active && tl < (LPG < 4 ? LPG : 4)) {
 #pragma unroll
                     for (int kq = 0; kq < TC::NQ; kq++) {
-                        const V x = cred[((bpk >> (2 * qv[kq])) & 3) * 4 + qv[kq]];
+                        const V x = cred[perm_pos<V>(bpk, qv[kq]) * 4 + qv[kq]];
                         xmax = max_v(xmax, x);
                         tmax = max_v(tmax, (int64_t)x * c.tscale[cls_in[kq]]);
                     }
@@ -1034,8 +1021,8 @@ vp_schedule_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand, co
                     s_cap[cl] = cp < kp.granule ? kp.granule : cp;
                     cap_max = max_v(cap_max, s_cap[cl]);
                 }
-                // granule units: capacities below 2^25 granules, every entry below 2^32 granules
-                const int units = cap_max / kp.granule < ((int64_t)1 << 25) && kp.granule >= 256;
+                // granule units: capacities below 2^22 granules (four credits and a permutation byte share 32 bits)
+                const int units = cap_max / kp.granule < ((int64_t)1 << 22) && kp.granule >= 256;
                 for (int cl = 0; cl < dc.n_classes; cl++) {
                     s_cap32[cl] = (uint32_t)(units ? s_cap[cl] / kp.granule : 0);
                     s_tscale[cl] = dc.class_wdiv[cl] * (units ? kp.granule : 1);

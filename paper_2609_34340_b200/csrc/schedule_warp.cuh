@@ -82,7 +82,7 @@ __device__ __forceinline__ void team_best_x(const unsigned (&tile)[kWT], int tl,
         for (int t = 0; t < kWT; t++) key[t] = max_v(key[t], other[t]);
     }
 #pragma unroll
-    for (int t = 0; t < kWT; t++) { bpk[t] = ws<uint8_t>(o_lut)[key[t] & 31u]; val[t] = key[t] >> 5; }
+    for (int t = 0; t < kWT; t++) { bpk[t] = ~key[t] & 255u; val[t] = key[t] >> 8; }      // the permutation byte, the sum
 }
 __device__ __forceinline__ void team_best_x(const unsigned (&tile)[kWT], int tl, const uint8_t (&pidx)[3][4], unsigned o_lut,
                                             unsigned (&bpk)[kWT], int64_t (&val)[kWT]) {
@@ -249,7 +249,7 @@ __device__ __forceinline__ void decompose_warp(const DevCat& dc, const KParams& 
                 team_best_x(tile, tl, pidx, c.o_lut, bpk, val);
 #pragma unroll
                 for (int t = 0; t < kWT; t++)
-                    if (writer && (alive >> t & 1)) ws<uint8_t>(o_src[t])[a * 4 + q] = (uint8_t)(a * 4 + ((bpk[t] >> (2 * q)) & 3));
+                    if (writer && (alive >> t & 1)) ws<uint8_t>(o_src[t])[a * 4 + q] = (uint8_t)(a * 4 + perm_pos<V>(bpk[t], q));
                 __syncwarp();
                 // destination half: credits into destination group a from the current sources of its in-slots
 #pragma unroll
@@ -265,7 +265,7 @@ __device__ __forceinline__ void decompose_warp(const DevCat& dc, const KParams& 
                 team_best_x(tile, tl, pidx, c.o_lut, bpk, val);
 #pragma unroll
                 for (int t = 0; t < kWT; t++)
-                    if (writer && (alive >> t & 1)) *ws<uint8_t>(o_rin_d[t]) = (uint8_t)(a * 4 + ((bpk[t] >> (2 * q)) & 3));
+                    if (writer && (alive >> t & 1)) *ws<uint8_t>(o_rin_d[t]) = (uint8_t)(a * 4 + perm_pos<V>(bpk[t], q));
                 int64_t Fn[kWT];
                 team_totals(val, active && tl == 0, Fn);                                  // Eq. (8)
 #pragma unroll
@@ -287,7 +287,7 @@ __device__ __forceinline__ void decompose_warp(const DevCat& dc, const KParams& 
 #pragma unroll
                 for (int t = 0; t < kWT; t++) {
                     x[t] = 0;
-                    if (writer && (valid >> t & 1)) x[t] = ws<V>(tile[t])[((bpk_fin[t] >> (2 * q)) & 3) * 4 + q];
+                    if (writer && (valid >> t & 1)) x[t] = ws<V>(tile[t])[perm_pos<V>(bpk_fin[t], q) * 4 + q];
                 }
                 if (sizeof(V) == 4 && dc.n_classes == 1) {      // one path rate: the slowest lane carries the largest volume
                     const int64_t ts = ws<int64_t>(c.o_tscale)[0];
@@ -515,8 +515,8 @@ vp_schedule_warp_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ deman
                 cap_max = max_v(cap_max, cp);
                 if (lane == 0) cap64[cl] = cp;
             }
-            // granule units: capacities below 2^25 granules, every entry below 2^32 granules
-            const bool units = cap_max / kp.granule < ((int64_t)1 << 25) && kp.granule >= 256;
+            // granule units: capacities below 2^22 granules (four credits and a permutation byte share 32 bits)
+            const bool units = cap_max / kp.granule < ((int64_t)1 << 22) && kp.granule >= 256;
             __syncwarp();
             if (lane < dc.n_classes) {
                 cap32[lane] = (uint32_t)(units ? cap64[lane] / kp.granule : 0);
