@@ -418,6 +418,15 @@ __device__ __forceinline__ void decompose(const DevCat& dc, const KParams& kp, c
     const int ns_shift = (kp.n_start & (kp.n_start - 1)) == 0 ? 31 - __clz(kp.n_start) : -1;     // n_start a power of two: shifts for divisions
 
     const bool inc = kp.incremental != 0;
+    // Small plain score tables (at most 16 D-hat cells, one shape per thread): the shape's lane counts are kept in a
+    // register, four bits per cell, and scoring needs no term loads (see phase A).  Cells beyond G*G have count 0.
+    const bool dense = LPG == 8 && !dc.sym && dc.tbl_size <= 16 && dc.n_shapes <= NT && ((uintptr_t)c.Dhat & 15) == 0;
+    unsigned long long shape_mask = 0;
+    if (LPG == 8 && dense && tid < dc.n_shapes)
+        for (int e = 0; e < dc.max_terms; e++) {
+            const uint32_t w = __ldg(&dc.term[(size_t)tid * dc.max_terms + e]);
+            shape_mask |= (unsigned long long)(w >> 16) << (4 * ((w & 0xffffu) >> 3));
+        }
     // a score is at most g x (what is left) and only shrinks: when that fits 32 bits the scores are kept as 32-bit
     // words, which shared memory can add to natively (64-bit adds are compare-and-swap loops)
     const bool s32 = inc && left * GS < ((int64_t)1 << 31);
@@ -472,6 +481,18 @@ __device__ __forceinline__ void decompose(const DevCat& dc, const KParams& kp, c
             const char* tb = (const char*)c.tbl;
             // a score is at most g x (what is left): when that fits 32 bits the low words of the table suffice
             const bool narrow = left * GS < ((int64_t)1 << 31);
+            if (LPG == 8 && dense && narrow) {
+                // one shape per thread, its lane counts in a register (a nibble per D-hat cell): sixteen multiply-adds
+                // on the low words of D-hat, which eight 16-byte loads (the same for every thread) bring in
+                const uint4* dh = (const uint4*)c.Dhat;
+                uint32_t sc = 0;
+#pragma unroll
+                for (int v = 0; v < 8; v++) {
+                    const uint4 x = dh[v];
+                    sc += x.x * (uint32_t)((shape_mask >> (8 * v)) & 15u) + x.z * (uint32_t)((shape_mask >> (8 * v + 4)) & 15u);
+                }
+                if (tid < dc.n_shapes) { best = (int64_t)sc; best_s = tid; }
+            } else
             for (int s = tid; s < dc.n_shapes; s += NT) {
                 const uint32_t* tp = c.p_term + (size_t)s * c.term_ss;
                 int64_t score = 0;
