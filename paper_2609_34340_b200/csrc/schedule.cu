@@ -565,53 +565,48 @@ __device__ __forceinline__ void decompose(const DevCat& dc, const KParams& kp, c
             bool tmax_done = false;
             if constexpr (LPG > 1) {
                 // team path: one rank group per team of LPG lanes (G <= 32 / LPG)
+                // Teams beyond the last group repeat the last group's work on a tile of their own (same values to the same
+                // binding entries), so the code below needs no per-team predicates; only the sum over teams leaves them out.
                 const bool active = team < G;
-                const int a = team;               // the team's group: source group, then destination group
+                const int a = active ? team : G - 1;        // the team's group: source group, then destination group
                 V cap_out[TC::NQ], cap_in[TC::NQ];
                 int r_in[TC::NQ], cls_in[TC::NQ];
 #pragma unroll
                 for (int kq = 0; kq < TC::NQ; kq++) {
-                    cap_out[kq] = 0; cap_in[kq] = 0; r_in[kq] = 0; cls_in[kq] = 0;
-                    if (active) {
-                        const unsigned w = fin[a * 4 + qv[kq]];
-                        cap_out[kq] = cap[fcls[a * 4 + qv[kq]]];
-                        cls_in[kq] = (int)(w >> 8);
-                        cap_in[kq] = cap[cls_in[kq]];
-                        r_in[kq] = (int)(w & 0xff);
-                    }
+                    const unsigned w = fin[a * 4 + qv[kq]];
+                    cap_out[kq] = cap[fcls[a * 4 + qv[kq]]];
+                    cls_in[kq] = (int)(w >> 8);
+                    cap_in[kq] = cap[cls_in[kq]];
+                    r_in[kq] = (int)(w & 0xff);
                 }
                 __syncwarp();
                 unsigned bpk = 0;
                 for (int sweep = 0; sweep < kp.i_aa; sweep++) {
-                    if (active) {                              // source half: credits of source group a
 #pragma unroll
-                        for (int kq = 0; kq < TC::NQ; kq++) {
-                            const int dq = dstb[a * 4 + qv[kq]];
+                    for (int kq = 0; kq < TC::NQ; kq++) {      // source half: credits of source group a
+                        const int dq = dstb[a * 4 + qv[kq]];
 #pragma unroll
-                            for (int m = 0; m < TC::NI; m++)
-                                cred[iv[m] * 4 + qv[kq]] = min_v(Drem[(size_t)(a * 4 + iv[m]) * N + dq], cap_out[kq]);
-                        }
+                        for (int m = 0; m < TC::NI; m++)
+                            cred[iv[m] * 4 + qv[kq]] = min_v(Drem[(size_t)(a * 4 + iv[m]) * N + dq], cap_out[kq]);
                     }
                     __syncwarp();
                     team_best<LPG>(cred, tl, mp, pidx, c.perm_lut, bpk);
-                    if (active && tl < (LPG < 4 ? LPG : 4)) {
+                    if (tl < (LPG < 4 ? LPG : 4)) {
 #pragma unroll
                         for (int kq = 0; kq < TC::NQ; kq++)
                             srcb[a * 4 + qv[kq]] = (uint8_t)(a * 4 + perm_pos<V>(bpk, qv[kq]));
                     }
                     __syncwarp();
-                    if (active) {                              // destination half: credits into group a
 #pragma unroll
-                        for (int kq = 0; kq < TC::NQ; kq++) {
-                            const int sq = srcb[r_in[kq]];
+                    for (int kq = 0; kq < TC::NQ; kq++) {      // destination half: credits into group a
+                        const int sq = srcb[r_in[kq]];
 #pragma unroll
-                            for (int m = 0; m < TC::NI; m++)
-                                cred[iv[m] * 4 + qv[kq]] = min_v(Drem[(size_t)sq * N + a * 4 + iv[m]], cap_in[kq]);
-                        }
+                        for (int m = 0; m < TC::NI; m++)
+                            cred[iv[m] * 4 + qv[kq]] = min_v(Drem[(size_t)sq * N + a * 4 + iv[m]], cap_in[kq]);
                     }
                     __syncwarp();
                     const V v = team_best<LPG>(cred, tl, mp, pidx, c.perm_lut, bpk);
-                    if (active && tl < (LPG < 4 ? LPG : 4)) {
+                    if (tl < (LPG < 4 ? LPG : 4)) {
 #pragma unroll
                         for (int kq = 0; kq < TC::NQ; kq++)
                             dstb[r_in[kq]] = (uint8_t)(a * 4 + perm_pos<V>(bpk, qv[kq]));
@@ -634,7 +629,7 @@ __device__ __forceinline__ void decompose(const DevCat& dc, const KParams& kp, c
                 }
                 // Eq. (9) volumes are the chosen credits of the last destination half; slowest lane of Eq. (10)
                 V xmax = 0;
-                if (active && tl < (LPG < 4 ? LPG : 4)) {
+                if (tl < (LPG < 4 ? LPG : 4)) {
 #pragma unroll
                     for (int kq = 0; kq < TC::NQ; kq++) {
                         const V x = cred[perm_pos<V>(bpk, qv[kq]) * 4 + qv[kq]];
