@@ -591,11 +591,9 @@ __device__ __forceinline__ void decompose(const DevCat& dc, const KParams& kp, c
                     }
                     __syncwarp();
                     team_best<LPG>(cred, tl, mp, pidx, c.perm_lut, bpk);
-                    if (tl < (LPG < 4 ? LPG : 4)) {
 #pragma unroll
-                        for (int kq = 0; kq < TC::NQ; kq++)
-                            srcb[a * 4 + qv[kq]] = (uint8_t)(a * 4 + perm_pos<V>(bpk, qv[kq]));
-                    }
+                    for (int kq = 0; kq < TC::NQ; kq++)          // (with eight lanes, lanes tl and tl + 4 write the same entry)
+                        srcb[a * 4 + qv[kq]] = (uint8_t)(a * 4 + perm_pos<V>(bpk, qv[kq]));
                     __syncwarp();
 #pragma unroll
                     for (int kq = 0; kq < TC::NQ; kq++) {      // destination half: credits into group a
@@ -606,11 +604,9 @@ __device__ __forceinline__ void decompose(const DevCat& dc, const KParams& kp, c
                     }
                     __syncwarp();
                     const V v = team_best<LPG>(cred, tl, mp, pidx, c.perm_lut, bpk);
-                    if (tl < (LPG < 4 ? LPG : 4)) {
 #pragma unroll
-                        for (int kq = 0; kq < TC::NQ; kq++)
-                            dstb[r_in[kq]] = (uint8_t)(a * 4 + perm_pos<V>(bpk, qv[kq]));
-                    }
+                    for (int kq = 0; kq < TC::NQ; kq++)
+                        dstb[r_in[kq]] = (uint8_t)(a * 4 + perm_pos<V>(bpk, qv[kq]));
                     // Eq. (8): sum over the teams.  Every lane of a team holds the team's value and the
                     // exchanges connect equal team lanes only, so all 32 lanes end with the same total.
                     if constexpr (sizeof(V) == 4) {
@@ -629,13 +625,11 @@ __device__ __forceinline__ void decompose(const DevCat& dc, const KParams& kp, c
                 }
                 // Eq. (9) volumes are the chosen credits of the last destination half; slowest lane of Eq. (10)
                 V xmax = 0;
-                if (tl < (LPG < 4 ? LPG : 4)) {
 #pragma unroll
-                    for (int kq = 0; kq < TC::NQ; kq++) {
-                        const V x = cred[perm_pos<V>(bpk, qv[kq]) * 4 + qv[kq]];
-                        xmax = max_v(xmax, x);
-                        tmax = max_v(tmax, (int64_t)x * c.tscale[cls_in[kq]]);
-                    }
+                for (int kq = 0; kq < TC::NQ; kq++) {
+                    const V x = cred[perm_pos<V>(bpk, qv[kq]) * 4 + qv[kq]];
+                    xmax = max_v(xmax, x);
+                    tmax = max_v(tmax, (int64_t)x * c.tscale[cls_in[kq]]);
                 }
                 if constexpr (sizeof(V) == 4) {
                     if (dc.n_classes == 1) {          // one path rate: the slowest lane carries the largest volume
