@@ -770,22 +770,17 @@ __device__ __forceinline__ void decompose(const DevCat& dc, const KParams& kp, c
                 const uint32_t w = slot[r];
                 const int i = srcb[r], j = dstb[r];
                 const V x = min_v(cap[(w >> 24) & 0xf], Drem[(size_t)i * N + j]);
-                int64_t sa = c.send_acc[i], ra = c.recv_acc[j];
-                if (x > 0) {
-                    const int64_t bytes = (int64_t)x * unit;
-                    c.lane_dst_b[row + i] = (int16_t)j;
-                    c.lane_inst_b[row + i] = (uint16_t)(w & 0xffffu);
-                    c.lane_bytes_b[row + i] = bytes;
-                    Drem[(size_t)i * N + j] -= x;
-                    atomicAdd((unsigned long long*)&c.Dhat[(i / GS) * G + (j / GS)], (unsigned long long)(-(int64_t)x));
-                    sa += bytes; ra += bytes;
-                    c.send_acc[i] = sa;
-                    c.recv_acc[j] = ra;
-                } else {
-                    c.lane_dst_b[row + i] = -1;
-                    c.lane_inst_b[row + i] = 0xFFFF;
-                    c.lane_bytes_b[row + i] = 0;
-                }
+                // straight-line: an idle lane (x = 0) writes the idle values and adds zero; only the D-hat update is skipped
+                const bool busy = x > 0;
+                const int64_t bytes = (int64_t)x * unit;
+                const int64_t sa = c.send_acc[i] + bytes, ra = c.recv_acc[j] + bytes;
+                c.lane_dst_b[row + i] = busy ? (int16_t)j : (int16_t)-1;
+                c.lane_inst_b[row + i] = busy ? (uint16_t)(w & 0xffffu) : (uint16_t)0xFFFF;
+                c.lane_bytes_b[row + i] = bytes;
+                Drem[(size_t)i * N + j] -= x;
+                c.send_acc[i] = sa;
+                c.recv_acc[j] = ra;
+                if (busy) atomicAdd((unsigned long long*)&c.Dhat[(i / GS) * G + (j / GS)], (unsigned long long)(-(int64_t)x));
                 c.send_off_b[orow + i] = sa;              // src and dst are permutations: every rank is written once
                 if (c.recv_off_b) c.recv_off_b[orow + j] = ra;
             }
