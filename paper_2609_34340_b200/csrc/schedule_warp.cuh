@@ -147,9 +147,8 @@ __device__ __forceinline__ void decompose_warp(const DevCat& dc, const KParams& 
     const int ns_pad = (dc.n_shapes + 31) & ~31;         // row stride of the transposed term table
     const int team = lane >> 3, tl = lane & 7;
     const bool active = team < G;
-    const int a = active ? team : 0;                     // the team's group: source group, then destination group
+    const int a = active ? team : G - 1;                 // the team's group (spare teams repeat the last group on their own tiles)
     const int q = tl & 3, i0 = tl >> 2, i1 = i0 + 2;     // the lane's credit elements: (i0, q) and (i1, q)
-    const bool writer = active && tl < 4;                // the lane that records slot q of its group
     const bool ns4 = kp.n_start == 4;
     V* const Drem = ws<V>(c.o_drem);
     const V* const cap = ws<V>(c.o_cap);
@@ -244,12 +243,12 @@ __device__ __forceinline__ void decompose_warp(const DevCat& dc, const KParams& 
                 }
 #pragma unroll
                 for (int t = 0; t < kWT; t++)
-                    if (active && (alive >> t & 1)) { ws<V>(tile[t])[i0 * 4 + q] = v0[t]; ws<V>(tile[t])[i1 * 4 + q] = v1[t]; }
+                    if (alive >> t & 1) { ws<V>(tile[t])[i0 * 4 + q] = v0[t]; ws<V>(tile[t])[i1 * 4 + q] = v1[t]; }
                 __syncwarp();
                 team_best_x(tile, tl, pidx, c.o_lut, bpk, val);
 #pragma unroll
                 for (int t = 0; t < kWT; t++)
-                    if (writer && (alive >> t & 1)) ws<uint8_t>(o_src[t])[a * 4 + q] = (uint8_t)(a * 4 + perm_pos<V>(bpk[t], q));
+                    if (alive >> t & 1) ws<uint8_t>(o_src[t])[a * 4 + q] = (uint8_t)(a * 4 + perm_pos<V>(bpk[t], q));
                 __syncwarp();
                 // destination half: credits into destination group a from the current sources of its in-slots
 #pragma unroll
@@ -260,12 +259,12 @@ __device__ __forceinline__ void decompose_warp(const DevCat& dc, const KParams& 
                 }
 #pragma unroll
                 for (int t = 0; t < kWT; t++)
-                    if (active && (alive >> t & 1)) { ws<V>(tile[t])[i0 * 4 + q] = v0[t]; ws<V>(tile[t])[i1 * 4 + q] = v1[t]; }
+                    if (alive >> t & 1) { ws<V>(tile[t])[i0 * 4 + q] = v0[t]; ws<V>(tile[t])[i1 * 4 + q] = v1[t]; }
                 __syncwarp();
                 team_best_x(tile, tl, pidx, c.o_lut, bpk, val);
 #pragma unroll
                 for (int t = 0; t < kWT; t++)
-                    if (writer && (alive >> t & 1)) *ws<uint8_t>(o_rin_d[t]) = (uint8_t)(a * 4 + perm_pos<V>(bpk[t], q));
+                    if (alive >> t & 1) *ws<uint8_t>(o_rin_d[t]) = (uint8_t)(a * 4 + perm_pos<V>(bpk[t], q));
                 int64_t Fn[kWT];
                 team_totals(val, active && tl == 0, Fn);                                  // Eq. (8)
 #pragma unroll
@@ -287,7 +286,7 @@ __device__ __forceinline__ void decompose_warp(const DevCat& dc, const KParams& 
 #pragma unroll
                 for (int t = 0; t < kWT; t++) {
                     x[t] = 0;
-                    if (writer && (valid >> t & 1)) x[t] = ws<V>(tile[t])[perm_pos<V>(bpk_fin[t], q) * 4 + q];
+                    if (valid >> t & 1) x[t] = ws<V>(tile[t])[perm_pos<V>(bpk_fin[t], q) * 4 + q];
                 }
                 if (sizeof(V) == 4 && dc.n_classes == 1) {      // one path rate: the slowest lane carries the largest volume
                     const int64_t ts = ws<int64_t>(c.o_tscale)[0];
@@ -325,21 +324,16 @@ __device__ __forceinline__ void decompose_warp(const DevCat& dc, const KParams& 
                 const uint32_t w = ws<uint32_t>(c.o_fam_slot)[(f0 + h) * N + r];
                 const int i = ws<uint8_t>(c.o_bind_src)[bt * N + r], j = ws<uint8_t>(c.o_bind_dst)[bt * N + r];
                 const V x = min_v(cap[(w >> 24) & 0xf], Drem[i * ld + j]);
-                int64_t sa = ws<int64_t>(c.o_send_acc)[i], ra = ws<int64_t>(c.o_recv_acc)[j];
-                if (x > 0) {
-                    const int64_t bytes = (int64_t)x * unit;
-                    c.lane_dst_b[row + i] = (int16_t)j;
-                    c.lane_inst_b[row + i] = (uint16_t)(w & 0xffffu);
-                    c.lane_bytes_b[row + i] = bytes;
-                    Drem[i * ld + j] -= x;
-                    sa += bytes; ra += bytes;
-                    ws<int64_t>(c.o_send_acc)[i] = sa;
-                    ws<int64_t>(c.o_recv_acc)[j] = ra;
-                } else {
-                    c.lane_dst_b[row + i] = -1;
-                    c.lane_inst_b[row + i] = 0xFFFF;
-                    c.lane_bytes_b[row + i] = 0;
-                }
+                // straight-line: an idle lane (x = 0) writes the idle values and adds zero
+                const bool busy = x > 0;
+                const int64_t bytes = (int64_t)x * unit;
+                const int64_t sa = ws<int64_t>(c.o_send_acc)[i] + bytes, ra = ws<int64_t>(c.o_recv_acc)[j] + bytes;
+                c.lane_dst_b[row + i] = busy ? (int16_t)j : (int16_t)-1;
+                c.lane_inst_b[row + i] = busy ? (uint16_t)(w & 0xffffu) : (uint16_t)0xFFFF;
+                c.lane_bytes_b[row + i] = bytes;
+                Drem[i * ld + j] -= x;
+                ws<int64_t>(c.o_send_acc)[i] = sa;
+                ws<int64_t>(c.o_recv_acc)[j] = ra;
                 c.send_off_b[orow + i] = sa;
                 if (c.recv_off_b) c.recv_off_b[orow + j] = ra;
             }
