@@ -475,12 +475,13 @@ __device__ __forceinline__ void decompose(const DevCat& dc, const KParams& kp, c
         if (k == kp.k_max) { st |= VP_ST_STEP_LIMIT; break; }
         // (A) Eq. (6): shape scores, first maximum
         if (dc.sym && !inc) build_table();
+        // a score is at most g x (what is left): when that fits 32 bits the low words of the table suffice, and a cell of
+        // D-hat can be decremented by a native 32-bit shared-memory add (a 64-bit one is a compare-and-swap loop)
+        const bool narrow = left * GS < ((int64_t)1 << 31);
         if (warp < n_score_warps) {
             int64_t best = -1;
             int best_s = 0x7fffffff;
             const char* tb = (const char*)c.tbl;
-            // a score is at most g x (what is left): when that fits 32 bits the low words of the table suffice
-            const bool narrow = left * GS < ((int64_t)1 << 31);
             if (LPG == 8 && dense && narrow) {
                 // one shape per thread, its lane counts in a register (a nibble per D-hat cell): sixteen multiply-adds
                 // on the low words of D-hat, which eight 16-byte loads (the same for every thread) bring in
@@ -780,7 +781,11 @@ __device__ __forceinline__ void decompose(const DevCat& dc, const KParams& kp, c
                 Drem[(size_t)i * N + j] -= x;
                 c.send_acc[i] = sa;
                 c.recv_acc[j] = ra;
-                if (busy) atomicAdd((unsigned long long*)&c.Dhat[(i / GS) * G + (j / GS)], (unsigned long long)(-(int64_t)x));
+                if (busy) {
+                    int64_t* cell = &c.Dhat[(i / GS) * G + (j / GS)];
+                    if (narrow) atomicSub((unsigned int*)cell, (unsigned int)x);        // high word is zero, low word >= x
+                    else atomicAdd((unsigned long long*)cell, (unsigned long long)(-(int64_t)x));
+                }
                 c.send_off_b[orow + i] = sa;              // src and dst are permutations: every rank is written once
                 if (c.recv_off_b) c.recv_off_b[orow + j] = ra;
             }
