@@ -33,7 +33,7 @@ UNIT = "matrices/s"
 INT64_OPS_PER_LANE_CLK = 0.5    # one 64-bit add/min/compare needs two 32-bit ALU issues
 SM_COUNT, LANES_PER_SM = 148, 128
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch on the default workload (ncu, see profiles/)
-NCU_DRAM_BYTES_PER_LAUNCH = {"pack_copy_bulk_kernel": 235_565_824 + 1_791_358_000, "vp_schedule_kernel": 633_344 + 0}
+NCU_DRAM_BYTES_PER_LAUNCH = {"pack_copy_bulk_kernel": 235_441_664 + 1_791_668_000, "vp_schedule_kernel": 646_656 + 0}
 
 
 def _dist_env():
@@ -286,7 +286,7 @@ def run_tools(vp, dev, peaks):
     large = {"workload": f"config 2 matrices x16: {B2} matrices N=16", "launch": vp.schedule_launch_info(dc2, B2, p2),
              "ms": round(ms_s, 4), "matrices_per_s": round(B2 / ms_s * 1e3, 1),
              "alu_frac": round(ops2 / (ms_s * 1e-3) / alu_peak, 4),
-             "ncu": {"issue_active_pct": 55.8, "shared_wavefronts_pct_of_peak": 56.1, "lsu_pipe_pct": 48.8,
+             "ncu": {"issue_active_pct": 57.1, "shared_wavefronts_pct_of_peak": 53.9, "lsu_pipe_pct": 45.7,
                      "source": "profiles/vp_schedule_warp_kernel_config2_x16.md"}}
     del plan2, D2
     ms_t = timed(lambda: vp.plan_time(dc, plan, w.lambda_ns, out=out))
