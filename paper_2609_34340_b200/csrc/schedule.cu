@@ -555,12 +555,19 @@ __device__ __forceinline__ void decompose(const DevCat& dc, const KParams& kp, c
             uint32_t slot_pre[(VP_MAX_N + 31) / 32];
             if (t == 0 && sub == 0) {
 #pragma unroll
-                for (int rr = 0; rr < (VP_MAX_N + 31) / 32; rr++)
+                for (int rr = 0; rr < (VP_MAX_N + 31) / 32; rr++) {
+                    if (rr * 32 >= N) break;
                     if (rr * 32 + lane < N) slot_pre[rr] = __ldg(&dc.fam_slot[(size_t)f * N + rr * 32 + lane]);
+                }
             }
-            for (int e = sub * 32 + lane; e < N; e += 32 * W) {      // in-slot e = d * GS + q: start t rotates q by t
-                const int q = e % GS;
+            if (N <= 32 && (N & (N - 1)) == 0) {                     // in-slot e = d * GS + q: start t rotates q by t
+                const int e = lane & (N - 1), q = e % GS;            // (lanes beyond N repeat the first N: no branch)
                 dstb[fin[e] & 0xff] = (uint8_t)(e - q + (q + t) % GS);
+            } else {
+                for (int e = sub * 32 + lane; e < N; e += 32 * W) {
+                    const int q = e % GS;
+                    dstb[fin[e] & 0xff] = (uint8_t)(e - q + (q + t) % GS);
+                }
             }
             int64_t F_old = -1, F_new = -1, tmax = 0;
             bool tmax_done = false;
@@ -711,8 +718,10 @@ __device__ __forceinline__ void decompose(const DevCat& dc, const KParams& kp, c
             if (sub == 0) cnt.tasks++;
             if (t == 0 && sub == 0) {
 #pragma unroll
-                for (int rr = 0; rr < (VP_MAX_N + 31) / 32; rr++)
+                for (int rr = 0; rr < (VP_MAX_N + 31) / 32; rr++) {
+                    if (rr * 32 >= N) break;
                     if (rr * 32 + lane < N) c.slotw[h * N + rr * 32 + lane] = slot_pre[rr];
+                }
             }
             if (lane == 0 && sub == 0) {
                 c.task_f[task] = F_new;
