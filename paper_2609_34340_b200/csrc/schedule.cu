@@ -556,18 +556,23 @@ __device__ __forceinline__ void decompose(const DevCat& dc, const KParams& kp, c
             if (t == 0 && sub == 0) {
 #pragma unroll
                 for (int rr = 0; rr < (VP_MAX_N + 31) / 32; rr++) {
-                    if (rr * 32 >= N) break;
+                    if (LPG > 1 && rr * 32 >= N) break;              // (lane teams: N <= 64, mostly one round)
                     if (rr * 32 + lane < N) slot_pre[rr] = __ldg(&dc.fam_slot[(size_t)f * N + rr * 32 + lane]);
                 }
             }
-            if (N <= 32 && (N & (N - 1)) == 0) {                     // in-slot e = d * GS + q: start t rotates q by t
+            // initial destination binding: in-slot e = d * GS + q, start t rotates q by t
+            if (LPG > 1 && N <= 32 && (N & (N - 1)) == 0) {
                 const int e = lane & (N - 1), q = e % GS;            // (lanes beyond N repeat the first N: no branch)
                 dstb[fin[e] & 0xff] = (uint8_t)(e - q + (q + t) % GS);
-            } else {
-                for (int e = sub * 32 + lane; e < N; e += 32 * W) {
+            } else if (LPG > 1) {
+                for (int e = lane; e < N; e += 32) {
                     const int q = e % GS;
                     dstb[fin[e] & 0xff] = (uint8_t)(e - q + (q + t) % GS);
                 }
+            } else {
+                for (int d = sub * 32 + lane; d < G; d += 32 * W)
+#pragma unroll
+                    for (int q = 0; q < GS; q++) dstb[fin[d * GS + q] & 0xff] = (uint8_t)(d * GS + (q + t) % GS);
             }
             int64_t F_old = -1, F_new = -1, tmax = 0;
             bool tmax_done = false;
@@ -719,7 +724,7 @@ __device__ __forceinline__ void decompose(const DevCat& dc, const KParams& kp, c
             if (t == 0 && sub == 0) {
 #pragma unroll
                 for (int rr = 0; rr < (VP_MAX_N + 31) / 32; rr++) {
-                    if (rr * 32 >= N) break;
+                    if (LPG > 1 && rr * 32 >= N) break;
                     if (rr * 32 + lane < N) c.slotw[h * N + rr * 32 + lane] = slot_pre[rr];
                 }
             }
@@ -787,10 +792,10 @@ __device__ __forceinline__ void decompose(const DevCat& dc, const KParams& kp, c
                 c.lane_dst_b[row + i] = busy ? (int16_t)j : (int16_t)-1;
                 c.lane_inst_b[row + i] = busy ? (uint16_t)(w & 0xffffu) : (uint16_t)0xFFFF;
                 c.lane_bytes_b[row + i] = bytes;
-                Drem[(size_t)i * N + j] -= x;
                 c.send_acc[i] = sa;
                 c.recv_acc[j] = ra;
                 if (busy) {
+                    Drem[(size_t)i * N + j] -= x;           // (for N = 256 this is a read-modify-write in L2: not for idle lanes)
                     int64_t* cell = &c.Dhat[(i / GS) * G + (j / GS)];
                     if (narrow) atomicSub((unsigned int*)cell, (unsigned int)x);        // high word is zero, low word >= x
                     else atomicAdd((unsigned long long*)cell, (unsigned long long)(-(int64_t)x));
