@@ -357,8 +357,10 @@ static int64_t best_assignment(const int64_t credit[VPO_MAX_G][VPO_MAX_G], int g
 /* ------------------------------------------------------- MultiStartAA */
 
 typedef struct {
-    int64_t *trace; int cap; int len;   /* optional records: (step, family, start, sweep, F) per AA sweep and
-                                           (step, family, -1, sum of volumes, W * duration) per candidate */
+    int64_t *trace; int cap; int len;   /* optional records: (step, family, start, sweep, F) per AA sweep,
+                                           (step, family, -2 - start, slot, src * 65536 + dst) for the binding a run
+                                           ends with, and (step, family, -1, sum of volumes, W * duration) per
+                                           candidate */
 } vpo_trace;
 
 /*
@@ -421,6 +423,11 @@ static int64_t multistart_aa(const vpo_catalog *c, int fam, const int64_t *Drem,
             if (F_new <= F_old) break;
             F_old = F_new;
         }
+        if (tr && tr->trace)                             /* tracing only: the binding this run ends with */
+            for (int r = 0; r < N && tr->len < tr->cap; r++) {
+                int64_t *o = &tr->trace[5 * (size_t)tr->len++];
+                o[0] = step; o[1] = fam; o[2] = -2 - t; o[3] = r; o[4] = (int64_t)src[r] * 65536 + dst[r];
+            }
         if (F_new > F_best) {
             F_best = F_new;
             memcpy(src_best, src, sizeof(int) * N);

@@ -178,7 +178,9 @@ class OracleCatalog:
         return out
 
     def schedule(self, D, params, tau_in: int = 0, trace_cap: int = 0) -> dict:
-        """One matrix; with ``trace_cap`` > 0 also returns (step, family, start, sweep, F) records."""
+        """One matrix; with ``trace_cap`` > 0 also returns the trace records: (step, family, start, sweep, F) per
+        AA sweep, (step, family, -2 - start, slot, src * 65536 + dst) for the binding each run ends with, and
+        (step, family, -1, sum of volumes, W * duration) per candidate."""
         lib = _load()
         D = np.ascontiguousarray(D, dtype=np.int64)
         N = self.N

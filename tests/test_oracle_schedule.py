@@ -278,3 +278,81 @@ def test_round_counts_on_the_configs(oracle_lib):
         single = oc.schedule_batch(c["demand"].numpy(), c["params"], threads=1)
         for k in ("n_steps", "chan_id", "lane_dst", "lane_inst", "lane_bytes", "send_off", "recv_off"):
             assert (out[k] == single[k]).all()
+
+
+def _aa_cases():
+    """(catalog, demand, params, tau) where the starts of MultiStartAA really differ: two or more groups and
+    sparse demand in a handful of small values, so that runs end at different sweeps, with different F and,
+    among equal F, with different bindings."""
+    rng = np.random.default_rng(77)
+    u = 64
+    for name, i_aa in [("node8", 1), ("node8", 5), ("two_nodes", 3), ("two_nodes", 5), ("g2_two_nodes", 5),
+                       ("node8_64_50", 2), ("template_4_nodes", 4)]:
+        cat = TOPOS[name]()
+        N = cat.topology.N
+        for density, hi in [(0.25, 2), (0.4, 5), (0.15, 9)]:
+            D = _random_demand(rng, N, u, hi, density)
+            if D.any():
+                yield cat, D, SchedParams(lambda_ns=100, granule_bytes=u, n_start=4, i_aa=i_aa).resolved(N), 2
+
+
+def test_multistart_aa_stop_rule_and_best_start(oracle_lib):
+    """Section 4.2, Step 2: a run of the Alternating Algorithm ends after I_AA sweeps or after the first
+    complete sweep that does not raise F_B, and MultiStartAA returns its highest-scoring run (lowest start
+    among equals, this build's convention).  Checked from the trace: every run's sweep records end exactly
+    where the rule says; the binding a run ends with scores the F of its last sweep on the residual demand
+    (recomputed here in numpy); each candidate's volume is the largest such F; and the emitted activation is
+    the binding of the lowest start that reaches it."""
+    seen = dict(early=0, limit=0, later_start=0, tie_other_binding=0, runs=0)
+    for cat, D, p, tau in _aa_cases():
+        oc = _oc(oracle_lib, cat)
+        N, u = oc.N, p.granule_bytes
+        plan = oc.schedule(D, p, tau_in=tau, trace_cap=2_000_000)
+        assert plan["status"] == 0 and len(plan["trace"]) < 2_000_000
+        cap = _caps(oc, tau, u)
+        fam = oc.families()
+        tr = plan["trace"]
+        rem = D.copy()
+        for k in range(int(plan["n_steps"])):
+            rows = tr[tr[:, 0] == k]
+            cands = rows[rows[:, 2] == -1]
+            assert len(cands) >= 1
+            for f, vol in zip(cands[:, 1].tolist(), cands[:, 3].tolist()):
+                fr = rows[rows[:, 1] == f]
+                last_f, binds = [], []
+                for t in range(p.n_start):
+                    F = fr[fr[:, 2] == t]
+                    assert F[:, 3].tolist() == list(range(len(F))) and 1 <= len(F) <= p.i_aa
+                    Fv = [-1] + F[:, 4].tolist()
+                    m = len(F)
+                    assert all(Fv[s + 1] > Fv[s] for s in range(m - 1))       # it went on only after an improvement
+                    assert m == p.i_aa or Fv[m] <= Fv[m - 1]                  # it ended at the limit or at no gain
+                    seen["early" if m < p.i_aa else "limit"] += 1
+                    b = fr[fr[:, 2] == -2 - t]
+                    assert b[:, 3].tolist() == list(range(N))
+                    src, dst = b[:, 4] // 65536, b[:, 4] % 65536
+                    assert sorted(src.tolist()) == list(range(N)) and sorted(dst.tolist()) == list(range(N))
+                    credit = np.minimum(rem[src, dst], cap[fam[f]])           # Eq. (7) x tau, Eq. (8)
+                    assert credit.sum() == Fv[m]                              # the binding as it stands scores the last F
+                    last_f.append(Fv[m]); binds.append((src, dst, credit))
+                    seen["runs"] += 1
+                assert vol == max(last_f)                                     # returns the highest-scoring run
+                if f == plan["chan_id"][k]:
+                    t_star = last_f.index(max(last_f))
+                    seen["later_start"] += t_star > 0
+                    src, dst, x = binds[t_star]
+                    exp_dst = np.full(N, -1, np.int64); exp_x = np.zeros(N, np.int64); exp_i = np.full(N, 0xFFFF, np.int64)
+                    busy = x > 0
+                    exp_dst[src[busy]] = dst[busy]; exp_x[src[busy]] = x[busy]; exp_i[src[busy]] = fam[f][busy]
+                    assert (plan["lane_dst"][k] == exp_dst).all() and (plan["lane_bytes"][k] == exp_x).all()
+                    assert (plan["lane_inst"][k] == exp_i).all()
+                    for t in range(t_star + 1, p.n_start):                    # an equal run that would emit something else
+                        if last_f[t] == last_f[t_star]:
+                            s2, d2, x2 = binds[t]
+                            o_dst = np.full(N, -1, np.int64); o_dst[s2[x2 > 0]] = d2[x2 > 0]
+                            seen["tie_other_binding"] += int((o_dst != exp_dst).any())
+            act = plan["lane_dst"][k] >= 0
+            rem[np.nonzero(act)[0], plan["lane_dst"][k][act]] -= plan["lane_bytes"][k][act]
+        assert not rem.any()
+    # the cases exercise every branch of the rule
+    assert seen["early"] > 100 and seen["limit"] > 100 and seen["later_start"] > 10 and seen["tie_other_binding"] > 10
