@@ -382,7 +382,12 @@ int vp_unpack_tokens(const int32_t* n_steps_b, const int16_t* lane_dst_b, const 
  * How vp_schedule_batch would launch for a batch of B matrices (for benchmarks and tests): out4 (host) receives
  * {kernel, CTAs, threads per CTA, dynamic shared memory bytes}.  kernel 0 = one CTA per matrix; kernel 1 = one
  * warp per matrix, chosen for topologies of at most four groups of four ranks once B exceeds the number of CTAs
- * that fit the GPU at once.  Both kernels produce identical plans.
+ * that fit the GPU at once; kernel 2 = one CTA per matrix with 16-bit saturating credits in shared memory, chosen
+ * for node-symmetric catalogs of more than sixteen groups of four ranks (a second launch of kernel 0 then takes the
+ * matrices whose capacities or totals do not fit that representation).  All kernels produce identical plans.
+ * CTAs is also the number of matrices in flight at once: a caller that splits a large batch into sub-batches
+ * wastes least when each sub-batch is several times this number (the CTAs pull matrices from a shared counter, so
+ * only the last matrix of each CTA can leave the others waiting).
  */
 int vp_schedule_launch_info(const vp_catalog* catalog, int B, const vp_sched_params* params, int32_t* out4);
 

@@ -136,7 +136,8 @@ def schedule_launch_info(catalog: "Catalog", B: int, params: "SchedParams") -> d
     out = (C.c_int32 * 4)()
     p = params._c(catalog.N)
     _check(_load().vp_schedule_launch_info(catalog._h, int(B), C.byref(p), out), "vp_schedule_launch_info")
-    return dict(kernel="warp per matrix" if out[0] else "CTA per matrix", ctas=int(out[1]), threads=int(out[2]), smem=int(out[3]))
+    kernel = {0: "CTA per matrix", 1: "warp per matrix", 2: "CTA per matrix, 16-bit credits"}[int(out[0])]
+    return dict(kernel=kernel, ctas=int(out[1]), threads=int(out[2]), smem=int(out[3]))
 
 
 def schedule_read_stats(workspace: torch.Tensor, stream=None) -> dict:

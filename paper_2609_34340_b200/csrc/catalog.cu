@@ -2,11 +2,12 @@
 // Eq. (3) and Eq. (4) of Section 4.1 and builds the device image the kernels read.
 #include <algorithm>
 #include <cstring>
+#include <map>
 #include <new>
 
 #include "vp_internal.h"
 
-long long g_vp_launches = 0;
+std::atomic<long long> g_vp_launches{0};
 
 namespace {
 
@@ -248,6 +249,8 @@ extern "C" int vp_load_catalog(const void* topology, size_t topo_bytes, const vo
     vp_catalog* c = new (std::nothrow) vp_catalog();
     if (!c) return VP_E_NOMEM;
     c->device = device;
+    memset(c->memo, 0, sizeof(c->memo));
+    c->memo_next = 0;
     int prev = -1;
     cudaGetDevice(&prev);
     if (cudaSetDevice(device) != cudaSuccess) { delete c; return VP_E_CUDA; }
@@ -278,6 +281,43 @@ extern "C" int vp_load_catalog(const void* topology, size_t topo_bytes, const vo
         for (int s = 0; s < n_shapes; s++)
             for (int e = 0; e < max_terms; e++) term_t[(size_t)e * ns_pad + s] = term_pad[(size_t)s * max_terms + e];
         if (!rc) rc = upload(c, term_t, &dc.term_t);
+    }
+    if (sym) {   // row patterns: the terms of each shape split by source rail, distinct rows numbered
+        std::map<std::vector<uint32_t>, int> ids;
+        std::vector<std::vector<uint32_t>> rows;
+        const int ns_pad = (n_shapes + 31) & ~31, words = (S + 1) / 2;
+        std::vector<uint32_t> shape_pat((size_t)ns_pad * words, 0);
+        size_t max_row = 1;
+        bool fits = true;
+        for (int s = 0; s < n_shapes && fits; s++)
+            for (int q = 0; q < S; q++) {
+                std::vector<uint32_t> row;
+                for (uint32_t e = term_ptr[s]; e < term_ptr[s + 1]; e++) {
+                    const uint32_t idx = (term[e] & 0xffffu) / 8;
+                    if ((int)((idx / S) % S) == q) row.push_back(idx | (term[e] & 0xffff0000u));
+                }
+                auto it = ids.find(row);
+                int id;
+                if (it == ids.end()) {
+                    id = (int)rows.size();
+                    ids.emplace(row, id);
+                    rows.push_back(row);
+                    max_row = std::max(max_row, row.size());
+                } else {
+                    id = it->second;
+                }
+                if (id >= 65536) { fits = false; break; }
+                shape_pat[(size_t)(q / 2) * ns_pad + s] |= (uint32_t)id << (16 * (q & 1));
+            }
+        if (fits) {
+            std::vector<uint32_t> pat_term(rows.size() * max_row, 0);
+            for (size_t p = 0; p < rows.size(); p++)
+                for (size_t t = 0; t < rows[p].size(); t++) pat_term[p * max_row + t] = rows[p][t];
+            dc.n_patterns = (int)rows.size();
+            dc.max_row_terms = (int)max_row;
+            if (!rc) rc = upload(c, pat_term, &dc.pat_term);
+            if (!rc) rc = upload(c, shape_pat, &dc.shape_pat);
+        }
     }
     if (!rc) rc = upload(c, bucket_ptr, &dc.bucket_ptr);
     if (!rc) rc = upload(c, fam_slot, &dc.fam_slot);
@@ -315,7 +355,7 @@ extern "C" int vp_load_catalog(const void* topology, size_t topo_bytes, const vo
     return VP_OK;
 }
 
-extern "C" int64_t vp_kernel_launch_count(void) { return g_vp_launches; }
+extern "C" int64_t vp_kernel_launch_count(void) { return g_vp_launches.load(); }
 
 extern "C" const char* vp_strerror(int code) {
     switch (code) {

@@ -30,6 +30,7 @@
 //      the next row of the running send / receive offsets.
 #include <cuda_runtime.h>
 
+#include <cstring>
 #include <utility>
 
 #include "bulk_copy.cuh"
@@ -854,7 +855,9 @@ vp_schedule_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand, co
                    int32_t* __restrict__ n_steps, int32_t* __restrict__ chan_id, int16_t* __restrict__ lane_dst,
                    uint16_t* __restrict__ lane_inst, int64_t* __restrict__ lane_bytes, int64_t* __restrict__ send_off,
                    int64_t* __restrict__ recv_off, int64_t* __restrict__ tau_out, int32_t* __restrict__ status,
-                   int64_t* ws_drem, unsigned int* counter) {
+                   int64_t* ws_drem, unsigned int* counter, const int* __restrict__ todo) {
+    // With a to-do list (left by the kernel for large node-symmetric catalogs) the CTAs work through the matrices
+    // todo[0 .. counter[1]) and pull positions from counter[2]; without one, through 0 .. B-1 from counter[0].
     static_assert(LPG == 1 || GS == 4, "lane teams are defined for groups of four ranks");
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int N = dc.N, G = dc.G, tid = threadIdx.x, NT = blockDim.x;
@@ -961,7 +964,15 @@ vp_schedule_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand, co
     }
 
     for (;;) {
-        if (tid == 0) { s_b = (int)atomicAdd(counter, 1u); s_flags = 0; }
+        if (tid == 0) {
+            if (todo) {
+                const unsigned at = atomicAdd(counter + 2, 1u);
+                s_b = at < counter[1] ? todo[at] : B;
+            } else {
+                s_b = (int)atomicAdd(counter, 1u);
+            }
+            s_flags = 0;
+        }
         __syncthreads();
         const int b = s_b;
         if (b >= B) break;
@@ -1099,18 +1110,26 @@ vp_schedule_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand, co
 }  // namespace
 
 #include "schedule_warp.cuh"
+#include "schedule_big.cuh"
 
 namespace {
 
 struct Launch {
     int threads, grid, lpg;
-    int warp_kernel;          // 1: one warp per matrix (vp_schedule_warp_kernel), 0: one CTA per matrix
+    int kernel;               // 0: one CTA per matrix (vp_schedule_kernel), 1: one warp per matrix (vp_schedule_warp_kernel),
+                              // 2: vp_schedule_big_kernel, followed by vp_schedule_kernel on the matrices it left
     size_t smem;
     KParams kp;
+    int big_w, big_threads, big_grid;     // kernel 2: warps per task, threads and CTAs of the first launch
+    size_t big_smem;
+    int wave;                 // CTAs of the chosen kernel that are resident at once (the grid is min(B, wave) or less)
 };
+static_assert(sizeof(Launch) <= sizeof(((vp_launch_memo*)0)->launch), "the launch memo is too small");
 
 typedef void (*KernelFn)(DevCat, KParams, const int64_t*, const int64_t*, int, int32_t*, int32_t*, int16_t*, uint16_t*,
-                         int64_t*, int64_t*, int64_t*, int64_t*, int32_t*, int64_t*, unsigned int*);
+                         int64_t*, int64_t*, int64_t*, int64_t*, int32_t*, int64_t*, unsigned int*, const int*);
+typedef void (*BigKernelFn)(DevCat, KParams, const int64_t*, const int64_t*, int, int32_t*, int32_t*, int16_t*, uint16_t*,
+                            int64_t*, int64_t*, int64_t*, int64_t*, int32_t*, int64_t*, unsigned int*, int*);
 
 KernelFn pick_kernel(int g, int lpg) {
     switch (g) {
@@ -1127,6 +1146,7 @@ KernelFn pick_kernel(int g, int lpg) {
     }
     return nullptr;
 }
+BigKernelFn pick_big_kernel(int w) { return w == 2 ? vp_schedule_big_kernel<2> : vp_schedule_big_kernel<1>; }
 
 int resolve_params(const vp_catalog* c, const vp_sched_params* p, KParams* kp) {
     if (!c || !p) return VP_E_BAD_ARG;
@@ -1141,12 +1161,15 @@ int resolve_params(const vp_catalog* c, const vp_sched_params* p, KParams* kp) {
     return VP_OK;
 }
 
-int plan_launch(const vp_catalog* c, int B, const vp_sched_params* p, Launch* out) {
+// Works out kernel, launch shape and shared-memory layout for a batch of B matrices.  This sets function attributes
+// and asks the runtime for occupancies, so vp_catalog keeps the last few results (see plan_launch).
+int plan_launch_uncached(const vp_catalog* c, int B, const vp_sched_params* p, Launch* out) {
     const DevCat& dc = c->dc;
     Launch L;
+    memset(&L, 0, sizeof(L));
     int rc = resolve_params(c, p, &L.kp);
     if (rc) return rc;
-    L.warp_kernel = 0;
+    L.kernel = 0;
     L.lpg = 1;
     if (dc.g == 4) L.lpg = dc.G <= 4 ? 8 : (dc.G <= 8 ? 4 : (dc.G <= 16 ? 2 : 1));
     L.threads = dc.N <= 64 ? 128 : 512;
@@ -1176,7 +1199,26 @@ int plan_launch(const vp_catalog* c, int B, const vp_sched_params* p, Launch* ou
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, L.threads, L.smem) != cudaSuccess || per_sm < 1)
         return VP_E_CUDA;
     long long cap = (long long)per_sm * c->sm_count;
+    L.wave = (int)cap;
     L.grid = (int)(B < cap ? B : cap);
+#ifndef VP_NO_BIG_KERNEL
+    // Large node-symmetric catalogs (groups of four, more than sixteen groups): 16-bit credits in shared memory and
+    // scores on the per-node-offset table; the general kernel then takes whatever matrices that kernel left.
+    if (dc.g == 4 && dc.G > 16 && dc.G <= 64 && dc.sym && dc.shape_pat && dc.n_patterns <= 2048 && dc.n_classes <= 15) {
+        const size_t smem = (size_t)big_smem_layout(dc, L.kp).total;
+        if (smem + 2048 <= (size_t)c->max_smem_optin) {
+            const int w = dc.G > 32 ? 2 : 1;
+            BigKernelFn bf = pick_big_kernel(w);
+            if (cudaFuncSetAttribute(bf, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return VP_E_CUDA;
+            int bper_sm = 0;
+            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&bper_sm, bf, 512, smem) != cudaSuccess || bper_sm < 1) return VP_E_CUDA;
+            const long long bcap = (long long)bper_sm * c->sm_count;
+            L.kernel = 2; L.big_w = w; L.big_threads = 512; L.big_smem = smem;
+            L.big_grid = (int)(B < bcap ? B : bcap);
+            L.wave = (int)bcap;
+        }
+    }
+#endif
 #ifndef VP_NO_WARP_KERNEL
     // Small topologies (groups of four, at most four groups, plain D-hat scores) and more matrices than the
     // CTAs of one wave: one warp per matrix gives up latency per matrix for three to four times as many
@@ -1191,9 +1233,10 @@ int plan_launch(const vp_catalog* c, int B, const vp_sched_params* p, Launch* ou
             if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&wper_sm, vp_schedule_warp_kernel, warps * 32, smem) != cudaSuccess || wper_sm < 1)
                 return VP_E_CUDA;
             const long long wcap = (long long)wper_sm * c->sm_count, want = ((long long)B + warps - 1) / warps;
-            L.warp_kernel = 1; L.lpg = 8; L.threads = warps * 32; L.smem = smem;
+            L.kernel = 1; L.lpg = 8; L.threads = warps * 32; L.smem = smem;
             L.kp.drem_in_smem = 1; L.kp.stage_terms = L.kp.stage_fam = L.kp.stage_bucket = 1;
             L.grid = (int)(want < wcap ? want : wcap);
+            L.wave = (int)wcap * warps;
         }
     }
 #endif
@@ -1201,9 +1244,41 @@ int plan_launch(const vp_catalog* c, int B, const vp_sched_params* p, Launch* ou
     return VP_OK;
 }
 
-size_t workspace_bytes(const vp_catalog* c, const Launch& L) {
-    size_t drem = L.kp.drem_in_smem ? 0 : (size_t)L.grid * c->dc.N * c->dc.N * 8;
-    return vp_align256(256 + drem);
+// plan_launch_uncached through the catalog's memo.  A launch depends on B only through min(B, one wave) -- except for
+// the switch to the warp kernel, which happens exactly when B exceeds the general kernel's wave -- so batches are
+// keyed by min(B, 65536) and a cached launch is reused when its own grid rule gives the same answer.  The memo is not
+// locked: calls that share a catalog handle from several host threads must be serialised by the caller (as must
+// anything else that shares a workspace).
+int plan_launch(const vp_catalog* cc, int B, const vp_sched_params* p, Launch* out) {
+    vp_catalog* c = const_cast<vp_catalog*>(cc);
+    if (!c || !p) return VP_E_BAD_ARG;
+    for (vp_launch_memo& m : c->memo) {
+        if (!m.valid || m.B_class != B || m.k_target != p->k_target || m.n_start != p->n_start || m.i_aa != p->i_aa ||
+            m.k_max != p->k_max || m.lambda_ns != p->lambda_ns || m.granule != p->granule_bytes)
+            continue;
+        memcpy(out, m.launch, sizeof(Launch));
+        return VP_OK;
+    }
+    Launch L;
+    const int rc = plan_launch_uncached(c, B, p, &L);
+    if (rc) return rc;
+    vp_launch_memo& m = c->memo[c->memo_next];
+    c->memo_next = (c->memo_next + 1) % (int)(sizeof(c->memo) / sizeof(c->memo[0]));
+    m.valid = 1; m.B_class = B;
+    m.k_target = p->k_target; m.n_start = p->n_start; m.i_aa = p->i_aa; m.k_max = p->k_max;
+    m.lambda_ns = p->lambda_ns; m.granule = p->granule_bytes;
+    memcpy(m.launch, &L, sizeof(Launch));
+    *out = L;
+    return VP_OK;
+}
+
+size_t workspace_bytes(const vp_catalog* c, const Launch& L, int B) {
+    // 256 bytes of counters; one residual slot per CTA when the residual does not fit shared memory; with the kernel
+    // for large node-symmetric catalogs also the list of matrices left to the general kernel
+    const int slots = L.kernel == 2 ? (L.grid > L.big_grid ? L.grid : L.big_grid) : L.grid;
+    size_t drem = L.kp.drem_in_smem ? 0 : (size_t)slots * c->dc.N * c->dc.N * 8;
+    size_t list = L.kernel == 2 ? vp_align256((size_t)B * 4) : 0;
+    return vp_align256(256 + drem) + list;
 }
 
 }  // namespace
@@ -1213,10 +1288,10 @@ extern "C" size_t vp_schedule_workspace_bytes(const vp_catalog* c, int B, const 
     if (B <= 0 || !c || !p) return 0;
     int prev = -1;
     cudaGetDevice(&prev);
-    cudaSetDevice(c->device);
+    if (prev != c->device) cudaSetDevice(c->device);
     int rc = plan_launch(c, B, p, &L);
-    if (prev >= 0) cudaSetDevice(prev);
-    return rc == VP_OK ? workspace_bytes(c, L) : 0;
+    if (prev >= 0 && prev != c->device) cudaSetDevice(prev);
+    return rc == VP_OK ? workspace_bytes(c, L, B) : 0;
 }
 
 extern "C" int vp_schedule_batch(const vp_catalog* c, const vp_sched_params* p, const int64_t* demand,
@@ -1229,10 +1304,10 @@ extern "C" int vp_schedule_batch(const vp_catalog* c, const vp_sched_params* p, 
         return VP_E_BAD_ARG;
     int prev = -1;
     cudaGetDevice(&prev);
-    if (cudaSetDevice(c->device) != cudaSuccess) return VP_E_CUDA;
+    if (prev != c->device && cudaSetDevice(c->device) != cudaSuccess) return VP_E_CUDA;
     Launch L;
     int rc = plan_launch(c, B, p, &L);
-    if (!rc && (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes_given < workspace_bytes(c, L))) rc = VP_E_WORKSPACE;
+    if (!rc && (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes_given < workspace_bytes(c, L, B))) rc = VP_E_WORKSPACE;
     if (!rc) {
         cudaStream_t stream = (cudaStream_t)cuda_stream;
         unsigned int* counter = (unsigned int*)workspace;
@@ -1240,20 +1315,31 @@ extern "C" int vp_schedule_batch(const vp_catalog* c, const vp_sched_params* p, 
         if (cudaMemsetAsync(counter, 0, 256, stream) != cudaSuccess) rc = VP_E_CUDA;
         if (!rc) {
             vp_prof_mark(0, 0, stream);
-            if (L.warp_kernel)
+            if (L.kernel == 1) {
                 vp_schedule_warp_kernel<<<L.grid, L.threads, L.smem, stream>>>(
                     c->dc, L.kp, demand, tau_ns_in, B, n_steps, chan_id, lane_dst, lane_inst, lane_bytes, send_off, recv_off,
                     tau_ns_out, status, counter);
-            else
+            } else if (L.kernel == 2) {
+                const int slots = L.grid > L.big_grid ? L.grid : L.big_grid;
+                int* todo = (int*)((char*)workspace + vp_align256(256 + (size_t)slots * c->dc.N * c->dc.N * 8));
+                pick_big_kernel(L.big_w)<<<L.big_grid, L.big_threads, L.big_smem, stream>>>(
+                    c->dc, L.kp, demand, tau_ns_in, B, n_steps, chan_id, lane_dst, lane_inst, lane_bytes, send_off, recv_off,
+                    tau_ns_out, status, ws_drem, counter, todo);
+                g_vp_launches++;
                 pick_kernel(c->dc.g, L.lpg)<<<L.grid, L.threads, L.smem, stream>>>(
                     c->dc, L.kp, demand, tau_ns_in, B, n_steps, chan_id, lane_dst, lane_inst, lane_bytes, send_off, recv_off,
-                    tau_ns_out, status, ws_drem, counter);
+                    tau_ns_out, status, ws_drem, counter, todo);
+            } else {
+                pick_kernel(c->dc.g, L.lpg)<<<L.grid, L.threads, L.smem, stream>>>(
+                    c->dc, L.kp, demand, tau_ns_in, B, n_steps, chan_id, lane_dst, lane_inst, lane_bytes, send_off, recv_off,
+                    tau_ns_out, status, ws_drem, counter, nullptr);
+            }
             g_vp_launches++;
             if (cudaGetLastError() != cudaSuccess) rc = VP_E_CUDA;
             vp_prof_mark(0, 1, stream);
         }
     }
-    if (prev >= 0) cudaSetDevice(prev);
+    if (prev >= 0 && prev != c->device) cudaSetDevice(prev);
     return rc;
 }
 
@@ -1262,11 +1348,14 @@ extern "C" int vp_schedule_launch_info(const vp_catalog* c, int B, const vp_sche
     Launch L;
     int prev = -1;
     cudaGetDevice(&prev);
-    if (cudaSetDevice(c->device) != cudaSuccess) return VP_E_CUDA;
+    if (prev != c->device && cudaSetDevice(c->device) != cudaSuccess) return VP_E_CUDA;
     const int rc = plan_launch(c, B, p, &L);
-    if (prev >= 0) cudaSetDevice(prev);
+    if (prev >= 0 && prev != c->device) cudaSetDevice(prev);
     if (rc) return rc;
-    out4[0] = L.warp_kernel; out4[1] = L.grid; out4[2] = L.threads; out4[3] = (int32_t)L.smem;
+    out4[0] = L.kernel;
+    out4[1] = L.kernel == 2 ? L.big_grid : L.grid;
+    out4[2] = L.kernel == 2 ? L.big_threads : L.threads;
+    out4[3] = (int32_t)(L.kernel == 2 ? L.big_smem : L.smem);
     return VP_OK;
 }
 

@@ -2,6 +2,8 @@
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
+
+#include <atomic>
 #include <vector>
 
 #include "variopath.h"
@@ -23,6 +25,14 @@ struct DevCat {
     const uint32_t* term;
     const uint32_t* term_t;       // the same, transposed: term e of shape s at term_t[e * ((n_shapes + 31) & ~31) + s]
     int max_terms;
+    // Row patterns (node-symmetric catalogs): the terms of a shape whose source group is rail q of node 0 form the
+    // shape's row q; Eq. (6) is the sum of its S row scores, and distinct rows are few (127 per rail for 4,095 shapes on
+    // 32 nodes).  pat_term[p * max_row_terms + t] = table index | count << 16 (zero padded) lists the terms of row
+    // pattern p; shape_pat[w * ((n_shapes + 31) & ~31) + s] holds the pattern ids of rows 2w and 2w + 1 of shape s
+    // (16 bits each).  Null unless there are fewer than 65,536 patterns.
+    const uint32_t* pat_term;
+    const uint32_t* shape_pat;
+    int n_patterns, max_row_terms;
     const uint32_t* bucket_ptr;
     // family f, slot r: instance id | destination group << 16 | rate class << 24
     const uint32_t* fam_slot;
@@ -46,6 +56,15 @@ struct DevCat {
     int64_t bw_max, W;
 };
 
+// A launch shape worked out once per (catalog, batch class, parameters) and reused by later calls.
+struct vp_launch_memo {
+    int valid;
+    int B_class;                  // min(B, CTAs of one wave + 1): batches of one class launch alike up to the grid size
+    int32_t k_target, n_start, i_aa, k_max;
+    int64_t lambda_ns, granule;
+    unsigned char launch[160];    // the scheduler's Launch record
+};
+
 struct vp_catalog {
     int device;
     vp_info info;
@@ -53,9 +72,11 @@ struct vp_catalog {
     std::vector<void*> allocs;
     int sm_count;
     int max_smem_optin;
+    vp_launch_memo memo[4];
+    int memo_next;
 };
 
-extern long long g_vp_launches;
+extern std::atomic<long long> g_vp_launches;
 
 // Profiling hook: when enabled, records a CUDA event on `stream` before (edge 0) / after (edge 1)
 // the kernels of one kind (0 schedule kernel, 1 pack index kernels, 2 pack copy kernel).
