@@ -1,22 +1,28 @@
 #!/usr/bin/env python
 """Benchmark of the VarioPath online scheduler + pack on B200.
 
-A *step* is one pass of the whole hot path over one batch of synthetic input:
-``vp_schedule_batch`` over the N=16 batch of 256 MoE demand matrices (config 2) followed by
-``vp_pack`` of one rank's 16384 x top-8 routed rows of 7168 bf16 (config 5).  ``value`` is
-matrices per second over whole steps (inputs resident in HBM); ``e2e`` is the same step through
-the host-buffer entry points with pinned host memory, copies inside the timed region.
+A *step* is one pass of the whole hot path over one batch of synthetic input: ``vp_schedule_batch`` over the
+N=256 batch of 4096 demand matrices (config 4, in sub-batches that reuse the plan buffers) followed by ``vp_pack``
+of one rank's 16384 x top-8 routed rows of 7168 bf16 (config 5).  ``value`` is matrices per second over whole
+steps with inputs resident in HBM; ``e2e`` is the same step through the host-buffer entry points with pinned host
+memory, copies inside the timed region.  Beside the headline the line carries
+
+* ``sched_configs``: the scheduler alone on configs 1, 2 and 3 (L2 flushed between launches),
+* ``peaks``: integer-issue, shared-memory and write-only rates measured in this run by the library's probes,
+* ``roofline`` (scheduler, the dominant kernel) and ``roofline_other`` (pack copy kernel),
+* ``cpu_baseline``: the CPU oracle on a bounded sample of the same workload.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--sched-config 1|2|3|4]
 
-With N > 1 (torchrun) every rank runs its own replica of the step (the path has no exchange
-step: matrices are independent and a rank packs only its own rows), times are max-reduced.
-``--impl reference`` times the CPU oracle on the host cores instead (rank 0 only).
+With N > 1 (torchrun) every rank runs its own replica of the step (the path has no exchange step: matrices are
+independent and a rank packs only its own rows); times are max-reduced.  ``--impl reference`` times the CPU oracle
+on the host cores instead (rank 0 only).
 """
 from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
 import statistics
 import subprocess
@@ -30,10 +36,8 @@ if ROOT not in sys.path:
 
 METRIC = "matrices_scheduled_per_sec"
 UNIT = "matrices/s"
-INT64_OPS_PER_LANE_CLK = 0.5    # one 64-bit add/min/compare needs two 32-bit ALU issues
-SM_COUNT, LANES_PER_SM = 148, 128
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch on the default workload (ncu, see profiles/)
-NCU_DRAM_BYTES_PER_LAUNCH = {"pack_copy_bulk_kernel": 235_441_664 + 1_791_668_000, "vp_schedule_kernel": 646_656 + 0}
+SM_COUNT, SCHEDULERS_PER_SM = 148, 4
+COUNTERS_JSON = os.path.join(ROOT, "profiles", "ncu_counters.json")
 
 
 def _dist_env():
@@ -64,6 +68,16 @@ def load_peaks():
             p = json.load(f)
         return dict(hbm_gbs=float(p["hbm_gbs"]), source="measured", sm_max_mhz=float(p.get("sm_max_mhz", 1965.0)))
     return dict(hbm_gbs=6650.0, source="fallback", sm_max_mhz=1965.0)
+
+
+def load_counters() -> dict:
+    """Per-kernel ncu counters of earlier captures (warp instructions and shared-memory wavefronts per activation,
+    DRAM bytes per launch), kept under profiles/ with the commit they were captured at."""
+    try:
+        with open(COUNTERS_JSON) as f:
+            return json.load(f)
+    except (OSError, ValueError):
+        return {}
 
 
 class ClockSampler:
@@ -128,20 +142,150 @@ def build_workload(args, device: str):
     return sched, pack
 
 
+def workload_string(args, sched, pk) -> str:
+    """Names the step's workload; both arms build it from the same inputs, so the strings are identical."""
+    cat = sched["catalog"]
+    B, N = sched["demand"].shape[0], cat.topology.N
+    T, topk = pk["expert_idx"].shape
+    R = int(pk["demand"][0, pk["rank"]].sum().item() // pk["row_bytes"])
+    kind = {1: "MoE", 2: "MoE", 3: "MoE", 4: "MoE + sequence-parallel"}[args.sched_config]
+    rep = " x%d" % args.sched_repeat if args.sched_repeat > 1 else ""
+    return (f"config {args.sched_config}{rep}: {B} {kind} demand matrices N={N} ({cat.n_shapes} shapes / "
+            f"{cat.n_families} families) + config 5 pack: rank {pk['rank']} of 16, {T} tokens x top-{topk}, "
+            f"{pk['row_bytes']}-B rows, {R} staged rows")
+
+
 def vp_params(vp, w):
     return vp.SchedParams(lambda_ns=w.lambda_ns, granule_bytes=w.granule_bytes, k_target=w.k_target,
                           n_start=w.n_start, i_aa=w.i_aa, k_max=w.k_max)
 
 
 def sched_ops(cat, stats: dict, n_start: int) -> float:
-    """Algorithmic 64-bit integer operations of a measured batch (Section 4.2, planning complexity,
-    with sparse shapes): per activation one multiply-add per shape term and N subtract/offset updates;
-    per AA sweep 2G assignments of g! permutations x g terms (min + add); per task 2N for Evaluate."""
-    import math
+    """Algorithmic integer operations of a measured batch (Section 4.2, planning complexity, with sparse
+    shapes): per activation one multiply-add per shape term and N subtract/offset updates; per AA sweep 2G
+    assignments of g! permutations x g terms (min + add); per task 2N for Evaluate."""
     topo = cat.topology
     terms = sum(len(s) for s in cat.shapes)
     per_sweep = 2 * topo.G * math.factorial(topo.g) * topo.g
     return stats["activations"] * (terms + topo.N) + stats["sweeps"] * per_sweep + stats["tasks"] * 2 * topo.N
+
+
+class SchedRun:
+    """One scheduler workload on the device: the batch goes through ``vp_schedule_batch`` in sub-batches that
+    reuse one set of plan buffers (a config-4 plan is 29 MB per matrix)."""
+
+    def __init__(self, vp, torch, sched, dev, local_rank, sub_batch):
+        self.vp, self.torch = vp, torch
+        cat, w = sched["catalog"], sched["params"]
+        self.cat, self.w = cat, w
+        self.dc = vp.load_catalog(cat.topology.blob(), cat.blob(), device=local_rank)
+        self.params = vp_params(vp, w)
+        self.demand = sched["demand"].to(dev).contiguous()
+        self.B, self.N = self.demand.shape[0], cat.topology.N
+        per_matrix = w.k_max * self.N * 12 + 2 * (w.k_max + 1) * self.N * 8
+        fit = max(1, int(40e9 // per_matrix))                    # at most ~40 GB of plan buffers
+        self.sub = min(self.B, sub_batch or self.B, fit)
+        self.plan = vp.Plan.empty(self.sub, self.N, w.k_max, dev)
+        self.ws = torch.empty(vp.schedule_workspace_bytes(self.dc, self.sub, self.params), dtype=torch.uint8, device=dev)
+        self.launch = vp.schedule_launch_info(self.dc, self.sub, self.params)
+        self.calls = (self.B + self.sub - 1) // self.sub
+
+    def run(self):
+        for lo in range(0, self.B, self.sub):
+            self.vp.schedule_batch(self.dc, self.params, self.demand[lo:lo + self.sub], plan=self.plan, workspace=self.ws)
+
+    def stats_whole_batch(self) -> dict:
+        """Work counters of the whole batch: the workspace holds those of the last call, so one extra pass reads
+        them call by call (outside any timed region)."""
+        total = dict(activations=0, tasks=0, sweeps=0)
+        for lo in range(0, self.B, self.sub):
+            self.vp.schedule_batch(self.dc, self.params, self.demand[lo:lo + self.sub], plan=self.plan, workspace=self.ws)
+            st = self.vp.schedule_read_stats(self.ws)
+            assert int(self.plan.status[: min(self.sub, self.B - lo)].max().item()) == 0, "workload did not schedule cleanly"
+            for k in total:
+                total[k] += st[k]
+        return total
+
+
+def event_pair(torch):
+    return torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+
+def measure_peaks(vp, torch, dev, staged) -> dict:
+    """Integer-issue and shared-memory rates from the library's probes, and the write-only rate of a
+    ``cudaMemsetAsync`` over the staged buffer.  Best of five launches each, CUDA events."""
+    sink = torch.zeros(1, dtype=torch.int64, device=dev)
+    out = {}
+    for name, kind, iters, scale, unit in (("int32_add_min_tops", 0, 400, 1e12, "Tops/s"), ("int64_add_min_tops", 1, 200, 1e12, "Tops/s"),
+                                           ("smem_load32_tbs", 2, 400, 1e12, "TB/s"), ("smem_load64_tbs", 3, 400, 1e12, "TB/s")):
+        best = 0.0
+        vp.microbench(kind, iters, sink)
+        for _ in range(5):
+            e0, e1 = event_pair(torch)
+            e0.record()
+            units = vp.microbench(kind, iters, sink)
+            e1.record()
+            torch.cuda.synchronize()
+            best = max(best, units / (e0.elapsed_time(e1) * 1e-3) / scale)
+        out[name] = round(best, 3)
+    best = 0.0
+    for _ in range(6):
+        e0, e1 = event_pair(torch)
+        e0.record()
+        n = vp.memset_probe(staged)
+        e1.record()
+        torch.cuda.synchronize()
+        best = max(best, n / (e0.elapsed_time(e1) * 1e-3) / 1e9)
+    out["write_only_gbs"] = round(best, 1)
+    out["how"] = ("vp_microbench kinds 0-3 (every warp slot of every SM busy, eight independent chains per thread) and "
+                  "cudaMemsetAsync over the staged buffer; best of 5, CUDA events, at the clock sampled in this run")
+    return out
+
+
+def time_sched_config(vp, torch, idx, dev, local_rank, flush, peaks_now, counters, reps=20) -> dict:
+    """The scheduler alone on config ``idx``: L2 flushed (a 256 MB fill) before every timed launch."""
+    from workloads.configs import build_config
+    sched = build_config(idx, device=dev)
+    run = SchedRun(vp, torch, sched, dev, local_rank, None)
+    for _ in range(3):
+        run.run()
+    torch.cuda.synchronize()
+    times = []
+    for _ in range(reps):
+        flush.zero_()
+        e0, e1 = event_pair(torch)
+        e0.record()
+        run.run()
+        e1.record()
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1))
+    stats = run.stats_whole_batch()
+    ms = statistics.median(times)
+    act = stats["activations"]
+    ops = sched_ops(run.cat, stats, run.w.n_start)
+    out = {"workload": f"config {idx}: {run.B} matrices N={run.N} ({run.cat.n_shapes} shapes / {run.cat.n_families} families)",
+           "launch": run.launch, "ms": round(ms, 4), "ms_best": round(min(times), 4),
+           "matrices_per_s": round(run.B / ms * 1e3, 1), "activations": act,
+           "activations_per_s": round(act / ms * 1e3, 1), "us_per_activation": round(ms * 1e3 / max(act, 1), 4),
+           "algorithmic_int_ops": int(ops),
+           "alu_frac_of_measured_int32_peak": round(ops / (ms * 1e-3) / 1e12 / peaks_now["int32_add_min_tops"], 5)}
+    out.update(issue_fraction(counters, f"config{idx}", act, ms, peaks_now.get("sm_mhz")))
+    return out
+
+
+def issue_fraction(counters: dict, key: str, activations: int, ms: float, sm_mhz) -> dict:
+    """Issue-slot and shared-memory-pipe use from the warp instructions / wavefronts per activation that an ncu
+    capture of the same kernel and config recorded (profiles/ncu_counters.json), over this run's time and clock."""
+    c = (counters.get("scheduler") or {}).get(key)
+    if not c or not sm_mhz:
+        return {"issue_slot_frac": None, "shared_wavefront_frac": None}
+    cycles = ms * 1e-3 * sm_mhz * 1e6
+    inst = c["warp_inst_per_activation"] * activations
+    wave = c["shared_wavefronts_per_activation"] * activations
+    return {"issue_slot_frac": round(inst / (cycles * SM_COUNT * SCHEDULERS_PER_SM), 4),
+            "shared_wavefront_frac": round(wave / (cycles * SM_COUNT), 4),
+            "counters_from": f"profiles/ncu_counters.json ({c.get('source', '?')}, commit {counters.get('commit', '?')})",
+            "ncu_issue_active_pct": c.get("issue_active_pct"), "ncu_shared_wavefront_pct": c.get("shared_wavefront_pct")}
 
 
 def run_ours(args):
@@ -157,15 +301,8 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device(dev))
 
     sched, pk = build_workload(args, dev)
-    cat, w = sched["catalog"], sched["params"]
-    dc = vp.load_catalog(cat.topology.blob(), cat.blob(), device=local_rank)
-    params = vp_params(vp, w)
-    demand = sched["demand"].to(dev).contiguous()
-    B, N = demand.shape[0], cat.topology.N
-    sub = min(B, 256) if N > 64 else B          # N=256 plans are 30 MB each: sub-batches reuse the output buffers
-    plan = vp.Plan.empty(sub, N, w.k_max, dev)
-    ws = torch.empty(vp.schedule_workspace_bytes(dc, sub, params), dtype=torch.uint8, device=dev)
-    sched["_launch"] = vp.schedule_launch_info(dc, sub, params)
+    run = SchedRun(vp, torch, sched, dev, local_rank, args.sub_batch)
+    cat, w, B, N = run.cat, run.w, run.B, run.N
 
     # pack case: its own one-matrix plan on the config-2 topology
     pcat, pw = pk["catalog"], pk["params"]
@@ -186,8 +323,7 @@ def run_ours(args):
     copy_bytes = T * row_bytes + R * row_bytes + 4 * T * topk              # what the copy kernel itself must move
 
     def step():
-        for lo in range(0, B, sub):
-            vp.schedule_batch(dc, params, demand[lo:lo + sub], plan=plan, workspace=ws)
+        run.run()
         vp.pack(pplan, 0, prank, idx, pk["experts_per_rank"], rows, staged, src_map, pstatus, pws)
 
     def barrier():
@@ -205,13 +341,13 @@ def run_ours(args):
         if n_warm % 16 == 0:
             torch.cuda.synchronize()
     barrier()
-    assert int(pstatus.item()) == 0 and int(plan.status.max().item()) == 0, "workload did not schedule cleanly"
+    assert int(pstatus.item()) == 0 and int(run.plan.status.max().item()) == 0, "workload did not schedule cleanly"
 
     vp.profile_enable(True)
     for k in range(3):
         vp.profile_read(k)
     launches0 = vp.kernel_launch_count()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0, ev1 = event_pair(torch)
     barrier()
     ev0.record()
     for _ in range(args.steps):
@@ -225,30 +361,43 @@ def run_ours(args):
     copy_ms, n_copy = vp.profile_read(2)
     vp.profile_enable(False)
     clocks = sampler.stop()
-    stats = vp.schedule_read_stats(ws)
-    if sub < B:                                    # counters cover the last sub-batch only: scale to the batch
-        stats = {k: v * (B // sub) for k, v in stats.items()}
+    stats = run.stats_whole_batch()
 
     ms_per_step = reduce_max(total_ms / args.steps, world)
     value = aggregate_value(B, world, ms_per_step / 1e3)
+    sched_per_step = sched_ms / max(args.steps, 1)               # all scheduler launches of one step
+    sched_per_launch = sched_ms / max(n_sched, 1)
 
-    sched_avg = sched_ms / max(n_sched, 1) * (B // sub)
-    if sub < B or args.no_e2e:
-        e2e_ms, h2d, d2h, e2e_steps = None, 0, 0, 0
+    extras = {}
+    if rank == 0 and world == 1 and not args.no_extras:
+        sampler2 = ClockSampler(local_rank)
+        sampler2.start()
+        peaks_now = measure_peaks(vp, torch, dev, staged)
+        peaks_now["sm_mhz"] = clocks.get("sm_mhz") or load_peaks()["sm_max_mhz"]
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+        counters = load_counters()
+        extras["peaks"] = peaks_now
+        extras["sched_configs"] = {}
+        for idx_cfg in (1, 2, 3):
+            if idx_cfg != args.sched_config:
+                extras["sched_configs"][f"config{idx_cfg}"] = time_sched_config(vp, torch, idx_cfg, dev, local_rank, flush, peaks_now, counters)
+        extras["clocks_extras"] = sampler2.stop()
+        del flush
+    if args.no_e2e:
+        e2e = None
     else:
-        e2e_ms, h2d, d2h, e2e_steps = run_e2e(vp, args, world, local_rank, dev, sched, pk, dc, params, pplan, idx, rows,
-                                              R, barrier)
+        e2e = run_e2e(vp, args, world, local_rank, dev, run, pk, pplan, idx, rows, R, barrier)
     tools = run_tools(vp, dev, load_peaks()) if args.tools and rank == 0 else None
     if rank != 0:
         return
-    sched["_tools"] = tools
-    finish(args, world, cat, w, B, N, T, topk, R, prank, row_bytes, pack_bytes, copy_bytes, stats, clocks, launches,
-           sched_avg, index_ms, copy_ms, n_copy, ms_per_step, value, e2e_ms, h2d, d2h, e2e_steps, sched, pk)
+    finish(args, world, run, sched, pk, T, topk, R, pack_bytes, copy_bytes, stats, clocks, launches, sched_per_step,
+           sched_per_launch, n_sched, index_ms, copy_ms, n_copy, ms_per_step, value, e2e, extras, tools)
 
 
 def run_tools(vp, dev, peaks):
-    """The two kernels around the scheduler (`--tools`): Eq. (2) plan time over the config-3 plans and the
-    demand rows of 16 ranks from config-5-sized routing.  Device-resident, CUDA-event timed."""
+    """The kernels around the scheduler (`--tools`): Eq. (2) plan time over the config-3 plans, the demand rows of
+    16 ranks from config-5-sized routing, both unpack directions, and the warp-per-matrix kernel beyond one wave.
+    Device-resident, CUDA-event timed."""
     import torch
     from workloads.configs import build_config
     from workloads.demand import moe_routing
@@ -281,13 +430,8 @@ def run_tools(vp, dev, peaks):
     plan2 = vp.Plan.empty(B2, cat2.topology.N, w2.k_max, dev)
     ws2 = torch.empty(vp.schedule_workspace_bytes(dc2, B2, p2), dtype=torch.uint8, device=dev)
     ms_s = timed(lambda: vp.schedule_batch(dc2, p2, D2, plan=plan2, workspace=ws2), reps=10)
-    ops2 = sched_ops(cat2, vp.schedule_read_stats(ws2), w2.n_start)
-    alu_peak = SM_COUNT * LANES_PER_SM * INT64_OPS_PER_LANE_CLK * peaks["sm_max_mhz"] * 1e6
     large = {"workload": f"config 2 matrices x16: {B2} matrices N=16", "launch": vp.schedule_launch_info(dc2, B2, p2),
-             "ms": round(ms_s, 4), "matrices_per_s": round(B2 / ms_s * 1e3, 1),
-             "alu_frac": round(ops2 / (ms_s * 1e-3) / alu_peak, 4),
-             "ncu": {"issue_active_pct": 57.1, "shared_wavefronts_pct_of_peak": 53.9, "lsu_pipe_pct": 45.7,
-                     "source": "profiles/vp_schedule_warp_kernel_config2_x16.md"}}
+             "ms": round(ms_s, 4), "matrices_per_s": round(B2 / ms_s * 1e3, 1)}
     del plan2, D2
     ms_t = timed(lambda: vp.plan_time(dc, plan, w.lambda_ns, out=out))
     bytes_t = steps * cat.topology.N * 10                       # lane_bytes (8) + lane_inst (2) of every emitted step
@@ -352,15 +496,20 @@ def run_tools(vp, dev, peaks):
                                     "ms": round(ms_d, 4), "gb_per_s": round(bytes_d / ms_d / 1e6, 1)}}
 
 
-def run_e2e(vp, args, world, local_rank, dev, sched, pk, dc, params, pplan, idx, rows, R, barrier):
+def run_e2e(vp, args, world, local_rank, dev, run, pk, pplan, idx, rows, R, barrier):
+    """The same step through the host-buffer entry points: demand, routing and rows start in pinned host memory,
+    plans and the staged buffer end there; every copy is inside the timed region.  The scheduler batch goes
+    through ``vp_schedule_batch_host`` in sub-batches that reuse one pinned plan buffer."""
+    import ctypes
     import torch
-    cat, w, pw = sched["catalog"], sched["params"], pk["params"]
-    B, N = sched["demand"].shape[0], cat.topology.N
+    cat, w, pw = run.cat, run.w, pk["params"]
+    B, N = run.B, run.N
     T, topk = idx.shape
     prank, row_bytes = pk["rank"], pk["row_bytes"]
-    # ---- end to end through the host-buffer entry points (pinned memory, copies timed)
-    h_demand = sched["demand"].cpu().contiguous().pin_memory()
-    h_plan = vp.Plan.empty(B, N, w.k_max, "cpu", pin=True)
+    per_matrix = w.k_max * N * 12 + 2 * (w.k_max + 1) * N * 8
+    sub = max(1, min(B, int(4e9 // per_matrix)))                 # at most ~4 GB pinned at a time
+    h_demand = run.demand.cpu().contiguous().pin_memory()
+    h_plan = vp.Plan.empty(sub, N, w.k_max, "cpu", pin=True)
     h_pplan = vp.Plan.empty(1, 16, pw.k_max, "cpu", pin=True)
     for name in ("n_steps", "chan_id", "lane_dst", "lane_inst", "lane_bytes", "send_off", "recv_off", "tau_ns", "status"):
         getattr(h_pplan, name).copy_(getattr(pplan, name).cpu())
@@ -368,19 +517,23 @@ def run_e2e(vp, args, world, local_rank, dev, sched, pk, dc, params, pplan, idx,
     h_staged = torch.empty((R, rows.shape[1]), dtype=rows.dtype).pin_memory()
     h_map = torch.empty(R, dtype=torch.int32).pin_memory()
     h_status = torch.zeros(1, dtype=torch.int32).pin_memory()
-    need = int(vp.binding._load().vp_schedule_host_scratch_bytes(dc._h, B, __import__("ctypes").byref(params._c(N))))
+    need = int(vp.binding._load().vp_schedule_host_scratch_bytes(run.dc._h, sub, ctypes.byref(run.params._c(N))))
     sscr = torch.empty(need, dtype=torch.uint8, device=dev)
     need = int(vp.binding._load().vp_pack_host_scratch_bytes(16, T, topk, pw.k_max, row_bytes, R * row_bytes))
     pscr = torch.empty(need, dtype=torch.uint8, device=dev)
 
     def e2e_step():
-        vp.schedule_batch_host(dc, params, h_demand, plan=h_plan, scratch=sscr)
+        bad = 0
+        for lo in range(0, B, sub):
+            n = min(sub, B - lo)
+            vp.schedule_batch_host(run.dc, run.params, h_demand[lo:lo + n], plan=h_plan, scratch=sscr)
+            bad |= int(h_plan.status[:n].max().item())           # the step's result is read on the host
         vp.pack_host(h_pplan, 0, prank, h_idx, pk["experts_per_rank"], h_rows, h_staged, h_map, h_status, pscr,
                      device=local_rank)
-        return int(h_status.item())
+        return bad | int(h_status.item())
 
-    e2e_steps = max(3, min(args.steps, 10))
-    e2e_step()
+    e2e_steps = max(1, min(args.steps, args.e2e_steps))
+    assert e2e_step() == 0
     barrier()
     t0 = time.perf_counter()
     for _ in range(e2e_steps):
@@ -390,81 +543,75 @@ def run_e2e(vp, args, world, local_rank, dev, sched, pk, dc, params, pplan, idx,
     K1 = w.k_max
     h2d = (B * N * N * 8) + (4 + pw.k_max * 16 * 10 + (pw.k_max + 1) * 16 * 8 + T * topk * 4 + T * row_bytes)
     d2h = (B * (4 + K1 * 4 + K1 * N * 12 + 2 * (K1 + 1) * N * 8 + 8 + 4)) + (4 + R * row_bytes + R * 4)
-    return e2e_ms, h2d, d2h, e2e_steps
+    return {"value": round(B * world / (e2e_ms / 1e3), 1), "unit": UNIT, "ms_per_step": round(e2e_ms, 3),
+            "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": e2e_steps,
+            "host_sub_batch": sub}
 
 
-def finish(args, world, cat, w, B, N, T, topk, R, prank, row_bytes, pack_bytes, copy_bytes, stats, clocks, launches,
-           sched_avg, index_ms, copy_ms, n_copy, ms_per_step, value, e2e_ms, h2d, d2h, e2e_steps, sched, pk):
+def finish(args, world, run, sched, pk, T, topk, R, pack_bytes, copy_bytes, stats, clocks, launches, sched_per_step,
+           sched_per_launch, n_sched, index_ms, copy_ms, n_copy, ms_per_step, value, e2e, extras, tools):
     peaks = load_peaks()
+    counters = load_counters()
+    cat, w, B, N = run.cat, run.w, run.B, run.N
     copy_avg = copy_ms / max(n_copy, 1)
     index_avg = index_ms / max(n_copy, 1)
     pack_gbs = copy_bytes / (copy_avg * 1e-3) / 1e9
     ops = sched_ops(cat, stats, w.n_start)
     sm_mhz = clocks.get("sm_mhz") or peaks["sm_max_mhz"]
-    alu_peak_max = SM_COUNT * LANES_PER_SM * INT64_OPS_PER_LANE_CLK * peaks["sm_max_mhz"] * 1e6 / 1e12
-    alu_peak_now = SM_COUNT * LANES_PER_SM * INT64_OPS_PER_LANE_CLK * sm_mhz * 1e6 / 1e12
-    sched_tops = ops / (sched_avg * 1e-3) / 1e12
-    # DRAM bytes per launch from the ncu captures summarised under profiles/ (default workload only)
-    default_workload = args.sched_config == 2 and args.batch is None and args.pack_tokens == 16384 and args.sched_repeat == 1
-    traffic_copy = NCU_DRAM_BYTES_PER_LAUNCH["pack_copy_bulk_kernel"] if default_workload else None
-    traffic_sched = NCU_DRAM_BYTES_PER_LAUNCH["vp_schedule_kernel"] if default_workload else None
+    p_now = extras.get("peaks") or {}
+    int_peak = p_now.get("int32_add_min_tops")
+    sched_tops = ops / (sched_per_step * 1e-3) / 1e12
+    pack_counters = (counters.get("pack_copy_bulk_kernel") or {}) if args.pack_tokens == 16384 else {}
     roof_pack = dict(kernel="pack_copy_bulk_kernel", bound="hbm", achieved=round(pack_gbs, 1), peak=peaks["hbm_gbs"],
-                     unit="GB/s", frac=round(pack_gbs / peaks["hbm_gbs"], 4), traffic=traffic_copy,
-                     peak_source=peaks["source"], ms_per_launch=round(copy_avg, 4),
-                     algorithmic_bytes_per_launch=copy_bytes)
-    launch = sched.get("_launch") or {}
-    roof_sched = dict(kernel="vp_schedule_warp_kernel" if launch.get("kernel") == "warp per matrix" else "vp_schedule_kernel",
-                      launch=launch, bound="alu", achieved=round(sched_tops, 4), peak=round(alu_peak_max, 2),
-                      unit="Tops/s (64-bit integer)", frac=round(sched_tops / alu_peak_max, 5), traffic=traffic_sched,
-                      peak_source="derived: 148 SMs x 128 lanes x 0.5 64-bit ops/clk x max SM clock",
-                      frac_at_sampled_clock=round(sched_tops / alu_peak_now, 5), ms_per_launch=round(sched_avg, 4),
-                      algorithmic_ops_per_launch=int(ops))
-    dominant, other = (roof_pack, roof_sched) if copy_avg >= sched_avg else (roof_sched, roof_pack)
+                     unit="GB/s", frac=round(pack_gbs / peaks["hbm_gbs"], 4), traffic=pack_counters.get("dram_bytes_per_launch"),
+                     peak_source=peaks["source"] + " copy peak (MEASURED_PEAKS.json)", ms_per_launch=round(copy_avg, 4),
+                     algorithmic_bytes_per_launch=copy_bytes,
+                     frac_of_nominal_8tbs=round(pack_gbs / 8000.0, 4),
+                     whole_call_gb_per_s=round(pack_bytes / ((copy_avg + index_avg) * 1e-3) / 1e9, 1),
+                     whole_call_frac=round(pack_bytes / ((copy_avg + index_avg) * 1e-3) / 1e9 / peaks["hbm_gbs"], 4),
+                     write_only_peak_gbs=p_now.get("write_only_gbs"))
+    key = f"config{args.sched_config}"
+    sc = (counters.get("scheduler") or {}).get(key) or {}
+    calls = run.calls
+    roof_sched = dict(kernel={"warp per matrix": "vp_schedule_warp_kernel", "CTA per matrix": "vp_schedule_kernel"}.get(
+                          run.launch.get("kernel"), "vp_schedule_big_kernel"),
+                      launch=run.launch, bound="alu", achieved=round(sched_tops, 4), peak=int_peak,
+                      unit="Tops/s (integer add/min, algorithmic)",
+                      frac=round(sched_tops / int_peak, 5) if int_peak else None,
+                      traffic=(sc.get("dram_bytes_per_activation") or 0) * stats["activations"] / calls if sc.get("dram_bytes_per_activation") else None,
+                      peak_source="measured in this run: vp_microbench kind 0 (32-bit add + min, all warp slots busy)",
+                      ms_per_launch=round(sched_per_launch, 4), launches_per_step=calls,
+                      algorithmic_ops_per_launch=int(ops / calls))
+    roof_sched.update(issue_fraction(counters, key, stats["activations"], sched_per_step, sm_mhz))
+    dominant, other = (roof_pack, roof_sched) if copy_avg >= sched_per_step else (roof_sched, roof_pack)
     act = stats["activations"]
     line = {
         "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": round(ms_per_step, 4), "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "int64", "data": "synthetic",
-        "config": {"workload": f"config {args.sched_config}{' x%d' % args.sched_repeat if args.sched_repeat > 1 else ''}: {B} MoE demand matrices N={N} "
-                               f"({cat.n_shapes} shapes / {cat.n_families} families) + config 5 pack: rank {prank} of 16, "
-                               f"{T} tokens x top-{topk}, {row_bytes}-B rows, {R} staged rows",
-                   "batch_per_gpu": B, "parallelism": f"replicas x{world}, no collective",
-                   "l2": "each step's pack streams %.2f GB (> 126 MB L2) between two schedule launches" % (pack_bytes / 1e9)},
-        "sched": {"matrices_per_s": round(B / (sched_avg * 1e-3), 1), "ms": round(sched_avg, 4),
-                  "activations_per_batch": act, "us_per_activation_amortized": round(sched_avg * 1e3 / max(act, 1), 4),
-                  "activations_per_s": round(act / (sched_avg * 1e-3), 1)},
+        "config": {"workload": workload_string(args, sched, pk),
+                   "value_is": "matrices of the scheduler batch per second of whole step (all sub-batches + one pack)",
+                   "batch_per_gpu": B, "sub_batch": run.sub, "parallelism": f"replicas x{world}, no collective",
+                   "l2": "inputs larger than L2: %.2f GB of demand per step, and each step's pack streams %.2f GB"
+                         % (B * N * N * 8 / 1e9, pack_bytes / 1e9)},
+        "sched": {"matrices_per_s": round(B / (sched_per_step * 1e-3), 1), "ms": round(sched_per_step, 4),
+                  "activations_per_batch": act, "us_per_activation_amortized": round(sched_per_step * 1e3 / max(act, 1), 4),
+                  "activations_per_s": round(act / (sched_per_step * 1e-3), 1)},
         "pack": {"gb_per_s": round(pack_gbs, 1), "copy_ms": round(copy_avg, 4), "index_ms": round(index_avg, 4),
                  "gb_per_s_incl_index": round(pack_bytes / ((copy_avg + index_avg) * 1e-3) / 1e9, 1)},
         "roofline": dominant, "roofline_other": other,
-        "e2e": ({"value": round(B * world / (e2e_ms / 1e3), 1), "unit": UNIT, "ms_per_step": round(e2e_ms, 3),
-                 "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": e2e_steps}
-                if e2e_ms else None),
-        "gpu_launches": int(launches), "clocks": clocks,
+        "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
     }
-    if sched.get("_tools"):
-        line["next_rows"] = sched["_tools"]
-    line["cpu_baseline"] = cpu_baseline(sched, pk, budget_s=20.0) if world == 1 and not args.no_cpu_baseline else None
+    line.update(extras)
+    if tools:
+        line["next_rows"] = tools
+    line["cpu_baseline"] = cpu_baseline(args, sched, pk, budget_s=20.0) if world == 1 and not args.no_cpu_baseline else None
     print(json.dumps(line))
 
 
 # ------------------------------------------------------------------------------------------
 # CPU oracle legs
 # ------------------------------------------------------------------------------------------
-
-def _oracle_step(oc, poc, sched, pk, plan_one, threads, tokens):
-    """One oracle step: schedule the whole batch, pack the first ``tokens`` tokens' worth of plan."""
-    import numpy as np
-    t0 = time.perf_counter()
-    oc.schedule_batch(sched["demand"].numpy(), sched["params"], threads=threads)
-    t1 = time.perf_counter()
-    rows = pk["_rows_np"]
-    R = pk["_R"]
-    if pk.get("_staged") is None:
-        pk["_staged"] = np.zeros((R, rows.shape[1] * rows.itemsize), np.uint8)
-    poc.pack(plan_one, pk["rank"], pk["_idx_np"], pk["experts_per_rank"], rows, R, staged=pk["_staged"])
-    t2 = time.perf_counter()
-    return t1 - t0, t2 - t1
-
 
 def _oracle_setup(sched, pk):
     import numpy as np
@@ -481,21 +628,56 @@ def _oracle_setup(sched, pk):
     return oc, poc, plan_one
 
 
-def cpu_baseline(sched, pk, budget_s: float) -> dict:
-    """The oracle as it stands, timed on this machine's host cores on the same workload."""
+def oracle_sample(sched, limit: int):
+    """The bounded sample the oracle schedules per step: the whole batch when it is small, else ``limit`` matrices
+    spread evenly over the seeded batch (so that every class of the recipe is in it).  Returns (matrices, note)."""
+    import numpy as np
+    D = sched["demand"].cpu().numpy()
+    B = D.shape[0]
+    if B <= limit:
+        return D, B, f"all {B} matrices"
+    pick = np.linspace(0, B - 1, limit).astype(np.int64)
+    return np.ascontiguousarray(D[pick]), limit, f"{limit} of the {B} matrices (evenly spaced), scaled to {B}"
+
+
+def _oracle_sched(oc, D, params, threads):
+    """Schedules the sample on ``threads`` host threads (interleaved split: equal mixes of long and short matrices)."""
+    import numpy as np
+    n = D.shape[0]
+    order = np.concatenate([np.arange(t, n, threads) for t in range(threads)]) if threads > 1 else np.arange(n)
+    t0 = time.perf_counter()
+    oc.schedule_batch(np.ascontiguousarray(D[order]), params, threads=threads)
+    return time.perf_counter() - t0
+
+
+def _oracle_pack(poc, pk, plan_one):
+    import numpy as np
+    rows, R = pk["_rows_np"], pk["_R"]
+    if pk.get("_staged") is None:
+        pk["_staged"] = np.zeros((R, rows.shape[1] * rows.itemsize), np.uint8)
+    t0 = time.perf_counter()
+    poc.pack(plan_one, pk["rank"], pk["_idx_np"], pk["experts_per_rank"], rows, R, staged=pk["_staged"])
+    return time.perf_counter() - t0
+
+
+def cpu_baseline(args, sched, pk, budget_s: float) -> dict:
+    """The oracle as it stands, timed on this machine's host cores on a bounded sample of the same workload."""
     cores = os.cpu_count() or 1
     oc, poc, plan_one = _oracle_setup(sched, pk)
     B = sched["demand"].shape[0]
-    ts, tp, n = 0.0, 0.0, 0
-    t_start = time.perf_counter()
-    while n < 1 or (time.perf_counter() - t_start < budget_s and n < 5):
-        a, b = _oracle_step(oc, poc, sched, pk, plan_one, cores, None)
-        ts += a; tp += b; n += 1
-    step_s = (ts + tp) / n
+    D, n, note = oracle_sample(sched, args.oracle_sample)
+    t_all = _oracle_sched(oc, D, sched["params"], cores)
+    n1 = max(1, min(n, n // cores if t_all > 1.0 else n))        # the one-thread figure on a smaller slice
+    t_one = _oracle_sched(oc, D[:n1], sched["params"], 1)
+    t_pack = _oracle_pack(poc, pk, plan_one)
+    sched_s = t_all * B / n
+    step_s = sched_s + t_pack
+    pack_bytes = pk["_rows_np"].nbytes + pk["_R"] * pk["row_bytes"]
     return {"value": round(B / step_s, 2), "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": f"{n} full step(s): all {B} matrices split over {cores} threads + the whole pack on 1 thread",
-            "sched_matrices_per_s": round(B / (ts / n), 2), "pack_gb_per_s": round(
-                (pk["_rows_np"].nbytes + pk["_R"] * pk["row_bytes"]) / (tp / n) / 1e9, 3)}
+            "sample": f"scheduler: {note}, over {cores} threads; pack: the whole pack on 1 thread",
+            "sched_matrices_per_s": round(n / t_all, 2),
+            "sched_matrices_per_s_one_thread": round(n1 / t_one, 3), "one_thread_sample": f"first {n1} matrices of the sample",
+            "pack_gb_per_s_one_thread": round(pack_bytes / t_pack / 1e9, 3)}
 
 
 def run_reference(args):
@@ -507,21 +689,26 @@ def run_reference(args):
     cores = os.cpu_count() or 1
     oc, poc, plan_one = _oracle_setup(sched, pk)
     B = sched["demand"].shape[0]
+    D, n, note = oracle_sample(sched, args.oracle_sample)
+
+    def step():
+        return _oracle_sched(oc, D, sched["params"], cores), _oracle_pack(poc, pk, plan_one)
+
     for _ in range(args.warmup):
-        _oracle_step(oc, poc, sched, pk, plan_one, cores, None)
-    t0 = time.perf_counter()
+        step()
+    ts = tp = 0.0
     for _ in range(args.steps):
-        _oracle_step(oc, poc, sched, pk, plan_one, cores, None)
-    ms = (time.perf_counter() - t0) * 1e3 / args.steps
+        a, b = step()
+        ts += a; tp += b
+    sched_s = ts / args.steps * B / n                            # the sample's time scaled to the whole batch
+    ms = (sched_s + tp / args.steps) * 1e3
     value = B / (ms / 1e3)
-    N = sched["catalog"].topology.N
+    sample = f"every step: scheduler on {note}, over {cores} threads; the whole pack on 1 thread"
     line = {"impl": "reference", "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(ms, 3), "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "int64", "data": "synthetic",
-            "config": {"workload": f"config {args.sched_config}: {B} MoE demand matrices N={N} + config 5 pack "
-                                   f"(CPU oracle, whole workload per step)"},
-            "cpu_baseline": {"value": round(value, 2), "unit": UNIT, "cores": cores, "kind": "oracle",
-                             "sample": f"every step: all {B} matrices over {cores} threads + the whole pack on 1 thread"},
+            "config": {"workload": workload_string(args, sched, pk)},
+            "cpu_baseline": {"value": round(value, 2), "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
             "e2e": {"value": round(value, 2), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line))
@@ -538,21 +725,27 @@ def _has_cuda() -> bool:
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--sched-config", type=int, default=2, choices=[1, 2, 3, 4])
+    ap.add_argument("--sched-config", type=int, default=4, choices=[1, 2, 3, 4])
+    ap.add_argument("--sub-batch", type=int, default=1024,
+                    help="matrices per vp_schedule_batch call (the plan buffers are reused); the batch when smaller")
     ap.add_argument("--batch", type=int, default=None, help="truncate the scheduler batch (tests)")
     ap.add_argument("--sched-repeat", type=int, default=1,
                     help="schedule the batch this many times over in one call (a batch beyond one wave; not the default benchmark)")
     ap.add_argument("--token-scale", type=float, default=1.0, help="scale token counts (tests)")
     ap.add_argument("--pack-tokens", type=int, default=16384, help="tokens of the packed rank (tests)")
+    ap.add_argument("--oracle-sample", type=int, default=64,
+                    help="matrices the CPU oracle schedules per step when the batch is larger (reference arm, cpu_baseline)")
     ap.add_argument("--min-warmup-s", type=float, default=1.0,
                     help="keep warming up (beyond --warmup steps) until this many seconds have passed, so that "
                          "clocks settle and nvidia-smi has samples under load")
-    ap.add_argument("--tools", action="store_true", help="also time vp_plan_time and vp_demand_from_routing")
+    ap.add_argument("--e2e-steps", type=int, default=2, help="steps of the host-buffer leg (each moves the whole plan over PCIe)")
+    ap.add_argument("--tools", action="store_true", help="also time the kernels around the scheduler (unpack, plan time, demand rows)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the CPU oracle leg (profiling runs)")
+    ap.add_argument("--no-extras", action="store_true", help="skip the peak probes and the other scheduler configs (profiling runs)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":

@@ -392,6 +392,24 @@ int vp_unpack_tokens(const int32_t* n_steps_b, const int16_t* lane_dst_b, const 
 int vp_schedule_launch_info(const vp_catalog* catalog, int B, const vp_sched_params* params, int32_t* out4);
 
 /*
+ * Peak-rate probes (no counterpart in the paper; measurement support for Section 4.2's operation counts).  Launches
+ * one kernel on `cuda_stream` of the current device that keeps every warp slot of every SM busy with
+ *   kind 0: 32-bit integer add + min on eight independent chains per thread (units = integer operations),
+ *   kind 1: the same on 64-bit integers (units = 64-bit operations),
+ *   kind 2 / 3: conflict-free 32-bit / 64-bit shared-memory loads (units = bytes loaded),
+ * for `iters` loop iterations, and stores the number of units one launch performs in *units_per_launch (host).
+ * The caller times the launch (CUDA events on the same stream) and divides.  `sink_device` is 8 bytes of device
+ * memory that the kernel never writes in practice.  Returns VP_E_BAD_ARG for an unknown kind or iters <= 0.
+ */
+int vp_microbench(int kind, int iters, void* sink_device, int64_t* units_per_launch, void* cuda_stream);
+
+/*
+ * Write-only bandwidth probe (no counterpart in the paper): enqueues one cudaMemsetAsync of `bytes` zero bytes over
+ * the caller's device buffer on `cuda_stream`; the caller times it.
+ */
+int vp_memset_probe(void* device_buffer, size_t bytes, void* cuda_stream);
+
+/*
  * Work counters of the last vp_schedule_batch that used `workspace` (device): copies three
  * uint64 to host `out3` after synchronising the stream: activations emitted, (family, start)
  * binding tasks run, AA sweeps run over all tasks.  Used to count the algorithmic operations

@@ -30,6 +30,8 @@ from .binding import (  # noqa: F401
     demand_from_routing,
     schedule_read_stats,
     schedule_launch_info,
+    microbench,
+    memset_probe,
     profile_enable,
     profile_read,
     library_path,

@@ -101,6 +101,8 @@ def _load():
     lib.vp_demand_from_routing.argtypes = [P, i32, i32, i32, i32, i32, i32, i64, P, P, P]
     lib.vp_schedule_read_stats.argtypes = [P, P, P]
     lib.vp_schedule_launch_info.argtypes = [vp, i32, C.POINTER(_Params), P]
+    lib.vp_microbench.argtypes = [i32, i32, P, C.POINTER(i64), P]
+    lib.vp_memset_probe.argtypes = [P, sz, P]
     lib.vp_profile_enable.argtypes = [i32]
     lib.vp_profile_read.argtypes = [i32, C.POINTER(C.c_double), C.POINTER(i64)]
     lib.vp_strerror.argtypes = [i32]
@@ -145,6 +147,21 @@ def schedule_read_stats(workspace: torch.Tensor, stream=None) -> dict:
     out = (C.c_uint64 * 3)()
     _check(_load().vp_schedule_read_stats(_ptr(workspace), _stream(stream), out), "vp_schedule_read_stats")
     return dict(activations=int(out[0]), tasks=int(out[1]), sweeps=int(out[2]))
+
+
+def microbench(kind: int, iters: int, sink: torch.Tensor, stream=None) -> int:
+    """``vp_microbench``: launches peak-rate probe ``kind`` on the current stream; returns the units (integer
+    operations or bytes) one launch performs.  ``sink`` is an 8-byte device tensor."""
+    units = C.c_int64(0)
+    _check(_load().vp_microbench(int(kind), int(iters), _ptr(sink), C.byref(units), _stream(stream)), "vp_microbench")
+    return int(units.value)
+
+
+def memset_probe(buf: torch.Tensor, stream=None) -> int:
+    """``vp_memset_probe``: one ``cudaMemsetAsync`` over ``buf``; returns the bytes written."""
+    n = buf.numel() * buf.element_size()
+    _check(_load().vp_memset_probe(_ptr(buf), n, _stream(stream)), "vp_memset_probe")
+    return n
 
 
 def profile_enable(on: bool) -> None:
