@@ -1204,7 +1204,7 @@ int plan_launch_uncached(const vp_catalog* c, int B, const vp_sched_params* p, L
 #ifndef VP_NO_BIG_KERNEL
     // Large node-symmetric catalogs (groups of four, more than sixteen groups): 16-bit credits in shared memory and
     // scores on the per-node-offset table; the general kernel then takes whatever matrices that kernel left.
-    if (dc.g == 4 && dc.G > 16 && dc.G <= 64 && dc.sym && dc.shape_pat && dc.n_patterns <= 2048 && dc.n_classes <= 15) {
+    if (dc.g == 4 && dc.G > 16 && dc.G <= 64 && dc.sym && dc.shape_pat && dc.n_patterns < 1024 && dc.n_classes <= 15) {
         const size_t smem = (size_t)big_smem_layout(dc, L.kp).total;
         if (smem + 2048 <= (size_t)c->max_smem_optin) {
             const int w = dc.G > 32 ? 2 : 1;

@@ -17,18 +17,26 @@
 //    then every shape is the sum of S looked-up row scores -- two loads and an addition instead of six
 //    multiply-adds.  The row scores are kept in eight copies so that the lanes of a warp rarely meet in a bank.
 //
-// A matrix that does not meet the conditions (granule below 256 bytes, a capacity of 2^16 granules or more, 2^32
-// granules or more in total) is appended to a list that the general kernel works through afterwards.
+//  * Large capacities.  When a lane capacity reaches 2^16 granules (skewed MoE matrices with many tokens), the few
+//    columns that hold cells of 65,535 granules or more -- the destinations of the popular experts -- become "hot
+//    columns": their cells are kept exactly, low 16 bits in the credit matrix and high 16 bits in a side array of up
+//    to 32 columns, and the credits that touch them are patched after the ordinary 16-bit pass.  Every other cell of
+//    such a matrix is below 65,535 granules, so its 16-bit copy is exact.  No L2 traffic is needed in this mode.
+//
+// A matrix that does not meet the conditions (granule below 256 bytes, a capacity of 2^22 granules or more, 2^32
+// granules or more in total, more than 32 hot columns) is appended to a list that the general kernel works through
+// afterwards.
 #pragma once
 
 namespace {
 
 // Scoring reads the row scores at data-dependent positions; with one copy per lane class (lane mod 8) the lanes of a
 // warp meet in a bank only when they share a class and read different patterns of equal parity.
-constexpr int BIG_RS_COPIES = 8;
+constexpr int BIG_RS_COPIES = 1;
+constexpr int BIG_HOT_MAX = 32;       // columns whose cells are kept beyond 16 bits
 
 struct BigSmem {
-    int cs, tbl, rs, pat, gnode, send_acc, recv_acc, red, pair, task_f, task_den, slotw, bind_src, bind_dst, term, bucket, total;
+    int cs, tbl, rs, pat, bnd, hi, colmap, gnode, send_acc, recv_acc, red, pair, task_f, task_den, slotw, bind_src, bind_dst, term, bucket, total;
     int cs_stride;            // credits per row of the 16-bit matrix (N + 2: rows start in different banks)
     int pat_words;            // 32-bit words of row-pattern ids per shape (two ids per word)
 };
@@ -37,16 +45,19 @@ __host__ __device__ inline BigSmem big_smem_layout(const DevCat& dc, const KPara
     BigSmem L;
     int o = 0;
     L.cs_stride = dc.N + 2;
-    const int cs_bytes = dc.N * L.cs_stride * 2, dhat_bytes = dc.G * dc.G * 8 + dc.N * 16;
+    const int cs_bytes = dc.N * L.cs_stride * 2, dhat_bytes = dc.G * dc.G * 8 + dc.N * 24;
     L.cs = o;        o += align16(cs_bytes > dhat_bytes ? cs_bytes : dhat_bytes);   // set-up: D-hat, row and column sums
+    L.hi = o;        o += BIG_HOT_MAX * dc.N * 2;                  // high halves of the hot columns' cells
+    L.colmap = o;    o += align16(dc.N);                          // hot-column index of every rank, 0xFF = none
     L.tbl = o;       o += align16(dc.tbl_size * 4);
     L.rs = o;        o += dc.n_patterns * 8 * BIG_RS_COPIES;      // row scores, one copy per lane class
     L.pat = o;       o += align16(dc.n_patterns * dc.max_row_terms * 4);
+    L.bnd = o;       o += ((dc.n_shapes + 31) & ~31) * 4;          // upper bounds on (score >> 2) of every shape
     L.gnode = o;     o += align16(dc.G * 2);
     L.send_acc = o;  o += dc.N * 8;
     L.recv_acc = o;  o += dc.N * 8;
     L.red = o;       o += 64 * 8;
-    L.pair = o;      o += 16 * 6 * 8;
+    L.pair = o;      o += 16 * 8 * 8;
     L.task_f = o;    o += align16(kp.max_tasks * 8);
     L.task_den = o;  o += align16(kp.max_tasks * 8);
     L.slotw = o;     o += align16(dc.max_bucket * dc.N * 4);
@@ -59,25 +70,98 @@ __host__ __device__ inline BigSmem big_smem_layout(const DevCat& dc, const KPara
     return L;
 }
 
-// Exact 4 x 4 assignment on credits that arrive shifted left by eight bits (a sum of four stays below 2^26):
-// maximise key = 255 + sum_q (c[phi(q)][q] - (phi(q) << (6 - 2q))) over the permutations phi.  The subtracted part is
-// the permutation written as a byte (position 0 in the two highest bits), so the largest key belongs to the largest
-// credit sum and, among equal sums, to the first permutation in lexicographic order, exactly as an enumeration in
-// that order that keeps the first maximum.  Because the key is a sum over positions it is maximised by dynamic
-// programming over the set of rows already placed (positions 0, 1, 2, 3 in turn): 28 additions and 17 maxima
-// instead of 24 sums of four.  The permutation byte is ~key & 255, the credit sum key >> 8.
-__device__ __forceinline__ uint32_t big_best_key(const uint32_t (&c)[4][4]) {
-#define VP_V(r, q) ((int32_t)c[r][q] - ((r) << (6 - 2 * (q))))
-    const int32_t a0 = 255 + VP_V(0, 0), a1 = 255 + VP_V(1, 0), a2 = 255 + VP_V(2, 0), a3 = 255 + VP_V(3, 0);
-    const int32_t b01 = max_v(a0 + VP_V(1, 1), a1 + VP_V(0, 1)), b02 = max_v(a0 + VP_V(2, 1), a2 + VP_V(0, 1));
-    const int32_t b03 = max_v(a0 + VP_V(3, 1), a3 + VP_V(0, 1)), b12 = max_v(a1 + VP_V(2, 1), a2 + VP_V(1, 1));
-    const int32_t b13 = max_v(a1 + VP_V(3, 1), a3 + VP_V(1, 1)), b23 = max_v(a2 + VP_V(3, 1), a3 + VP_V(2, 1));
-    const int32_t c012 = max_v(max_v(b01 + VP_V(2, 2), b02 + VP_V(1, 2)), b12 + VP_V(0, 2));
-    const int32_t c013 = max_v(max_v(b01 + VP_V(3, 2), b03 + VP_V(1, 2)), b13 + VP_V(0, 2));
-    const int32_t c023 = max_v(max_v(b02 + VP_V(3, 2), b03 + VP_V(2, 2)), b23 + VP_V(0, 2));
-    const int32_t c123 = max_v(max_v(b12 + VP_V(3, 2), b13 + VP_V(2, 2)), b23 + VP_V(1, 2));
-    return (uint32_t)max_v(max_v(c012 + VP_V(3, 3), c013 + VP_V(2, 3)), max_v(c023 + VP_V(1, 3), c123 + VP_V(0, 3)));
-#undef VP_V
+// Tag of row r at position q of a 4 x 4 assignment: (3 - r) in the two bits that position q owns in a byte whose
+// two highest bits belong to position 0.  The four tags of a permutation add up to 255 minus the permutation written
+// as a byte, so a credit sum carried as (sum << 8) + tags is largest for the largest sum and, among equal sums, for
+// the first permutation in lexicographic order -- the same winner as an enumeration that keeps the first maximum.
+__host__ __device__ constexpr uint32_t big_tag(int r, int q) { return (uint32_t)(3 - r) << (6 - 2 * q); }
+
+__device__ __forceinline__ uint32_t add_max(uint32_t a, uint32_t b, uint32_t c) { return __viaddmax_u32(a, b, c); }   // max(a + b, c)
+
+// Exact 4 x 4 assignment: v[r][q] = (credit of row r at position q) << 8 | big_tag(r, q).  Returns the largest
+// sum_q v[phi(q)][q] over the permutations phi, by dynamic programming over the set of rows placed so far (positions
+// 0, 1, 2, 3 in turn), 28 add / add-max operations.  The permutation byte is ~key & 255, the credit sum key >> 8.
+__device__ __forceinline__ uint32_t big_best_key(const uint32_t (&v)[4][4]) {
+    const uint32_t b01 = add_max(v[0][0], v[1][1], v[1][0] + v[0][1]), b02 = add_max(v[0][0], v[2][1], v[2][0] + v[0][1]);
+    const uint32_t b03 = add_max(v[0][0], v[3][1], v[3][0] + v[0][1]), b12 = add_max(v[1][0], v[2][1], v[2][0] + v[1][1]);
+    const uint32_t b13 = add_max(v[1][0], v[3][1], v[3][0] + v[1][1]), b23 = add_max(v[2][0], v[3][1], v[3][0] + v[2][1]);
+    const uint32_t c012 = add_max(b01, v[2][2], add_max(b02, v[1][2], b12 + v[0][2]));
+    const uint32_t c013 = add_max(b01, v[3][2], add_max(b03, v[1][2], b13 + v[0][2]));
+    const uint32_t c023 = add_max(b02, v[3][2], add_max(b03, v[2][2], b23 + v[0][2]));
+    const uint32_t c123 = add_max(b12, v[3][2], add_max(b13, v[2][2], b23 + v[1][2]));
+    return add_max(c012, v[3][3], add_max(c013, v[2][3], add_max(c023, v[1][3], c123 + v[0][3])));
+}
+
+// Maximum of distinct 64-bit keys over the warp: the largest high word, then the largest low word among its holders.
+__device__ __forceinline__ uint64_t big_warp_max64(uint64_t key) {
+    const uint32_t hi = (uint32_t)(key >> 32), lo = (uint32_t)key;
+    const uint32_t mhi = __reduce_max_sync(0xffffffffu, hi);
+    const uint32_t mlo = __reduce_max_sync(0xffffffffu, hi == mhi ? lo : 0u);
+    return (uint64_t)mhi << 32 | mlo;
+}
+
+// Fills bytes [lo, hi) of dst with a repeated byte, by 16-byte stores where the address allows (all threads of the CTA).
+__device__ __forceinline__ void big_fill_bytes(unsigned char* dst, size_t lo, size_t hi, unsigned char byte, int tid, int NT) {
+    if (lo >= hi) return;
+    const size_t head = min((size_t)((16 - ((uintptr_t)(dst + lo) & 15)) & 15), hi - lo);
+    for (size_t e = lo + tid; e < lo + head; e += NT) dst[e] = byte;
+    const size_t vlo = lo + head, nvec = (hi - vlo) / 16;
+    const uint32_t w = 0x01010101u * byte;
+    uint4* v = (uint4*)(dst + vlo);
+    for (size_t e = tid; e < nvec; e += NT) v[e] = make_uint4(w, w, w, w);
+    for (size_t e = vlo + nvec * 16 + tid; e < hi; e += NT) dst[e] = byte;
+}
+
+// Step 3 when several families compete (kept out of line: most shapes have one family, and the main loop should
+// stay small for the instruction cache): best start per family (largest F, lowest start), then the family of largest
+// utility F / duration by exact cross-multiplication, lowest family first among equals.  Whole warp.
+__device__ __noinline__ void big_select_family(const int64_t* task_f, const int64_t* task_den, int H, int n_start, int lane,
+                                               int& wtask, int64_t& wF) {
+    int64_t bf = -1, bd = 1;
+    int bt = 0x7fffffff;
+    for (int h = lane; h < H; h += 32) {
+        int64_t ff = -1; int tt = 0;
+        for (int t = 0; t < n_start; t++)
+            if (task_f[h * n_start + t] > ff) { ff = task_f[h * n_start + t]; tt = h * n_start + t; }
+        if (bt == 0x7fffffff || util_greater(ff, task_den[tt], bf, bd)) { bf = ff; bd = task_den[tt]; bt = tt; }
+    }
+#pragma unroll 1
+    for (int o = 16; o; o >>= 1) {
+        const int64_t of = __shfl_xor_sync(0xffffffffu, bf, o), od = __shfl_xor_sync(0xffffffffu, bd, o);
+        const int ot = __shfl_xor_sync(0xffffffffu, bt, o);
+        bool take = false;
+        if (ot != 0x7fffffff) {
+            if (bt == 0x7fffffff) take = true;
+            else if (util_greater(of, od, bf, bd)) take = true;
+            else if (!util_greater(bf, bd, of, od) && ot < bt) take = true;
+        }
+        if (take) { bf = of; bd = od; bt = ot; }
+    }
+    wtask = __shfl_sync(0xffffffffu, bt, 0);
+    wF = __shfl_sync(0xffffffffu, bf, 0);
+}
+
+// Eq. (9) volumes of a binding as it stands (the credit of every in-slot of this lane's group) and the slowest lane of
+// Eq. (10) over the warp, in rate-lcm time units.  Only needed when several families compete.  Whole warp.
+__device__ __noinline__ int64_t big_slowest_lane(const uint16_t* Cs, int CS, const uint16_t* Hi, const uint8_t* colmap, int N,
+                                                 bool hot_mode, const uint8_t* srcb, const uint8_t* dstb,
+                                                 const int (&rq)[4], const uint32_t (&cap_in)[4], const int (&cls_in)[4],
+                                                 const int64_t* tscale, int n_classes, bool active) {
+    int64_t tmax = 0;
+    uint32_t xmax = 0;
+    if (active) {
+#pragma unroll 1
+        for (int q = 0; q < 4; q++) {
+            const int sq = srcb[rq[q]], dq = dstb[rq[q]];
+            uint32_t val = Cs[sq * CS + dq];
+            if (hot_mode && colmap[dq] != 0xFF) val |= (uint32_t)Hi[(int)colmap[dq] * N + sq] << 16;
+            const uint32_t x = min_v(val, cap_in[q]);
+            xmax = max_v(xmax, x);
+            if (n_classes > 1) tmax = max_v(tmax, (int64_t)x * tscale[cls_in[q]]);
+        }
+    }
+    if (n_classes == 1) return (int64_t)__reduce_max_sync(0xffffffffu, xmax) * tscale[0];
+    return warp_max_i64(tmax);
 }
 
 // W = warps per (family, start) task: one lane per rank group, 32 W >= G.
@@ -95,8 +179,11 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
     const int CS = L.cs_stride;
     uint16_t* Cs = (uint16_t*)(smem_raw + L.cs);
     uint32_t* tbl = (uint32_t*)(smem_raw + L.tbl);
+    uint16_t* Hi = (uint16_t*)(smem_raw + L.hi);
+    uint8_t* colmap = smem_raw + L.colmap;
     uint64_t* rs = (uint64_t*)(smem_raw + L.rs);
     uint32_t* pat = (uint32_t*)(smem_raw + L.pat);
+    uint32_t* bnd = (uint32_t*)(smem_raw + L.bnd);
     uint8_t* gnode = smem_raw + L.gnode;                 // per group: node index, then (at G) rail index
     int64_t* send_acc = (int64_t*)(smem_raw + L.send_acc);
     int64_t* recv_acc = (int64_t*)(smem_raw + L.recv_acc);
@@ -110,7 +197,7 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
     uint32_t* spat = (uint32_t*)(smem_raw + L.term);      // row-pattern ids per shape
     uint32_t* bucket = (uint32_t*)(smem_raw + L.bucket);
     uint32_t* Dg = (uint32_t*)(ws_drem + (size_t)blockIdx.x * N * N);      // exact residual, granules
-    __shared__ int s_b, s_flags, s_ok;
+    __shared__ int s_b, s_flags, s_mode, s_nhot;           // s_mode: 0 leave to the general kernel, 1 plain, 2 hot columns
     __shared__ int64_t s_tau, s_left;
     __shared__ int64_t s_tscale[VP_MAX_CLASSES];
     __shared__ uint32_t s_cap[VP_MAX_CLASSES];
@@ -148,9 +235,14 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
         }
         for (int a = tid; a < G; a += NT) { gnode[a] = (uint8_t)(a / S); gnode[G + a] = (uint8_t)(a % S); }
         __syncthreads();
+        // pattern ids become byte offsets into the row scores (fewer than 1,024 patterns, so they still fit 16 bits)
+        for (int e = tid; e < ns_pad * L.pat_words; e += NT) {
+            const uint32_t w = spat[e];
+            spat[e] = (w & 0xffffu) * (8 * BIG_RS_COPIES) | ((w >> 16) * (8 * BIG_RS_COPIES)) << 16;
+        }
+        __syncthreads();
     }
     const int ns_shift = (kp.n_start & (kp.n_start - 1)) == 0 ? 31 - __clz(kp.n_start) : -1;
-    const int n_score_warps = min(n_warps, (dc.n_shapes + 31) >> 5);
 
     for (;;) {
         if (tid == 0) { s_b = (int)atomicAdd(counter, 1u); s_flags = 0; }
@@ -173,20 +265,21 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
         int64_t* Dhat = (int64_t*)(smem_raw + L.cs);
         int64_t* rowsum = Dhat + G * G;
         int64_t* colsum = rowsum + N;
-        for (int i = tid; i < N; i += NT) { colsum[i] = 0; send_acc[i] = 0; recv_acc[i] = 0; }
+        int64_t* colmax = colsum + N;
+        for (int i = tid; i < N; i += NT) { colsum[i] = 0; colmax[i] = 0; rowsum[i] = 0; send_acc[i] = 0; recv_acc[i] = 0; colmap[i] = 0xFF; }
+        if (tid == 0) s_nhot = 0;
+        for (int e = tid; e < G * G; e += NT) Dhat[e] = 0;
         __syncthreads();
         int flags = 0;
+        // (kept as small rolled loops: this code runs once per matrix and must not crowd the instruction cache)
         for (int a = warp; a < G; a += n_warps) {            // one warp per source group: four rows, eight columns per lane
-            int64_t cell0 = 0, cell1 = 0, col[8];
-#pragma unroll
-            for (int m = 0; m < 8; m++) col[m] = 0;
-#pragma unroll
-            for (int i4 = 0; i4 < 4; i4++) {
-                const int i = a * 4 + i4;
-                int64_t rs = 0;
-#pragma unroll
-                for (int m = 0; m < 8; m++) {
-                    const int j = lane * 8 + m;
+#pragma unroll 1
+            for (int m = 0; m < 8; m++) {
+                const int j = lane * 8 + m;
+                int64_t colv = 0, colm = 0;
+#pragma unroll 1
+                for (int i4 = 0; i4 < 4; i4++) {
+                    const int i = a * 4 + i4;
                     int64_t v = 0;
                     if (j < N) {
                         v = D[(size_t)i * N + j];
@@ -197,18 +290,17 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
                             if (v % kp.granule) flags |= VP_ST_NOT_GRANULE;
                         }
                     }
-                    rs += v;
-                    col[m] += v;
-                    if (m < 4) cell0 += v; else cell1 += v;
+                    colv += v;
+                    colm = max_v(colm, v);
+                    const int64_t rs1 = warp_sum_i64(v);
+                    if (lane == 0) rowsum[i] += rs1;         // (rows of this group belong to this warp alone)
                 }
-                rs = warp_sum_i64(rs);
-                if (lane == 0) rowsum[i] = rs;
+                if (j < N) {
+                    atomicAdd((unsigned long long*)&colsum[j], (unsigned long long)colv);
+                    atomicMax((long long*)&colmax[j], (long long)colm);
+                    atomicAdd((unsigned long long*)&Dhat[a * G + (j >> 2)], (unsigned long long)colv);
+                }
             }
-            if (lane * 2 < G) Dhat[a * G + lane * 2] = cell0;
-            if (lane * 2 + 1 < G) Dhat[a * G + lane * 2 + 1] = cell1;
-#pragma unroll
-            for (int m = 0; m < 8; m++)
-                if (lane * 8 + m < N) atomicAdd((unsigned long long*)&colsum[lane * 8 + m], (unsigned long long)col[m]);
         }
         const int64_t tau_given = tau_in ? tau_in[b] : 0;
         if (tid == 0 && (tau_given < 0 || tau_given > VP_ENTRY_LIMIT)) flags |= VP_ST_BAD_TAU;
@@ -252,13 +344,25 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
                     s_cap[cl] = (uint32_t)min_v(cp / kp.granule, (int64_t)0xffffffffll);
                     s_tscale[cl] = dc.class_wdiv[cl] * kp.granule;
                 }
-                // 16-bit credits need capacities below 2^16 granules; the 32-bit table needs fewer than 2^32 granules in all
-                s_ok = kp.granule >= 256 && cap_max / kp.granule < 65535 && t / kp.granule < ((int64_t)1 << 32);
+                // 16-bit credits need capacities below 2^16 granules, hot columns capacities below 2^22 (four credits and
+                // a tag share 32 bits); the 32-bit table needs fewer than 2^32 granules in all
+                const bool fits = kp.granule >= 256 && t / kp.granule < ((int64_t)1 << 32);
+                s_mode = !fits ? 0 : (cap_max / kp.granule < 65535 ? 1 : (cap_max / kp.granule < ((int64_t)1 << 22) ? 2 : 0));
                 s_tau = tq; s_left = t / kp.granule;
             }
             __syncthreads();
             tau = s_tau;
-            deferred = !s_ok;
+            if (s_mode == 2) {                               // hot columns: those with a cell of 65,535 granules or more
+                for (int j = tid; j < N; j += NT)
+                    if (colmax[j] / kp.granule >= 65535) {
+                        const int at = atomicAdd(&s_nhot, 1);
+                        if (at < BIG_HOT_MAX) colmap[j] = (uint8_t)at;
+                    }
+                __syncthreads();
+                if (tid == 0 && s_nhot > BIG_HOT_MAX) s_mode = 0;
+                __syncthreads();
+            }
+            deferred = s_mode == 0;
         }
         if (deferred) {
             // the general kernel takes this matrix (it validates and derives the quantum again)
@@ -279,51 +383,86 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
             }
             __syncthreads();
             // ---- pass 2 over D: the residual in granules (workspace slot) and its saturating 16-bit copy
+            const bool hot_mode = s_mode == 2;
             for (int e = tid; e < N * N; e += NT) {
                 const uint32_t v = (uint32_t)(D[e] / kp.granule);
                 const int i = e / N, j = e - i * N;
-                Dg[e] = v;
-                Cs[i * CS + j] = (uint16_t)min_v(v, 65535u);
+                if (!hot_mode) {
+                    Dg[e] = v;
+                    Cs[i * CS + j] = (uint16_t)min_v(v, 65535u);
+                } else {                                     // exact: 32 bits in a hot column, below 65,535 elsewhere
+                    Cs[i * CS + j] = (uint16_t)v;
+                    if (colmap[j] != 0xFF) Hi[(int)colmap[j] * N + i] = (uint16_t)(v >> 16);
+                }
             }
             __syncthreads();
             int64_t left = s_left;
+            int last_s = -1;                                 // shape chosen in the last iteration
+            for (int s = tid; s < dc.n_shapes; s += NT) bnd[s] = 0xffffffffu;
+            uint16_t* sat_cell = nullptr;                    // a saturated cell whose exact residual is on its way from L2
+            uint32_t sat_left = 0;
+            int f_cached = -1;                               // family whose tables this lane still holds (first task only)
+            uint32_t c_co = 0;
+            uint2 c_fi = make_uint2(0u, 0u);
             VP_TICK(0);
 
             for (;;) {
                 if (left == 0) break;
                 if (k == kp.k_max) { st |= VP_ST_STEP_LIMIT; break; }
-                // (A) Eq. (6): shape scores on the table, first maximum
-                for (int p = tid; p < dc.n_patterns; p += NT) {       // row scores: at most max_row_terms products each
+                // (A) Eq. (6).  Row scores first: at most max_row_terms products each, stored shifted left by 16 bits.
+                for (int p = tid; p < dc.n_patterns; p += NT) {
                     uint64_t v = 0;
+#pragma unroll 1
                     for (int t = 0; t < dc.max_row_terms; t++) {
                         const uint32_t tw = pat[p * dc.max_row_terms + t];
                         v += (uint64_t)tbl[tw & 0xffffu] * (tw >> 16);
                     }
-#pragma unroll
-                    for (int r = 0; r < BIG_RS_COPIES; r++) rs[p * BIG_RS_COPIES + r] = v;
+                    rs[p] = v << 16;
                 }
                 __syncthreads();
-                if (warp < n_score_warps) {
-                    int64_t best = -1;
-                    int best_s = 0x7fffffff;
-                    const uint64_t* rl = rs + (lane & (BIG_RS_COPIES - 1));
-                    for (int s = tid; s < dc.n_shapes; s += NT) {
-                        uint64_t score = 0;
-                        for (int w = 0; w < L.pat_words; w++) {
-                            const uint32_t pw = spat[w * ns_pad + s];
-                            score += rl[(pw & 0xffffu) * BIG_RS_COPIES];
-                            if (2 * w + 1 < S) score += rl[(pw >> 16) * BIG_RS_COPIES];
-                        }
-                        if ((int64_t)score > best) { best = (int64_t)score; best_s = s; }
+                // A score is below 2^34 (g x fewer than 2^32 granules) and there are fewer than 2^16 shapes, so
+                // key = score << 16 | (65535 - shape) orders by score first and lower shape index second: the first
+                // maximum of Eq. (6) is a plain maximum of keys.
+                //
+                // Lazy evaluation.  Table entries only ever shrink while a matrix is decomposed, so the score a shape had
+                // when it was last computed bounds its score now.  The shape chosen last time, scored again, is a lower
+                // bound on the maximum; a shape whose old score lies below that bound (both compared after dropping their
+                // two lowest bits, so that they fit 32 bits) cannot be the maximum, nor tie with it, and is skipped.
+                auto score_key = [&](int s) {
+                    uint64_t key = (uint64_t)(65535 - s);
+                    for (int w = 0; w < L.pat_words; w++) {
+                        const uint32_t pw = spat[w * ns_pad + s];              // two byte offsets into the row scores
+                        key += *(const uint64_t*)((const char*)rs + (pw & 0xffffu));
+                        if (2 * w + 1 < S) key += *(const uint64_t*)((const char*)rs + (pw >> 16));
                     }
-                    warp_argmax_first(best, best_s);
-                    if (lane == 0) { red[warp] = best; red[32 + warp] = best_s; }
+                    return key;
+                };
+                uint64_t best = 0;
+                {
+                    uint32_t floor32 = 0;
+                    if (last_s >= 0) {
+                        best = score_key(last_s);                              // (the same in every thread)
+                        floor32 = (uint32_t)(best >> 18);
+                    }
+#pragma unroll 1
+                    for (int s = tid; s < dc.n_shapes; s += NT) {
+                        if (bnd[s] < floor32) continue;
+                        const uint64_t key = score_key(s);
+                        bnd[s] = (uint32_t)(key >> 18);
+                        best = max_v(best, key);
+                    }
+                    best = big_warp_max64(best);
+                    if (lane == 0) red[warp] = (int64_t)best;
+                }
+                if (sat_cell) {                                  // (requested by the last emit step; back from L2 by now)
+                    *sat_cell = (uint16_t)min_v(sat_left, 65535u);
+                    sat_cell = nullptr;
                 }
                 __syncthreads();
-                int64_t best = lane < n_score_warps ? red[lane] : -1;
-                int best_s = lane < n_score_warps ? (int)red[32 + lane] : 0x7fffffff;
-                warp_argmax_first(best, best_s);
-                if (best <= 0) { st |= VP_ST_UNCOVERED; break; }
+                const uint64_t bkey = big_warp_max64(lane < n_warps ? (uint64_t)red[lane] : 0ull);
+                if ((bkey >> 16) == 0) { st |= VP_ST_UNCOVERED; break; }
+                const int best_s = 65535 - (int)(bkey & 0xffffu);
+                last_s = best_s;
                 const int f0 = (int)bucket[best_s], H = (int)bucket[best_s + 1] - f0;
                 const int n_tasks = H * kp.n_start;
                 VP_TICK(1);
@@ -340,90 +479,160 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
                     const int h = ns_shift >= 0 ? task >> ns_shift : task / kp.n_start, f = f0 + h, t = task - h * kp.n_start;
                     uint8_t* srcb = bind_src + (size_t)task * N;
                     uint8_t* dstb = bind_dst + (size_t)task * N;
+                    int64_t* pair = pairs + wgroup * 8;
                     uint32_t cap_out[4], cap_in[4];
                     int rq[4], cls_in[4];
+                    uint32_t my_dst = 0, my_src = 0;             // what this lane last wrote to the two bindings
+                    uint32_t hot_in = 0xffffffffu;               // hot-column indices of this group's four ranks (0xFF = none)
+                    if (hot_mode && active) hot_in = *((const uint32_t*)colmap + a);
                     if (active) {
-                        const uint32_t co = __ldg((const uint32_t*)(dc.fam_cls + (size_t)f * N) + a);
-                        const uint2 fi = __ldg((const uint2*)(dc.fam_in + (size_t)f * N) + a);
+                        uint32_t co;
+                        uint2 fi;
+                        const bool first = task == wgroup;
+                        if (first && f == f_cached) {             // the same family as in the last iteration: tables still held
+                            co = c_co; fi = c_fi;
+                        } else {
+                            co = __ldg((const uint32_t*)(dc.fam_cls + (size_t)f * N) + a);
+                            fi = __ldg((const uint2*)(dc.fam_in + (size_t)f * N) + a);
+                            if (t == 0) {                         // the family's slot words, parked for step (D)
+                                const uint4 sw = __ldg((const uint4*)(dc.fam_slot + (size_t)f * N) + a);
+                                *((uint4*)(slotw + h * N) + a) = sw;
+                            }
+                            if (first) { c_co = co; c_fi = fi; }
+                        }
+                        if (first) f_cached = f;
                         const uint32_t fw[4] = {fi.x & 0xffffu, fi.x >> 16, fi.y & 0xffffu, fi.y >> 16};
 #pragma unroll
                         for (int q = 0; q < 4; q++) {
-                            cap_out[q] = s_cap[(co >> (8 * q)) & 0xffu] << 8;
+                            cap_out[q] = s_cap[(co >> (8 * q)) & 0xffu];
                             rq[q] = (int)(fw[q] & 0xffu);
                             cls_in[q] = (int)(fw[q] >> 8);
-                            cap_in[q] = s_cap[cls_in[q]] << 8;
-                            dstb[rq[q]] = (uint8_t)(a * 4 + ((q + t) & 3));      // start t rotates the in-slots
-                        }
-                        if (t == 0) {                             // the family's slot words, parked for step (D)
-                            const uint4 sw = __ldg((const uint4*)(dc.fam_slot + (size_t)f * N) + a);
-                            *((uint4*)(slotw + h * N) + a) = sw;
+                            cap_in[q] = s_cap[cls_in[q]];
+                            const uint32_t d = (uint32_t)(a * 4 + ((q + t) & 3));   // start t rotates the in-slots
+                            dstb[rq[q]] = (uint8_t)d;
+                            my_dst |= d << (8 * q);
                         }
                     }
                     task_sync();
                     int64_t F_old = -1, F_new = -1;
-                    uint32_t xmax = 0;
-                    int64_t tmax = 0;
-                    int64_t* pair = pairs + wgroup * 6;
                     for (int sweep = 0; sweep < kp.i_aa; sweep++) {
+                        bool moved = false;
                         if (active) {                             // source half: one exact assignment per source group
                             const uint32_t d4 = *((const uint32_t*)dstb + a);
-                            uint32_t cr[4][4];
+                            uint32_t v[4][4];
 #pragma unroll
                             for (int q = 0; q < 4; q++) {
                                 const uint16_t* colp = Cs + (a * 4) * CS + ((d4 >> (8 * q)) & 0xffu);
 #pragma unroll
-                                for (int i = 0; i < 4; i++) cr[i][q] = min_v((uint32_t)colp[i * CS] << 8, cap_out[q]);
+                                for (int i = 0; i < 4; i++) v[i][q] = min_v((uint32_t)colp[i * CS], cap_out[q]) * 256u + big_tag(i, q);
                             }
-                            const uint32_t pb = ~big_best_key(cr) & 255u;
-                            *((uint32_t*)srcb + a) = (uint32_t)(a * 4) * 0x01010101u +
-                                                     (((pb >> 6) & 3u) | (((pb >> 4) & 3u) << 8) | (((pb >> 2) & 3u) << 16) | ((pb & 3u) << 24));
-                        }
-                        task_sync();
-                        uint32_t part = 0;
-                        if (active) {                             // destination half
-                            uint32_t cr[4][4];
+                            if (hot_mode) {                       // out-slots bound to a hot column: exact 32-bit cells
 #pragma unroll
-                            for (int q = 0; q < 4; q++) {
-                                const uint32_t* rowp = (const uint32_t*)(Cs + (int)srcb[rq[q]] * CS + a * 4);
-                                const uint32_t lo = rowp[0], hi = rowp[1];
-                                cr[0][q] = min_v(__byte_perm(lo, 0, 0x4104), cap_in[q]);     // (low half) << 8
-                                cr[1][q] = min_v(__byte_perm(lo, 0, 0x4324), cap_in[q]);     // (high half) << 8
-                                cr[2][q] = min_v(__byte_perm(hi, 0, 0x4104), cap_in[q]);
-                                cr[3][q] = min_v(__byte_perm(hi, 0, 0x4324), cap_in[q]);
+                                for (int q = 0; q < 4; q++) {
+                                    const int dq = (int)((d4 >> (8 * q)) & 0xffu), hc = colmap[dq];
+                                    if (hc != 0xFF) {
+#pragma unroll
+                                        for (int i = 0; i < 4; i++) {
+                                            const uint32_t val = (uint32_t)Cs[(a * 4 + i) * CS + dq] | (uint32_t)Hi[hc * N + a * 4 + i] << 16;
+                                            v[i][q] = min_v(val, cap_out[q]) * 256u + big_tag(i, q);
+                                        }
+                                    }
+                                }
                             }
-                            const uint32_t key = big_best_key(cr);
-                            const uint32_t pb = ~key & 255u;
-                            part = key >> 8;                      // key = (sum of credits) << 8 | tag
-#pragma unroll
-                            for (int q = 0; q < 4; q++) dstb[rq[q]] = (uint8_t)(a * 4 + ((pb >> (6 - 2 * q)) & 3u));
+                            const uint32_t pb = ~big_best_key(v) & 255u;
+                            const uint32_t word = (uint32_t)(a * 4) * 0x01010101u +
+                                                  (((pb >> 6) & 3u) | (((pb >> 4) & 3u) << 8) | (((pb >> 2) & 3u) << 16) | ((pb & 3u) << 24));
+                            moved = sweep == 0 || word != my_src;
+                            my_src = word;
+                            *((uint32_t*)srcb + a) = word;
                         }
-                        F_new = (int64_t)__reduce_add_sync(0xffffffffu, part);          // Eq. (8); at most 2^8 lanes of < 2^16
-                        if (W == 2) {                             // add the partner warp's half (slots alternate by sweep)
-                            if (lane == 0) pair[(sweep & 1) * 2 + sub] = F_new;
+                        // If no source binding moved, the destination half would see what it saw last sweep and return the
+                        // same binding and the same F: the run ends here exactly as it would after computing that.
+                        bool any_moved = __any_sync(0xffffffffu, moved);
+                        if (W == 2) {
+                            if (lane == 0) ((int32_t*)(pair + 6))[sub] = any_moved;
                             task_sync();
-                            F_new = pair[(sweep & 1) * 2] + pair[(sweep & 1) * 2 + 1];
+                            any_moved = (((const int32_t*)(pair + 6))[0] | ((const int32_t*)(pair + 6))[1]) != 0;
                         } else {
                             __syncwarp();
                         }
+                        if (!any_moved) {
+                            if (sub == 0 && lane == 0) n_sweeps++;
+                            F_new = F_old;
+                            break;
+                        }
+                        uint32_t part = 0;
+                        moved = false;
+                        if (active) {                             // destination half
+                            uint32_t v[4][4];
+#pragma unroll
+                            for (int q = 0; q < 4; q++) {
+                                const uint32_t* rowp = (const uint32_t*)(Cs + (int)srcb[rq[q]] * CS + a * 4);
+                                const uint32_t c2 = min_v(cap_in[q], 65535u) * 0x00010001u;   // the capacity in both halves
+                                const uint32_t lo = __vminu2(rowp[0], c2), hi = __vminu2(rowp[1], c2);
+                                v[0][q] = __byte_perm(lo, big_tag(0, q), 0x5104);  // (low half) << 8 | tag
+                                v[1][q] = __byte_perm(lo, big_tag(1, q), 0x5324);  // (high half) << 8 | tag
+                                v[2][q] = __byte_perm(hi, big_tag(2, q), 0x5104);
+                                v[3][q] = __byte_perm(hi, big_tag(3, q), 0x5324);
+                            }
+                            if (hot_in != 0xffffffffu) {          // some rank of this group is a hot column: exact 32-bit cells
+#pragma unroll
+                                for (int j = 0; j < 4; j++) {
+                                    const int hc = (int)((hot_in >> (8 * j)) & 0xffu);
+                                    if (hc != 0xFF) {
+#pragma unroll
+                                        for (int q = 0; q < 4; q++) {
+                                            const int sq = srcb[rq[q]];
+                                            const uint32_t val = (uint32_t)Cs[sq * CS + a * 4 + j] | (uint32_t)Hi[hc * N + sq] << 16;
+                                            v[j][q] = min_v(val, cap_in[q]) * 256u + big_tag(j, q);
+                                        }
+                                    }
+                                }
+                            }
+                            const uint32_t key = big_best_key(v);
+                            const uint32_t pb = ~key & 255u;
+                            part = key >> 8;
+                            uint32_t word = 0;
+#pragma unroll
+                            for (int q = 0; q < 4; q++) {
+                                const uint32_t d = (uint32_t)(a * 4) + ((pb >> (6 - 2 * q)) & 3u);
+                                dstb[rq[q]] = (uint8_t)d;
+                                word |= d << (8 * q);
+                            }
+                            moved = word != my_dst;
+                            my_dst = word;
+                        }
+                        // Eq. (8): at most 2^8 lanes of less than 2^18 granules.  The low bit carries "a destination
+                        // binding moved": if none did, the next sweep would be a repetition of this one (same sources, same
+                        // destinations, same F) and would end the run, so it is counted and skipped.
+                        uint32_t fm = __reduce_add_sync(0xffffffffu, part) << 1 | (uint32_t)__any_sync(0xffffffffu, moved);
+                        if (W == 2) {
+                            if (lane == 0) ((uint32_t*)(pair + (sweep & 1) * 2))[sub] = fm;
+                            task_sync();
+                            const uint32_t f0w = ((const uint32_t*)(pair + (sweep & 1) * 2))[0], f1w = ((const uint32_t*)(pair + (sweep & 1) * 2))[1];
+                            fm = ((f0w >> 1) + (f1w >> 1)) << 1 | ((f0w | f1w) & 1u);
+                        } else {
+                            __syncwarp();
+                        }
+                        F_new = (int64_t)(fm >> 1);
                         if (sub == 0 && lane == 0) n_sweeps++;
                         if (F_new <= F_old) break;
                         F_old = F_new;
-                    }
-                    // Eq. (9) volumes of the binding as it stands: the credit of every in-slot; slowest lane of Eq. (10)
-                    if (active) {
-#pragma unroll
-                        for (int q = 0; q < 4; q++) {
-                            const uint32_t x = min_v((uint32_t)Cs[(int)srcb[rq[q]] * CS + (int)dstb[rq[q]]], cap_in[q] >> 8);
-                            xmax = max_v(xmax, x);
-                            if (dc.n_classes > 1) tmax = max_v(tmax, (int64_t)x * s_tscale[cls_in[q]]);
+                        if (!(fm & 1u) && sweep + 1 < kp.i_aa) {
+                            if (sub == 0 && lane == 0) n_sweeps++;
+                            break;
                         }
                     }
-                    if (dc.n_classes == 1) tmax = (int64_t)__reduce_max_sync(0xffffffffu, xmax) * s_tscale[0];
-                    else tmax = warp_max_i64(tmax);
-                    if (W == 2) {
-                        if (lane == 0) pair[4 + sub] = tmax;
-                        task_sync();
-                        tmax = max_v(pair[4], pair[5]);
+                    // Eq. (9) volumes of the binding as it stands (the credit of every in-slot) and the slowest lane of
+                    // Eq. (10): only needed when several families compete on utility
+                    int64_t tmax = 0;
+                    if (H > 1) {
+                        tmax = big_slowest_lane(Cs, CS, Hi, colmap, N, hot_mode, srcb, dstb, rq, cap_in, cls_in, s_tscale, dc.n_classes, active);
+                        if (W == 2) {
+                            if (lane == 0) pair[4 + sub] = tmax;
+                            task_sync();
+                            tmax = max_v(pair[4], pair[5]);
+                        }
                     }
                     if (lane == 0 && sub == 0) {
                         n_tasks_done++;
@@ -437,53 +646,40 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
                 // (C) best start per family (largest F, lowest t), then largest utility, lowest family
                 int wtask;
                 int64_t wF;
-                if (H == 1 && kp.n_start <= 32) {
-                    int64_t ff = lane < kp.n_start ? task_f[lane] : -1;
-                    int tt = lane;
-                    warp_argmax_first(ff, tt);
-                    wtask = tt; wF = ff;
+                if (H == 1 && kp.n_start == 4) {                 // one family, four starts: best start, no utilities to compare
+                    const int64_t f0v = task_f[0], f1v = task_f[1], f2v = task_f[2], f3v = task_f[3];
+                    const int64_t m01 = max_v(f0v, f1v), m23 = max_v(f2v, f3v);
+                    wF = max_v(m01, m23);
+                    wtask = m01 >= m23 ? (f0v >= f1v ? 0 : 1) : (f2v >= f3v ? 2 : 3);
+                } else if (H == 1) {
+                    wtask = 0; wF = task_f[0];
+                    for (int t = 1; t < kp.n_start; t++)
+                        if (task_f[t] > wF) { wF = task_f[t]; wtask = t; }
                 } else {
-                    int64_t bf = -1, bd = 1;
-                    int bt = 0x7fffffff;
-                    for (int h = lane; h < H; h += 32) {
-                        int64_t ff = -1; int tt = 0;
-                        for (int t = 0; t < kp.n_start; t++)
-                            if (task_f[h * kp.n_start + t] > ff) { ff = task_f[h * kp.n_start + t]; tt = h * kp.n_start + t; }
-                        if (bt == 0x7fffffff || util_greater(ff, task_den[tt], bf, bd)) { bf = ff; bd = task_den[tt]; bt = tt; }
-                    }
-                    for (int o = 16; o; o >>= 1) {
-                        const int64_t of = __shfl_xor_sync(0xffffffffu, bf, o), od = __shfl_xor_sync(0xffffffffu, bd, o);
-                        const int ot = __shfl_xor_sync(0xffffffffu, bt, o);
-                        bool take = false;
-                        if (ot != 0x7fffffff) {
-                            if (bt == 0x7fffffff) take = true;
-                            else if (util_greater(of, od, bf, bd)) take = true;
-                            else if (!util_greater(bf, bd, of, od) && ot < bt) take = true;
-                        }
-                        if (take) { bf = of; bd = od; bt = ot; }
-                    }
-                    wtask = __shfl_sync(0xffffffffu, bt, 0);
-                    wF = __shfl_sync(0xffffffffu, bf, 0);
+                    big_select_family(task_f, task_den, H, kp.n_start, lane, wtask, wF);
                 }
                 if (wF <= 0) { st |= VP_ST_NO_PROGRESS; break; }
                 VP_TICK(3);
 
                 // (D) emit activation k: volumes off the residual and off the score table, next offset row
-                {
+                if (warp * 32 < N) {
                     const int h = ns_shift >= 0 ? wtask >> ns_shift : wtask / kp.n_start;
                     const uint32_t* slot = slotw + h * N;
                     const uint8_t* srcb = bind_src + (size_t)wtask * N;
                     const uint8_t* dstb = bind_dst + (size_t)wtask * N;
                     const size_t row = (size_t)k * N, orow = (size_t)(k + 1) * N;
-                    for (int r0 = warp * 32; r0 < N; r0 += NT) {  // whole warps: the sums below need every lane
-                        const int r = r0 + lane;
-                        const bool live = r < N;
-                        uint32_t x = 0, mine = 0xffffffffu;
-                        if (live) {
+                    for (int r = tid; r < N; r += NT) {
+                        uint32_t x = 0;
+                        {
                             const uint32_t w = slot[r];
                             const int i = srcb[r], j = dstb[r];
                             uint16_t* cell = Cs + i * CS + j;
-                            const uint32_t c = *cell;
+                            uint32_t c = *cell;
+                            uint16_t* hcell = nullptr;
+                            if (hot_mode && colmap[j] != 0xFF) {  // a hot column: the exact 32-bit cell
+                                hcell = Hi + (int)colmap[j] * N + i;
+                                c |= (uint32_t)*hcell << 16;
+                            }
                             x = min_v(s_cap[(w >> 24) & 0xf], c);
                             const bool busy = x > 0;
                             const int64_t bytes = (int64_t)x * kp.granule;
@@ -496,47 +692,53 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
                             send_off_b[orow + i] = sa;            // src and dst are permutations: every rank is written once
                             if (recv_off_b) recv_off_b[orow + j] = ra;
                             if (busy) {
-                                uint32_t nv = c - x;
-                                if (c == 65535u) {                // saturated: the exact residual is in the workspace slot
-                                    nv = atomicSub(&Dg[(size_t)i * N + j], x) - x;
-                                    nv = min_v(nv, 65535u);
+                                if (hcell) {
+                                    *cell = (uint16_t)(c - x);
+                                    *hcell = (uint16_t)((c - x) >> 16);
+                                } else if (c == 65535u && !hot_mode) {   // saturated: the exact residual is in the workspace slot;
+                                    sat_cell = cell;              // its new value is put in place before the next Step 2
+                                    sat_left = atomicSub(&Dg[(size_t)i * N + j], x) - x;
+                                } else {
+                                    *cell = (uint16_t)(c - x);
                                 }
-                                *cell = (uint16_t)nv;
+                                // the volume leaves the table entry of its group pair
                                 const int ga = i >> 2, gd = j >> 2;
                                 int delta = (int)gnode[gd] - (int)gnode[ga];
                                 if (delta < 0) delta += P;
-                                mine = (uint32_t)((delta * S + gnode[G + ga]) * S + gnode[G + gd]);
-                            }
-                        }
-                        // the volumes leave the table entries of their group pairs: the lanes of an activation fall into
-                        // the entries of the chosen shape's terms, so one warp sum per such entry, then one atomic each
-                        for (int q = 0; q < S; q++) {
-                            const uint32_t pid = (spat[(q >> 1) * ns_pad + best_s] >> (16 * (q & 1))) & 0xffffu;
-                            for (int t = 0; t < dc.max_row_terms; t++) {
-                                const uint32_t tw = pat[pid * dc.max_row_terms + t];
-                                if (!(tw >> 16)) continue;                // (the same word in every thread)
-                                const uint32_t sum = __reduce_add_sync(0xffffffffu, mine == (tw & 0xffffu) ? x : 0u);
-                                if (lane == 0 && sum) atomicSub(&tbl[tw & 0xffffu], sum);
+                                atomicSub(&tbl[(delta * S + gnode[G + ga]) * S + gnode[G + gd]], x);
                             }
                         }
                     }
                     if (tid == 0) chan_id_b[k] = f0 + h;
-                    left -= wF;
                 }
+                left -= wF;
                 k++;
                 __syncthreads();
                 VP_TICK(4);
             }
         }
         __syncthreads();
-        // ---- idle rows beyond n_steps; offset rows repeat the totals
-        for (size_t e = (size_t)k * N + tid; e < (size_t)kp.k_max * N; e += NT) {
-            lane_dst_b[e] = -1;
-            lane_inst_b[e] = 0xFFFF;
-            lane_bytes_b[e] = 0;
-            const int i = (int)(e % N);
-            send_off_b[N + e] = send_acc[i];
-            if (recv_off_b) recv_off_b[N + e] = recv_acc[i];
+        // ---- idle rows beyond n_steps (16-byte stores); offset rows repeat the totals
+        {
+            const size_t lo = (size_t)k * N, hi = (size_t)kp.k_max * N;
+            big_fill_bytes((unsigned char*)lane_dst_b, lo * 2, hi * 2, 0xff, tid, NT);
+            big_fill_bytes((unsigned char*)lane_inst_b, lo * 2, hi * 2, 0xff, tid, NT);
+            big_fill_bytes((unsigned char*)lane_bytes_b, lo * 8, hi * 8, 0x00, tid, NT);
+            const bool vec = (((uintptr_t)send_off_b | (uintptr_t)(recv_off_b ? recv_off_b : send_off_b)) & 15) == 0;
+            if (vec) {                                       // N is a multiple of four: rows are whole 16-byte pairs
+                const int half = N / 2;
+                for (size_t e = lo / 2 + tid; e < hi / 2; e += NT) {
+                    const int i2 = (int)(e % half);
+                    ((longlong2*)(send_off_b + N))[e] = ((const longlong2*)send_acc)[i2];
+                    if (recv_off_b) ((longlong2*)(recv_off_b + N))[e] = ((const longlong2*)recv_acc)[i2];
+                }
+            } else {
+                for (size_t e = lo + tid; e < hi; e += NT) {
+                    const int i = (int)(e % N);
+                    send_off_b[N + e] = send_acc[i];
+                    if (recv_off_b) recv_off_b[N + e] = recv_acc[i];
+                }
+            }
         }
         for (int kk = k + tid; kk < kp.k_max; kk += NT) chan_id_b[kk] = -1;
         if (tid == 0) {

@@ -370,6 +370,37 @@ def test_mid_size_template_catalogs(vp, oracle_lib, nodes):
         _assert_same(got, want)
 
 
+@pytest.mark.parametrize("nodes", [9, 32])
+def test_large_capacities_and_hot_columns(vp, oracle_lib, nodes):
+    """Node-symmetric catalogs of more than sixteen groups with lane capacities of 2^16 granules and more: a few columns
+    (popular destinations) hold cells far above 65,535 granules and are kept exactly beside the 16-bit credits; with
+    too many such columns, or capacities of 2^22 granules and more, the general kernel takes the matrix.  Mixed in one
+    batch with ordinary matrices, uniform and mixed rates."""
+    cat = node_template_catalog(tree_topology(nodes, pcie_bw=64, nic_bw=50 if nodes == 9 else 64))
+    N = cat.topology.N
+    rng = np.random.default_rng(100 + nodes)
+    u = 256
+    B = 7
+    D = (rng.integers(0, 3000, size=(B, N, N)) * (rng.random((B, N, N)) < 0.5)).astype(np.int64)
+    hot = rng.choice(N, size=5, replace=False)
+    D[0][:, hot] = rng.integers(60_000, 3_000_000, size=(N, 5))          # five hot columns, capacity well above 2^16
+    D[1][:, hot[:2]] = rng.integers(65_535, 65_540, size=(N, 2))         # cells right at the 16-bit boundary
+    D[2][:, rng.choice(N, size=40, replace=False)] = 200_000             # more hot columns than are kept: general kernel
+    D[3][:, hot[:1]] = rng.integers(1 << 27, 1 << 28, size=(N, 1))       # capacity of 2^22 granules and more: general kernel
+    D[4][hot[:3], :] = rng.integers(60_000, 900_000, size=(3, N))        # hot rows instead: every column is hot or none
+    D[5] = 0
+    D *= u
+    for b in range(B):
+        np.fill_diagonal(D[b], 0)
+    for extra in ({}, {"n_start": 2, "i_aa": 5, "lambda_ns": 0}):
+        w = WParams(granule_bytes=u, k_max=12 * N, **extra).resolved(N)
+        got, want, *_ = _both(vp, oracle_lib, cat, D, w)
+        _assert_same(got, want)
+    tau = np.array([0, 70_000 * u // 50, 0, 0, 0, 1, 0], np.int64)       # a given quantum that puts matrix 1 in hot mode
+    got, want, *_ = _both(vp, oracle_lib, cat, D, WParams(granule_bytes=u, k_max=12 * N).resolved(N), tau=tau)
+    _assert_same(got, want)
+
+
 def test_batches_around_one_wave(vp, oracle_lib):
     """Batch sizes just below and above the number of resident CTAs: the kernel changes, the plans do not."""
     c = build_config(2)
