@@ -1129,7 +1129,7 @@ static_assert(sizeof(Launch) <= sizeof(((vp_launch_memo*)0)->launch), "the launc
 typedef void (*KernelFn)(DevCat, KParams, const int64_t*, const int64_t*, int, int32_t*, int32_t*, int16_t*, uint16_t*,
                          int64_t*, int64_t*, int64_t*, int64_t*, int32_t*, int64_t*, unsigned int*, const int*);
 typedef void (*BigKernelFn)(DevCat, KParams, const int64_t*, const int64_t*, int, int32_t*, int32_t*, int16_t*, uint16_t*,
-                            int64_t*, int64_t*, int64_t*, int64_t*, int32_t*, int64_t*, unsigned int*, int*);
+                            int64_t*, int64_t*, int64_t*, int64_t*, int32_t*, int64_t*, unsigned int*, int*, const int*);
 
 KernelFn pick_kernel(int g, int lpg) {
     switch (g) {
@@ -1277,7 +1277,7 @@ size_t workspace_bytes(const vp_catalog* c, const Launch& L, int B) {
     // for large node-symmetric catalogs also the list of matrices left to the general kernel
     const int slots = L.kernel == 2 ? (L.grid > L.big_grid ? L.grid : L.big_grid) : L.grid;
     size_t drem = L.kp.drem_in_smem ? 0 : (size_t)slots * c->dc.N * c->dc.N * 8;
-    size_t list = L.kernel == 2 ? vp_align256((size_t)B * 4) : 0;
+    size_t list = L.kernel == 2 ? 3 * vp_align256((size_t)B * 4) : 0;     // left-over list, work order, its keys
     return vp_align256(256 + drem) + list;
 }
 
@@ -1322,9 +1322,17 @@ extern "C" int vp_schedule_batch(const vp_catalog* c, const vp_sched_params* p, 
             } else if (L.kernel == 2) {
                 const int slots = L.grid > L.big_grid ? L.grid : L.big_grid;
                 int* todo = (int*)((char*)workspace + vp_align256(256 + (size_t)slots * c->dc.N * c->dc.N * 8));
+                int* order = nullptr;
+                if (B > L.big_grid && B <= 16384) {          // more matrices than CTAs: longest first (see big_rank_kernel)
+                    order = todo + vp_align256((size_t)B * 4) / 4;
+                    int* key = order + vp_align256((size_t)B * 4) / 4;
+                    big_count_nonzero_kernel<<<(B + 7) / 8, 256, 0, stream>>>(demand, B, c->dc.N * c->dc.N, key);
+                    big_rank_kernel<<<(B + 255) / 256, 256, 0, stream>>>(key, B, order);
+                    g_vp_launches += 2;
+                }
                 pick_big_kernel(L.big_w)<<<L.big_grid, L.big_threads, L.big_smem, stream>>>(
                     c->dc, L.kp, demand, tau_ns_in, B, n_steps, chan_id, lane_dst, lane_inst, lane_bytes, send_off, recv_off,
-                    tau_ns_out, status, ws_drem, counter, todo);
+                    tau_ns_out, status, ws_drem, counter, todo, order);
                 g_vp_launches++;
                 pick_kernel(c->dc.g, L.lpg)<<<L.grid, L.threads, L.smem, stream>>>(
                     c->dc, L.kp, demand, tau_ns_in, B, n_steps, chan_id, lane_dst, lane_inst, lane_bytes, send_off, recv_off,

@@ -164,6 +164,32 @@ __device__ __noinline__ int64_t big_slowest_lane(const uint16_t* Cs, int CS, con
     return warp_max_i64(tmax);
 }
 
+// Work order for a batch whose matrices differ a lot in length: the number of non-zero cells predicts the number of
+// activations well (dense cross-node MoE demand takes several times as many as block-diagonal sequence-parallel
+// demand), and CTAs that take the long matrices first leave a short tail.  One warp counts one matrix ...
+__global__ void __launch_bounds__(256) big_count_nonzero_kernel(const int64_t* __restrict__ demand, int B, int cells, int* __restrict__ key) {
+    const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (b >= B) return;
+    const int64_t* D = demand + (size_t)b * cells;
+    int n = 0;
+    for (int e = lane; e < cells; e += 32) n += D[e] != 0;
+    n = __reduce_add_sync(0xffffffffu, n);
+    if (lane == 0) key[b] = n;
+}
+// ... and every matrix finds its place by counting the matrices that go before it (more non-zero cells, or as many
+// and a lower index): B^2 comparisons over the whole grid, a few microseconds for a few thousand matrices.
+__global__ void __launch_bounds__(256) big_rank_kernel(const int* __restrict__ key, int B, int* __restrict__ order) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= B) return;
+    const int mine = key[b];
+    int before = 0;
+    for (int o = 0; o < B; o++) {
+        const int other = __ldg(&key[o]);
+        before += other > mine || (other == mine && o < b);
+    }
+    order[before] = b;
+}
+
 // W = warps per (family, start) task: one lane per rank group, 32 W >= G.
 template <int W>
 __global__ void __launch_bounds__(512, 1)
@@ -171,7 +197,8 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
                        int32_t* __restrict__ n_steps, int32_t* __restrict__ chan_id, int16_t* __restrict__ lane_dst,
                        uint16_t* __restrict__ lane_inst, int64_t* __restrict__ lane_bytes, int64_t* __restrict__ send_off,
                        int64_t* __restrict__ recv_off, int64_t* __restrict__ tau_out, int32_t* __restrict__ status,
-                       int64_t* ws_drem, unsigned int* counter, int* __restrict__ todo) {
+                       int64_t* ws_drem, unsigned int* counter, int* __restrict__ todo, const int* __restrict__ order) {
+    // `order` (may be null) lists the matrices in the order in which the CTAs should take them: longest first.
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int N = dc.N, G = dc.G, tid = threadIdx.x, NT = blockDim.x;
     const int lane = tid & 31, warp = tid >> 5, n_warps = NT >> 5;
@@ -245,7 +272,11 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
     const int ns_shift = (kp.n_start & (kp.n_start - 1)) == 0 ? 31 - __clz(kp.n_start) : -1;
 
     for (;;) {
-        if (tid == 0) { s_b = (int)atomicAdd(counter, 1u); s_flags = 0; }
+        if (tid == 0) {
+            const unsigned at = atomicAdd(counter, 1u);
+            s_b = at < (unsigned)B ? (order ? order[at] : (int)at) : B;
+            s_flags = 0;
+        }
         __syncthreads();
         const int b = s_b;
         if (b >= B) break;
