@@ -56,6 +56,11 @@ extern "C" {
 #define VP_ST_STEP_LIMIT    128   /* k_max activations emitted, residual demand left              */
 #define VP_ST_PACK_MISMATCH 256   /* vp_pack: routed copies disagree with the plan's byte counts  */
 #define VP_ST_PACK_CAPACITY 512   /* vp_pack: staged buffer smaller than the plan's send volume   */
+/* Row-copy kernels (vp_pack, vp_pack_static, vp_unpack, vp_unpack_tokens): a bounded wait for an asynchronous
+ * copy into shared memory gave up (2^22 polls; never seen in practice).  The kernel then issues no further
+ * loads, lets the stores it already issued finish and returns; the output buffer is INCOMPLETE and the call
+ * must be repeated.  Nothing faults and the context stays usable. */
+#define VP_ST_INTERNAL_TIMEOUT (1 << 30)
 /* Bits 1..16 reject the matrix before scheduling: n_steps[b] = 0 and an empty plan. */
 
 typedef struct vp_catalog vp_catalog;   /* opaque, owned by the library */
@@ -242,8 +247,10 @@ int vp_pack(const int32_t* n_steps_b, const int16_t* lane_dst_b, const int64_t* 
  * given the input and output buffers and nothing else; it owns no allocator, and calling cudaMalloc there
  * is off the table (the call synchronises the whole device, may fail under the engine's memory cap, and
  * bypasses the engine's own accounting).  For these callers the library carries its own scratch: one
- * block of VP_PACK_STATIC_SCRATCH_BYTES of device memory that every GPU which loads the library sets
- * aside at load time and keeps until the process exits.  The call allocates nothing, on host or device.
+ * block of VP_PACK_STATIC_SCRATCH_BYTES of device memory per GPU, which the CUDA runtime sets aside when the
+ * library's pack code is first used on that GPU (with lazy module loading that can be inside the first
+ * vp_pack_static call itself) and keeps until the process exits.  Calls after the first one on a device
+ * allocate nothing, on host or device.
  *
  * Arguments, results and status bits are those of vp_pack; inputs and outputs are still the caller's.
  * Limits and rules:

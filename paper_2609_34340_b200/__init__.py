@@ -36,6 +36,6 @@ from .binding import (  # noqa: F401
     profile_read,
     library_path,
     ST_NEGATIVE, ST_OVERFLOW_RISK, ST_DIAG_NONZERO, ST_NOT_GRANULE, ST_BAD_TAU, ST_UNCOVERED,
-    ST_NO_PROGRESS, ST_STEP_LIMIT, ST_PACK_MISMATCH, ST_PACK_CAPACITY,
+    ST_NO_PROGRESS, ST_STEP_LIMIT, ST_PACK_MISMATCH, ST_PACK_CAPACITY, ST_INTERNAL_TIMEOUT,
     E_BAD_ARG, E_BAD_CATALOG, E_NOMEM, E_CUDA, E_WORKSPACE, E_UNSUPPORTED,
 )

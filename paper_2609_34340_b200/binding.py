@@ -18,6 +18,7 @@ E_BAD_ARG, E_BAD_CATALOG, E_NOMEM, E_CUDA, E_WORKSPACE, E_UNSUPPORTED = -1, -2, 
 ST_NEGATIVE, ST_OVERFLOW_RISK, ST_DIAG_NONZERO, ST_NOT_GRANULE = 1, 2, 4, 8
 ST_BAD_TAU, ST_UNCOVERED, ST_NO_PROGRESS, ST_STEP_LIMIT = 16, 32, 64, 128
 ST_PACK_MISMATCH, ST_PACK_CAPACITY = 256, 512
+ST_INTERNAL_TIMEOUT = 1 << 30    # a row-copy kernel gave up a bounded wait: the output buffer is incomplete
 
 
 class VpError(RuntimeError):

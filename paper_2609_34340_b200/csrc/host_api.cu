@@ -53,6 +53,17 @@ SchedBufs carve_sched(void* base, const vp_catalog* c, int B, const vp_sched_par
             return VP_E_CUDA;                                                                 \
     } while (0)
 
+// Makes a device current for the lifetime of a call and puts the caller's device back on every way out.
+struct DeviceScope {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceScope(int device) {
+        cudaGetDevice(&prev);
+        if (prev != device) ok = cudaSetDevice(device) == cudaSuccess;
+    }
+    ~DeviceScope() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
 }  // namespace
 
 extern "C" size_t vp_schedule_host_scratch_bytes(const vp_catalog* c, int B, const vp_sched_params* p) {
@@ -75,9 +86,8 @@ extern "C" int vp_schedule_batch_host(const vp_catalog* c, const vp_sched_params
     if (device_scratch_bytes < s.total) return VP_E_WORKSPACE;
     cudaStream_t stream = (cudaStream_t)cuda_stream;
     const size_t N = (size_t)c->info.N, K = (size_t)p->k_max, b = (size_t)B;
-    int prev = -1;
-    cudaGetDevice(&prev);
-    if (cudaSetDevice(c->device) != cudaSuccess) return VP_E_CUDA;
+    DeviceScope scope(c->device);
+    if (!scope.ok) return VP_E_CUDA;
     VP_COPY(s.demand, demand, b * N * N * 8, cudaMemcpyHostToDevice);
     if (tau_ns_in) VP_COPY(s.tau_in, tau_ns_in, b * 8, cudaMemcpyHostToDevice);
     int rc = vp_schedule_batch(c, p, s.demand, tau_ns_in ? s.tau_in : nullptr, B, s.n_steps, s.chan_id, s.lane_dst,
@@ -94,7 +104,6 @@ extern "C" int vp_schedule_batch_host(const vp_catalog* c, const vp_sched_params
     if (tau_ns_out) VP_COPY(tau_ns_out, s.tau_out, b * 8, cudaMemcpyDeviceToHost);
     VP_COPY(status, s.status, b * 4, cudaMemcpyDeviceToHost);
     if (cudaStreamSynchronize(stream) != cudaSuccess) return VP_E_CUDA;
-    if (prev >= 0) cudaSetDevice(prev);
     return VP_OK;
 }
 

@@ -10,12 +10,18 @@ namespace {
 constexpr int kKinds = 4;
 bool g_on = false;
 std::vector<cudaEvent_t> g_begin[kKinds], g_end[kKinds];
+std::vector<cudaEvent_t> g_pool;       // events handed back by vp_profile_read, reused by later marks
 }  // namespace
 
 void vp_prof_mark(int kind, int edge, cudaStream_t stream) {
     if (!g_on || kind < 0 || kind >= kKinds) return;
     cudaEvent_t ev;
-    if (cudaEventCreate(&ev) != cudaSuccess) return;
+    if (!g_pool.empty()) {
+        ev = g_pool.back();
+        g_pool.pop_back();
+    } else if (cudaEventCreate(&ev) != cudaSuccess) {
+        return;
+    }
     cudaEventRecord(ev, stream);
     (edge ? g_end : g_begin)[kind].push_back(ev);
 }
@@ -38,8 +44,8 @@ extern "C" int vp_profile_read(int kind, double* total_ms, int64_t* launches) {
             rc = VP_E_CUDA;
         else { total += ms; n++; }
     }
-    for (cudaEvent_t e : g_begin[kind]) cudaEventDestroy(e);
-    for (cudaEvent_t e : g_end[kind]) cudaEventDestroy(e);
+    for (cudaEvent_t e : g_begin[kind]) g_pool.push_back(e);
+    for (cudaEvent_t e : g_end[kind]) g_pool.push_back(e);
     g_begin[kind].clear();
     g_end[kind].clear();
     *total_ms = total;

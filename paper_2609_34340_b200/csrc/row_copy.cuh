@@ -15,7 +15,6 @@ namespace {
 constexpr int kPiece = 16384;              // bytes per bulk transfer (rows longer than this are split)
 constexpr int kMinBulkRow = 2048;          // shorter rows use the plain-load kernel
 constexpr unsigned kSpinLimit = 1u << 22;  // bounded mbarrier wait
-constexpr int VP_ST_INTERNAL_TIMEOUT = 1 << 30;
 
 // One warp per CTA.  A "unit" is one piece (<= kPiece bytes) of one source row.  Units are dealt to CTAs round
 // robin.  Unit u is loaded into stage u % S, kLook units ahead of its stores.  The destination rows of a unit
@@ -96,6 +95,7 @@ pack_copy_bulk_kernel(const char* __restrict__ rows, char* __restrict__ staged, 
                 }
                 failed = __any_sync(0xffffffffu, failed);
                 phase ^= 1u << s;
+                if (!failed) loaded &= ~(1u << s);   // this stage's load has landed
                 if (!failed) {
                     const unsigned bytes = (unsigned)min((long long)kPiece, row_bytes - (long long)p * kPiece);
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -118,7 +118,19 @@ pack_copy_bulk_kernel(const char* __restrict__ rows, char* __restrict__ staged, 
         }
     }
     bulk_wait_all();                                 // stores must finish before shared memory is released
-    if (failed && lane == 0) atomicOr(status, VP_ST_INTERNAL_TIMEOUT);
+    if (failed) {
+        // Give-up path: no further loads were issued.  Loads already in flight must not land in shared memory that
+        // the next CTA owns, so each is given one more bounded wait (the stage whose wait gave up had its parity
+        // flipped: put it back first).  Then the status bit tells the caller that the output is incomplete.
+        for (int s = 0; s < S; s++) {
+            if (!(loaded & (1u << s))) continue;
+            unsigned spins = 0;
+            while (!mbar_try_wait(smem_u32(&bars[s]), ((phase >> s) & 1u) ^ 1u) && !mbar_try_wait(smem_u32(&bars[s]), (phase >> s) & 1u) &&
+                   ++spins < (1u << 18)) {
+            }
+        }
+        if (lane == 0) atomicOr(status, VP_ST_INTERNAL_TIMEOUT);
+    }
 }
 
 // Plain-load path (short or unaligned rows): one warp per token, V-byte vectors.
@@ -157,16 +169,27 @@ pack_copy_plain_kernel(const char* __restrict__ rows, char* __restrict__ staged,
 // `flags[0] != 0` (device) turns the copy into a no-op.  Returns VP_OK or VP_E_CUDA.
 inline int launch_row_copy(const void* rows, void* out, const int32_t* dst_row, const int32_t* flags, int n_src, int fanout,
                            long long row_bytes, int32_t* status, cudaStream_t stream) {
-    int dev = 0, sms = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-        return VP_E_CUDA;
+    // per device, once: the SM count and the bulk kernel's shared-memory limit (kept out of the per-call path)
+    static int s_sms[64] = {0};
+    static bool s_attr_set[64] = {false};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return VP_E_CUDA;
+    const bool cached = dev >= 0 && dev < 64;
+    int sms = cached ? s_sms[dev] : 0;
+    if (!sms) {
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return VP_E_CUDA;
+        if (cached) s_sms[dev] = sms;
+    }
     const bool aligned16 = row_bytes % 16 == 0 && ((uintptr_t)rows & 15) == 0 && ((uintptr_t)out & 15) == 0;
     if (aligned16 && row_bytes >= kMinBulkRow) {
         constexpr int S = 6;
         const int pieces = (int)((row_bytes + kPiece - 1) / kPiece);
         const size_t smem = (size_t)S * kPiece;
-        if (cudaFuncSetAttribute(pack_copy_bulk_kernel<S>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-            return VP_E_CUDA;
+        if (!cached || !s_attr_set[dev]) {
+            if (cudaFuncSetAttribute(pack_copy_bulk_kernel<S>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+                return VP_E_CUDA;
+            if (cached) s_attr_set[dev] = true;
+        }
         pack_copy_bulk_kernel<S><<<sms * 2, 32, smem, stream>>>((const char*)rows, (char*)out, dst_row, flags, n_src, fanout,
                                                                 row_bytes, pieces, status);
     } else {

@@ -1112,6 +1112,10 @@ vp_schedule_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand, co
 #include "schedule_warp.cuh"
 #include "schedule_big.cuh"
 
+#ifndef VP_BIG_MIN_GROUPS
+#define VP_BIG_MIN_GROUPS 16      // node-symmetric catalogs with at least this many groups of four take vp_schedule_big_kernel
+#endif
+
 namespace {
 
 struct Launch {
@@ -1204,16 +1208,20 @@ int plan_launch_uncached(const vp_catalog* c, int B, const vp_sched_params* p, L
 #ifndef VP_NO_BIG_KERNEL
     // Large node-symmetric catalogs (groups of four, more than sixteen groups): 16-bit credits in shared memory and
     // scores on the per-node-offset table; the general kernel then takes whatever matrices that kernel left.
-    if (dc.g == 4 && dc.G > 16 && dc.G <= 64 && dc.sym && dc.shape_pat && dc.n_patterns < 1024 && dc.n_classes <= 15) {
+    const int big_min_groups = VP_BIG_MIN_GROUPS;
+    if (dc.g == 4 && dc.G >= big_min_groups && dc.G <= 64 && dc.sym && dc.shape_pat && dc.n_patterns < 1024 && dc.n_classes <= 15) {
         const size_t smem = (size_t)big_smem_layout(dc, L.kp).total;
         if (smem + 2048 <= (size_t)c->max_smem_optin) {
+            // one lane per group: two warps per task beyond 32 groups, and then sixteen warps for shape scoring and the
+            // emit step; up to 32 groups a task is one warp and four to eight warps per CTA leave room for several CTAs per SM
             const int w = dc.G > 32 ? 2 : 1;
+            const int threads = w == 2 ? 512 : (dc.G > 16 ? 256 : 128);
             BigKernelFn bf = pick_big_kernel(w);
             if (cudaFuncSetAttribute(bf, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return VP_E_CUDA;
             int bper_sm = 0;
-            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&bper_sm, bf, 512, smem) != cudaSuccess || bper_sm < 1) return VP_E_CUDA;
+            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&bper_sm, bf, threads, smem) != cudaSuccess || bper_sm < 1) return VP_E_CUDA;
             const long long bcap = (long long)bper_sm * c->sm_count;
-            L.kernel = 2; L.big_w = w; L.big_threads = 512; L.big_smem = smem;
+            L.kernel = 2; L.big_w = w; L.big_threads = threads; L.big_smem = smem;
             L.big_grid = (int)(B < bcap ? B : bcap);
             L.wave = (int)bcap;
         }
@@ -1272,14 +1280,23 @@ int plan_launch(const vp_catalog* cc, int B, const vp_sched_params* p, Launch* o
     return VP_OK;
 }
 
-size_t workspace_bytes(const vp_catalog* c, const Launch& L, int B) {
-    // 256 bytes of counters; one residual slot per CTA when the residual does not fit shared memory; with the kernel
-    // for large node-symmetric catalogs also the list of matrices left to the general kernel
+// Workspace: 256 bytes of counters; one residual slot per CTA when a kernel keeps the residual outside shared memory
+// (the kernel for large node-symmetric catalogs always has one, for its saturated cells); with that kernel also the
+// list of matrices left to the general kernel, the work order and its keys.
+struct WsLayout { size_t drem, todo, order, key, total; };
+WsLayout ws_layout(const vp_catalog* c, const Launch& L, int B) {
+    WsLayout w;
     const int slots = L.kernel == 2 ? (L.grid > L.big_grid ? L.grid : L.big_grid) : L.grid;
-    size_t drem = L.kp.drem_in_smem ? 0 : (size_t)slots * c->dc.N * c->dc.N * 8;
-    size_t list = L.kernel == 2 ? 3 * vp_align256((size_t)B * 4) : 0;     // left-over list, work order, its keys
-    return vp_align256(256 + drem) + list;
+    const size_t slot_bytes = (L.kernel == 2 || !L.kp.drem_in_smem) ? (size_t)slots * c->dc.N * c->dc.N * 8 : 0;
+    w.drem = 256;
+    w.todo = vp_align256(256 + slot_bytes);
+    const size_t list = L.kernel == 2 ? vp_align256((size_t)B * 4) : 0;
+    w.order = w.todo + list;
+    w.key = w.order + list;
+    w.total = w.key + list;
+    return w;
 }
+size_t workspace_bytes(const vp_catalog* c, const Launch& L, int B) { return ws_layout(c, L, B).total; }
 
 }  // namespace
 
@@ -1320,12 +1337,12 @@ extern "C" int vp_schedule_batch(const vp_catalog* c, const vp_sched_params* p, 
                     c->dc, L.kp, demand, tau_ns_in, B, n_steps, chan_id, lane_dst, lane_inst, lane_bytes, send_off, recv_off,
                     tau_ns_out, status, counter);
             } else if (L.kernel == 2) {
-                const int slots = L.grid > L.big_grid ? L.grid : L.big_grid;
-                int* todo = (int*)((char*)workspace + vp_align256(256 + (size_t)slots * c->dc.N * c->dc.N * 8));
+                const WsLayout w = ws_layout(c, L, B);
+                int* todo = (int*)((char*)workspace + w.todo);
                 int* order = nullptr;
                 if (B > L.big_grid && B <= 16384) {          // more matrices than CTAs: longest first (see big_rank_kernel)
-                    order = todo + vp_align256((size_t)B * 4) / 4;
-                    int* key = order + vp_align256((size_t)B * 4) / 4;
+                    order = (int*)((char*)workspace + w.order);
+                    int* key = (int*)((char*)workspace + w.key);
                     big_count_nonzero_kernel<<<(B + 7) / 8, 256, 0, stream>>>(demand, B, c->dc.N * c->dc.N, key);
                     big_rank_kernel<<<(B + 255) / 256, 256, 0, stream>>>(key, B, order);
                     g_vp_launches += 2;

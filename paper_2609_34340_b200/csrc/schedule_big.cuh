@@ -191,8 +191,11 @@ __global__ void __launch_bounds__(256) big_rank_kernel(const int* __restrict__ k
 }
 
 // W = warps per (family, start) task: one lane per rank group, 32 W >= G.
+#ifndef VP_BIG_W1_CTAS
+#define VP_BIG_W1_CTAS 2
+#endif
 template <int W>
-__global__ void __launch_bounds__(512, 1)
+__global__ void __launch_bounds__(W == 2 ? 512 : 256, W == 2 ? 1 : VP_BIG_W1_CTAS)
 vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand, const int64_t* __restrict__ tau_in, int B,
                        int32_t* __restrict__ n_steps, int32_t* __restrict__ chan_id, int16_t* __restrict__ lane_dst,
                        uint16_t* __restrict__ lane_inst, int64_t* __restrict__ lane_bytes, int64_t* __restrict__ send_off,

@@ -98,3 +98,16 @@ def test_binding_fails_loudly_without_library(monkeypatch):
     monkeypatch.setattr(b, "_LIB_PATH", "/nonexistent/libvariopath.so")
     with pytest.raises(RuntimeError, match="no CPU fallback"):
         b.kernel_launch_count()
+
+
+def test_status_bits_are_distinct_and_the_timeout_bit_is_declared():
+    """Every status bit the header declares is mirrored by the binding, no two share a value, and the row-copy
+    kernels' give-up bit (the output buffer is incomplete) is among them."""
+    import paper_2609_34340_b200 as vp
+    header = open(os.path.join(ROOT, "include", "variopath.h")).read()
+    declared = dict(re.findall(r"#define (VP_ST_[A-Z_]+)\s+\(?([0-9 <]+)\)?", header))
+    values = {k: eval(v) for k, v in declared.items()}
+    assert len(set(values.values())) == len(values) and "VP_ST_INTERNAL_TIMEOUT" in values
+    for name, v in values.items():
+        assert getattr(vp, name[3:]) == v, name
+    assert vp.ST_INTERNAL_TIMEOUT == 1 << 30 and vp.ST_INTERNAL_TIMEOUT & (vp.ST_PACK_MISMATCH | vp.ST_PACK_CAPACITY) == 0
