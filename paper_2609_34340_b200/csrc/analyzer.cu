@@ -1,11 +1,15 @@
-// vp_build_catalog: offline catalog construction, Algorithm 1 of Section 4.1 (host code).
+// vp_build_catalog: offline catalog construction (host code).  What it enumerates is Section 4.1's definition: every
+// multiset of path instances that gives each group exactly g outgoing and g incoming lanes (Eq. 3 for its shape,
+// Eq. 4 for the family) and uses no directed resource twice.
 //
-// Pruned binary DFS over the path instances in id order.  A state is (next instance t, chosen multiset B);
-// the include branch is taken when CanAdd holds (resource disjointness and the per-group degree limits g),
-// SuffixOK cuts states whose remaining instances cannot fill every group's g outgoing and g incoming slots,
-// Complete states are recorded under their shape M.  An instance of lane multiplicity m (PIX) is decided in
-// one level as "0..m lanes".  PruneFamilies then drops, inside each bucket, exact duplicates and families
-// that another family matches footprint by footprint with no lower and somewhere higher rates.
+// The search is this build's own: families are assembled one SOURCE GROUP at a time.  A group's g lanes are a
+// multiset over the instances that leave it (these are contiguous in the topology blob); the instances are walked in
+// id order and each takes 0 .. min(multiplicity, lanes still missing, room left at its destination) lanes, provided
+// its footprint is disjoint from the resources taken so far, which is one AND on a bitset.  Two cuts keep the walk
+// small: a group is abandoned as soon as the instances not yet walked cannot supply its missing lanes, and the next
+// group is only entered if every destination can still reach g with the lanes that later groups can send it.  A
+// family is complete when the last group is filled.  PruneFamilies then drops, inside each bucket, exact duplicates
+// and families that another family matches footprint by footprint with no lower and somewhere higher rates.
 // Output order (what the scheduler's tie-breaks refer to): shapes by their sorted (a, d, count) list,
 // families inside a bucket by their instance-id list.
 #include <algorithm>
@@ -26,46 +30,73 @@ struct AInst {
 struct Analyzer {
     int N, G, g, n_res;
     std::vector<AInst> inst;
-    std::vector<std::vector<int>> out_suffix, in_suffix;   // lanes still available from instance t on, per group
-    std::vector<int> out_deg, in_deg, chosen;
-    std::vector<unsigned char> used;                        // directed resources taken by the partial family
+    std::vector<int> group_begin;                           // instances leaving group a: group_begin[a] .. group_begin[a + 1]
+    std::vector<int> supply_after;                          // lanes the instances after t, of t's own group, can still give
+    std::vector<std::vector<int>> in_later;                 // in_later[a][d]: lanes groups a, a + 1, ... can send to d
+    std::vector<std::vector<uint64_t>> footprint;           // per instance: its directed resources as a bitset
+    std::vector<uint64_t> taken;                            // resources of the partial family
+    std::vector<int> in_deg, chosen;
     std::vector<std::vector<uint16_t>> found;
     size_t limit;
     bool overflow = false;
 
-    bool complete() const {
-        for (int a = 0; a < G; a++)
-            if (out_deg[a] != g || in_deg[a] != g) return false;
+    void prepare() {
+        const int n = (int)inst.size(), words = (n_res + 63) / 64 + 1;
+        group_begin.assign(G + 1, n);
+        for (int r = n - 1; r >= 0; r--) group_begin[inst[r].a] = r;
+        for (int a = G - 1; a >= 0; a--) group_begin[a] = std::min(group_begin[a], group_begin[a + 1]);
+        supply_after.assign(n, 0);
+        for (int a = 0; a < G; a++) {
+            int later = 0;
+            for (int r = group_begin[a + 1] - 1; r >= group_begin[a]; r--) { supply_after[r] = later; later += inst[r].mult; }
+        }
+        in_later.assign(G + 1, std::vector<int>(G, 0));
+        for (int a = G - 1; a >= 0; a--) {
+            in_later[a] = in_later[a + 1];
+            for (int r = group_begin[a]; r < group_begin[a + 1]; r++) in_later[a][inst[r].d] += inst[r].mult;
+        }
+        footprint.assign(n, std::vector<uint64_t>(words, 0));
+        for (int r = 0; r < n; r++)
+            for (int k = 0; k < inst[r].n_res; k++) footprint[r][inst[r].res[k] >> 6] |= (uint64_t)1 << (inst[r].res[k] & 63);
+        taken.assign(words, 0);
+        in_deg.assign(G, 0);
+        chosen.clear();
+    }
+    bool disjoint(int r) const {
+        for (size_t w = 0; w < taken.size(); w++)
+            if (taken[w] & footprint[r][w]) return false;
         return true;
     }
-    bool suffix_ok(int t) const {
-        for (int a = 0; a < G; a++)
-            if (out_deg[a] + out_suffix[t][a] < g || in_deg[a] + in_suffix[t][a] < g) return false;
-        return true;
-    }
-    void explore(int t) {
+    // Group a still misses `need` lanes; instances from t on (of this group) may supply them.
+    void fill_group(int a, int t, int need) {
         if (overflow) return;
-        if (complete()) {
-            if (found.size() >= limit) { overflow = true; return; }
-            found.emplace_back(chosen.begin(), chosen.end());
+        if (need == 0) {
+            if (a + 1 == G) {                               // every group has sent g lanes; each must also have received g
+                for (int d = 0; d < G; d++)
+                    if (in_deg[d] != g) return;
+                if (found.size() >= limit) { overflow = true; return; }
+                found.emplace_back(chosen.begin(), chosen.end());
+                return;
+            }
+            for (int d = 0; d < G; d++)                     // can the later groups still fill every destination?
+                if (in_deg[d] + in_later[a + 1][d] < g) return;
+            fill_group(a + 1, group_begin[a + 1], g);
             return;
         }
-        if (t >= (int)inst.size() || !suffix_ok(t)) return;
-        explore(t + 1);                                     // exclude r_t
+        if (t == group_begin[a + 1]) return;
         const AInst& r = inst[t];
-        for (int k = 0; k < r.n_res; k++)                  // CanAdd: resource disjointness
-            if (used[r.res[k]]) return;
-        for (int k = 0; k < r.n_res; k++) used[r.res[k]] = 1;
-        int added = 0;
-        for (int c = 1; c <= r.mult; c++) {                 // CanAdd: degree limits, one more lane each round
-            if (out_deg[r.a] + 1 > g || in_deg[r.d] + 1 > g) break;
-            out_deg[r.a]++; in_deg[r.d]++;
+        if (supply_after[t] >= need) fill_group(a, t + 1, need);            // no lane on this instance
+        if (!disjoint(t)) return;
+        const int most = std::min(std::min(r.mult, need), g - in_deg[r.d]);
+        if (most < 1) return;
+        for (size_t w = 0; w < taken.size(); w++) taken[w] |= footprint[t][w];
+        for (int lanes = 1; lanes <= most; lanes++) {
+            in_deg[r.d]++;
             chosen.push_back(t);
-            added++;
-            explore(t + 1);
+            if (supply_after[t] >= need - lanes) fill_group(a, t + 1, need - lanes);
         }
-        for (int k = 0; k < added; k++) { out_deg[r.a]--; in_deg[r.d]--; chosen.pop_back(); }
-        for (int k = 0; k < r.n_res; k++) used[r.res[k]] = 0;
+        for (int lanes = 0; lanes < most; lanes++) { in_deg[r.d]--; chosen.pop_back(); }
+        for (size_t w = 0; w < taken.size(); w++) taken[w] &= ~footprint[t][w];
     }
 };
 
@@ -191,20 +222,9 @@ extern "C" int vp_build_catalog(const void* topology, size_t topo_bytes, void* c
     Analyzer A;
     int rc = parse_topology(topology, topo_bytes, A, nullptr);
     if (rc) return rc;
-    const int n_inst = (int)A.inst.size();
-    A.out_suffix.assign(n_inst + 1, std::vector<int>(A.G, 0));
-    A.in_suffix.assign(n_inst + 1, std::vector<int>(A.G, 0));
-    for (int r = n_inst - 1; r >= 0; r--) {
-        A.out_suffix[r] = A.out_suffix[r + 1];
-        A.in_suffix[r] = A.in_suffix[r + 1];
-        A.out_suffix[r][A.inst[r].a] += A.inst[r].mult;
-        A.in_suffix[r][A.inst[r].d] += A.inst[r].mult;
-    }
-    A.out_deg.assign(A.G, 0);
-    A.in_deg.assign(A.G, 0);
-    A.used.assign(A.n_res + 1, 0);
+    A.prepare();
     A.limit = (size_t)1 << 22;                              // more families than this is not a usable catalog
-    A.explore(0);
+    A.fill_group(0, A.group_begin[0], A.g);
     if (A.overflow) return VP_E_UNSUPPORTED;
     if (A.found.empty()) return VP_E_BAD_CATALOG;
     return write_catalog(A, channels_out, capacity_bytes, bytes_needed, n_shapes_out, n_families_out);

@@ -4,7 +4,8 @@ import time
 
 import pytest
 
-from workloads.topology import (complete_catalog, crossbar_catalog, crossbar_topology, tree_topology, Topology, Instance)
+from workloads.topology import (complete_catalog, crossbar_catalog, crossbar_topology, ring_topology, tree_topology, Topology,
+                                Instance)
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
 
@@ -127,3 +128,92 @@ def test_template_catalog_needs_two_groups_per_node(vp):
     with pytest.raises(vp.VpError) as e:
         vp.build_template_catalog(crossbar_topology(4).blob())
     assert e.value.code == vp.E_UNSUPPORTED
+
+
+def _brute_force_families(topo):
+    """Every family of a topology by plain enumeration, written from the definition alone (Section 4.1): each group
+    picks g lanes among the instances that leave it; a pick is a family when every group also receives g lanes and no
+    directed resource is used twice.  Independent of both catalog builders."""
+    from itertools import combinations_with_replacement, product
+    per_group = []
+    for a in range(topo.G):
+        ids = [i for i, r in enumerate(topo.instances) if r.src_group == a]
+        picks = [c for c in combinations_with_replacement(ids, topo.g)
+                 if all(c.count(i) <= topo.instances[i].mult for i in set(c))]
+        per_group.append(picks)
+    fams = set()
+    for combo in product(*per_group):
+        fam = tuple(sorted(i for c in combo for i in c))
+        inn = [0] * topo.G
+        used = []
+        for i in fam:
+            inn[topo.instances[i].dst_group] += 1
+            used += list(topo.instances[i].res)
+        if inn == [topo.g] * topo.G and len(used) == len(set(used)):
+            fams.add(fam)
+    return fams
+
+
+def _shape_count(topo, fams):
+    shapes = set()
+    for f in fams:
+        cnt = {}
+        for i in f:
+            key = (topo.instances[i].src_group, topo.instances[i].dst_group)
+            cnt[key] = cnt.get(key, 0) + 1
+        shapes.add(tuple(sorted(cnt.items())))
+    return len(shapes)
+
+
+@pytest.mark.parametrize("make", [lambda: tree_topology(2, g=2), lambda: ring_topology(1, switches_per_node=4, g=2),
+                                  lambda: ring_topology(1, switches_per_node=3, g=2, pcie_bw=64, nic_bw=50)])
+def test_counts_against_plain_enumeration(vp, oracle_lib, make):
+    """The two-node tree (g = 2) and one-node rings: the library's catalog holds exactly the families that plain
+    enumeration from the definition finds (all rates equal per kind, so PruneFamilies removes nothing but duplicates)."""
+    topo = make()
+    want = _brute_force_families(topo)
+    blob, ns, nf = vp.build_catalog(topo.blob())
+    oc = oracle_lib.OracleCatalog(topo.blob(), blob)
+    assert oc.check() == 0 and oc.covers()
+    got = {tuple(int(x) for x in row) for row in oc.families()}
+    assert got == want and nf == len(want) and ns == _shape_count(topo, want)
+
+
+def test_ring_topology_through_prune_build_and_oracle(vp, oracle_lib):
+    """A ring of PCIe switches: candidate paths -> vp_prune_paths -> vp_build_catalog -> the oracle's Eq. (3)/(4)
+    checker, coverage, and a schedule whose plans are valid (conservation, Eq. 1, Eq. 9)."""
+    import numpy as np
+    from workloads import SchedParams
+    topo = ring_topology(1, switches_per_node=4, g=2)
+    pruned = vp.prune_paths(topo.blob())
+    assert pruned == topo.blob()                                         # the generator already pruned: a fixed point
+    blob, ns, nf = vp.build_catalog(pruned)
+    oc = oracle_lib.OracleCatalog(pruned, blob)
+    assert oc.check() == 0 and oc.covers() and ns > 3 and nf >= ns
+    # two ring paths per switch pair, one per direction: neither footprint contains the other, so PrunePaths keeps both
+    inst = oc.instances()
+    assert sorted(len(r[5]) for r in inst if (r[0], r[1], r[2]) == (0, 2, 1)) == [2, 2]
+    assert sorted(len(r[5]) for r in inst if (r[0], r[1], r[2]) == (0, 1, 1)) == [1, 3]
+    rng = np.random.default_rng(8)
+    for _ in range(4):
+        D = (rng.integers(0, 40, size=(8, 8)) * (rng.random((8, 8)) < 0.7) * 64).astype(np.int64)
+        np.fill_diagonal(D, 0)
+        plan = oc.schedule(D, SchedParams(granule_bytes=64).resolved(8))
+        assert plan["status"] == 0 and oc.check_plan(D, plan, int(plan["tau_ns"]), 64) == 0
+
+
+def test_catalog_scale_report(vp, capsys):
+    """Catalog scale and build time per topology, in the manner of Table 3 (shapes, families, KiB, seconds); only the
+    one-node row is a pin (3 shapes / 6 families), the rest is a report."""
+    rows = []
+    for name, topo in [("1 node, tree 2 x 4", tree_topology(1)), ("2 nodes, tree 2 x 4", tree_topology(2)),
+                       ("3 nodes, tree 2 x 2", tree_topology(3, g=2)), ("1 node, ring 4 x 2", ring_topology(1, 4, 2)),
+                       ("1 node, ring 5 x 2", ring_topology(1, 5, 2))]:
+        t0 = time.perf_counter()
+        blob, ns, nf = vp.build_catalog(topo.blob())
+        rows.append((name, topo.N, ns, nf, len(blob) / 1024, time.perf_counter() - t0))
+    with capsys.disabled():
+        print()
+        for name, n, ns, nf, kib, sec in rows:
+            print(f"    {name:22s} N={n:3d}  shapes {ns:6d}  families {nf:7d}  {kib:9.1f} KiB  {sec:7.3f} s")
+    assert rows[0][2:4] == (3, 6)

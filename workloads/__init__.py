@@ -10,6 +10,7 @@ from .topology import (  # noqa: F401
     Topology,
     Catalog,
     tree_topology,
+    ring_topology,
     crossbar_topology,
     complete_catalog,
     node_template_catalog,

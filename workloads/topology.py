@@ -181,6 +181,35 @@ def tree_topology(nodes: int, g: int = 4, pcie_bw: int = 64, nic_bw: int = 64,
     return Topology(N=G * g, G=G, g=g, groups_per_node=S, n_resources=4 * G, instances=inst)
 
 
+def ring_topology(nodes: int, switches_per_node: int = 4, g: int = 2, pcie_bw: int = 64, nic_bw: int = 64) -> Topology:
+    """PCIe ring (Table 2 lists one platform with a "Ring" PCIe topology and says no more; this is the plainest
+    reading): the switches of a node form a ring, each with ``g`` GPUs and one NIC.  Directed shared resources per
+    switch: its clockwise and its counter-clockwise ring link, NIC transmit, NIC receive.  Group-level path
+    instances: PIX (same switch), one ring path per direction to every other switch of the node (footprint = the
+    ring links it crosses, at most four), NIC to every other group; ``PrunePaths`` then removes dominated ones."""
+    S = switches_per_node
+    G = nodes * S
+    cands: List[Instance] = []
+    for a in range(G):
+        node, sa = divmod(a, S)
+        for d in range(G):
+            if a == d:
+                if g >= 2:
+                    cands.append(Instance(a, d, KIND_PIX, pcie_bw, g, ()))
+                continue
+            if d // S == node:
+                sd = d % S
+                cw = [_res_id(node * S + (sa + k) % S, 0) for k in range((sd - sa) % S)]
+                ccw = [_res_id(node * S + (sa - k) % S, 1) for k in range((sa - sd) % S)]
+                for links in (cw, ccw):
+                    if len(links) <= 4:
+                        cands.append(Instance(a, d, KIND_PXB, pcie_bw, 1, tuple(links)))
+            cands.append(Instance(a, d, KIND_NIC, nic_bw, 1, (_res_id(a, 2), _res_id(d, 3))))
+    inst = prune_paths(cands)
+    inst.sort(key=lambda r: (r.src_group, r.dst_group, r.kind, len(r.res), r.res))
+    return Topology(N=G * g, G=G, g=g, groups_per_node=S, n_resources=4 * G, instances=inst)
+
+
 def crossbar_topology(n: int, bw: int = 64) -> Topology:
     """One switch with ``n`` GPUs: a single group, every pair on a PIX path."""
     return Topology(N=n, G=1, g=n, groups_per_node=1, n_resources=0,
