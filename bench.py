@@ -578,7 +578,7 @@ def finish(args, world, run, sched, pk, T, topk, R, pack_bytes, copy_bytes, stat
                       launch=run.launch, bound="alu", achieved=round(sched_tops, 4), peak=int_peak,
                       unit="Tops/s (integer add/min, algorithmic)",
                       frac=round(sched_tops / int_peak, 5) if int_peak else None,
-                      traffic=(sc.get("dram_bytes_per_activation") or 0) * stats["activations"] / calls if sc.get("dram_bytes_per_activation") else None,
+                      traffic=int(sc["dram_bytes_per_matrix"] * B / calls) if sc.get("dram_bytes_per_matrix") else None,
                       peak_source="measured in this run: vp_microbench kind 0 (32-bit add + min, all warp slots busy)",
                       ms_per_launch=round(sched_per_launch, 4), launches_per_step=calls,
                       algorithmic_ops_per_launch=int(ops / calls))
@@ -714,6 +714,49 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def run_quality(args):
+    """Plan-quality report (`--quality`): Eq. (2) over a grid of (lambda, K_target) on config 2's 256 matrices
+    (vp_sweep_plan_time), the same with the two-node node-template catalog (15 shapes / 20 families) in place of
+    the complete one (89 / 152), and the ratio to the link-load lower bound on a sample (the bound is oracle-side
+    Python, test infrastructure, so the sample is small)."""
+    import numpy as np
+    import torch
+    import oracle
+    import paper_2609_34340_b200 as vp
+    from paper_2609_34340_b200.build import build
+    from workloads.configs import build_config
+    from workloads.topology import node_template_catalog, tree_topology
+    build()
+    dev = "cuda:0"
+    c = build_config(2, device=dev)
+    w = c["params"]
+    D = c["demand"].to(dev).contiguous()
+    N = c["catalog"].topology.N
+    lambdas, k_targets = [0, 2000, 8000, 32000], [N, 2 * N, 3 * N, 4 * N]
+    cats = {"complete 89/152": c["catalog"], "node-template 15/20": node_template_catalog(tree_topology(2))}
+    res = {}
+    for name, cat in cats.items():
+        dc = vp.load_catalog(cat.topology.blob(), cat.blob(), device=0)
+        T, K, st = vp.sweep_plan_time(dc, vp_params(vp, w), D, lambdas, k_targets)
+        torch.cuda.synchronize()
+        assert int(st.max().item()) == 0
+        res[name] = (T.cpu().numpy().astype(np.float64) / dc.rate_lcm, K.cpu().numpy())
+    Tc, Kc = res["complete 89/152"]
+    Tt, Kt = res["node-template 15/20"]
+    oc = oracle.OracleCatalog(c["catalog"].topology.blob(), c["catalog"].blob())
+    sample = list(range(0, D.shape[0], 8))
+    lb = np.array([float(oc.lower_bound(c["demand"][b].numpy())) for b in sample])
+    out = {"workload": "config 2: 256 MoE demand matrices N=16", "lambda_ns": lambdas, "k_target": k_targets,
+           "mean_T_us_complete": np.round(Tc.mean(axis=2) / 1e3, 1).tolist(),
+           "mean_activations_complete": np.round(Kc.mean(axis=2), 1).tolist(),
+           "mean_T_us_template": np.round(Tt.mean(axis=2) / 1e3, 1).tolist(),
+           "template_over_complete_mean_ratio": np.round((Tt / Tc).mean(axis=2), 4).tolist(),
+           "template_over_complete_max_ratio": np.round((Tt / Tc).max(axis=2), 4).tolist(),
+           "T_over_lower_bound_at_lambda0": {"sample": f"{len(sample)} matrices (every 8th)",
+                                             "mean_per_k_target": np.round((Tc[0][:, sample] / lb).mean(axis=1), 4).tolist()}}
+    print(json.dumps({"plan_quality": out}))
+
+
 def _has_cuda() -> bool:
     try:
         import torch
@@ -742,13 +785,16 @@ def main():
                     help="keep warming up (beyond --warmup steps) until this many seconds have passed, so that "
                          "clocks settle and nvidia-smi has samples under load")
     ap.add_argument("--e2e-steps", type=int, default=2, help="steps of the host-buffer leg (each moves the whole plan over PCIe)")
+    ap.add_argument("--quality", action="store_true", help="print the plan-quality report (Eq. 2 sweep, template vs complete catalog) and exit")
     ap.add_argument("--tools", action="store_true", help="also time the kernels around the scheduler (unpack, plan time, demand rows)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the CPU oracle leg (profiling runs)")
     ap.add_argument("--no-extras", action="store_true", help="skip the peak probes and the other scheduler configs (profiling runs)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
-    if args.impl == "reference":
+    if args.quality:
+        run_quality(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

@@ -306,6 +306,22 @@ int vp_plan_time(const vp_catalog* catalog, int B, int k_max, const int32_t* n_s
                  const int64_t* lane_bytes, int64_t lambda_ns, int64_t* time_xw, void* cuda_stream);
 
 /*
+ * vp_sweep_plan_time - plan quality over a grid of parameters: for every pair (lambda_ns[i], k_target[j]) the batch
+ * is decomposed with those two parameters in place of params' (Algorithm 2; Section 5 "Global execution
+ * granularity": K_target sets the time quantum) and Eq. (2) is evaluated with that lambda.  Results, device arrays
+ * indexed [(i * n_k + j) * B + b]: time_xw = rate_lcm x T(S_b) in nanoseconds, n_steps_out (may be NULL) the
+ * activation counts, status_out (may be NULL) the per-matrix status bits.  lambda_ns and k_target are HOST arrays
+ * (k_target 0 = 2N).  The plans themselves live in `workspace` (device, 256-byte aligned,
+ * vp_sweep_workspace_bytes(catalog, B, params) bytes) and are overwritten from pair to pair.  Everything is
+ * enqueued on cuda_stream; nothing is synchronised.
+ */
+size_t vp_sweep_workspace_bytes(const vp_catalog* catalog, int B, const vp_sched_params* params);
+int vp_sweep_plan_time(const vp_catalog* catalog, const vp_sched_params* params, const int64_t* demand, int B,
+                       const int64_t* lambda_ns, int n_lambda, const int32_t* k_target, int n_k, int64_t* time_xw,
+                       int32_t* n_steps_out, int32_t* status_out, void* workspace, size_t workspace_bytes,
+                       void* cuda_stream);
+
+/*
  * vp_demand_from_routing - the demand rows of n_src source ranks from their top-k routing indices
  * (Section 6 "Workloads": demand matrices derived from top-k MoE routing; Section 3: D_ii = 0).
  *   expert_idx  device int32 [n_src][T][topk]; < 0 = dropped copy; expert e lives on rank e / experts_per_rank

@@ -200,6 +200,28 @@ class OracleCatalog:
         out["trace"] = trace[: int(tl[0])]
         return out
 
+    def sweep_plan_time(self, demand, params, lambdas, k_targets, threads: int = 1):
+        """Eq. (2) over a grid: for every (lambda, K_target) decompose the batch with those two parameters and evaluate
+        rate_lcm x T(S) with that lambda.  Returns (time_xw int64 [n_lambda, n_k, B], n_steps int32 of the same shape)."""
+        import copy
+        D = np.ascontiguousarray(demand, dtype=np.int64)
+        B = D.shape[0]
+        T = np.zeros((len(lambdas), len(k_targets), B), np.int64)
+        K = np.zeros((len(lambdas), len(k_targets), B), np.int32)
+        for i, lam in enumerate(lambdas):
+            for j, kt in enumerate(k_targets):
+                q = copy.copy(params)
+                if isinstance(q, dict):
+                    q = dict(q, lambda_ns=int(lam), k_target=int(kt))
+                else:
+                    q.lambda_ns, q.k_target = int(lam), int(kt)
+                out = self.schedule_batch(D, q, threads=threads)
+                K[i, j] = out["n_steps"]
+                for b in range(B):
+                    one = {k: out[k][b] for k in ("n_steps", "lane_dst", "lane_inst", "lane_bytes")}
+                    T[i, j, b] = self.modeled_time_xw(one, int(lam))
+        return T, K
+
     # ---- plan-level quantities ----------------------------------------
     def modeled_time(self, plan: dict, lambda_ns: int) -> Fraction:
         """Eq. (2): modeled completion time of a one-matrix plan, in nanoseconds."""

@@ -27,6 +27,7 @@ from .binding import (  # noqa: F401
     unpack_tokens,
     kernel_launch_count,
     plan_time,
+    sweep_plan_time,
     demand_from_routing,
     schedule_read_stats,
     schedule_launch_info,

@@ -100,6 +100,9 @@ def _load():
     lib.vp_prune_paths.argtypes = [P, sz, P, sz, C.POINTER(sz), C.POINTER(C.c_int32)]
     lib.vp_plan_time.argtypes = [vp, i32, i32, P, P, P, i64, P, P]
     lib.vp_demand_from_routing.argtypes = [P, i32, i32, i32, i32, i32, i32, i64, P, P, P]
+    lib.vp_sweep_workspace_bytes.argtypes = [vp, i32, C.POINTER(_Params)]
+    lib.vp_sweep_workspace_bytes.restype = sz
+    lib.vp_sweep_plan_time.argtypes = [vp, C.POINTER(_Params), P, i32, P, i32, P, i32, P, P, P, P, sz, P]
     lib.vp_schedule_read_stats.argtypes = [P, P, P]
     lib.vp_schedule_launch_info.argtypes = [vp, i32, C.POINTER(_Params), P]
     lib.vp_microbench.argtypes = [i32, i32, P, C.POINTER(i64), P]
@@ -312,6 +315,24 @@ def plan_time(catalog: Catalog, plan: Plan, lambda_ns: int, out: Optional[torch.
     _check(_load().vp_plan_time(catalog._h, int(B), int(plan.k_max), _ptr(plan.n_steps), _ptr(plan.lane_inst),
                                 _ptr(plan.lane_bytes), int(lambda_ns), _ptr(out), _stream(stream)), "vp_plan_time")
     return out
+
+
+def sweep_plan_time(catalog: Catalog, params: SchedParams, demand: torch.Tensor, lambdas, k_targets, stream=None):
+    """``vp_sweep_plan_time``: returns (time_xw int64 ``[n_lambda, n_k, B]``, n_steps int32, status int32), all on device."""
+    assert demand.is_cuda and demand.dtype == torch.int64 and demand.is_contiguous()
+    B, N = demand.shape[0], catalog.N
+    p = params._c(N)
+    lam = (C.c_int64 * len(lambdas))(*[int(x) for x in lambdas])
+    kt = (C.c_int32 * len(k_targets))(*[int(x) for x in k_targets])
+    shape = (len(lambdas), len(k_targets), B)
+    out = torch.empty(shape, dtype=torch.int64, device=demand.device)
+    n_steps = torch.empty(shape, dtype=torch.int32, device=demand.device)
+    status = torch.empty(shape, dtype=torch.int32, device=demand.device)
+    need = int(_load().vp_sweep_workspace_bytes(catalog._h, B, C.byref(p)))
+    ws = torch.empty(need, dtype=torch.uint8, device=demand.device)
+    _check(_load().vp_sweep_plan_time(catalog._h, C.byref(p), _ptr(demand), B, lam, len(lambdas), kt, len(k_targets), _ptr(out),
+                                      _ptr(n_steps), _ptr(status), _ptr(ws), need, _stream(stream)), "vp_sweep_plan_time")
+    return out, n_steps, status
 
 
 def demand_from_routing(expert_idx: torch.Tensor, experts_per_rank: int, N: int, row_bytes: int, src0: int = 0,

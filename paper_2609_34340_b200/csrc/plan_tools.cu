@@ -118,3 +118,73 @@ extern "C" int vp_demand_from_routing(const int32_t* expert_idx, int n_src, int 
     g_vp_launches++;
     return cudaGetLastError() == cudaSuccess ? VP_OK : VP_E_CUDA;
 }
+
+// ---- plan-quality sweep: Eq. (2) over a grid of (lambda, K_target) ---------------------------------------------------
+
+namespace {
+
+struct SweepBufs {
+    int32_t *n_steps, *chan_id, *status;
+    int16_t* lane_dst;
+    uint16_t* lane_inst;
+    int64_t *lane_bytes, *send_off, *tau;
+    void* ws;
+    size_t ws_bytes, total;
+};
+
+SweepBufs carve_sweep(char* base, const vp_catalog* c, int B, const vp_sched_params* p) {
+    const size_t N = (size_t)c->info.N, K = (size_t)p->k_max, b = (size_t)B;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { char* at = base ? base + off : nullptr; off += vp_align256(bytes); return (void*)at; };
+    SweepBufs s;
+    s.n_steps = (int32_t*)take(b * 4);
+    s.chan_id = (int32_t*)take(b * K * 4);
+    s.status = (int32_t*)take(b * 4);
+    s.lane_dst = (int16_t*)take(b * K * N * 2);
+    s.lane_inst = (uint16_t*)take(b * K * N * 2);
+    s.lane_bytes = (int64_t*)take(b * K * N * 8);
+    s.send_off = (int64_t*)take(b * (K + 1) * N * 8);
+    s.tau = (int64_t*)take(b * 8);
+    s.ws_bytes = vp_schedule_workspace_bytes(c, B, p);
+    s.ws = take(s.ws_bytes);
+    s.total = off;
+    return s;
+}
+
+}  // namespace
+
+extern "C" size_t vp_sweep_workspace_bytes(const vp_catalog* c, int B, const vp_sched_params* p) {
+    if (!c || !p || B <= 0 || p->k_max <= 0) return 0;
+    SweepBufs s = carve_sweep(nullptr, c, B, p);
+    return s.ws_bytes ? s.total : 0;
+}
+
+extern "C" int vp_sweep_plan_time(const vp_catalog* c, const vp_sched_params* p, const int64_t* demand, int B,
+                                  const int64_t* lambda_ns, int n_lambda, const int32_t* k_target, int n_k, int64_t* time_xw,
+                                  int32_t* n_steps_out, int32_t* status_out, void* workspace, size_t workspace_bytes,
+                                  void* cuda_stream) {
+    if (!c || !p || !demand || !lambda_ns || !k_target || !time_xw || B <= 0 || n_lambda <= 0 || n_k <= 0 || p->k_max <= 0)
+        return VP_E_BAD_ARG;
+    if (!workspace || ((uintptr_t)workspace & 255)) return VP_E_WORKSPACE;
+    SweepBufs s = carve_sweep((char*)workspace, c, B, p);
+    if (!s.ws_bytes) return VP_E_BAD_ARG;
+    if (workspace_bytes < s.total) return VP_E_WORKSPACE;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    for (int i = 0; i < n_lambda; i++)
+        for (int j = 0; j < n_k; j++) {
+            vp_sched_params q = *p;
+            q.lambda_ns = lambda_ns[i];
+            q.k_target = k_target[j];
+            int rc = vp_schedule_batch(c, &q, demand, nullptr, B, s.n_steps, s.chan_id, s.lane_dst, s.lane_inst, s.lane_bytes, s.send_off,
+                                       nullptr, s.tau, s.status, s.ws, s.ws_bytes, cuda_stream);
+            if (rc) return rc;
+            const size_t at = ((size_t)i * n_k + j) * B;
+            rc = vp_plan_time(c, B, p->k_max, s.n_steps, s.lane_inst, s.lane_bytes, q.lambda_ns, time_xw + at, cuda_stream);
+            if (rc) return rc;
+            if (n_steps_out && cudaMemcpyAsync(n_steps_out + at, s.n_steps, (size_t)B * 4, cudaMemcpyDeviceToDevice, stream) != cudaSuccess)
+                return VP_E_CUDA;
+            if (status_out && cudaMemcpyAsync(status_out + at, s.status, (size_t)B * 4, cudaMemcpyDeviceToDevice, stream) != cudaSuccess)
+                return VP_E_CUDA;
+        }
+    return VP_OK;
+}

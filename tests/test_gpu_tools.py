@@ -75,3 +75,25 @@ def test_plan_time_with_mixed_rates(vp, oracle_lib):
         one = {k: (v[b] if isinstance(v, np.ndarray) else v) for k, v in host.items()}
         assert int(got[b]) == oc.modeled_time_xw(one, 123)
     assert got[4] == 0
+
+
+def test_sweep_plan_time_matches_oracle(vp, oracle_lib):
+    """vp_sweep_plan_time over a grid of (lambda, K_target): rate_lcm x T(S) and the activation counts of every grid
+    point equal the oracle's, integer for integer; every value is at least the link-load lower bound at lambda = 0."""
+    from workloads.configs import build_config
+    c = build_config(2, device="cuda", batch=6, token_scale=0.25)
+    cat, w = c["catalog"], c["params"]
+    oc = oracle_lib.OracleCatalog(cat.topology.blob(), cat.blob())
+    dc = vp.load_catalog(cat.topology.blob(), cat.blob())
+    p = vp.SchedParams(lambda_ns=w.lambda_ns, granule_bytes=w.granule_bytes, k_target=w.k_target, n_start=w.n_start,
+                       i_aa=w.i_aa, k_max=w.k_max)
+    lambdas, k_targets = [0, 8000], [16, 32, 48]
+    T, K, st = vp.sweep_plan_time(dc, p, c["demand"].cuda().contiguous(), lambdas, k_targets)
+    torch.cuda.synchronize()
+    wantT, wantK = oc.sweep_plan_time(c["demand"].numpy(), w, lambdas, k_targets, threads=4)
+    assert (st.cpu().numpy() == 0).all()
+    assert np.array_equal(K.cpu().numpy(), wantK)
+    assert np.array_equal(T.cpu().numpy(), wantT)
+    for b in range(6):
+        lb = oc.lower_bound(c["demand"][b].numpy())
+        assert all(int(T[0, j, b]) >= lb * oc.W for j in range(len(k_targets)))

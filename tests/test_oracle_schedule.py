@@ -356,3 +356,27 @@ def test_multistart_aa_stop_rule_and_best_start(oracle_lib):
         assert not rem.any()
     # the cases exercise every branch of the rule
     assert seen["early"] > 100 and seen["limit"] > 100 and seen["later_start"] > 10 and seen["tie_other_binding"] > 10
+
+
+@pytest.mark.parametrize("n", [4, 7])
+def test_sweep_of_lambda_and_k_target_against_the_crossbar_closed_form(oracle_lib, n):
+    """Eq. (2) over a grid of (lambda, K_target) (Section 5: K_target sets the quantum).  Uniform demand c on a crossbar:
+    est = (N-1) c / bw, tau = ceil(est / K_target), cap = max(u, floor(tau bw / u) u), then (N-1) ceil(c / cap) rounds of
+    full lanes, the last round of each pair carrying the remainder -- a closed form for every grid point."""
+    bw, u, c = 64, 64, 64 * 1000
+    oc = _oc(oracle_lib, crossbar_catalog(crossbar_topology(n, bw=bw)))
+    D = uniform_demand(n, c).numpy()[None]
+    lambdas, k_targets = [0, 500, 8000], [1, 3, n, 2 * n, 5 * n, 1000 * n]
+    T, K = oc.sweep_plan_time(D, SchedParams(granule_bytes=u, k_max=1200 * n).resolved(n), lambdas, k_targets)
+    for i, lam in enumerate(lambdas):
+        for j, kt in enumerate(k_targets):
+            est = -(-(n - 1) * c // bw)
+            tau = max(1, -(-est // kt))
+            cap = max(u, tau * bw // u * u)
+            full, rest = divmod(c, cap)
+            rounds = full + (1 if rest else 0)
+            want = (n - 1) * (full * (lam + Fraction(cap, bw)) + (1 if rest else 0) * (lam + Fraction(rest, bw)))
+            assert K[i, j, 0] == (n - 1) * rounds
+            assert Fraction(int(T[i, j, 0]), oc.W) == want
+    # more rounds cost more overhead and never less transfer time: T grows with lambda at every K_target
+    assert (np.diff(T[:, :, 0], axis=0) >= 0).all()
