@@ -286,6 +286,19 @@ int vp_schedule_batch_host(const vp_catalog* catalog, const vp_sched_params* par
                            int64_t* lane_bytes, int64_t* send_off, int64_t* recv_off,
                            int64_t* tau_ns_out, int32_t* status,
                            void* device_scratch, size_t device_scratch_bytes, void* cuda_stream);
+/*
+ * vp_schedule_batch_host_used - vp_schedule_batch_host that brings back only what a plan uses: of every matrix b the
+ * rows k < n_steps[b] of chan_id, lane_dst, lane_inst and lane_bytes and the rows k <= n_steps[b] of send_off / recv_off
+ * (row n_steps[b] holds the totals).  Rows beyond keep whatever the host buffers held.  With k_max sized for the
+ * longest plan this is a small part of the arrays (config 4: 26 GB instead of 122 GB per 4096 matrices).  Same
+ * arguments, scratch and errors as vp_schedule_batch_host; it synchronises the stream once more (to read n_steps).
+ */
+int vp_schedule_batch_host_used(const vp_catalog* catalog, const vp_sched_params* params,
+                                const int64_t* demand, const int64_t* tau_ns_in, int B,
+                                int32_t* n_steps, int32_t* chan_id, int16_t* lane_dst, uint16_t* lane_inst,
+                                int64_t* lane_bytes, int64_t* send_off, int64_t* recv_off,
+                                int64_t* tau_ns_out, int32_t* status,
+                                void* device_scratch, size_t device_scratch_bytes, void* cuda_stream);
 size_t vp_pack_host_scratch_bytes(int N, int T, int topk, int k_max, int64_t row_bytes,
                                   int64_t staged_capacity_bytes);
 int vp_pack_host(const int32_t* n_steps_b, const int16_t* lane_dst_b, const int64_t* lane_bytes_b,

@@ -80,6 +80,7 @@ def _load():
     lib.vp_schedule_host_scratch_bytes.argtypes = [vp, i32, C.POINTER(_Params)]
     lib.vp_schedule_host_scratch_bytes.restype = sz
     lib.vp_schedule_batch_host.argtypes = sched_args + [P, sz, P]
+    lib.vp_schedule_batch_host_used.argtypes = sched_args + [P, sz, P]
     lib.vp_pack_workspace_bytes.argtypes = [i32, i32, i32, i32]
     lib.vp_pack_workspace_bytes.restype = sz
     pack_args = [P, P, P, P, i32, i32, i32, P, i32, i32, i32, P, i64, P, i64, P, P]
@@ -292,8 +293,9 @@ def schedule_batch(catalog: Catalog, params: SchedParams, demand: torch.Tensor,
 
 def schedule_batch_host(catalog: Catalog, params: SchedParams, demand: torch.Tensor,
                         tau_ns_in: Optional[torch.Tensor] = None, plan: Optional[Plan] = None,
-                        scratch: Optional[torch.Tensor] = None, stream=None) -> Plan:
-    """``vp_schedule_batch_host``: host tensors in and out (pinned memory recommended)."""
+                        scratch: Optional[torch.Tensor] = None, stream=None, used_only: bool = False) -> Plan:
+    """``vp_schedule_batch_host``: host tensors in and out (pinned memory recommended).  ``used_only`` selects
+    ``vp_schedule_batch_host_used``: only the rows below each matrix's ``n_steps`` come back."""
     assert not demand.is_cuda and demand.dtype == torch.int64 and demand.is_contiguous()
     B, N = demand.shape[0], catalog.N
     p = params._c(N)
@@ -302,8 +304,8 @@ def schedule_batch_host(catalog: Catalog, params: SchedParams, demand: torch.Ten
     if scratch is None:
         need = int(_load().vp_schedule_host_scratch_bytes(catalog._h, B, C.byref(p)))
         scratch = torch.empty(need, dtype=torch.uint8, device=f"cuda:{catalog.device}")
-    _check(_sched_call(_load().vp_schedule_batch_host, catalog, p, demand, tau_ns_in, B, plan, scratch, stream),
-           "vp_schedule_batch_host")
+    fn = _load().vp_schedule_batch_host_used if used_only else _load().vp_schedule_batch_host
+    _check(_sched_call(fn, catalog, p, demand, tau_ns_in, B, plan, scratch, stream), "vp_schedule_batch_host")
     return plan
 
 

@@ -72,11 +72,14 @@ extern "C" size_t vp_schedule_host_scratch_bytes(const vp_catalog* c, int B, con
     return s.ws_bytes ? s.total : 0;
 }
 
-extern "C" int vp_schedule_batch_host(const vp_catalog* c, const vp_sched_params* p, const int64_t* demand,
-                                      const int64_t* tau_ns_in, int B, int32_t* n_steps, int32_t* chan_id,
-                                      int16_t* lane_dst, uint16_t* lane_inst, int64_t* lane_bytes, int64_t* send_off,
-                                      int64_t* recv_off, int64_t* tau_ns_out, int32_t* status, void* device_scratch,
-                                      size_t device_scratch_bytes, void* cuda_stream) {
+namespace {
+
+// Both host-buffer scheduler calls: copy in, run vp_schedule_batch, copy out.  With used_only the plan arrays come back
+// only up to each matrix's n_steps (one copy per matrix and array, after n_steps itself has been read).
+int schedule_host(const vp_catalog* c, const vp_sched_params* p, const int64_t* demand, const int64_t* tau_ns_in, int B,
+                  int32_t* n_steps, int32_t* chan_id, int16_t* lane_dst, uint16_t* lane_inst, int64_t* lane_bytes,
+                  int64_t* send_off, int64_t* recv_off, int64_t* tau_ns_out, int32_t* status, void* device_scratch,
+                  size_t device_scratch_bytes, void* cuda_stream, bool used_only) {
     if (!c || !p || B <= 0 || p->k_max <= 0 || !demand || !n_steps || !chan_id || !lane_dst || !lane_inst || !lane_bytes ||
         !send_off || !status)
         return VP_E_BAD_ARG;
@@ -95,16 +98,49 @@ extern "C" int vp_schedule_batch_host(const vp_catalog* c, const vp_sched_params
                                tau_ns_out ? s.tau_out : nullptr, s.status, s.ws, s.ws_bytes, cuda_stream);
     if (rc) return rc;
     VP_COPY(n_steps, s.n_steps, b * 4, cudaMemcpyDeviceToHost);
-    VP_COPY(chan_id, s.chan_id, b * K * 4, cudaMemcpyDeviceToHost);
-    VP_COPY(lane_dst, s.lane_dst, b * K * N * 2, cudaMemcpyDeviceToHost);
-    VP_COPY(lane_inst, s.lane_inst, b * K * N * 2, cudaMemcpyDeviceToHost);
-    VP_COPY(lane_bytes, s.lane_bytes, b * K * N * 8, cudaMemcpyDeviceToHost);
-    VP_COPY(send_off, s.send_off, b * (K + 1) * N * 8, cudaMemcpyDeviceToHost);
-    if (recv_off) VP_COPY(recv_off, s.recv_off, b * (K + 1) * N * 8, cudaMemcpyDeviceToHost);
     if (tau_ns_out) VP_COPY(tau_ns_out, s.tau_out, b * 8, cudaMemcpyDeviceToHost);
     VP_COPY(status, s.status, b * 4, cudaMemcpyDeviceToHost);
+    if (!used_only) {
+        VP_COPY(chan_id, s.chan_id, b * K * 4, cudaMemcpyDeviceToHost);
+        VP_COPY(lane_dst, s.lane_dst, b * K * N * 2, cudaMemcpyDeviceToHost);
+        VP_COPY(lane_inst, s.lane_inst, b * K * N * 2, cudaMemcpyDeviceToHost);
+        VP_COPY(lane_bytes, s.lane_bytes, b * K * N * 8, cudaMemcpyDeviceToHost);
+        VP_COPY(send_off, s.send_off, b * (K + 1) * N * 8, cudaMemcpyDeviceToHost);
+        if (recv_off) VP_COPY(recv_off, s.recv_off, b * (K + 1) * N * 8, cudaMemcpyDeviceToHost);
+    } else {
+        if (cudaStreamSynchronize(stream) != cudaSuccess) return VP_E_CUDA;      // n_steps is needed on the host now
+        for (size_t m = 0; m < b; m++) {
+            const size_t k = n_steps[m] < 0 ? 0 : ((size_t)n_steps[m] > K ? K : (size_t)n_steps[m]);
+            VP_COPY(chan_id + m * K, s.chan_id + m * K, k * 4, cudaMemcpyDeviceToHost);
+            VP_COPY(lane_dst + m * K * N, s.lane_dst + m * K * N, k * N * 2, cudaMemcpyDeviceToHost);
+            VP_COPY(lane_inst + m * K * N, s.lane_inst + m * K * N, k * N * 2, cudaMemcpyDeviceToHost);
+            VP_COPY(lane_bytes + m * K * N, s.lane_bytes + m * K * N, k * N * 8, cudaMemcpyDeviceToHost);
+            VP_COPY(send_off + m * (K + 1) * N, s.send_off + m * (K + 1) * N, (k + 1) * N * 8, cudaMemcpyDeviceToHost);
+            if (recv_off) VP_COPY(recv_off + m * (K + 1) * N, s.recv_off + m * (K + 1) * N, (k + 1) * N * 8, cudaMemcpyDeviceToHost);
+        }
+    }
     if (cudaStreamSynchronize(stream) != cudaSuccess) return VP_E_CUDA;
     return VP_OK;
+}
+
+}  // namespace
+
+extern "C" int vp_schedule_batch_host(const vp_catalog* c, const vp_sched_params* p, const int64_t* demand,
+                                      const int64_t* tau_ns_in, int B, int32_t* n_steps, int32_t* chan_id,
+                                      int16_t* lane_dst, uint16_t* lane_inst, int64_t* lane_bytes, int64_t* send_off,
+                                      int64_t* recv_off, int64_t* tau_ns_out, int32_t* status, void* device_scratch,
+                                      size_t device_scratch_bytes, void* cuda_stream) {
+    return schedule_host(c, p, demand, tau_ns_in, B, n_steps, chan_id, lane_dst, lane_inst, lane_bytes, send_off, recv_off,
+                         tau_ns_out, status, device_scratch, device_scratch_bytes, cuda_stream, false);
+}
+
+extern "C" int vp_schedule_batch_host_used(const vp_catalog* c, const vp_sched_params* p, const int64_t* demand,
+                                           const int64_t* tau_ns_in, int B, int32_t* n_steps, int32_t* chan_id,
+                                           int16_t* lane_dst, uint16_t* lane_inst, int64_t* lane_bytes, int64_t* send_off,
+                                           int64_t* recv_off, int64_t* tau_ns_out, int32_t* status, void* device_scratch,
+                                           size_t device_scratch_bytes, void* cuda_stream) {
+    return schedule_host(c, p, demand, tau_ns_in, B, n_steps, chan_id, lane_dst, lane_inst, lane_bytes, send_off, recv_off,
+                         tau_ns_out, status, device_scratch, device_scratch_bytes, cuda_stream, true);
 }
 
 namespace {

@@ -173,6 +173,34 @@ def test_host_buffer_variant(vp, oracle_lib):
     _assert_same(plan.cpu(), want)
 
 
+def test_host_buffer_variant_used_rows_only(vp, oracle_lib):
+    """vp_schedule_batch_host_used: rows below n_steps (and offset row n_steps) equal the oracle's; rows beyond keep what
+    the host buffers held before the call."""
+    c = build_config(2, device="cuda", batch=9, token_scale=0.5)
+    cat = c["catalog"]
+    oc = oracle_lib.OracleCatalog(cat.topology.blob(), cat.blob())
+    dc = vp.load_catalog(cat.topology.blob(), cat.blob())
+    p = _params(vp, c["params"])
+    plan = vp.Plan.empty(9, 16, p.k_max, "cpu", pin=True)
+    marks = dict(chan_id=-77, lane_dst=-55, lane_inst=1234, lane_bytes=-99, send_off=-11, recv_off=-13)
+    for name, v in marks.items():
+        getattr(plan, name).fill_(v)
+    vp.schedule_batch_host(dc, p, c["demand"].pin_memory(), plan=plan, used_only=True)
+    want = oc.schedule_batch(c["demand"].numpy(), c["params"])
+    got = plan.cpu()
+    assert np.array_equal(got["n_steps"], want["n_steps"]) and np.array_equal(got["status"], want["status"])
+    assert np.array_equal(got["tau_ns"], want["tau_ns"])
+    for b in range(9):
+        K = int(want["n_steps"][b])
+        assert 0 < K < p.k_max - 1
+        for name in ("chan_id", "lane_dst", "lane_inst", "lane_bytes"):
+            assert np.array_equal(got[name][b][:K], want[name][b][:K]), (name, b)
+            assert (got[name][b][K:] == (marks[name] if name != "lane_inst" else 1234)).all(), (name, b)
+        for name in ("send_off", "recv_off"):
+            assert np.array_equal(got[name][b][:K + 1], want[name][b][:K + 1]), (name, b)
+            assert (got[name][b][K + 1:] == marks[name]).all(), (name, b)
+
+
 @pytest.mark.parametrize("idx", [1, 2])
 def test_config_full_batch(vp, oracle_lib, idx):
     c = build_config(idx, device="cuda")
