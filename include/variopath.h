@@ -56,6 +56,7 @@ extern "C" {
 #define VP_ST_STEP_LIMIT    128   /* k_max activations emitted, residual demand left              */
 #define VP_ST_PACK_MISMATCH 256   /* vp_pack: routed copies disagree with the plan's byte counts  */
 #define VP_ST_PACK_CAPACITY 512   /* vp_pack: staged buffer smaller than the plan's send volume   */
+#define VP_ST_EXCHANGE_TIMEOUT 2048 /* vp_exchange_wait: the arrival counter did not reach the plan's byte count in max_polls polls */
 /* Row-copy kernels (vp_pack, vp_pack_static, vp_unpack, vp_unpack_tokens): a bounded wait for an asynchronous
  * copy into shared memory gave up (2^22 polls; never seen in practice).  The kernel then issues no further
  * loads, lets the stores it already issued finish and returns; the output buffer is INCOMPLETE and the call
@@ -317,6 +318,42 @@ int vp_pack_host(const int32_t* n_steps_b, const int16_t* lane_dst_b, const int6
  */
 int vp_plan_time(const vp_catalog* catalog, int B, int k_max, const int32_t* n_steps, const uint16_t* lane_inst,
                  const int64_t* lane_bytes, int64_t lambda_ns, int64_t* time_xw, void* cuda_stream);
+
+/*
+ * vp_exchange_put / vp_exchange_wait - executing a plan over peer memory (Section 5, "Device-resident buffer layout":
+ * one contiguous chunk per peer and activation in the send buffer; arrival signalled through device-resident counters
+ * instead of a global barrier; two buffer slots alternate between invocations).  This is the step between vp_pack and
+ * vp_unpack.
+ *
+ * vp_exchange_put, the sender side of rank `rank`: for every step k < n_steps with j = lane_dst[k][rank] >= 0 the bytes
+ * [send_off[k][rank], send_off[k+1][rank]) of `staged` (device; what vp_pack wrote) are stored into
+ * recv_bufs[j] + recv_off[k][j].  The plan pointers are one matrix's device arrays (row stride N), as for vp_pack.
+ *   recv_bufs            device array [N] of device pointers: the receive buffer of every rank for the current slot.
+ *                        Ordinary device memory when ranks share a GPU; peer-mapped memory of the other GPUs otherwise
+ *                        (the kernel only issues ordinary loads and stores, never multicast or cluster-scope copies)
+ *   recv_capacity_bytes  device int64 [N]: size of each receive buffer; a chunk that would overrun it is not copied and
+ *                        VP_ST_PACK_CAPACITY is set in status
+ *   arrived              device array [N] of pointers to uint64 counters (NULL array or NULL entries: no signalling):
+ *                        after a part of a chunk has been stored and fenced system-wide its byte count is added to
+ *                        *arrived[j] with a system-scope atomic.  A rank's counter ends at base + recv_off[n_steps][rank]
+ *   status               device int32[1], bits are OR-ed in (not cleared)
+ * The call only enqueues one kernel on cuda_stream of the current device; it never waits.
+ *
+ * vp_exchange_wait, the receiver side: one thread polls *arrived_counter (acquire, system scope) until it is at least
+ * counter_base + recv_off[n_steps][rank], at most max_polls times 200 ns apart; if it is not, VP_ST_EXCHANGE_TIMEOUT is
+ * OR-ed into status and the kernel returns -- it never spins unbounded, and the context stays usable.  Kernels enqueued
+ * after it on the same stream (vp_unpack) then see the delivered bytes.  counter_base is the counter's value before this
+ * invocation's puts (0 after a reset; counters may also be left to grow from invocation to invocation).
+ *
+ * Several ranks on ONE GPU: enqueue every rank's put before any wait (or puts and waits on one stream in that order);
+ * kernels of one GPU must not wait for kernels that have not been enqueued before them.
+ */
+int vp_exchange_put(const int32_t* n_steps_b, const int16_t* lane_dst_b, const int64_t* send_off_b, const int64_t* recv_off_b,
+                    int N, int rank, int k_max, const void* staged, void* const* recv_bufs,
+                    const int64_t* recv_capacity_bytes, uint64_t* const* arrived, int32_t* status, void* cuda_stream);
+int vp_exchange_wait(const int32_t* n_steps_b, const int64_t* recv_off_b, int N, int rank, int k_max,
+                     const uint64_t* arrived_counter, uint64_t counter_base, uint32_t max_polls, int32_t* status,
+                     void* cuda_stream);
 
 /*
  * vp_sweep_plan_time - plan quality over a grid of parameters: for every pair (lambda_ns[i], k_target[j]) the batch

@@ -743,6 +743,33 @@ int vpo_demand_from_routing(const int32_t *idx, int n_src, int T, int topk, int 
     return bad;
 }
 
+/* ---------------------------------------------------------- exchange */
+
+/*
+ * What the transport does between pack and unpack (Section 5, "Device-resident buffer layout": one contiguous
+ * chunk per peer and activation).  Sender side for one rank: in step k the lane_bytes[k][rank] bytes at offset
+ * send_off[k][rank] of its staged buffer go to rank j = lane_dst[k][rank], where they land at offset recv_off[k][j]
+ * of j's receive buffer (recv_bufs[j]); arrived[j] (optional) counts the bytes delivered to j.  A chunk that would
+ * overrun recv_capacity[j] is not copied and the function returns VPO_ST_PACK_CAPACITY.
+ */
+int vpo_exchange_put(const int32_t *n_steps, const int16_t *lane_dst, const int64_t *lane_bytes, const int64_t *send_off,
+                     const int64_t *recv_off, int N, int rank, int k_max, const uint8_t *staged,
+                     uint8_t *const *recv_bufs, const int64_t *recv_capacity, uint64_t *arrived)
+{
+    int K = *n_steps < 0 ? 0 : (*n_steps > k_max ? k_max : *n_steps);
+    int st = 0;
+    for (int k = 0; k < K; k++) {
+        int j = lane_dst[(size_t)k * N + rank];
+        int64_t n = lane_bytes[(size_t)k * N + rank];
+        if (j < 0 || n <= 0) continue;
+        int64_t from = send_off[(size_t)k * N + rank], to = recv_off[(size_t)k * N + j];
+        if (to + n > recv_capacity[j]) { st |= VPO_ST_PACK_CAPACITY; continue; }
+        memcpy(recv_bufs[j] + to, staged + from, (size_t)n);
+        if (arrived) arrived[j] += (uint64_t)n;
+    }
+    return st;
+}
+
 /* ------------------------------------------------------------ unpack */
 
 /*

@@ -59,6 +59,7 @@ def _load():
                                     + [C.c_void_p] * 4)
         _lib.vpo_unpack_tokens.argtypes = ([C.c_void_p] * 4 + [C.c_int] * 3 + [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p,
                                             C.c_int64, C.c_int64, C.c_void_p, C.c_void_p])
+        _lib.vpo_exchange_put.argtypes = [C.c_void_p] * 5 + [C.c_int] * 3 + [C.c_void_p] * 4
         _lib.vpo_pack.argtypes = ([C.c_void_p] * 4 + [C.c_int] * 3 + [C.c_void_p, C.c_int, C.c_int, C.c_int,
                                   C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p])
     return _lib
@@ -302,6 +303,26 @@ class OracleCatalog:
                               _p(idx), T, topk, int(experts_per_rank), _p(rows_b), row_bytes, _p(staged),
                               capacity_rows * row_bytes, _p(src_map))
         return staged, src_map, int(st)
+
+    # ---- exchange -------------------------------------------------------
+    def exchange(self, plan: dict, staged_by_src: dict, row_bytes: int = 1):
+        """Every rank in ``staged_by_src`` (rank -> staged bytes, 2-D or flat uint8) sends its chunks as the one-matrix
+        plan says.  Returns (receive buffers per rank as flat uint8 arrays sized by the plan's receive totals,
+        arrived bytes per rank, status)."""
+        N, K = self.N, int(plan["n_steps"])
+        cap = np.ascontiguousarray(plan["recv_off"][K], dtype=np.int64)
+        bufs = [np.zeros(max(int(cap[j]), 1), np.uint8) for j in range(N)]
+        ptrs = (C.c_void_p * N)(*[b.ctypes.data for b in bufs])
+        arrived = np.zeros(N, np.uint64)
+        n_steps = np.asarray([plan["n_steps"]], dtype=np.int32)
+        st = 0
+        for i, staged in staged_by_src.items():
+            flat = np.ascontiguousarray(staged).view(np.uint8).reshape(-1)
+            st |= _load().vpo_exchange_put(_p(n_steps), _p(np.ascontiguousarray(plan["lane_dst"])),
+                                           _p(np.ascontiguousarray(plan["lane_bytes"])), _p(np.ascontiguousarray(plan["send_off"])),
+                                           _p(np.ascontiguousarray(plan["recv_off"])), N, int(i), int(plan["k_max"]),
+                                           _p(flat), ptrs, _p(cap), _p(arrived))
+        return [b[: int(cap[j])] for j, b in enumerate(bufs)], arrived, int(st)
 
     # ---- unpack ---------------------------------------------------------
     def unpack_tokens(self, plan: dict, rank: int, expert_idx, experts_per_rank: int, recv, out=None):

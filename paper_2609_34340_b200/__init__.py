@@ -32,11 +32,14 @@ from .binding import (  # noqa: F401
     schedule_read_stats,
     schedule_launch_info,
     microbench,
+    exchange_put,
+    exchange_wait,
+    gather_exchange_tables,
     memset_probe,
     profile_enable,
     profile_read,
     library_path,
     ST_NEGATIVE, ST_OVERFLOW_RISK, ST_DIAG_NONZERO, ST_NOT_GRANULE, ST_BAD_TAU, ST_UNCOVERED,
-    ST_NO_PROGRESS, ST_STEP_LIMIT, ST_PACK_MISMATCH, ST_PACK_CAPACITY, ST_INTERNAL_TIMEOUT,
+    ST_NO_PROGRESS, ST_STEP_LIMIT, ST_PACK_MISMATCH, ST_PACK_CAPACITY, ST_EXCHANGE_TIMEOUT, ST_INTERNAL_TIMEOUT,
     E_BAD_ARG, E_BAD_CATALOG, E_NOMEM, E_CUDA, E_WORKSPACE, E_UNSUPPORTED,
 )

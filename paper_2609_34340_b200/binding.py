@@ -18,6 +18,7 @@ E_BAD_ARG, E_BAD_CATALOG, E_NOMEM, E_CUDA, E_WORKSPACE, E_UNSUPPORTED = -1, -2, 
 ST_NEGATIVE, ST_OVERFLOW_RISK, ST_DIAG_NONZERO, ST_NOT_GRANULE = 1, 2, 4, 8
 ST_BAD_TAU, ST_UNCOVERED, ST_NO_PROGRESS, ST_STEP_LIMIT = 16, 32, 64, 128
 ST_PACK_MISMATCH, ST_PACK_CAPACITY = 256, 512
+ST_EXCHANGE_TIMEOUT = 2048
 ST_INTERNAL_TIMEOUT = 1 << 30    # a row-copy kernel gave up a bounded wait: the output buffer is incomplete
 
 
@@ -107,6 +108,8 @@ def _load():
     lib.vp_schedule_read_stats.argtypes = [P, P, P]
     lib.vp_schedule_launch_info.argtypes = [vp, i32, C.POINTER(_Params), P]
     lib.vp_microbench.argtypes = [i32, i32, P, C.POINTER(i64), P]
+    lib.vp_exchange_put.argtypes = [P, P, P, P, i32, i32, i32, P, P, P, P, P, P]
+    lib.vp_exchange_wait.argtypes = [P, P, i32, i32, i32, P, C.c_uint64, C.c_uint32, P, P]
     lib.vp_memset_probe.argtypes = [P, sz, P]
     lib.vp_profile_enable.argtypes = [i32]
     lib.vp_profile_read.argtypes = [i32, C.POINTER(C.c_double), C.POINTER(i64)]
@@ -152,6 +155,39 @@ def schedule_read_stats(workspace: torch.Tensor, stream=None) -> dict:
     out = (C.c_uint64 * 3)()
     _check(_load().vp_schedule_read_stats(_ptr(workspace), _stream(stream), out), "vp_schedule_read_stats")
     return dict(activations=int(out[0]), tasks=int(out[1]), sweeps=int(out[2]))
+
+
+def exchange_put(plan: "Plan", b: int, rank: int, staged: torch.Tensor, recv_bufs: torch.Tensor, recv_capacity: torch.Tensor,
+                 arrived: Optional[torch.Tensor], status: torch.Tensor, stream=None) -> None:
+    """``vp_exchange_put`` for matrix ``b`` of a device plan: ``recv_bufs`` / ``arrived`` are int64 device tensors ``[N]`` holding
+    device addresses (``tensor.data_ptr()`` of every rank's receive buffer / counter), ``recv_capacity`` int64 ``[N]`` bytes."""
+    N = plan.lane_dst.shape[2]
+    _check(_load().vp_exchange_put(_ptr(plan.n_steps[b:]), _ptr(plan.lane_dst[b]), _ptr(plan.send_off[b]), _ptr(plan.recv_off[b]),
+                                   int(N), int(rank), int(plan.k_max), _ptr(staged), _ptr(recv_bufs), _ptr(recv_capacity),
+                                   _ptr(arrived), _ptr(status), _stream(stream)), "vp_exchange_put")
+
+
+def exchange_wait(plan: "Plan", b: int, rank: int, counter: torch.Tensor, base: int, max_polls: int, status: torch.Tensor,
+                  stream=None) -> None:
+    """``vp_exchange_wait``: bounded wait for rank ``rank``'s arrival counter (an int64/uint64 device tensor of one element)."""
+    N = plan.lane_dst.shape[2]
+    _check(_load().vp_exchange_wait(_ptr(plan.n_steps[b:]), _ptr(plan.recv_off[b]), int(N), int(rank), int(plan.k_max),
+                                    _ptr(counter), int(base), int(max_polls), _ptr(status), _stream(stream)), "vp_exchange_wait")
+
+
+def gather_exchange_tables(recv_ptr: int, counter_ptr: int, capacity_bytes: int, device=None):
+    """The three tables ``vp_exchange_put`` takes, assembled over ``torch.distributed``: every rank contributes the address
+    of its receive buffer and of its arrival counter (addresses that are valid on the other ranks' GPUs: peer-mapped or
+    symmetric memory) and its buffer size; every rank gets all of them, indexed by rank.  Returns int64 tensors
+    (recv_bufs ``[world]``, arrived ``[world]``, recv_capacity ``[world]``) on ``device`` (default: CPU, for gloo groups)."""
+    import torch.distributed as dist
+    world = dist.get_world_size()
+    on = torch.device("cuda", torch.cuda.current_device()) if dist.get_backend() == "nccl" else torch.device("cpu")
+    mine = torch.tensor([int(recv_ptr), int(counter_ptr), int(capacity_bytes)], dtype=torch.int64, device=on)
+    every = [torch.empty_like(mine) for _ in range(world)]
+    dist.all_gather(every, mine)
+    table = torch.stack(every).to(device if device is not None else "cpu")
+    return table[:, 0].contiguous(), table[:, 1].contiguous(), table[:, 2].contiguous()
 
 
 def microbench(kind: int, iters: int, sink: torch.Tensor, stream=None) -> int:

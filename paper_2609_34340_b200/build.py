@@ -9,7 +9,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libvariopath.so")
-SOURCES = ["catalog.cu", "schedule.cu", "pack.cu", "host_api.cu", "profile.cu", "plan_tools.cu", "analyzer.cu", "unpack.cu", "microbench.cu"]
+SOURCES = ["catalog.cu", "schedule.cu", "pack.cu", "host_api.cu", "profile.cu", "plan_tools.cu", "analyzer.cu", "unpack.cu", "microbench.cu", "exchange.cu"]
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC"]
 

@@ -58,3 +58,20 @@ def test_reference_arm_runs_on_rank0_only():
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["e2e"]["d2h_bytes_per_step"] == 0
     for key in ("metric", "unit", "steps", "warmup", "ms_per_step", "higher_is_better", "config"):
         assert key in line
+
+
+def test_exchange_tables_over_two_gloo_ranks():
+    """Host side of a multi-rank exchange: every rank learns every rank's receive-buffer address, counter address and
+    capacity, indexed by rank (two gloo ranks on CPU; the addresses are stand-ins)."""
+    code = (
+        "import torch.distributed as dist\n"
+        "import paper_2609_34340_b200 as vp\n"
+        "dist.init_process_group('gloo')\n"
+        "r = dist.get_rank()\n"
+        "bufs, ctrs, caps = vp.gather_exchange_tables(0x1000 * (r + 1), 0x2000 * (r + 1) + 8, 4096 * (r + 3))\n"
+        "import json; print(json.dumps([bufs.tolist(), ctrs.tolist(), caps.tolist()]))\n"
+        "dist.destroy_process_group()\n")
+    res = _spawn(code, 2)
+    for rc, out, err in res:
+        assert rc == 0, err
+        assert json.loads(out.strip().splitlines()[-1]) == [[0x1000, 0x2000], [0x2008, 0x4008], [4096 * 3, 4096 * 4]]

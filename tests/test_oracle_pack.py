@@ -127,8 +127,14 @@ def test_pack_exchange_unpack_round_trip(oracle_lib):
         s, m, st = oc.pack(plan, i, idx[i], epr, rows[i], R)
         assert st == 0
         staged[i], meta[i] = s, idx[i].reshape(-1)[m] % epr          # local expert id travels with each row
+    # the oracle's exchange (sender side, rank by rank) delivers the payload; the metadata travels by the numpy helper.
+    # Both must give the receiver the same rows, and every rank must receive exactly its demand column.
+    bufs, arrived, xst = oc.exchange(plan, staged)
+    assert xst == 0 and arrived.tolist() == D.sum(0).tolist()
     for j in (0, 5):
         recv, recv_expert = deliver(plan, j, staged, rb, meta)
+        assert np.array_equal(bufs[j].reshape(-1, rb), recv)
+        recv = bufs[j].reshape(-1, rb)
         out, expert_off, out_src, out_map, st = oc.unpack(plan, j, recv, recv_expert, epr)
         assert st == 0
         want_rows, want_src, want_off = [], [], [0]
