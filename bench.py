@@ -488,7 +488,23 @@ def run_tools(vp, dev, peaks):
            "copy_kernel_gb_per_s": round(bytes_r / (ms_rcopy / max(n_rcopy, 1)) / 1e6, 1),
            "copy_kernel_frac_of_hbm_peak": round(bytes_r / (ms_rcopy / max(n_rcopy, 1)) / 1e6 / peaks["hbm_gbs"], 4)}
     del rrecv, tout
-    return {"schedule_large_batch": large, "unpack_tokens": ret, "unpack": {"workload": f"config 5 receive side: rank {prank}, {R} rows x {pk['row_bytes']} B, {epr} local experts",
+    # plan execution, sender side: rank 8 puts its staged buffer (1.85 GB) into the 15 receivers' buffers on this GPU
+    Rs = int(pk["demand"][0, prank, :].sum().item() // pk["row_bytes"])
+    xstaged = torch.randint(-32768, 32768, (Rs, pk["row_bytes"] // 2), dtype=torch.int16, device=dev, generator=gen)
+    capv = [int(pk["demand"][0, :, j].sum().item()) for j in range(16)]
+    xbufs = [torch.empty(max(cj, 16), dtype=torch.uint8, device=dev) for cj in capv]
+    xcnt = torch.zeros(16, dtype=torch.int64, device=dev)
+    xptr = torch.tensor([t_.data_ptr() for t_ in xbufs], dtype=torch.int64, device=dev)
+    xcptr = torch.tensor([xcnt[j:].data_ptr() for j in range(16)], dtype=torch.int64, device=dev)
+    xcap = torch.tensor(capv, dtype=torch.int64, device=dev)
+    xst = torch.zeros(1, dtype=torch.int32, device=dev)
+    ms_x = timed(lambda: vp.exchange_put(pplan, 0, prank, xstaged, xptr, xcap, xcptr, xst))
+    assert int(xst.item()) == 0
+    bytes_x = 2 * Rs * pk["row_bytes"]
+    xput = {"workload": f"config 5 sender side: rank {prank} puts {Rs} rows x {pk['row_bytes']} B into 15 receive buffers on the same GPU",
+            "ms": round(ms_x, 4), "gb_per_s": round(bytes_x / ms_x / 1e6, 1), "frac_of_hbm_peak": round(bytes_x / ms_x / 1e6 / peaks["hbm_gbs"], 4)}
+    del xstaged, xbufs
+    return {"schedule_large_batch": large, "exchange_put": xput, "unpack_tokens": ret, "unpack": {"workload": f"config 5 receive side: rank {prank}, {R} rows x {pk['row_bytes']} B, {epr} local experts",
                        "ms": round(ms_u, 4), "copy_kernel_ms": round(ms_copy / max(n_copy, 1), 4),
                        "gb_per_s": round(bytes_u / ms_u / 1e6, 1),
                        "copy_kernel_gb_per_s": round(bytes_u / (ms_copy / max(n_copy, 1)) / 1e6, 1),

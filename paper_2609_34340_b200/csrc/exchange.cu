@@ -52,7 +52,14 @@ exchange_put_kernel(const int32_t* __restrict__ n_steps, const int16_t* __restri
         const long long n = to - from;
         if ((((uintptr_t)src | (uintptr_t)dst) & 15) == 0) {
             const long long vecs = n >> 4;
-            for (long long e = threadIdx.x; e < vecs; e += kPutThreads) ((uint4*)dst)[e] = ((const uint4*)src)[e];
+            long long e = threadIdx.x;
+            for (; e + 3 * kPutThreads < vecs; e += 4 * kPutThreads) {      // four 16-byte loads in flight per thread
+                const uint4 v0 = ((const uint4*)src)[e], v1 = ((const uint4*)src)[e + kPutThreads];
+                const uint4 v2 = ((const uint4*)src)[e + 2 * kPutThreads], v3 = ((const uint4*)src)[e + 3 * kPutThreads];
+                ((uint4*)dst)[e] = v0; ((uint4*)dst)[e + kPutThreads] = v1;
+                ((uint4*)dst)[e + 2 * kPutThreads] = v2; ((uint4*)dst)[e + 3 * kPutThreads] = v3;
+            }
+            for (; e < vecs; e += kPutThreads) ((uint4*)dst)[e] = ((const uint4*)src)[e];
             for (long long e = (vecs << 4) + threadIdx.x; e < n; e += kPutThreads) dst[e] = src[e];
         } else {
             for (long long e = threadIdx.x; e < n; e += kPutThreads) dst[e] = src[e];
@@ -98,7 +105,7 @@ extern "C" int vp_exchange_put(const int32_t* n_steps_b, const int16_t* lane_dst
         if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return VP_E_CUDA;
         if (dev >= 0 && dev < 64) s_sms[dev] = sms;
     }
-    exchange_put_kernel<<<sms * 4, kPutThreads, 0, (cudaStream_t)cuda_stream>>>(
+    exchange_put_kernel<<<sms * 8, kPutThreads, 0, (cudaStream_t)cuda_stream>>>(
         n_steps_b, lane_dst_b, send_off_b, recv_off_b, N, rank, k_max, (const unsigned char*)staged,
         (unsigned char* const*)recv_bufs, recv_capacity_bytes, (unsigned long long* const*)arrived, status);
     g_vp_launches++;
