@@ -317,6 +317,67 @@ extern "C" int vp_load_catalog(const void* topology, size_t topo_bytes, const vo
             dc.max_row_terms = (int)max_row;
             if (!rc) rc = upload(c, pat_term, &dc.pat_term);
             if (!rc) rc = upload(c, shape_pat, &dc.shape_pat);
+            // Two rails: when the shapes that share a first row are consecutive, and first rows fall into few classes
+            // with the same list of second rows, the first maximum of Eq. (6) can be taken class by class.
+            if (S == 2 && !rc) {
+                std::vector<int> run_row, run_start;                       // first row and first shape of every run
+                std::vector<std::vector<uint32_t>> run_list;               // its second rows, in shape order
+                std::vector<char> seen(rows.size(), 0);
+                bool ok = true;
+                for (int s = 0; s < n_shapes && ok; s++) {
+                    const int p0 = (int)(shape_pat[s] & 0xffffu), p1 = (int)(shape_pat[s] >> 16);
+                    if (run_row.empty() || run_row.back() != p0) {
+                        if (seen[p0]) ok = false;                           // a first row with two separate runs
+                        seen[p0] = 1;
+                        run_row.push_back(p0); run_start.push_back(s); run_list.emplace_back();
+                    }
+                    run_list.back().push_back((uint32_t)p1);
+                }
+                std::map<std::vector<uint32_t>, int> cls_of;
+                std::vector<std::vector<uint32_t>> members, lists;          // per class: first row | run start << 16; second rows
+                for (size_t r = 0; r < run_row.size() && ok; r++) {
+                    auto it = cls_of.find(run_list[r]);
+                    int cl;
+                    if (it == cls_of.end()) {
+                        cl = (int)members.size();
+                        cls_of.emplace(run_list[r], cl);
+                        members.emplace_back();
+                        lists.push_back(run_list[r]);
+                    } else {
+                        cl = it->second;
+                    }
+                    members[cl].push_back((uint32_t)run_row[r] | (uint32_t)run_start[r] << 16);
+                }
+                // Units: 2 cl = the first rows of class cl, 2 cl + 1 = its second rows; each unit's entries fill whole
+                // chunks of 32 (one warp each).  An entry carries the row's terms and its place within the unit.
+                const int n = (int)members.size(), stride = (int)max_row + 1;
+                size_t n_chunks = 0;
+                for (int cl = 0; cl < n; cl++) n_chunks += (members[cl].size() + 31) / 32 + (lists[cl].size() + 31) / 32;
+                if (ok && n <= 16 && n_chunks <= 32) {
+                    constexpr int kHeader = 72;                            // 3 + (2 n + 1) + up to 32 chunk units <= 72
+                    std::vector<uint32_t> dec(kHeader + n_chunks * 32 * stride, 0);
+                    dec[0] = (uint32_t)n_chunks; dec[1] = (uint32_t)stride; dec[2] = kHeader;
+                    size_t chunk = 0;
+                    for (int unit = 0; unit < 2 * n; unit++) {
+                        dec[3 + unit] = (uint32_t)chunk;
+                        const std::vector<uint32_t>& src = unit & 1 ? lists[unit >> 1] : members[unit >> 1];
+                        const size_t padded = (src.size() + 31) / 32 * 32;
+                        for (size_t i = 0; i < padded; i++) {
+                            uint32_t* ent = &dec[kHeader + (chunk * 32 + i) * stride];
+                            if (i >= src.size()) { ent[stride - 1] = 0xffffffffu; continue; }    // padding: never wins
+                            const std::vector<uint32_t>& row = rows[src[i] & 0xffffu];
+                            for (size_t t = 0; t < row.size(); t++) ent[t] = row[t];
+                            ent[stride - 1] = (uint32_t)i | (src[i] & 0xffff0000u);              // place | run start << 16
+                        }
+                        for (size_t cc = chunk; cc < chunk + padded / 32; cc++) dec[3 + 2 * n + 1 + cc] = (uint32_t)unit;
+                        chunk += padded / 32;
+                    }
+                    dec[3 + 2 * n] = (uint32_t)chunk;
+                    dc.dec_classes = n;
+                    dc.dec_words = (int)dec.size();
+                    rc = upload(c, dec, &dc.dec);
+                }
+            }
         }
     }
     if (!rc) rc = upload(c, bucket_ptr, &dc.bucket_ptr);

@@ -1152,7 +1152,7 @@ static_assert(sizeof(Launch) <= sizeof(((vp_launch_memo*)0)->launch), "the launc
 typedef void (*KernelFn)(DevCat, KParams, const int64_t*, const int64_t*, int, int32_t*, int32_t*, int16_t*, uint16_t*,
                          int64_t*, int64_t*, int64_t*, int64_t*, int32_t*, int64_t*, unsigned int*, const int*);
 typedef void (*BigKernelFn)(DevCat, KParams, const int64_t*, const int64_t*, int, int32_t*, int32_t*, int16_t*, uint16_t*,
-                            int64_t*, int64_t*, int64_t*, int64_t*, int32_t*, int64_t*, unsigned int*, int*, const int*);
+                            int64_t*, int64_t*, int64_t*, int64_t*, int32_t*, unsigned int*, int*, const int*);
 
 KernelFn pick_kernel(int g, int lpg) {
     switch (g) {
@@ -1169,7 +1169,10 @@ KernelFn pick_kernel(int g, int lpg) {
     }
     return nullptr;
 }
-BigKernelFn pick_big_kernel(int w) { return w == 2 ? vp_schedule_big_kernel<2> : vp_schedule_big_kernel<1>; }
+BigKernelFn pick_big_kernel(int w, bool dec) {
+    if (dec) return w == 2 ? vp_schedule_big_kernel<2, true> : vp_schedule_big_kernel<1, true>;
+    return w == 2 ? vp_schedule_big_kernel<2, false> : vp_schedule_big_kernel<1, false>;
+}
 
 int resolve_params(const vp_catalog* c, const vp_sched_params* p, KParams* kp) {
     if (!c || !p) return VP_E_BAD_ARG;
@@ -1235,7 +1238,7 @@ int plan_launch_uncached(const vp_catalog* c, int B, const vp_sched_params* p, L
             // emit step; up to 32 groups a task is one warp and four to eight warps per CTA leave room for several CTAs per SM
             const int w = dc.G > 32 ? 2 : 1;
             const int threads = w == 2 ? 512 : (dc.G > 16 ? 256 : 128);
-            BigKernelFn bf = pick_big_kernel(w);
+            BigKernelFn bf = pick_big_kernel(w, big_use_dec(dc));
             if (cudaFuncSetAttribute(bf, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return VP_E_CUDA;
             int bper_sm = 0;
             if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&bper_sm, bf, threads, smem) != cudaSuccess || bper_sm < 1) return VP_E_CUDA;
@@ -1299,14 +1302,13 @@ int plan_launch(const vp_catalog* cc, int B, const vp_sched_params* p, Launch* o
     return VP_OK;
 }
 
-// Workspace: 256 bytes of counters; one residual slot per CTA when a kernel keeps the residual outside shared memory
-// (the kernel for large node-symmetric catalogs always has one, for its saturated cells); with that kernel also the
-// list of matrices left to the general kernel, the work order and its keys.
+// Workspace: 256 bytes of counters; one residual slot per CTA of the general kernel when it keeps the residual outside
+// shared memory; with the kernel for large node-symmetric catalogs also the list of matrices left to the general
+// kernel, the work order and its keys.
 struct WsLayout { size_t drem, todo, order, key, total; };
 WsLayout ws_layout(const vp_catalog* c, const Launch& L, int B) {
     WsLayout w;
-    const int slots = L.kernel == 2 ? (L.grid > L.big_grid ? L.grid : L.big_grid) : L.grid;
-    const size_t slot_bytes = (L.kernel == 2 || !L.kp.drem_in_smem) ? (size_t)slots * c->dc.N * c->dc.N * 8 : 0;
+    const size_t slot_bytes = !L.kp.drem_in_smem ? (size_t)L.grid * c->dc.N * c->dc.N * 8 : 0;
     w.drem = 256;
     w.todo = vp_align256(256 + slot_bytes);
     const size_t list = L.kernel == 2 ? vp_align256((size_t)B * 4) : 0;
@@ -1366,9 +1368,9 @@ extern "C" int vp_schedule_batch(const vp_catalog* c, const vp_sched_params* p, 
                     big_rank_kernel<<<(B + 255) / 256, 256, 0, stream>>>(key, B, order);
                     g_vp_launches += 2;
                 }
-                pick_big_kernel(L.big_w)<<<L.big_grid, L.big_threads, L.big_smem, stream>>>(
+                pick_big_kernel(L.big_w, big_use_dec(c->dc))<<<L.big_grid, L.big_threads, L.big_smem, stream>>>(
                     c->dc, L.kp, demand, tau_ns_in, B, n_steps, chan_id, lane_dst, lane_inst, lane_bytes, send_off, recv_off,
-                    tau_ns_out, status, ws_drem, counter, todo, order);
+                    tau_ns_out, status, counter, todo, order);
                 g_vp_launches++;
                 pick_kernel(c->dc.g, L.lpg)<<<L.grid, L.threads, L.smem, stream>>>(
                     c->dc, L.kp, demand, tau_ns_in, B, n_steps, chan_id, lane_dst, lane_inst, lane_bytes, send_off, recv_off,

@@ -3,11 +3,11 @@
 //
 // One CTA decomposes one matrix at a time.  What differs from the general kernel is where the state lives:
 //
-//  * Credits.  Step 2 only ever looks at min(D_rem[i][j], cap_r) (Eq. 7).  When every lane capacity is below 2^16
-//    granules, a 16-bit copy of the residual that saturates at 65,535 granules gives exactly the same credits, and
-//    N x N of those fit shared memory (128 KB at N = 256) where the residual itself (256 KB in 32-bit granules) does
-//    not.  The exact residual of a cell is kept in an L2-resident workspace slot and is touched only while the cell
-//    is still saturated; once a cell has dropped below 65,535 granules the 16-bit copy *is* the residual.
+//  * Credits.  Step 2 only ever looks at min(D_rem[i][j], cap_r) (Eq. 7).  N x N 16-bit cells fit shared memory (128 KB
+//    at N = 256) where the residual in 32-bit granules (256 KB) does not.  A cell below F = 65,536 - M granules is
+//    kept as it is; a cell of F granules or more holds F + (its index in a side list of M = 4,096 exact 32-bit
+//    values).  As long as every lane capacity is below F, such a cell yields the same credit as its exact value
+//    (the capacity), and the emit step keeps the side list exact until the cell drops below F and becomes ordinary.
 //  * Scores.  Eq. (6) on a node-symmetric catalog is a sum of at most max_terms products count x C[e], where
 //    C[delta][q][q'] = sum_n D-hat[(n,q)][(n+delta,q')] (the same integer as the full sum over D-hat).  The table C
 //    (P S S entries, 32-bit granules) is kept in shared memory and every activation subtracts its lane volumes from
@@ -24,7 +24,7 @@
 //    such a matrix is below 65,535 granules, so its 16-bit copy is exact.  No L2 traffic is needed in this mode.
 //
 // A matrix that does not meet the conditions (granule below 256 bytes, a capacity of 2^22 granules or more, 2^32
-// granules or more in total, more than 32 hot columns) is appended to a list that the general kernel works through
+// granules or more in total, more than 32 hot columns, more big cells than the side list holds) is appended to a list that the general kernel works through
 // afterwards.
 #pragma once
 
@@ -36,13 +36,18 @@ constexpr int BIG_RS_COPIES = 1;
 constexpr int BIG_HOT_MAX = 32;       // columns whose cells are kept beyond 16 bits
 
 struct BigSmem {
-    int cs, tbl, rs, pat, bnd, hi, colmap, gnode, send_acc, recv_acc, red, pair, task_f, task_den, slotw, bind_src, bind_dst, term, bucket, total;
+    int cs, tbl, rs, pat, bnd, dec, hi, colmap, gnode, send_acc, recv_acc, red, pair, task_f, task_den, slotw, bind_src, bind_dst, term, bucket, total;
     int cs_stride;            // credits per row of the 16-bit matrix (N + 2: rows start in different banks)
     int pat_words;            // 32-bit words of row-pattern ids per shape (two ids per word)
 };
 
+// The arg-max is taken class by class when the catalog allows it and has enough shapes for that to pay: a few hundred
+// shapes are scanned faster than two rounds of class maxima.
+__host__ __device__ inline bool big_use_dec(const DevCat& dc) { return dc.dec != nullptr && dc.n_shapes >= 1024; }
+
 __host__ __device__ inline BigSmem big_smem_layout(const DevCat& dc, const KParams& kp) {
     BigSmem L;
+    const bool dec = big_use_dec(dc);
     int o = 0;
     L.cs_stride = dc.N + 2;
     const int cs_bytes = dc.N * L.cs_stride * 2, dhat_bytes = dc.G * dc.G * 8 + dc.N * 24;
@@ -52,7 +57,8 @@ __host__ __device__ inline BigSmem big_smem_layout(const DevCat& dc, const KPara
     L.tbl = o;       o += align16(dc.tbl_size * 4);
     L.rs = o;        o += dc.n_patterns * 8 * BIG_RS_COPIES;      // row scores, one copy per lane class
     L.pat = o;       o += align16(dc.n_patterns * dc.max_row_terms * 4);
-    L.bnd = o;       o += ((dc.n_shapes + 31) & ~31) * 4;          // upper bounds on (score >> 2) of every shape
+    L.bnd = o;       o += dec ? 0 : ((dc.n_shapes + 31) & ~31) * 4;     // upper bounds on (score >> 2) of every shape
+    L.dec = o;       o += dec ? align16(dc.dec_words * 4) : 0;     // class decomposition of the arg-max, if any
     L.gnode = o;     o += align16(dc.G * 2);
     L.send_acc = o;  o += dc.N * 8;
     L.recv_acc = o;  o += dc.N * 8;
@@ -64,7 +70,7 @@ __host__ __device__ inline BigSmem big_smem_layout(const DevCat& dc, const KPara
     L.bind_src = o;  o += align16(kp.max_tasks * dc.N);
     L.bind_dst = o;  o += align16(kp.max_tasks * dc.N);
     L.pat_words = (dc.S + 1) / 2;
-    L.term = o;      o += ((dc.n_shapes + 31) & ~31) * L.pat_words * 4;
+    L.term = o;      o += dec ? 0 : ((dc.n_shapes + 31) & ~31) * L.pat_words * 4;
     L.bucket = o;    o += align16((dc.n_shapes + 1) * 4);
     L.total = o;
     return L;
@@ -194,13 +200,14 @@ __global__ void __launch_bounds__(256) big_rank_kernel(const int* __restrict__ k
 #ifndef VP_BIG_W1_CTAS
 #define VP_BIG_W1_CTAS 2
 #endif
-template <int W>
+// DEC: the arg-max of Eq. (6) is taken class by class (see big_use_dec).
+template <int W, bool DEC>
 __global__ void __launch_bounds__(W == 2 ? 512 : 256, W == 2 ? 1 : VP_BIG_W1_CTAS)
 vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand, const int64_t* __restrict__ tau_in, int B,
                        int32_t* __restrict__ n_steps, int32_t* __restrict__ chan_id, int16_t* __restrict__ lane_dst,
                        uint16_t* __restrict__ lane_inst, int64_t* __restrict__ lane_bytes, int64_t* __restrict__ send_off,
                        int64_t* __restrict__ recv_off, int64_t* __restrict__ tau_out, int32_t* __restrict__ status,
-                       int64_t* ws_drem, unsigned int* counter, int* __restrict__ todo, const int* __restrict__ order) {
+                       unsigned int* counter, int* __restrict__ todo, const int* __restrict__ order) {
     // `order` (may be null) lists the matrices in the order in which the CTAs should take them: longest first.
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int N = dc.N, G = dc.G, tid = threadIdx.x, NT = blockDim.x;
@@ -214,6 +221,8 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
     uint64_t* rs = (uint64_t*)(smem_raw + L.rs);
     uint32_t* pat = (uint32_t*)(smem_raw + L.pat);
     uint32_t* bnd = (uint32_t*)(smem_raw + L.bnd);
+    const uint32_t* decs = (const uint32_t*)(smem_raw + L.dec);
+    const int dec_n = DEC ? dc.dec_classes : 0;
     uint8_t* gnode = smem_raw + L.gnode;                 // per group: node index, then (at G) rail index
     int64_t* send_acc = (int64_t*)(smem_raw + L.send_acc);
     int64_t* recv_acc = (int64_t*)(smem_raw + L.recv_acc);
@@ -226,8 +235,11 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
     uint8_t* bind_dst = smem_raw + L.bind_dst;
     uint32_t* spat = (uint32_t*)(smem_raw + L.term);      // row-pattern ids per shape
     uint32_t* bucket = (uint32_t*)(smem_raw + L.bucket);
-    uint32_t* Dg = (uint32_t*)(ws_drem + (size_t)blockIdx.x * N * N);      // exact residual, granules
-    __shared__ int s_b, s_flags, s_mode, s_nhot;           // s_mode: 0 leave to the general kernel, 1 plain, 2 hot columns
+    // Big cells (16-bit mode): a cell of big_floor granules or more holds big_floor + its index in the side list, where
+    // its exact value is kept.  Every capacity is below big_floor, so such a cell gives the same credit as its value.
+    uint32_t* side = (uint32_t*)(smem_raw + L.hi);
+    const int big_max = min(BIG_HOT_MAX * N / 2, 4096), big_floor = 65536 - big_max;
+    __shared__ int s_b, s_flags, s_mode, s_nhot, s_nbig;           // s_mode: 0 leave to the general kernel, 1 plain, 2 hot columns
     __shared__ int64_t s_tau, s_left;
     __shared__ int64_t s_tscale[VP_MAX_CLASSES];
     __shared__ uint32_t s_cap[VP_MAX_CLASSES];
@@ -242,7 +254,7 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
     // ---- stage the catalog once per CTA: packed terms and bucket pointers by bulk asynchronous copies (TMA) onto one
     // mbarrier; should the bounded wait give up, plain loads fetch the same arrays
     {
-        const unsigned b_term = (unsigned)(ns_pad * L.pat_words * 4), b_bucket = (unsigned)align16((dc.n_shapes + 1) * 4);
+        const unsigned b_term = DEC ? 0u : (unsigned)(ns_pad * L.pat_words * 4), b_bucket = (unsigned)align16((dc.n_shapes + 1) * 4);
         const unsigned b_pat = (unsigned)align16(dc.n_patterns * dc.max_row_terms * 4);
         bool landed = false;
         if (b_term + b_bucket + b_pat < (1u << 20)) {
@@ -251,7 +263,7 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
                 mbar_init(bar, 1);
                 asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
                 mbar_expect_tx(bar, b_term + b_bucket + b_pat);
-                bulk_load(smem_u32(spat), dc.shape_pat, b_term, bar);
+                if (b_term) bulk_load(smem_u32(spat), dc.shape_pat, b_term, bar);
                 bulk_load(smem_u32(bucket), dc.bucket_ptr, b_bucket, bar);
                 bulk_load(smem_u32(pat), dc.pat_term, b_pat, bar);
             }
@@ -259,14 +271,15 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
             landed = __syncthreads_and(mbar_wait_bounded(bar, 0, 1u << 20)) != 0;
         }
         if (!landed) {
-            for (int e = tid; e < ns_pad * L.pat_words; e += NT) spat[e] = dc.shape_pat[e];
+            for (int e = tid; e < ns_pad * L.pat_words && !DEC; e += NT) spat[e] = dc.shape_pat[e];
             for (int e = tid; e <= dc.n_shapes; e += NT) bucket[e] = dc.bucket_ptr[e];
             for (int e = tid; e < dc.n_patterns * dc.max_row_terms; e += NT) pat[e] = dc.pat_term[e];
         }
         for (int a = tid; a < G; a += NT) { gnode[a] = (uint8_t)(a / S); gnode[G + a] = (uint8_t)(a % S); }
+        for (int e = tid; e < dc.dec_words && DEC; e += NT) ((uint32_t*)(smem_raw + L.dec))[e] = dc.dec[e];
         __syncthreads();
         // pattern ids become byte offsets into the row scores (fewer than 1,024 patterns, so they still fit 16 bits)
-        for (int e = tid; e < ns_pad * L.pat_words; e += NT) {
+        for (int e = tid; e < ns_pad * L.pat_words && !DEC; e += NT) {
             const uint32_t w = spat[e];
             spat[e] = (w & 0xffffu) * (8 * BIG_RS_COPIES) | ((w >> 16) * (8 * BIG_RS_COPIES)) << 16;
         }
@@ -301,7 +314,7 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
         int64_t* colsum = rowsum + N;
         int64_t* colmax = colsum + N;
         for (int i = tid; i < N; i += NT) { colsum[i] = 0; colmax[i] = 0; rowsum[i] = 0; send_acc[i] = 0; recv_acc[i] = 0; colmap[i] = 0xFF; }
-        if (tid == 0) s_nhot = 0;
+        if (tid == 0) { s_nhot = 0; s_nbig = 0; }
         for (int e = tid; e < G * G; e += NT) Dhat[e] = 0;
         __syncthreads();
         int flags = 0;
@@ -381,7 +394,7 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
                 // 16-bit credits need capacities below 2^16 granules, hot columns capacities below 2^22 (four credits and
                 // a tag share 32 bits); the 32-bit table needs fewer than 2^32 granules in all
                 const bool fits = kp.granule >= 256 && t / kp.granule < ((int64_t)1 << 32);
-                s_mode = !fits ? 0 : (cap_max / kp.granule < 65535 ? 1 : (cap_max / kp.granule < ((int64_t)1 << 22) ? 2 : 0));
+                s_mode = !fits ? 0 : (cap_max / kp.granule < big_floor ? 1 : (cap_max / kp.granule < ((int64_t)1 << 22) ? 2 : 0));
                 s_tau = tq; s_left = t / kp.granule;
             }
             __syncthreads();
@@ -416,25 +429,34 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
                 tbl[e] = (uint32_t)(s / kp.granule);
             }
             __syncthreads();
-            // ---- pass 2 over D: the residual in granules (workspace slot) and its saturating 16-bit copy
+            // ---- pass 2 over D: the residual in granules as 16-bit cells (big cells through the side list)
             const bool hot_mode = s_mode == 2;
+            if (DEC && tid < 2 * dec_n) red[tid] = 0;        // the units' best keys (see step A)
             for (int e = tid; e < N * N; e += NT) {
                 const uint32_t v = (uint32_t)(D[e] / kp.granule);
                 const int i = e / N, j = e - i * N;
                 if (!hot_mode) {
-                    Dg[e] = v;
-                    Cs[i * CS + j] = (uint16_t)min_v(v, 65535u);
+                    uint32_t code = v;
+                    if (v >= (uint32_t)big_floor) {             // a big cell: exact value in the side list, its index in the matrix
+                        const int at = atomicAdd(&s_nbig, 1);
+                        code = (uint32_t)big_floor + (uint32_t)min_v(at, big_max - 1);
+                        if (at < big_max) side[at] = v;
+                    }
+                    Cs[i * CS + j] = (uint16_t)code;
                 } else {                                     // exact: 32 bits in a hot column, below 65,535 elsewhere
                     Cs[i * CS + j] = (uint16_t)v;
                     if (colmap[j] != 0xFF) Hi[(int)colmap[j] * N + i] = (uint16_t)(v >> 16);
                 }
             }
             __syncthreads();
+            if (s_nbig > big_max) {                          // more big cells than the side list holds: the general kernel's
+                if (tid == 0) todo[atomicAdd(counter + 1, 1u)] = b;
+                __syncthreads();
+                continue;
+            }
             int64_t left = s_left;
             int last_s = -1;                                 // shape chosen in the last iteration
-            for (int s = tid; s < dc.n_shapes; s += NT) bnd[s] = 0xffffffffu;
-            uint16_t* sat_cell = nullptr;                    // a saturated cell whose exact residual is on its way from L2
-            uint32_t sat_left = 0;
+            for (int s = tid; s < dc.n_shapes && !DEC; s += NT) bnd[s] = 0xffffffffu;
             int f_cached = -1;                               // family whose tables this lane still holds (first task only)
             uint32_t c_co = 0;
             uint2 c_fi = make_uint2(0u, 0u);
@@ -444,16 +466,18 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
                 if (left == 0) break;
                 if (k == kp.k_max) { st |= VP_ST_STEP_LIMIT; break; }
                 // (A) Eq. (6).  Row scores first: at most max_row_terms products each, stored shifted left by 16 bits.
-                for (int p = tid; p < dc.n_patterns; p += NT) {
-                    uint64_t v = 0;
+                if (!DEC) {
+                    for (int p = tid; p < dc.n_patterns; p += NT) {
+                        uint64_t v = 0;
 #pragma unroll 1
-                    for (int t = 0; t < dc.max_row_terms; t++) {
-                        const uint32_t tw = pat[p * dc.max_row_terms + t];
-                        v += (uint64_t)tbl[tw & 0xffffu] * (tw >> 16);
+                        for (int t = 0; t < dc.max_row_terms; t++) {
+                            const uint32_t tw = pat[p * dc.max_row_terms + t];
+                            v += (uint64_t)tbl[tw & 0xffffu] * (tw >> 16);
+                        }
+                        rs[p] = v << 16;
                     }
-                    rs[p] = v << 16;
+                    __syncthreads();
                 }
-                __syncthreads();
                 // A score is below 2^34 (g x fewer than 2^32 granules) and there are fewer than 2^16 shapes, so
                 // key = score << 16 | (65535 - shape) orders by score first and lower shape index second: the first
                 // maximum of Eq. (6) is a plain maximum of keys.
@@ -472,7 +496,26 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
                     return key;
                 };
                 uint64_t best = 0;
-                {
+                if (DEC) {
+                    // Class by class (two rails).  A shape is a first row p0 and a second row p1 from the list of p0's
+                    // class, and its index grows with p0's place in shape order first, p1's place in the list second.
+                    // So within a class the first maximum is (first maximal p0, first maximal p1 of the list): two
+                    // independent maxima.  One warp per chunk of 32 rows: each lane scores its row from the table
+                    // (at most max_row_terms products) and the chunk's best key score << 16 | (65535 - place) is kept.
+                    const int n_chunks = (int)decs[0], stride = (int)decs[1];
+                    for (int c = warp; c < n_chunks; c += n_warps) {
+                        const uint32_t* ent = decs + decs[2] + (size_t)(c * 32 + lane) * stride;
+                        uint64_t v = 0;
+#pragma unroll 3
+                        for (int t = 0; t < stride - 1; t++) {
+                            const uint32_t tw = ent[t];
+                            v += (uint64_t)tbl[tw & 0xffffu] * (tw >> 16);
+                        }
+                        const uint32_t meta = ent[stride - 1];
+                        const uint64_t key = big_warp_max64(meta == 0xffffffffu ? 0ull : (v << 16 | (uint64_t)(65535u - (meta & 0xffffu))));
+                        if (lane == 0) atomicMax((unsigned long long*)&red[decs[3 + 2 * dec_n + 1 + c]], (unsigned long long)key);
+                    }
+                } else {
                     uint32_t floor32 = 0;
                     if (last_s >= 0) {
                         best = score_key(last_s);                              // (the same in every thread)
@@ -488,12 +531,21 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
                     best = big_warp_max64(best);
                     if (lane == 0) red[warp] = (int64_t)best;
                 }
-                if (sat_cell) {                                  // (requested by the last emit step; back from L2 by now)
-                    *sat_cell = (uint16_t)min_v(sat_left, 65535u);
-                    sat_cell = nullptr;
-                }
                 __syncthreads();
-                const uint64_t bkey = big_warp_max64(lane < n_warps ? (uint64_t)red[lane] : 0ull);
+                uint64_t bkey;
+                if (DEC) {                                     // the classes' candidates: largest score, lowest shape
+                    uint64_t cand = 0;
+                    if (lane < dec_n) {                          // (red[unit]: the best key of the unit's chunks)
+                        const uint64_t k0 = (uint64_t)red[2 * lane], k1 = (uint64_t)red[2 * lane + 1];
+                        const uint32_t place0 = 65535u - (uint32_t)(k0 & 0xffffu);
+                        const uint32_t first = decs[decs[2] + (size_t)(decs[3 + 2 * lane] * 32 + place0) * decs[1] + decs[1] - 1] >> 16;
+                        const uint32_t shape = first + (65535u - (uint32_t)(k1 & 0xffffu));
+                        cand = ((k0 >> 16) + (k1 >> 16)) << 16 | (uint64_t)(65535u - shape);
+                    }
+                    bkey = big_warp_max64(cand);
+                } else {
+                    bkey = big_warp_max64(lane < n_warps ? (uint64_t)red[lane] : 0ull);
+                }
                 if ((bkey >> 16) == 0) { st |= VP_ST_UNCOVERED; break; }
                 const int best_s = 65535 - (int)(bkey & 0xffffu);
                 last_s = best_s;
@@ -729,9 +781,10 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
                                 if (hcell) {
                                     *cell = (uint16_t)(c - x);
                                     *hcell = (uint16_t)((c - x) >> 16);
-                                } else if (c == 65535u && !hot_mode) {   // saturated: the exact residual is in the workspace slot;
-                                    sat_cell = cell;              // its new value is put in place before the next Step 2
-                                    sat_left = atomicSub(&Dg[(size_t)i * N + j], x) - x;
+                                } else if (c >= (uint32_t)big_floor && !hot_mode) {   // a big cell: exact value in the side list
+                                    const uint32_t now = side[c - big_floor] - x;
+                                    if (now >= (uint32_t)big_floor) side[c - big_floor] = now;
+                                    else *cell = (uint16_t)now;   // (an ordinary cell from here on)
                                 } else {
                                     *cell = (uint16_t)(c - x);
                                 }
@@ -744,6 +797,7 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
                         }
                     }
                     if (tid == 0) chan_id_b[k] = f0 + h;
+                    if (DEC && tid < 2 * dec_n) red[tid] = 0;    // the units' best keys start the next iteration at zero
                 }
                 left -= wF;
                 k++;

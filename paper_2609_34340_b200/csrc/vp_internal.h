@@ -33,6 +33,15 @@ struct DevCat {
     const uint32_t* pat_term;
     const uint32_t* shape_pat;
     int n_patterns, max_row_terms;
+    // Class decomposition of the arg-max (two rails): the shapes with first row p0 are consecutive, starting at shape
+    // run_start(p0), and first rows of one class share the list of second rows that complete them, in shape order, so
+    // shape(p0, p1) = run_start(p0) + place of p1 in the list of p0's class.  Unit 2 cl holds the first rows of class cl,
+    // unit 2 cl + 1 its second rows, each padded to whole chunks of 32 entries.  dec[0] = chunks, dec[1] = words per
+    // entry, dec[2] = offset of the entries, dec[3 .. 3 + 2 n] = first chunk of every unit, then the unit of every chunk; an entry is the row's terms
+    // (table index | count << 16, zero padded) followed by place | run_start << 16 (all ones marks padding).  Null
+    // when the catalog has no such structure.
+    const uint32_t* dec;
+    int dec_classes, dec_words;
     const uint32_t* bucket_ptr;
     // family f, slot r: instance id | destination group << 16 | rate class << 24
     const uint32_t* fam_slot;

@@ -429,6 +429,41 @@ def test_large_capacities_and_hot_columns(vp, oracle_lib, nodes):
     _assert_same(got, want)
 
 
+@pytest.mark.parametrize("nodes", [9, 32])
+def test_big_cells_beside_16_bit_credits(vp, oracle_lib, nodes):
+    """Capacities below 2^16 granules with cells far above: such cells are kept exactly in a side list (16 N entries, at
+    most 4,096) and the matrix holds their indices.  Cells right at the boundary value, a sparse block-diagonal matrix
+    whose every cell is big, cells that shrink below the boundary while the matrix is decomposed, and more big cells
+    than the list holds (the general kernel takes that matrix)."""
+    cat = node_template_catalog(tree_topology(nodes, pcie_bw=64, nic_bw=50 if nodes == 9 else 64))
+    N = cat.topology.N
+    side = min(16 * N, 4096)
+    floor = 65536 - side
+    rng = np.random.default_rng(300 + nodes)
+    u = 256
+    B = 6
+    D = (rng.integers(0, 3000, size=(B, N, N)) * (rng.random((B, N, N)) < 0.3)).astype(np.int64)
+    D[0] = 0
+    for i in range(N):                                                    # eight partners per rank, every cell big
+        D[0][i, [(i // 8) * 8 + m for m in range(8)]] = rng.integers(70_000, 200_000)
+    mask = rng.random((N, N)) < 0.02
+    D[1][mask] = rng.integers(floor - 2, floor + 3, size=int(mask.sum()))   # right at the boundary
+    over = rng.random((N, N)) < 1.3 * side / (N * N)                      # more big cells than the list holds
+    D[2][over] = rng.integers(66_000, 90_000, size=int(over.sum()))
+    assert int(over.sum()) - N > side
+    D[3][rng.random((N, N)) < min(0.9 * side / (N * N), 0.5)] = 1_000_000  # just within the list, far above the boundary
+    D[4][: N // 2] = rng.integers(floor - 500, floor + 500, size=(N // 2, N))
+    D *= u
+    for b in range(B):
+        np.fill_diagonal(D[b], 0)
+    for extra in ({}, {"k_target": 64}, {"n_start": 2, "i_aa": 5, "lambda_ns": 0}):
+        w = WParams(granule_bytes=u, k_max=40 * N, **extra).resolved(N)
+        got, want, *_ = _both(vp, oracle_lib, cat, D, w)
+        _assert_same(got, want)
+        if "n_start" not in extra:                     # (fewer starts than ranks per group can end in "no progress")
+            assert int(np.asarray(want["n_steps"]).min()) > 0 and (np.asarray(want["status"]) == 0).all()
+
+
 def test_batches_around_one_wave(vp, oracle_lib):
     """Batch sizes just below and above the number of resident CTAs: the kernel changes, the plans do not."""
     c = build_config(2)
