@@ -396,7 +396,8 @@ struct Ctx {
 struct Counters { unsigned long long tasks, sweeps; long long cyc[6], t_mark; };
 
 #ifdef VP_PHASE_TIMING
-#define VP_TICK(i) do { long long now_ = clock64(); cnt.cyc[i] += now_ - cnt.t_mark; cnt.t_mark = now_; } while (0)
+// (the "memory" clobber keeps loads and stores on their side of the clock read)
+#define VP_TICK(i) do { long long now_; asm volatile("mov.u64 %0, %%clock64;" : "=l"(now_) :: "memory"); cnt.cyc[i] += now_ - cnt.t_mark; cnt.t_mark = now_; } while (0)
 #else
 #define VP_TICK(i) do { } while (0)
 #endif

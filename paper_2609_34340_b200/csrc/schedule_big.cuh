@@ -118,6 +118,10 @@ __device__ __forceinline__ void big_fill_bytes(unsigned char* dst, size_t lo, si
     for (size_t e = vlo + nvec * 16 + tid; e < hi; e += NT) dst[e] = byte;
 }
 
+// (out of line: 64-bit division is long, and granules are powers of two in practice)
+__device__ __noinline__ bool big_not_multiple(int64_t x, int64_t granule) { return x % granule != 0; }
+__device__ __noinline__ uint32_t big_div_granule(int64_t x, int64_t granule) { return (uint32_t)(x / granule); }
+
 // Step 3 when several families compete (kept out of line: most shapes have one family, and the main loop should
 // stay small for the instruction cache): best start per family (largest F, lowest start), then the family of largest
 // utility F / duration by exact cross-multiplication, lowest family first among equals.  Whole warp.
@@ -318,34 +322,44 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
         for (int e = tid; e < G * G; e += NT) Dhat[e] = 0;
         __syncthreads();
         int flags = 0;
-        // (kept as small rolled loops: this code runs once per matrix and must not crowd the instruction cache)
-        for (int a = warp; a < G; a += n_warps) {            // one warp per source group: four rows, eight columns per lane
+        // One warp per source group.  A row is read 32 columns per load instruction, its loads (up to eight) all in
+        // flight at once; row sums need one warp reduction per row, column figures are carried over the group's four rows.
+        const int64_t gmask = (kp.granule & (kp.granule - 1)) == 0 ? kp.granule - 1 : -1;     // power-of-two granule
+        for (int a = warp; a < G; a += n_warps) {
+            int64_t colv[8], colm[8];
+#pragma unroll
+            for (int m = 0; m < 8; m++) { colv[m] = 0; colm[m] = 0; }
 #pragma unroll 1
-            for (int m = 0; m < 8; m++) {
-                const int j = lane * 8 + m;
-                int64_t colv = 0, colm = 0;
-#pragma unroll 1
-                for (int i4 = 0; i4 < 4; i4++) {
-                    const int i = a * 4 + i4;
-                    int64_t v = 0;
-                    if (j < N) {
-                        v = D[(size_t)i * N + j];
-                        if (v < 0) flags |= VP_ST_NEGATIVE;
-                        else if (v >= VP_ENTRY_LIMIT) flags |= VP_ST_OVERFLOW_RISK;
-                        else {
-                            if (i == j && v != 0) flags |= VP_ST_DIAG_NONZERO;
-                            if (v % kp.granule) flags |= VP_ST_NOT_GRANULE;
-                        }
+            for (int i4 = 0; i4 < 4; i4++) {
+                const int i = a * 4 + i4;
+                const int64_t* row = D + (size_t)i * N;
+                int64_t v[8];
+#pragma unroll
+                for (int m = 0; m < 8; m++) v[m] = m * 32 + lane < N ? row[m * 32 + lane] : 0;
+                int64_t rsum = 0;
+#pragma unroll
+                for (int m = 0; m < 8; m++) {
+                    const int64_t x = v[m];
+                    if (x < 0) flags |= VP_ST_NEGATIVE;
+                    else if (x >= VP_ENTRY_LIMIT) flags |= VP_ST_OVERFLOW_RISK;
+                    else {
+                        if (m * 32 + lane == i && x != 0) flags |= VP_ST_DIAG_NONZERO;
+                        if (gmask >= 0 ? (x & gmask) != 0 : big_not_multiple(x, kp.granule)) flags |= VP_ST_NOT_GRANULE;
                     }
-                    colv += v;
-                    colm = max_v(colm, v);
-                    const int64_t rs1 = warp_sum_i64(v);
-                    if (lane == 0) rowsum[i] += rs1;         // (rows of this group belong to this warp alone)
+                    rsum += x;
+                    colv[m] += x;
+                    colm[m] = max_v(colm[m], x);
                 }
+                rsum = warp_sum_i64(rsum);
+                if (lane == 0) rowsum[i] = rsum;             // (rows of this group belong to this warp alone)
+            }
+#pragma unroll
+            for (int m = 0; m < 8; m++) {
+                const int j = m * 32 + lane;
                 if (j < N) {
-                    atomicAdd((unsigned long long*)&colsum[j], (unsigned long long)colv);
-                    atomicMax((long long*)&colmax[j], (long long)colm);
-                    atomicAdd((unsigned long long*)&Dhat[a * G + (j >> 2)], (unsigned long long)colv);
+                    atomicAdd((unsigned long long*)&colsum[j], (unsigned long long)colv[m]);
+                    atomicMax((long long*)&colmax[j], (long long)colm[m]);
+                    atomicAdd((unsigned long long*)&Dhat[a * G + (j >> 2)], (unsigned long long)colv[m]);
                 }
             }
         }
@@ -432,8 +446,17 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
             // ---- pass 2 over D: the residual in granules as 16-bit cells (big cells through the side list)
             const bool hot_mode = s_mode == 2;
             if (DEC && tid < 2 * dec_n) red[tid] = 0;        // the units' best keys (see step A)
-            for (int e = tid; e < N * N; e += NT) {
-                const uint32_t v = (uint32_t)(D[e] / kp.granule);
+            const int gshift = gmask >= 0 ? 63 - __clzll(kp.granule) : -1;
+#pragma unroll 1
+            for (int e0 = tid; e0 < N * N; e0 += 4 * NT) {       // four loads in flight per thread
+                int64_t raw[4];
+#pragma unroll
+                for (int u = 0; u < 4; u++) raw[u] = e0 + u * NT < N * N ? D[e0 + u * NT] : 0;
+#pragma unroll 1
+                for (int u = 0; u < 4; u++) {
+                const int e = e0 + u * NT;
+                if (e >= N * N) break;
+                const uint32_t v = gshift >= 0 ? (uint32_t)(raw[u] >> gshift) : big_div_granule(raw[u], kp.granule);
                 const int i = e / N, j = e - i * N;
                 if (!hot_mode) {
                     uint32_t code = v;
@@ -446,6 +469,7 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
                 } else {                                     // exact: 32 bits in a hot column, below 65,535 elsewhere
                     Cs[i * CS + j] = (uint16_t)v;
                     if (colmap[j] != 0xFF) Hi[(int)colmap[j] * N + i] = (uint16_t)(v >> 16);
+                }
                 }
             }
             __syncthreads();

@@ -464,6 +464,33 @@ def test_big_cells_beside_16_bit_credits(vp, oracle_lib, nodes):
             assert int(np.asarray(want["n_steps"]).min()) > 0 and (np.asarray(want["status"]) == 0).all()
 
 
+@pytest.mark.parametrize("granule", [256, 768])
+def test_status_codes_on_large_catalogs(vp, oracle_lib, granule):
+    """Invalid entries in matrices that take the kernel for large node-symmetric catalogs, with a power-of-two granule
+    and with another one: the same status words as the oracle, in any combination, and untouched neighbours."""
+    cat = node_template_catalog(tree_topology(9, pcie_bw=64, nic_bw=50))
+    N = cat.topology.N
+    rng = np.random.default_rng(granule)
+    D = (rng.integers(0, 500, size=(9, N, N)) * (rng.random((9, N, N)) < 0.4)).astype(np.int64) * granule
+    for b in range(9):
+        np.fill_diagonal(D[b], 0)
+    D[1, 5, 5] = granule                       # diagonal
+    D[2, 70, 3] = -granule                     # negative
+    D[3, 33, 64] += 1                          # not a granule multiple
+    D[4, 71, 0] = 1 << 40                      # overflow risk
+    D[5, 0, 0] = -1; D[5, 40, 41] = 3; D[5, 8, 9] = (1 << 40) + 5; D[5, 7, 7] = granule
+    D[6, 2, 2] = (1 << 40) + 1                 # on the diagonal and over the limit: only the limit is reported
+    D[7, 3, 3] = -3                            # negative on the diagonal: only "negative"
+    w = WParams(granule_bytes=granule, k_max=12 * N).resolved(N)
+    got, want, _, dc = _both(vp, oracle_lib, cat, D, w)
+    _assert_same(got, want)
+    p = _params(vp, w)
+    assert vp.schedule_launch_info(dc, 9, p)["kernel"] == "CTA per matrix, 16-bit credits"
+    assert got["status"].tolist() == [0, vp.ST_DIAG_NONZERO, vp.ST_NEGATIVE, vp.ST_NOT_GRANULE, vp.ST_OVERFLOW_RISK,
+                                      vp.ST_NEGATIVE | vp.ST_NOT_GRANULE | vp.ST_OVERFLOW_RISK | vp.ST_DIAG_NONZERO,
+                                      vp.ST_OVERFLOW_RISK, vp.ST_NEGATIVE, 0]
+
+
 def test_batches_around_one_wave(vp, oracle_lib):
     """Batch sizes just below and above the number of resident CTAs: the kernel changes, the plans do not."""
     c = build_config(2)
