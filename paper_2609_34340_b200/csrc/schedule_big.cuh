@@ -33,10 +33,15 @@ namespace {
 // Scoring reads the row scores at data-dependent positions; with one copy per lane class (lane mod 8) the lanes of a
 // warp meet in a bank only when they share a class and read different patterns of equal parity.
 constexpr int BIG_RS_COPIES = 1;
+#ifndef BIG_FILL_LANES
+#define BIG_FILL_LANES 8              // bulk copies of the fill issued per iteration of the main loop (32 measured 2 % slower)
+#endif
 constexpr int BIG_HOT_MAX = 32;       // columns whose cells are kept beyond 16 bits
+constexpr int BIG_SMEM_LIMIT = 227 * 1024 - 2048;   // dynamic shared memory of one CTA, less room for the static variables
 
 struct BigSmem {
     int cs, tbl, rs, pat, bnd, dec, hi, colmap, gnode, send_acc, recv_acc, red, pair, task_f, task_den, slotw, bind_src, bind_dst, term, bucket, total;
+    int fill, fill_rows;      // source buffers of the asynchronous fill, offset rows per buffer (0: plain stores)
     int cs_stride;            // credits per row of the 16-bit matrix (N + 2: rows start in different banks)
     int pat_words;            // 32-bit words of row-pattern ids per shape (two ids per word)
 };
@@ -72,6 +77,15 @@ __host__ __device__ inline BigSmem big_smem_layout(const DevCat& dc, const KPara
     L.pat_words = (dc.S + 1) / 2;
     L.term = o;      o += dec ? 0 : ((dc.n_shapes + 31) & ~31) * L.pat_words * 4;
     L.bucket = o;    o += align16((dc.n_shapes + 1) * 4);
+    // Source buffers of the asynchronous fill: all ones, zeros (written once per CTA), the send totals and the receive
+    // totals repeated fill_rows times (per matrix); the idle rows of a plan are written from them by bulk asynchronous
+    // copies while the next matrix is decomposed.  Only for the one-CTA-per-SM shape (more than 32 groups), in
+    // whatever shared memory is left, and not below 4 KB per buffer.
+    L.fill = o;
+    L.fill_rows = dc.G > 32 ? (BIG_SMEM_LIMIT - o) / 4 / (dc.N * 8) : 0;
+    if (L.fill_rows > 8) L.fill_rows = 8;
+    if (L.fill_rows * dc.N * 8 < 4096) L.fill_rows = 0;
+    o += 4 * L.fill_rows * dc.N * 8;
     L.total = o;
     return L;
 }
@@ -248,6 +262,11 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
     __shared__ int64_t s_tscale[VP_MAX_CLASSES];
     __shared__ uint32_t s_cap[VP_MAX_CLASSES];
     __shared__ __align__(8) unsigned long long s_stage_bar;
+    // Pending fill: the idle rows of the last finished matrix.  Arrays 0 and 1 (lane_dst, lane_inst) take 4 fill_rows rows
+    // per bulk copy, arrays 2 to 4 (lane_bytes, send_off, recv_off) fill_rows rows; copies are numbered array by array.
+    __shared__ unsigned char* s_job_ptr[5];
+    __shared__ int s_job_rows, s_job_next, s_job_total;
+    constexpr int FILL_WARP = 8;                         // issues the copies, a batch per iteration of the main loop
     unsigned long long n_act = 0, n_tasks_done = 0, n_sweeps = 0;
     Counters cnt;                                        // phase cycle counts (only with VP_PHASE_TIMING)
     cnt.t_mark = 0;
@@ -280,6 +299,10 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
             for (int e = tid; e < dc.n_patterns * dc.max_row_terms; e += NT) pat[e] = dc.pat_term[e];
         }
         for (int a = tid; a < G; a += NT) { gnode[a] = (uint8_t)(a / S); gnode[G + a] = (uint8_t)(a % S); }
+        for (int e = tid; e < L.fill_rows * N * 8 / 16; e += NT) {       // fill buffers: all ones, then zeros
+            ((uint4*)(smem_raw + L.fill))[e] = make_uint4(0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu);
+            ((uint4*)(smem_raw + L.fill + L.fill_rows * N * 8))[e] = make_uint4(0u, 0u, 0u, 0u);
+        }
         for (int e = tid; e < dc.dec_words && DEC; e += NT) ((uint32_t*)(smem_raw + L.dec))[e] = dc.dec[e];
         __syncthreads();
         // pattern ids become byte offsets into the row scores (fewer than 1,024 patterns, so they still fit 16 bits)
@@ -290,6 +313,28 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
         __syncthreads();
     }
     const int ns_shift = (kp.n_start & (kp.n_start - 1)) == 0 ? 31 - __clz(kp.n_start) : -1;
+    // Issues up to `batches` x 32 of the pending copies (one per lane) and commits them; FILL_WARP only.
+    auto fill_step = [&](int batches) {
+        const int R = L.fill_rows, rows = s_job_rows, total = s_job_total;
+        const int na = (rows + 4 * R - 1) / (4 * R), nb = (rows + R - 1) / R;
+        const unsigned chunk = (unsigned)(R * N * 8), buf = smem_u32(smem_raw + L.fill);
+        int next = s_job_next;
+        for (int bt = 0; bt < batches && next < total; bt++, next += BIG_FILL_LANES) {
+            const int op = next + lane;
+            if (lane < BIG_FILL_LANES && op < total) {
+                int arr, r0, cnt, width;
+                if (op < 2 * na) { arr = op >= na; r0 = (op - arr * na) * 4 * R; cnt = min(4 * R, rows - r0); width = 2; }
+                else { const int o2 = op - 2 * na; arr = 2 + o2 / nb; r0 = (o2 - (arr - 2) * nb) * R; cnt = min(R, rows - r0); width = 8; }
+                unsigned char* base = s_job_ptr[arr];
+                if (base) bulk_store(base + (size_t)r0 * N * width, buf + (arr < 2 ? 0u : (unsigned)(arr - 1) * chunk), (unsigned)(cnt * N * width));
+            }
+            bulk_commit();
+        }
+        __syncwarp();
+        if (lane == 0) s_job_next = next;
+        __syncwarp();
+    };
+    if (tid == 0) { s_job_next = 0; s_job_total = 0; s_job_rows = 0; }
 
     for (;;) {
         if (tid == 0) {
@@ -577,6 +622,8 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
                 const int n_tasks = H * kp.n_start;
                 VP_TICK(1);
 
+                if (W == 2 && warp == FILL_WARP && s_job_next < s_job_total) fill_step(1);   // (this warp has no task as a rule)
+
                 // (B) MultiStartAA: W warps per (family, start), one lane per rank group
                 const int sub = W == 2 ? (warp & 1) : 0, wgroup = W == 2 ? (warp >> 1) : warp;
                 const int a = sub * 32 + lane;                   // this lane's group: source group, then destination group
@@ -830,14 +877,42 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
             }
         }
         __syncthreads();
-        // ---- idle rows beyond n_steps (16-byte stores); offset rows repeat the totals
-        {
+        // ---- idle rows beyond n_steps; offset rows repeat the totals
+        const bool off_aligned = (((uintptr_t)send_off_b | (uintptr_t)(recv_off_b ? recv_off_b : send_off_b)) & 15) == 0;
+        const bool lane_aligned = (((uintptr_t)lane_dst_b | (uintptr_t)lane_inst_b | (uintptr_t)lane_bytes_b) & 15) == 0 && N % 8 == 0;
+        if (W == 2 && L.fill_rows > 0 && off_aligned && lane_aligned) {
+            // Bulk asynchronous copies out of the fill buffers, issued a batch at a time while the next matrices are
+            // decomposed.  First the copies still pending from the last matrix: they read the totals that change now.
+            if (warp == FILL_WARP) {
+                fill_step(0x7fffffff);
+                bulk_wait_read<0>();
+            }
+            __syncthreads();
+            const unsigned chunk = (unsigned)(L.fill_rows * N * 8);
+            unsigned char* buf = smem_raw + L.fill;
+            for (unsigned e = tid; e < chunk / 16; e += NT) {
+                const int i2 = (int)(e % (unsigned)(N / 2));
+                ((longlong2*)(buf + 2 * chunk))[e] = ((const longlong2*)send_acc)[i2];
+                ((longlong2*)(buf + 3 * chunk))[e] = ((const longlong2*)recv_acc)[i2];
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            if (tid == 0) {
+                const int rows = kp.k_max - k, R = L.fill_rows;
+                s_job_ptr[0] = (unsigned char*)(lane_dst_b + (size_t)k * N);
+                s_job_ptr[1] = (unsigned char*)(lane_inst_b + (size_t)k * N);
+                s_job_ptr[2] = (unsigned char*)(lane_bytes_b + (size_t)k * N);
+                s_job_ptr[3] = (unsigned char*)(send_off_b + (size_t)(k + 1) * N);
+                s_job_ptr[4] = recv_off_b ? (unsigned char*)(recv_off_b + (size_t)(k + 1) * N) : nullptr;
+                s_job_rows = rows;
+                s_job_next = 0;
+                s_job_total = 2 * ((rows + 4 * R - 1) / (4 * R)) + 3 * ((rows + R - 1) / R);
+            }
+        } else {
             const size_t lo = (size_t)k * N, hi = (size_t)kp.k_max * N;
             big_fill_bytes((unsigned char*)lane_dst_b, lo * 2, hi * 2, 0xff, tid, NT);
             big_fill_bytes((unsigned char*)lane_inst_b, lo * 2, hi * 2, 0xff, tid, NT);
             big_fill_bytes((unsigned char*)lane_bytes_b, lo * 8, hi * 8, 0x00, tid, NT);
-            const bool vec = (((uintptr_t)send_off_b | (uintptr_t)(recv_off_b ? recv_off_b : send_off_b)) & 15) == 0;
-            if (vec) {                                       // N is a multiple of four: rows are whole 16-byte pairs
+            if (off_aligned) {                               // N is a multiple of four: rows are whole 16-byte pairs
                 const int half = N / 2;
                 for (size_t e = lo / 2 + tid; e < hi / 2; e += NT) {
                     const int i2 = (int)(e % half);
@@ -861,6 +936,10 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
         }
         __syncthreads();
         VP_TICK(5);
+    }
+    if (W == 2 && warp == FILL_WARP) {                   // what is left of the last fill
+        fill_step(0x7fffffff);
+        bulk_wait_all();
     }
     unsigned long long* stats = (unsigned long long*)(counter + 4);
     if (tid == 0 && n_act) atomicAdd(&stats[0], n_act);
