@@ -41,7 +41,7 @@ constexpr int BIG_SMEM_LIMIT = 227 * 1024 - 2048;   // dynamic shared memory of 
 
 struct BigSmem {
     int cs, tbl, rs, pat, bnd, dec, hi, colmap, gnode, send_acc, recv_acc, red, pair, task_f, task_den, slotw, bind_src, bind_dst, term, bucket, total;
-    int fill, fill_rows;      // source buffers of the asynchronous fill, offset rows per buffer (0: plain stores)
+    int emit, fill, fill_rows;      // source buffers of the asynchronous fill, offset rows per buffer (0: plain stores)
     int cs_stride;            // credits per row of the 16-bit matrix (N + 2: rows start in different banks)
     int pat_words;            // 32-bit words of row-pattern ids per shape (two ids per word)
 };
@@ -77,6 +77,8 @@ __host__ __device__ inline BigSmem big_smem_layout(const DevCat& dc, const KPara
     L.pat_words = (dc.S + 1) / 2;
     L.term = o;      o += dec ? 0 : ((dc.n_shapes + 31) & ~31) * L.pat_words * 4;
     L.bucket = o;    o += align16((dc.n_shapes + 1) * 4);
+    // Staging row of the emit step (lane_dst, lane_inst, lane_bytes, send_off, recv_off of one activation: 28 N bytes)
+    L.emit = o;      o += dc.N % 8 == 0 ? 28 * dc.N : 0;
     // Source buffers of the asynchronous fill: all ones, zeros (written once per CTA), the send totals and the receive
     // totals repeated fill_rows times (per matrix); the idle rows of a plan are written from them by bulk asynchronous
     // copies while the next matrix is decomposed.  Only for the one-CTA-per-SM shape (more than 32 groups), in
@@ -530,6 +532,27 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
             uint32_t c_co = 0;
             uint2 c_fi = make_uint2(0u, 0u);
             VP_TICK(0);
+            // Emit rows through shared memory: the five rows of an activation are staged there, and the upper half of the
+            // warps, which has no task in Step 2 as a rule, copies them out during Step 2 of the next iteration.  (Plain
+            // stores to global memory by the emitting warps, just before a CTA-wide barrier, made every iteration wait
+            // for them: 6 % of the run time.)
+            const bool rows_async = N % 8 == 0 && kp.n_start * W <= (n_warps >> 1) &&
+                (((uintptr_t)lane_dst_b | (uintptr_t)lane_inst_b | (uintptr_t)lane_bytes_b | (uintptr_t)send_off_b |
+                  (uintptr_t)(recv_off_b ? recv_off_b : send_off_b)) & 15) == 0;
+            int copied = 0;                                  // activations copied out (upper warps)
+            auto copy_row = [&](int kk) {
+                const unsigned char* sb = smem_raw + L.emit;
+                for (int e = tid - (NT >> 1); e < 28 * N / 16; e += NT >> 1) {
+                    const int at = e * 16;
+                    unsigned char* dst;
+                    if (at < 4 * N) dst = at < 2 * N ? (unsigned char*)(lane_dst_b + (size_t)kk * N) + at
+                                                     : (unsigned char*)(lane_inst_b + (size_t)kk * N) + (at - 2 * N);
+                    else if (at < 12 * N) dst = (unsigned char*)(lane_bytes_b + (size_t)kk * N) + (at - 4 * N);
+                    else if (at < 20 * N) dst = (unsigned char*)(send_off_b + (size_t)(kk + 1) * N) + (at - 12 * N);
+                    else dst = recv_off_b ? (unsigned char*)(recv_off_b + (size_t)(kk + 1) * N) + (at - 20 * N) : nullptr;
+                    if (dst) *(uint4*)dst = *(const uint4*)(sb + at);
+                }
+            };
 
             for (;;) {
                 if (left == 0) break;
@@ -623,6 +646,7 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
                 VP_TICK(1);
 
                 if (W == 2 && warp == FILL_WARP && s_job_next < s_job_total) fill_step(1);   // (this warp has no task as a rule)
+                if (rows_async && warp >= (n_warps >> 1) && copied < k) copy_row(copied++);  // the last activation's rows
 
                 // (B) MultiStartAA: W warps per (family, start), one lane per rank group
                 const int sub = W == 2 ? (warp & 1) : 0, wgroup = W == 2 ? (warp >> 1) : warp;
@@ -841,13 +865,23 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
                             const bool busy = x > 0;
                             const int64_t bytes = (int64_t)x * kp.granule;
                             const int64_t sa = send_acc[i] + bytes, ra = recv_acc[j] + bytes;
-                            lane_dst_b[row + i] = busy ? (int16_t)j : (int16_t)-1;
-                            lane_inst_b[row + i] = busy ? (uint16_t)(w & 0xffffu) : (uint16_t)0xFFFF;
-                            lane_bytes_b[row + i] = bytes;
                             send_acc[i] = sa;
                             recv_acc[j] = ra;
-                            send_off_b[orow + i] = sa;            // src and dst are permutations: every rank is written once
-                            if (recv_off_b) recv_off_b[orow + j] = ra;
+                            // (src and dst are permutations: every rank of every row is written once)
+                            if (rows_async) {
+                                unsigned char* sb = smem_raw + L.emit;
+                                ((int16_t*)sb)[i] = busy ? (int16_t)j : (int16_t)-1;
+                                ((uint16_t*)(sb + 2 * N))[i] = busy ? (uint16_t)(w & 0xffffu) : (uint16_t)0xFFFF;
+                                ((int64_t*)(sb + 4 * N))[i] = bytes;
+                                ((int64_t*)(sb + 12 * N))[i] = sa;
+                                ((int64_t*)(sb + 20 * N))[j] = ra;
+                            } else {
+                                lane_dst_b[row + i] = busy ? (int16_t)j : (int16_t)-1;
+                                lane_inst_b[row + i] = busy ? (uint16_t)(w & 0xffffu) : (uint16_t)0xFFFF;
+                                lane_bytes_b[row + i] = bytes;
+                                send_off_b[orow + i] = sa;
+                                if (recv_off_b) recv_off_b[orow + j] = ra;
+                            }
                             if (busy) {
                                 if (hcell) {
                                     *cell = (uint16_t)(c - x);
@@ -875,6 +909,7 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
                 __syncthreads();
                 VP_TICK(4);
             }
+            if (rows_async && warp >= (n_warps >> 1) && copied < k) copy_row(copied++);   // the last activation of the matrix
         }
         __syncthreads();
         // ---- idle rows beyond n_steps; offset rows repeat the totals
@@ -937,10 +972,8 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
         __syncthreads();
         VP_TICK(5);
     }
-    if (W == 2 && warp == FILL_WARP) {                   // what is left of the last fill
-        fill_step(0x7fffffff);
-        bulk_wait_all();
-    }
+    if (W == 2 && warp == FILL_WARP) fill_step(0x7fffffff);     // what is left of the last fill
+    bulk_wait_all();
     unsigned long long* stats = (unsigned long long*)(counter + 4);
     if (tid == 0 && n_act) atomicAdd(&stats[0], n_act);
     if (lane == 0 && n_tasks_done) { atomicAdd(&stats[1], n_tasks_done); atomicAdd(&stats[2], n_sweeps); }
