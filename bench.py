@@ -287,7 +287,7 @@ def issue_fraction(counters: dict, key: str, activations: int, ms: float, sm_mhz
     wave = c["shared_wavefronts_per_activation"] * activations
     return {"issue_slot_frac": round(inst / (cycles * SM_COUNT * SCHEDULERS_PER_SM), 4),
             "shared_wavefront_frac": round(wave / (cycles * SM_COUNT), 4),
-            "counters_from": f"profiles/ncu_counters.json ({c.get('source', '?')}, commit {counters.get('commit', '?')})",
+            "counters_from": f"profiles/ncu_counters.json ({c.get('source', '?')}, commit {c.get('commit', counters.get('commit', '?'))})",
             "ncu_issue_active_pct": c.get("issue_active_pct"), "ncu_shared_wavefront_pct": c.get("shared_wavefront_pct")}
 
 
