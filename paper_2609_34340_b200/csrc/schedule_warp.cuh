@@ -4,11 +4,10 @@
 // iteration is spent in block barriers and in hand-overs through shared memory.  Here a warp owns a matrix from
 // the first to the last activation and nothing but __syncwarp orders its phases:
 //  (A) each lane scores every 32nd shape (Eq. 6); a butterfly of shuffles leaves the first maximum in all lanes;
-//  (B) the (family, start) tasks of the bucket run four at a time IN THE SAME WARP as independent instruction
-//      streams: the lanes keep their role (a team of eight lanes per rank group, three permutations per lane) and
-//      issue every step of the Alternating Algorithm (Eq. 7, 8) for the four tasks back to back, so the four
-//      dependent chains overlap; a task that stops improving is frozen (its stores are predicated off) while
-//      the others finish; Evaluate (Eq. 9, 10) and the best start / best family follow in registers;
+//  (B) the (family, start) tasks of the bucket run eight at a time: a team of four lanes per task, one lane per rank
+//      group, and every lane solves its group's exact 4 x 4 assignments (Eq. 7) by itself; the two halves of a sweep
+//      exchange nothing but the bindings; a task that stops improving (Eq. 8) is frozen while the others finish;
+//      Evaluate (Eq. 9, 10) runs when several families compete; best start / best family follow in registers;
 //  (D) sixteen lanes emit the activation and subtract it; D-hat is then re-summed from D_rem by all lanes
 //      (two lanes per cell), which needs no atomics.
 // A CTA is one to four such warps that share only the staged catalog.  Included by schedule.cu.
@@ -16,7 +15,6 @@
 
 namespace {
 
-constexpr int kWT = 4;                      // tasks in flight per warp
 
 struct WarpSmem {                           // byte offsets; the per-warp block comes first, once per warp
     int drem, dhat, send_acc, recv_acc, cred, cap64, tscale, cap32, bind_src, bind_dst, per_warp;
@@ -30,7 +28,7 @@ __host__ __device__ inline WarpSmem warp_smem_layout(const DevCat& dc, const KPa
     L.dhat = o;      o += align16(dc.G * dc.G * 8);
     L.send_acc = o;  o += dc.N * 8;
     L.recv_acc = o;  o += dc.N * 8;
-    L.cred = o;      o += kWT * 4 * 17 * 8;
+    L.cred = o;
     L.cap64 = o;     o += VP_MAX_CLASSES * 8;
     L.tscale = o;    o += VP_MAX_CLASSES * 8;
     L.cap32 = o;     o += VP_MAX_CLASSES * 4;
@@ -65,78 +63,18 @@ struct WCtx {
 
 template <typename T> __device__ __forceinline__ T* ws(unsigned off) { return (T*)(vp_wsmem + off); }
 
-// team_best for kWT credit tiles at once, written level by level so that the shuffles of the four tasks are
-// issued back to back (shuffles are not reordered by the compiler).
-__device__ __forceinline__ void team_best_x(const unsigned (&tile)[kWT], int tl, const uint8_t (&pidx)[3][4], unsigned o_lut,
-                                            unsigned (&bpk)[kWT], uint32_t (&val)[kWT]) {
-    const Reg8Lane L = reg8_lane(tl);
-    uint32_t key[kWT];
-#pragma unroll
-    for (int t = 0; t < kWT; t++) key[t] = reg8_key(ws<uint32_t>(tile[t]), L);
-#pragma unroll
-    for (int o = 4; o; o >>= 1) {
-        uint32_t other[kWT];
-#pragma unroll
-        for (int t = 0; t < kWT; t++) other[t] = __shfl_xor_sync(0xffffffffu, key[t], o);
-#pragma unroll
-        for (int t = 0; t < kWT; t++) key[t] = max_v(key[t], other[t]);
-    }
-#pragma unroll
-    for (int t = 0; t < kWT; t++) { bpk[t] = ~key[t] & 255u; val[t] = key[t] >> 8; }      // the permutation byte, the sum
+// Sum over the four lanes of a team (lane & ~3 .. lane | 3); every lane gets it.
+__device__ __forceinline__ uint32_t team_sum(uint32_t v) {
+    v += __shfl_xor_sync(0xffffffffu, v, 1);
+    return v + __shfl_xor_sync(0xffffffffu, v, 2);
 }
-__device__ __forceinline__ void team_best_x(const unsigned (&tile)[kWT], int tl, const uint8_t (&pidx)[3][4], unsigned o_lut,
-                                            unsigned (&bpk)[kWT], int64_t (&val)[kWT]) {
-    int bp[kWT];
-#pragma unroll
-    for (int t = 0; t < kWT; t++) {
-        const int64_t* cred = ws<int64_t>(tile[t]);
-        val[t] = -1; bp[t] = 0;
-#pragma unroll
-        for (int pp = 0; pp < 3; pp++) {
-            const int64_t v = cred[pidx[pp][0]] + cred[pidx[pp][1]] + cred[pidx[pp][2]] + cred[pidx[pp][3]];
-            if (v > val[t]) { val[t] = v; bp[t] = tl * 3 + pp; }
-        }
-    }
-#pragma unroll
-    for (int o = 4; o; o >>= 1) {
-        int64_t ov[kWT];
-        int op[kWT];
-#pragma unroll
-        for (int t = 0; t < kWT; t++) { ov[t] = __shfl_xor_sync(0xffffffffu, val[t], o); op[t] = __shfl_xor_sync(0xffffffffu, bp[t], o); }
-#pragma unroll
-        for (int t = 0; t < kWT; t++)
-            if (ov[t] > val[t] || (ov[t] == val[t] && op[t] < bp[t])) { val[t] = ov[t]; bp[t] = op[t]; }
-    }
-#pragma unroll
-    for (int t = 0; t < kWT; t++) bpk[t] = ws<uint8_t>(o_lut)[31 - bp[t]];
+__device__ __forceinline__ int64_t team_sum(int64_t v) {
+    v += __shfl_xor_sync(0xffffffffu, v, 1);
+    return v + __shfl_xor_sync(0xffffffffu, v, 2);
 }
-
-// Eq. (8): sum over the teams of a per-team value (held by every lane of the team); every lane gets the totals.
-__device__ __forceinline__ void team_totals(const uint32_t (&v)[kWT], bool first_lane_of_active_team, int64_t (&F)[kWT]) {
-#pragma unroll
-    for (int t = 0; t < kWT; t++) F[t] = (int64_t)__reduce_add_sync(0xffffffffu, first_lane_of_active_team ? v[t] : 0u);
-}
-__device__ __forceinline__ void team_totals(const int64_t (&v)[kWT], bool first_lane_of_active_team, int64_t (&F)[kWT]) {
-#pragma unroll
-    for (int t = 0; t < kWT; t++) F[t] = first_lane_of_active_team ? v[t] : 0;
-#pragma unroll
-    for (int o = 16; o; o >>= 1) {
-        int64_t other[kWT];
-#pragma unroll
-        for (int t = 0; t < kWT; t++) other[t] = __shfl_xor_sync(0xffffffffu, F[t], o);
-#pragma unroll
-        for (int t = 0; t < kWT; t++) F[t] += other[t];
-    }
-}
-__device__ __forceinline__ void warp_max_x(int64_t (&v)[kWT]) {
-#pragma unroll
-    for (int o = 16; o; o >>= 1) {
-        int64_t other[kWT];
-#pragma unroll
-        for (int t = 0; t < kWT; t++) other[t] = __shfl_xor_sync(0xffffffffu, v[t], o);
-#pragma unroll
-        for (int t = 0; t < kWT; t++) v[t] = max_v(v[t], other[t]);
-    }
+__device__ __forceinline__ int64_t team_max(int64_t v) {
+    v = max_v(v, __shfl_xor_sync(0xffffffffu, v, 1));
+    return max_v(v, __shfl_xor_sync(0xffffffffu, v, 2));
 }
 
 template <typename V>
@@ -145,171 +83,179 @@ __device__ __forceinline__ void decompose_warp(const DevCat& dc, const KParams& 
     const int N = c.N, G = c.G, lane = c.lane;
     const int ld = N + 1;                                // row stride of D_rem
     const int ns_pad = (dc.n_shapes + 31) & ~31;         // row stride of the transposed term table
-    const int team = lane >> 3, tl = lane & 7;
-    const bool active = team < G;
-    const int a = active ? team : G - 1;                 // the team's group (spare teams repeat the last group on their own tiles)
-    const int q = tl & 3, i0 = tl >> 2, i1 = i0 + 2;     // the lane's credit elements: (i0, q) and (i1, q)
-    const bool ns4 = kp.n_start == 4;
+    // Step 2 runs eight (family, start) tasks at a time: a team of four lanes per task, one lane per rank group, which
+    // solves its group's exact 4 x 4 assignments on its own (best_assignment) -- no credit tiles, no hand-overs
+    // between lanes except the bindings themselves.
+    const int team = lane >> 2, a = lane & 3;
+    const bool active = a < G;
+    const int ns_shift = (kp.n_start & (kp.n_start - 1)) == 0 ? 31 - __clz(kp.n_start) : -1;
     V* const Drem = ws<V>(c.o_drem);
     const V* const cap = ws<V>(c.o_cap);
     int64_t* const Dhat = ws<int64_t>(c.o_dhat);
-    uint8_t pidx[3][4];
-#pragma unroll
-    for (int pp = 0; pp < 3; pp++) {
-        const unsigned pk = perm4_packed_rt(tl * 3 + pp);
-#pragma unroll
-        for (int qq = 0; qq < 4; qq++) pidx[pp][qq] = (uint8_t)(((pk >> (2 * qq)) & 3) * 4 + qq);
-    }
-    unsigned tile[kWT];                                  // this team's credit tile of each task in flight
-#pragma unroll
-    for (int t = 0; t < kWT; t++) tile[t] = c.o_cred + (unsigned)((t * 4 + team) * 17 * sizeof(V));
+    // Plain score tables of at most 16 D-hat cells and at most 128 shapes: a lane keeps the lane counts of its (up to
+    // four) shapes in registers, four bits per cell, and scoring needs no term loads.
+    const bool dense = dc.tbl_size <= 16 && dc.n_shapes <= 128;
+    unsigned long long smask[4] = {0ull, 0ull, 0ull, 0ull};
+    if (dense)
+        for (int u = 0; u < 4; u++) {
+            const int s = lane + 32 * u;
+            if (s < dc.n_shapes)
+                for (int e = 0; e < dc.max_terms; e++) {
+                    const uint32_t w = ws<uint32_t>(c.o_term)[e * ns_pad + s];
+                    smask[u] |= (unsigned long long)(w >> 16) << (4 * ((w & 0xffffu) >> 3));
+                }
+        }
 
     for (;;) {
         if (left == 0) break;
         if (k == kp.k_max) { st |= VP_ST_STEP_LIMIT; break; }
-        // (A) Eq. (6): shape scores, four shapes per lane in flight, first maximum
+        // (A) Eq. (6): shape scores, first maximum
         int64_t best = -1;
         int best_s = 0x7fffffff;
-        for (int s0 = lane; s0 < dc.n_shapes; s0 += 128) {
-            int64_t score[4] = {0, 0, 0, 0};
-            const uint32_t* tp = ws<uint32_t>(c.o_term) + s0;     // term e of shape s is at [e][s]: lanes read neighbours
-            const int last = dc.n_shapes - 1 - s0;               // shapes beyond the catalog re-read the last one
-            int du[4];
+        if (dense) {
+            const bool narrow = left * 4 < ((int64_t)1 << 31);   // a score is at most g x (what is left)
+            if (narrow) {
+                uint32_t sc[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
-            for (int u = 0; u < 4; u++) du[u] = min(32 * u, last);
-#pragma unroll 4
-            for (int e = 0; e < dc.max_terms; e++) {
+                for (int cell = 0; cell < 16; cell++) {
+                    if (cell < dc.tbl_size) {
+                        const uint32_t d = (uint32_t)Dhat[cell];
 #pragma unroll
-                for (int u = 0; u < 4; u++) {
-                    const uint32_t w = tp[e * ns_pad + du[u]];
-                    score[u] += *(const int64_t*)((const char*)Dhat + (w & 0xffffu)) * (int64_t)(w >> 16);
+                        for (int u = 0; u < 4; u++) sc[u] += d * (uint32_t)((smask[u] >> (4 * cell)) & 15ull);
+                    }
                 }
-            }
 #pragma unroll
-            for (int u = 0; u < 4; u++)
-                if (s0 + 32 * u < dc.n_shapes && score[u] > best) { best = score[u]; best_s = s0 + 32 * u; }
+                for (int u = 0; u < 4; u++)
+                    if (lane + 32 * u < dc.n_shapes && (int64_t)sc[u] > best) { best = (int64_t)sc[u]; best_s = lane + 32 * u; }
+            } else {
+                int64_t sc[4] = {0, 0, 0, 0};
+#pragma unroll
+                for (int cell = 0; cell < 16; cell++) {
+                    if (cell < dc.tbl_size) {
+                        const int64_t d = Dhat[cell];
+#pragma unroll
+                        for (int u = 0; u < 4; u++) sc[u] += d * (int64_t)((smask[u] >> (4 * cell)) & 15ull);
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < 4; u++)
+                    if (lane + 32 * u < dc.n_shapes && sc[u] > best) { best = sc[u]; best_s = lane + 32 * u; }
+            }
+        } else {
+            for (int s0 = lane; s0 < dc.n_shapes; s0 += 128) {     // four shapes per lane in flight
+                int64_t score[4] = {0, 0, 0, 0};
+                const uint32_t* tp = ws<uint32_t>(c.o_term) + s0;  // term e of shape s is at [e][s]: lanes read neighbours
+                const int last = dc.n_shapes - 1 - s0;             // shapes beyond the catalog re-read the last one
+                int du[4];
+#pragma unroll
+                for (int u = 0; u < 4; u++) du[u] = min(32 * u, last);
+#pragma unroll 4
+                for (int e = 0; e < dc.max_terms; e++) {
+#pragma unroll
+                    for (int u = 0; u < 4; u++) {
+                        const uint32_t w = tp[e * ns_pad + du[u]];
+                        score[u] += *(const int64_t*)((const char*)Dhat + (w & 0xffffu)) * (int64_t)(w >> 16);
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < 4; u++)
+                    if (s0 + 32 * u < dc.n_shapes && score[u] > best) { best = score[u]; best_s = s0 + 32 * u; }
+            }
         }
         warp_argmax_first(best, best_s);
         if (best <= 0) { st |= VP_ST_UNCOVERED; break; }
         const int f0 = (int)ws<uint32_t>(c.o_bucket)[best_s], H = (int)ws<uint32_t>(c.o_bucket)[best_s + 1] - f0;
         const int n_tasks = H * kp.n_start;
 
-        // (B) MultiStartAA, four (family, start) tasks at a time; (C) best start per family, best family
+        // (B) MultiStartAA, eight (family, start) tasks at a time; (C) best start per family, best family
         int64_t bf = -1, bd = 1, ff = -1, fd = 1;        // best family so far; best start of the current family
         int bt = -1, ft = -1, cur_h = -1;
-        for (int task0 = 0; task0 < n_tasks; task0 += kWT) {
-            unsigned alive = 0;
-            V cap_out[kWT], cap_in[kWT];
-            int cls_in[kWT];
-            unsigned o_src[kWT], o_dst[kWT], o_rin_s[kWT], o_rin_d[kWT];
-            // initial destination binding: start t rotates the in-slots of every group by t
-            for (int e = lane; e < kWT * 16; e += 32) {
-                const int t = e >> 4, d = (e >> 2) & 3, qq = e & 3, task = task0 + t;
-                if (task < n_tasks && d < G) {
-                    const int h = ns4 ? task >> 2 : task / kp.n_start, tt = task - h * kp.n_start;
-                    ws<uint8_t>(c.o_bind_dst)[task * N + (ws<uint16_t>(c.o_fam_in)[(f0 + h) * N + d * 4 + qq] & 0xff)] =
-                        (uint8_t)(d * 4 + ((qq + tt) & 3));
-                }
-            }
+        for (int task0 = 0; task0 < n_tasks; task0 += 8) {
+            const int task = min(task0 + team, n_tasks - 1);
+            const bool has = task0 + team < n_tasks && active;
+            const int h = ns_shift >= 0 ? task >> ns_shift : task / kp.n_start, tt = task - h * kp.n_start, f = f0 + h;
+            uint8_t* const srcb = ws<uint8_t>(c.o_bind_src) + task * N;
+            uint8_t* const dstb = ws<uint8_t>(c.o_bind_dst) + task * N;
+            V cap_out[4], cap_in[4];
+            int rq[4], cls_in[4];
+            const int ag = active ? a : 0;                   // (spare lanes read group 0's tables and write nothing)
 #pragma unroll
-            for (int t = 0; t < kWT; t++) {
-                const int task = task0 + t < n_tasks ? task0 + t : n_tasks - 1;
-                if (task0 + t < n_tasks) alive |= 1u << t;
-                const int f = f0 + (ns4 ? task >> 2 : task / kp.n_start);
-                const unsigned w = ws<uint16_t>(c.o_fam_in)[f * N + a * 4 + q];
-                cap_out[t] = cap[ws<uint8_t>(c.o_fam_cls)[f * N + a * 4 + q]];
-                cls_in[t] = (int)(w >> 8);
-                cap_in[t] = cap[cls_in[t]];
-                o_src[t] = c.o_bind_src + (unsigned)(task * N);
-                o_dst[t] = c.o_bind_dst + (unsigned)(task * N);
-                o_rin_s[t] = o_src[t] + (w & 0xff);          // binding entries of the in-slot this lane serves
-                o_rin_d[t] = o_dst[t] + (w & 0xff);
+            for (int q = 0; q < 4; q++) {
+                const unsigned w = ws<uint16_t>(c.o_fam_in)[f * N + ag * 4 + q];
+                cap_out[q] = cap[ws<uint8_t>(c.o_fam_cls)[f * N + ag * 4 + q]];
+                rq[q] = (int)(w & 0xffu);
+                cls_in[q] = (int)(w >> 8);
+                cap_in[q] = cap[cls_in[q]];
+                if (has) dstb[rq[q]] = (uint8_t)(a * 4 + ((q + tt) & 3));     // start t rotates the in-slots of every group
             }
-            const unsigned valid = alive;
             __syncwarp();
-            int64_t F_old[kWT], F_new[kWT];
-            unsigned bpk_fin[kWT];
+            int64_t F_old = -1, F_new = -1;
+            bool alive = has;
+            for (int sweep = 0; sweep < kp.i_aa && __any_sync(0xffffffffu, alive); sweep++) {
+                if (alive) {                                  // source half: credits of group a towards its out-slots' destinations
+                    const uint32_t d4 = *(const uint32_t*)(dstb + a * 4);
+                    V cm[4][4];
 #pragma unroll
-            for (int t = 0; t < kWT; t++) { F_old[t] = -1; F_new[t] = -1; bpk_fin[t] = 0; }
-            for (int sweep = 0; sweep < kp.i_aa && alive; sweep++) {
-                V v0[kWT], v1[kWT], val[kWT];
-                unsigned bpk[kWT];
-                // source half: credits of source group a towards the current destinations of its out-slots
+                    for (int q = 0; q < 4; q++) {
+                        const V* col = Drem + (a * 4) * ld + ((d4 >> (8 * q)) & 0xffu);
 #pragma unroll
-                for (int t = 0; t < kWT; t++) {
-                    const int dq = ws<uint8_t>(o_dst[t])[a * 4 + q];
-                    v0[t] = min_v(Drem[(a * 4 + i0) * ld + dq], cap_out[t]);
-                    v1[t] = min_v(Drem[(a * 4 + i1) * ld + dq], cap_out[t]);
+                        for (int i = 0; i < 4; i++) cm[i][q] = min_v(col[i * ld], cap_out[q]);
+                    }
+                    unsigned bpk;
+                    best_assignment<4, V>(cm, bpk);
+                    *(uint32_t*)(srcb + a * 4) = (uint32_t)(a * 4) * 0x01010101u +
+                        ((bpk & 3u) | ((bpk >> 2) & 3u) << 8 | ((bpk >> 4) & 3u) << 16 | ((bpk >> 6) & 3u) << 24);
                 }
-#pragma unroll
-                for (int t = 0; t < kWT; t++)
-                    if (alive >> t & 1) { ws<V>(tile[t])[i0 * 4 + q] = v0[t]; ws<V>(tile[t])[i1 * 4 + q] = v1[t]; }
                 __syncwarp();
-                team_best_x(tile, tl, pidx, c.o_lut, bpk, val);
+                V part = 0;
+                if (alive) {                                  // destination half: credits into group a from its in-slots' sources
+                    V cm[4][4];
 #pragma unroll
-                for (int t = 0; t < kWT; t++)
-                    if (alive >> t & 1) ws<uint8_t>(o_src[t])[a * 4 + q] = (uint8_t)(a * 4 + perm_pos<V>(bpk[t], q));
-                __syncwarp();
-                // destination half: credits into destination group a from the current sources of its in-slots
+                    for (int q = 0; q < 4; q++) {
+                        const V* row = Drem + (int)srcb[rq[q]] * ld + a * 4;
 #pragma unroll
-                for (int t = 0; t < kWT; t++) {
-                    const int sq = *ws<uint8_t>(o_rin_s[t]);
-                    v0[t] = min_v(Drem[sq * ld + a * 4 + i0], cap_in[t]);
-                    v1[t] = min_v(Drem[sq * ld + a * 4 + i1], cap_in[t]);
+                        for (int i = 0; i < 4; i++) cm[i][q] = min_v(row[i], cap_in[q]);
+                    }
+                    unsigned bpk;
+                    part = best_assignment<4, V>(cm, bpk);
+#pragma unroll
+                    for (int q = 0; q < 4; q++) dstb[rq[q]] = (uint8_t)(a * 4 + ((bpk >> (2 * q)) & 3u));
                 }
-#pragma unroll
-                for (int t = 0; t < kWT; t++)
-                    if (alive >> t & 1) { ws<V>(tile[t])[i0 * 4 + q] = v0[t]; ws<V>(tile[t])[i1 * 4 + q] = v1[t]; }
+                const int64_t Fn = (int64_t)team_sum(part);   // Eq. (8)
+                if (alive) {
+                    F_new = Fn;
+                    if (a == 0) cnt.sweeps++;
+                    if (Fn <= F_old) alive = false;           // the run ends; its bindings stay as this sweep left them
+                    else F_old = Fn;
+                }
                 __syncwarp();
-                team_best_x(tile, tl, pidx, c.o_lut, bpk, val);
+            }
+            // Evaluate (Eq. 9, 10), needed only when several families compete: the volume of every in-slot of this
+            // lane's group under the final bindings, the slowest lane over the team
+            int64_t den = 1;
+            if (H > 1) {
+                int64_t tmax = 0;
+                if (has) {
 #pragma unroll
-                for (int t = 0; t < kWT; t++)
-                    if (alive >> t & 1) *ws<uint8_t>(o_rin_d[t]) = (uint8_t)(a * 4 + perm_pos<V>(bpk[t], q));
-                int64_t Fn[kWT];
-                team_totals(val, active && tl == 0, Fn);                                  // Eq. (8)
-#pragma unroll
-                for (int t = 0; t < kWT; t++) {
-                    if (alive >> t & 1) {
-                        F_new[t] = Fn[t];
-                        bpk_fin[t] = bpk[t];
-                        cnt.sweeps++;
-                        if (Fn[t] <= F_old[t]) alive &= ~(1u << t);       // frozen: bindings and credits stay
-                        else F_old[t] = Fn[t];
+                    for (int q = 0; q < 4; q++) {
+                        const V x = min_v(Drem[(int)srcb[rq[q]] * ld + (int)dstb[rq[q]]], cap_in[q]);
+                        tmax = max_v(tmax, (int64_t)x * ws<int64_t>(c.o_tscale)[cls_in[q]]);
                     }
                 }
-                __syncwarp();
+                tmax = team_max(tmax);
+                den = F_new > 0 ? kp.lambda_ns * dc.W + tmax : 1;
             }
-            // Evaluate: Eq. (9) volumes are the chosen credits of the task's last destination half; Eq. (10)
-            int64_t den[kWT];
-            {
-                V x[kWT];
-#pragma unroll
-                for (int t = 0; t < kWT; t++) {
-                    x[t] = 0;
-                    if (valid >> t & 1) x[t] = ws<V>(tile[t])[perm_pos<V>(bpk_fin[t], q) * 4 + q];
-                }
-                if (sizeof(V) == 4 && dc.n_classes == 1) {      // one path rate: the slowest lane carries the largest volume
-                    const int64_t ts = ws<int64_t>(c.o_tscale)[0];
-#pragma unroll
-                    for (int t = 0; t < kWT; t++) den[t] = (int64_t)__reduce_max_sync(0xffffffffu, (uint32_t)x[t]) * ts;
-                } else {
-#pragma unroll
-                    for (int t = 0; t < kWT; t++) den[t] = (int64_t)x[t] * ws<int64_t>(c.o_tscale)[cls_in[t]];
-                    warp_max_x(den);
-                }
-#pragma unroll
-                for (int t = 0; t < kWT; t++) den[t] = F_new[t] > 0 ? kp.lambda_ns * dc.W + den[t] : 1;
-            }
-#pragma unroll
-            for (int t = 0; t < kWT; t++) {
-                if (!(valid >> t & 1)) continue;
-                const int task = task0 + t, h = ns4 ? task >> 2 : task / kp.n_start;
-                cnt.tasks++;
-                if (h != cur_h) {                          // a new family starts: settle the previous one
+            if (has && a == 0) cnt.tasks++;
+            // the teams' results in task order (every lane follows along)
+            const int in_round = min(8, n_tasks - task0);
+            for (int t = 0; t < in_round; t++) {
+                const int64_t Ft = __shfl_sync(0xffffffffu, F_new, t * 4), dt = __shfl_sync(0xffffffffu, den, t * 4);
+                const int tk = task0 + t, ht = ns_shift >= 0 ? tk >> ns_shift : tk / kp.n_start;
+                if (ht != cur_h) {                             // a new family starts: settle the previous one
                     if (cur_h >= 0 && (bt < 0 || util_greater(ff, fd, bf, bd))) { bf = ff; bd = fd; bt = ft; }
-                    cur_h = h; ff = -1; fd = 1; ft = -1;
+                    cur_h = ht; ff = -1; fd = 1; ft = -1;
                 }
-                if (F_new[t] > ff) { ff = F_new[t]; fd = den[t]; ft = task; }    // largest F, lowest start
+                if (Ft > ff) { ff = Ft; fd = dt; ft = tk; }    // largest F, lowest start
             }
         }
         if (cur_h >= 0 && (bt < 0 || util_greater(ff, fd, bf, bd))) { bf = ff; bd = fd; bt = ft; }   // lowest family on ties
@@ -317,7 +263,7 @@ __device__ __forceinline__ void decompose_warp(const DevCat& dc, const KParams& 
 
         // (D) emit activation k, D_rem -= X(E), write offset row k+1, re-sum D-hat
         {
-            const int h = ns4 ? bt >> 2 : bt / kp.n_start;
+            const int h = ns_shift >= 0 ? bt >> ns_shift : bt / kp.n_start;
             const size_t row = (size_t)k * N, orow = (size_t)(k + 1) * N;
             if (lane < N) {
                 const int r = lane;
@@ -360,7 +306,7 @@ __device__ __forceinline__ void decompose_warp(const DevCat& dc, const KParams& 
 }
 
 #ifndef VP_WARP_MIN_BLOCKS
-#define VP_WARP_MIN_BLOCKS 3
+#define VP_WARP_MIN_BLOCKS 4
 #endif
 __global__ void __launch_bounds__(128, VP_WARP_MIN_BLOCKS)
 vp_schedule_warp_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand, const int64_t* __restrict__ tau_in, int B,
@@ -551,6 +497,8 @@ vp_schedule_warp_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ deman
         __syncwarp();
     }
     unsigned long long* stats = (unsigned long long*)(counter + 4);
+    cnt.tasks = (unsigned long long)warp_sum_i64((int64_t)cnt.tasks);      // (counted by the first lane of every team)
+    cnt.sweeps = (unsigned long long)warp_sum_i64((int64_t)cnt.sweeps);
     if (lane == 0) {
         if (n_act) atomicAdd(&stats[0], n_act);
         if (cnt.tasks) { atomicAdd(&stats[1], cnt.tasks); atomicAdd(&stats[2], cnt.sweeps); }
