@@ -48,7 +48,10 @@ struct BigSmem {
 
 // The arg-max is taken class by class when the catalog allows it and has enough shapes for that to pay: a few hundred
 // shapes are scanned faster than two rounds of class maxima.
-__host__ __device__ inline bool big_use_dec(const DevCat& dc) { return dc.dec != nullptr && dc.n_shapes >= 1024; }
+#ifndef BIG_DEC_MIN_SHAPES
+#define BIG_DEC_MIN_SHAPES 1024
+#endif
+__host__ __device__ inline bool big_use_dec(const DevCat& dc) { return dc.dec != nullptr && dc.n_shapes >= BIG_DEC_MIN_SHAPES; }
 
 __host__ __device__ inline BigSmem big_smem_layout(const DevCat& dc, const KParams& kp) {
     BigSmem L;
