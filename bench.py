@@ -526,7 +526,9 @@ def run_e2e(vp, args, world, local_rank, dev, run, pk, pplan, idx, rows, R, barr
     T, topk = idx.shape
     prank, row_bytes = pk["rank"], pk["row_bytes"]
     per_matrix = w.k_max * N * 12 + 2 * (w.k_max + 1) * N * 8
-    sub = max(1, min(B, int(4e9 // per_matrix)))                 # at most ~4 GB pinned at a time
+    # at most ~16 GB pinned at a time: the host-buffer call works through such a sub-batch in chunks of about one matrix per
+    # SM, decomposing one chunk while the results of the chunk before it travel to the host
+    sub = max(1, min(B, int(16e9 // per_matrix)))
     h_demand = run.demand.cpu().contiguous().pin_memory()
     h_plan = vp.Plan.empty(sub, N, w.k_max, "cpu", pin=True)
     h_pplan = vp.Plan.empty(1, 16, pw.k_max, "cpu", pin=True)

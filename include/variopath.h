@@ -279,6 +279,12 @@ int vp_pack_static(const int32_t* n_steps_b, const int16_t* lane_dst_b, const in
  * device scratch, run the kernels above, copy the results back and return
  * after synchronising the stream.  device_scratch must hold
  * vp_schedule_host_scratch_bytes / vp_pack_host_scratch_bytes bytes.
+ *
+ * A scheduler batch of 64 matrices or more is worked through in chunks of about one matrix per SM (at least three
+ * chunks), two chunks in flight inside the same scratch: one is decomposed on cuda_stream while the results of the
+ * chunk before it are copied to the host on a second stream that the catalog handle owns (created on first use, freed
+ * with the handle).  The results are the same as for one chunk; the call still returns only when everything is in
+ * host memory.  Host-buffer calls that share a catalog handle must not run concurrently.
  */
 size_t vp_schedule_host_scratch_bytes(const vp_catalog* catalog, int B, const vp_sched_params* params);
 int vp_schedule_batch_host(const vp_catalog* catalog, const vp_sched_params* params,

@@ -59,8 +59,13 @@ extern "C" void vp_free_catalog(vp_catalog* c) {
     if (!c) return;
     int prev = -1;
     cudaGetDevice(&prev);
-    if (cudaSetDevice(c->device) == cudaSuccess)
+    if (cudaSetDevice(c->device) == cudaSuccess) {
         for (void* p : c->allocs) cudaFree(p);
+        if (c->host_pipe_ready) {
+            cudaStreamDestroy(c->copy_stream);
+            for (cudaEvent_t e : c->host_ev) cudaEventDestroy(e);
+        }
+    }
     if (prev >= 0) cudaSetDevice(prev);
     delete c;
 }
@@ -251,6 +256,7 @@ extern "C" int vp_load_catalog(const void* topology, size_t topo_bytes, const vo
     c->device = device;
     memset(c->memo, 0, sizeof(c->memo));
     c->memo_next = 0;
+    c->host_pipe_ready = 0;
     int prev = -1;
     cudaGetDevice(&prev);
     if (cudaSetDevice(device) != cudaSuccess) { delete c; return VP_E_CUDA; }

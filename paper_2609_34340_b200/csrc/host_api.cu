@@ -74,51 +74,112 @@ extern "C" size_t vp_schedule_host_scratch_bytes(const vp_catalog* c, int B, con
 
 namespace {
 
-// Both host-buffer scheduler calls: copy in, run vp_schedule_batch, copy out.  With used_only the plan arrays come back
-// only up to each matrix's n_steps (one copy per matrix and array, after n_steps itself has been read).
-int schedule_host(const vp_catalog* c, const vp_sched_params* p, const int64_t* demand, const int64_t* tau_ns_in, int B,
+// Copies of one chunk's results to host memory on `stream`.  With used_only the plan arrays come back only up to each
+// matrix's n_steps, which must already be in host memory.
+int copy_plan_out(const SchedBufs& s, size_t N, size_t K, size_t lo, size_t n, int32_t* n_steps, int32_t* chan_id,
+                  int16_t* lane_dst, uint16_t* lane_inst, int64_t* lane_bytes, int64_t* send_off, int64_t* recv_off,
+                  bool used_only, cudaStream_t stream) {
+    if (!used_only) {
+        VP_COPY(chan_id + lo * K, s.chan_id, n * K * 4, cudaMemcpyDeviceToHost);
+        VP_COPY(lane_dst + lo * K * N, s.lane_dst, n * K * N * 2, cudaMemcpyDeviceToHost);
+        VP_COPY(lane_inst + lo * K * N, s.lane_inst, n * K * N * 2, cudaMemcpyDeviceToHost);
+        VP_COPY(lane_bytes + lo * K * N, s.lane_bytes, n * K * N * 8, cudaMemcpyDeviceToHost);
+        VP_COPY(send_off + lo * (K + 1) * N, s.send_off, n * (K + 1) * N * 8, cudaMemcpyDeviceToHost);
+        if (recv_off) VP_COPY(recv_off + lo * (K + 1) * N, s.recv_off, n * (K + 1) * N * 8, cudaMemcpyDeviceToHost);
+        return VP_OK;
+    }
+    for (size_t m = 0; m < n; m++) {
+        const size_t g = lo + m;
+        const size_t k = n_steps[g] < 0 ? 0 : ((size_t)n_steps[g] > K ? K : (size_t)n_steps[g]);
+        VP_COPY(chan_id + g * K, s.chan_id + m * K, k * 4, cudaMemcpyDeviceToHost);
+        VP_COPY(lane_dst + g * K * N, s.lane_dst + m * K * N, k * N * 2, cudaMemcpyDeviceToHost);
+        VP_COPY(lane_inst + g * K * N, s.lane_inst + m * K * N, k * N * 2, cudaMemcpyDeviceToHost);
+        VP_COPY(lane_bytes + g * K * N, s.lane_bytes + m * K * N, k * N * 8, cudaMemcpyDeviceToHost);
+        VP_COPY(send_off + g * (K + 1) * N, s.send_off + m * (K + 1) * N, (k + 1) * N * 8, cudaMemcpyDeviceToHost);
+        if (recv_off) VP_COPY(recv_off + g * (K + 1) * N, s.recv_off + m * (K + 1) * N, (k + 1) * N * 8, cudaMemcpyDeviceToHost);
+    }
+    return VP_OK;
+}
+
+// Batches of at least this many matrices are worked through in chunks, two of them in flight: while one chunk is
+// decomposed on the caller's stream, the results of the chunk before it travel to the host on a second stream.
+constexpr int kPipeMinBatch = 64;
+
+// Both host-buffer scheduler calls: copy in, run vp_schedule_batch, copy out.
+int schedule_host(const vp_catalog* cc, const vp_sched_params* p, const int64_t* demand, const int64_t* tau_ns_in, int B,
                   int32_t* n_steps, int32_t* chan_id, int16_t* lane_dst, uint16_t* lane_inst, int64_t* lane_bytes,
                   int64_t* send_off, int64_t* recv_off, int64_t* tau_ns_out, int32_t* status, void* device_scratch,
                   size_t device_scratch_bytes, void* cuda_stream, bool used_only) {
+    vp_catalog* c = const_cast<vp_catalog*>(cc);
     if (!c || !p || B <= 0 || p->k_max <= 0 || !demand || !n_steps || !chan_id || !lane_dst || !lane_inst || !lane_bytes ||
         !send_off || !status)
         return VP_E_BAD_ARG;
     if (!device_scratch || ((uintptr_t)device_scratch & 255)) return VP_E_WORKSPACE;
-    SchedBufs s = carve_sched(device_scratch, c, B, p);
-    if (!s.ws_bytes) return VP_E_BAD_ARG;
-    if (device_scratch_bytes < s.total) return VP_E_WORKSPACE;
+    SchedBufs whole = carve_sched(nullptr, c, B, p);
+    if (!whole.ws_bytes) return VP_E_BAD_ARG;
+    if (device_scratch_bytes < whole.total) return VP_E_WORKSPACE;
     cudaStream_t stream = (cudaStream_t)cuda_stream;
-    const size_t N = (size_t)c->info.N, K = (size_t)p->k_max, b = (size_t)B;
+    const size_t N = (size_t)c->info.N, K = (size_t)p->k_max;
     DeviceScope scope(c->device);
     if (!scope.ok) return VP_E_CUDA;
-    VP_COPY(s.demand, demand, b * N * N * 8, cudaMemcpyHostToDevice);
-    if (tau_ns_in) VP_COPY(s.tau_in, tau_ns_in, b * 8, cudaMemcpyHostToDevice);
-    int rc = vp_schedule_batch(c, p, s.demand, tau_ns_in ? s.tau_in : nullptr, B, s.n_steps, s.chan_id, s.lane_dst,
-                               s.lane_inst, s.lane_bytes, s.send_off, recv_off ? s.recv_off : nullptr,
-                               tau_ns_out ? s.tau_out : nullptr, s.status, s.ws, s.ws_bytes, cuda_stream);
-    if (rc) return rc;
-    VP_COPY(n_steps, s.n_steps, b * 4, cudaMemcpyDeviceToHost);
-    if (tau_ns_out) VP_COPY(tau_ns_out, s.tau_out, b * 8, cudaMemcpyDeviceToHost);
-    VP_COPY(status, s.status, b * 4, cudaMemcpyDeviceToHost);
-    if (!used_only) {
-        VP_COPY(chan_id, s.chan_id, b * K * 4, cudaMemcpyDeviceToHost);
-        VP_COPY(lane_dst, s.lane_dst, b * K * N * 2, cudaMemcpyDeviceToHost);
-        VP_COPY(lane_inst, s.lane_inst, b * K * N * 2, cudaMemcpyDeviceToHost);
-        VP_COPY(lane_bytes, s.lane_bytes, b * K * N * 8, cudaMemcpyDeviceToHost);
-        VP_COPY(send_off, s.send_off, b * (K + 1) * N * 8, cudaMemcpyDeviceToHost);
-        if (recv_off) VP_COPY(recv_off, s.recv_off, b * (K + 1) * N * 8, cudaMemcpyDeviceToHost);
-    } else {
-        if (cudaStreamSynchronize(stream) != cudaSuccess) return VP_E_CUDA;      // n_steps is needed on the host now
-        for (size_t m = 0; m < b; m++) {
-            const size_t k = n_steps[m] < 0 ? 0 : ((size_t)n_steps[m] > K ? K : (size_t)n_steps[m]);
-            VP_COPY(chan_id + m * K, s.chan_id + m * K, k * 4, cudaMemcpyDeviceToHost);
-            VP_COPY(lane_dst + m * K * N, s.lane_dst + m * K * N, k * N * 2, cudaMemcpyDeviceToHost);
-            VP_COPY(lane_inst + m * K * N, s.lane_inst + m * K * N, k * N * 2, cudaMemcpyDeviceToHost);
-            VP_COPY(lane_bytes + m * K * N, s.lane_bytes + m * K * N, k * N * 8, cudaMemcpyDeviceToHost);
-            VP_COPY(send_off + m * (K + 1) * N, s.send_off + m * (K + 1) * N, (k + 1) * N * 8, cudaMemcpyDeviceToHost);
-            if (recv_off) VP_COPY(recv_off + m * (K + 1) * N, s.recv_off + m * (K + 1) * N, (k + 1) * N * 8, cudaMemcpyDeviceToHost);
+
+    // chunks: about one matrix per SM each, at least three, and two chunks' buffers must fit the scratch of the whole batch
+    int n_chunks = 1, chunk = B;
+    if (B >= kPipeMinBatch) {
+        n_chunks = B / (c->sm_count > 0 ? c->sm_count : 128);
+        if (n_chunks < 3) n_chunks = 3;
+        chunk = (B + n_chunks - 1) / n_chunks;
+        n_chunks = (B + chunk - 1) / chunk;
+        const SchedBufs one = carve_sched(nullptr, c, chunk, p);
+        if (!one.ws_bytes || 2 * one.total > device_scratch_bytes) { n_chunks = 1; chunk = B; }
+    }
+    if (n_chunks > 1 && !c->host_pipe_ready) {
+        if (cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking) != cudaSuccess) return VP_E_CUDA;
+        for (cudaEvent_t& e : c->host_ev)
+            if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return VP_E_CUDA;
+        c->host_pipe_ready = 1;
+    }
+    const size_t slot_bytes = n_chunks > 1 ? carve_sched(nullptr, c, chunk, p).total : 0;
+    SchedBufs slot[2];
+    slot[0] = carve_sched(device_scratch, c, chunk, p);
+    slot[1] = n_chunks > 1 ? carve_sched((char*)device_scratch + slot_bytes, c, chunk, p) : slot[0];
+    cudaStream_t copy = n_chunks > 1 ? c->copy_stream : stream;
+    cudaEvent_t* done = c->host_ev;          // [0], [1]: chunk decomposed;  [2], [3]: its results copied out
+    cudaEvent_t* copied = c->host_ev + 2;
+
+    for (int i = 0; i <= n_chunks; i++) {
+        if (i < n_chunks) {                  // ---- chunk i: copy in and decompose, on the caller's stream
+            const SchedBufs& s = slot[i & 1];
+            const size_t lo = (size_t)i * chunk, n = (size_t)(B - (int)lo < chunk ? B - (int)lo : chunk);
+            if (n_chunks > 1 && i >= 2 && cudaStreamWaitEvent(stream, copied[i & 1], 0) != cudaSuccess) return VP_E_CUDA;
+            VP_COPY(s.demand, demand + lo * N * N, n * N * N * 8, cudaMemcpyHostToDevice);
+            if (tau_ns_in) VP_COPY(s.tau_in, tau_ns_in + lo, n * 8, cudaMemcpyHostToDevice);
+            const int rc = vp_schedule_batch(c, p, s.demand, tau_ns_in ? s.tau_in : nullptr, (int)n, s.n_steps, s.chan_id,
+                                             s.lane_dst, s.lane_inst, s.lane_bytes, s.send_off, recv_off ? s.recv_off : nullptr,
+                                             tau_ns_out ? s.tau_out : nullptr, s.status, s.ws, s.ws_bytes, cuda_stream);
+            if (rc) return rc;
+            if (n_chunks > 1 && cudaEventRecord(done[i & 1], stream) != cudaSuccess) return VP_E_CUDA;
+        }
+        if (i >= 1 || n_chunks == 1) {       // ---- chunk i - 1 (the only chunk when there is one): results to the host
+            const int j = n_chunks == 1 ? 0 : i - 1;
+            if (n_chunks == 1 && i == 1) break;
+            const SchedBufs& s = slot[j & 1];
+            const size_t lo = (size_t)j * chunk, n = (size_t)(B - (int)lo < chunk ? B - (int)lo : chunk);
+            if (n_chunks > 1 && cudaStreamWaitEvent(copy, done[j & 1], 0) != cudaSuccess) return VP_E_CUDA;
+            {
+                cudaStream_t stream = copy;  // (VP_COPY issues on `stream`)
+                VP_COPY(n_steps + lo, s.n_steps, n * 4, cudaMemcpyDeviceToHost);
+                if (tau_ns_out) VP_COPY(tau_ns_out + lo, s.tau_out, n * 8, cudaMemcpyDeviceToHost);
+                VP_COPY(status + lo, s.status, n * 4, cudaMemcpyDeviceToHost);
+                if (used_only && cudaStreamSynchronize(copy) != cudaSuccess) return VP_E_CUDA;   // n_steps is needed on the host now
+                const int rc = copy_plan_out(s, N, K, lo, n, n_steps, chan_id, lane_dst, lane_inst, lane_bytes, send_off, recv_off,
+                                             used_only, copy);
+                if (rc) return rc;
+            }
+            if (n_chunks > 1 && cudaEventRecord(copied[j & 1], copy) != cudaSuccess) return VP_E_CUDA;
         }
     }
+    if (n_chunks > 1 && cudaStreamSynchronize(copy) != cudaSuccess) return VP_E_CUDA;
     if (cudaStreamSynchronize(stream) != cudaSuccess) return VP_E_CUDA;
     return VP_OK;
 }

@@ -83,6 +83,10 @@ struct vp_catalog {
     int max_smem_optin;
     vp_launch_memo memo[4];
     int memo_next;
+    // the host-buffer scheduler call's own copy stream and events (created on first use, see host_api.cu)
+    cudaStream_t copy_stream;
+    cudaEvent_t host_ev[4];
+    int host_pipe_ready;
 };
 
 extern std::atomic<long long> g_vp_launches;

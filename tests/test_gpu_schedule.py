@@ -201,6 +201,43 @@ def test_host_buffer_variant_used_rows_only(vp, oracle_lib):
             assert (got[name][b][K + 1:] == marks[name]).all(), (name, b)
 
 
+@pytest.mark.parametrize("used_only", [False, True])
+def test_host_buffer_variant_in_chunks(vp, oracle_lib, used_only):
+    """Batches of 64 matrices and more go through the host-buffer call in chunks, two in flight on two streams (ragged
+    last chunk, tau given per matrix, one invalid matrix): the same plans as the oracle's, chunk by chunk."""
+    c = build_config(2, device="cuda", batch=203, token_scale=0.25)
+    cat = c["catalog"]
+    oc = oracle_lib.OracleCatalog(cat.topology.blob(), cat.blob())
+    dc = vp.load_catalog(cat.topology.blob(), cat.blob())
+    p = _params(vp, c["params"])
+    D = c["demand"].clone()
+    D[77, 3, 3] = c["params"].granule_bytes              # an invalid matrix in the middle chunk
+    tau = torch.zeros(203, dtype=torch.int64)
+    tau[::5] = 40_000                                   # a given quantum for every fifth matrix
+    plan = vp.Plan.empty(203, 16, p.k_max, "cpu", pin=True)
+    for name in ("chan_id", "lane_dst", "lane_inst", "lane_bytes", "send_off", "recv_off"):
+        getattr(plan, name).fill_(-7 if name != "lane_inst" else 777)
+    for _ in range(2):                                  # the second call reuses the streams and events of the first
+        vp.schedule_batch_host(dc, p, D.pin_memory(), tau.pin_memory(), plan=plan, used_only=used_only)
+    want = oc.schedule_batch(D.numpy(), c["params"], tau_in=tau.numpy(), threads=os.cpu_count())
+    got = plan.cpu()
+    assert got["status"][77] == vp.ST_DIAG_NONZERO and got["n_steps"][77] == 0
+    assert (np.delete(got["status"], 77)[np.delete(tau.numpy(), 77) == 0] == 0).all()   # (a small given quantum may hit k_max)
+    if not used_only:
+        _assert_same(got, want)
+        return
+    for key in ("n_steps", "status", "tau_ns"):
+        assert np.array_equal(got[key], want[key]), key
+    for b in range(203):
+        K = int(want["n_steps"][b])
+        for name in ("chan_id", "lane_dst", "lane_inst", "lane_bytes"):
+            assert np.array_equal(got[name][b][:K], want[name][b][:K]), (name, b)
+            assert (got[name][b][K:] == (-7 if name != "lane_inst" else 777)).all(), (name, b)
+        for name in ("send_off", "recv_off"):
+            assert np.array_equal(got[name][b][:K + 1], want[name][b][:K + 1]), (name, b)
+            assert (got[name][b][K + 1:] == -7).all(), (name, b)
+
+
 @pytest.mark.parametrize("idx", [1, 2])
 def test_config_full_batch(vp, oracle_lib, idx):
     c = build_config(idx, device="cuda")
