@@ -528,6 +528,43 @@ def test_status_codes_on_large_catalogs(vp, oracle_lib, granule):
                                       vp.ST_OVERFLOW_RISK, vp.ST_NEGATIVE, 0]
 
 
+def test_plan_arrays_at_odd_addresses(vp, oracle_lib):
+    """Plan arrays that are aligned to their element size only (2, 8 bytes), not to 16: the kernel for large catalogs
+    then writes emit rows and idle rows with plain stores instead of staged 16-byte copies and bulk copies.  Also the
+    demand at an address that is 8 bytes off a 16-byte boundary."""
+    cat = node_template_catalog(tree_topology(32))
+    N = cat.topology.N
+    rng = np.random.default_rng(77)
+    B = 5
+    D = (rng.integers(0, 4000, size=(B, N, N)) * (rng.random((B, N, N)) < 0.3)).astype(np.int64) * 256
+    for b in range(B):
+        np.fill_diagonal(D[b], 0)
+    w = WParams(granule_bytes=256, k_max=6 * N).resolved(N)
+    oc = oracle_lib.OracleCatalog(cat.topology.blob(), cat.blob())
+    dc = vp.load_catalog(cat.topology.blob(), cat.blob())
+    want = oc.schedule_batch(D, w, threads=B)
+    p = _params(vp, w)
+    K = p.k_max
+
+    def off(shape, dtype, elems):            # a contiguous tensor whose first element sits `elems` elements into an allocation
+        n = int(np.prod(shape))
+        return torch.empty(n + elems, dtype=dtype, device="cuda")[elems:].view(shape)
+
+    plan = vp.Plan(n_steps=torch.empty(B, dtype=torch.int32, device="cuda"), chan_id=off((B, K), torch.int32, 1),
+                   lane_dst=off((B, K, N), torch.int16, 1), lane_inst=off((B, K, N), torch.uint16, 3),
+                   lane_bytes=off((B, K, N), torch.int64, 1), send_off=off((B, K + 1, N), torch.int64, 1),
+                   recv_off=off((B, K + 1, N), torch.int64, 1), tau_ns=torch.empty(B, dtype=torch.int64, device="cuda"),
+                   status=torch.empty(B, dtype=torch.int32, device="cuda"), k_max=K)
+    assert plan.lane_dst.data_ptr() % 16 == 2 and plan.lane_bytes.data_ptr() % 16 == 8
+    demand = off((B, N, N), torch.int64, 1)
+    demand.copy_(torch.from_numpy(D))
+    assert demand.data_ptr() % 16 == 8
+    vp.schedule_batch(dc, p, demand, plan=plan)
+    torch.cuda.synchronize()
+    _assert_same(plan.cpu(), want)
+    assert vp.schedule_launch_info(dc, B, p)["kernel"] == "CTA per matrix, 16-bit credits"
+
+
 def test_batches_around_one_wave(vp, oracle_lib):
     """Batch sizes just below and above the number of resident CTAs: the kernel changes, the plans do not."""
     c = build_config(2)
