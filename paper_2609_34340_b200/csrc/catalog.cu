@@ -373,7 +373,8 @@ extern "C" int vp_load_catalog(const void* topology, size_t topo_bytes, const vo
                             if (i >= src.size()) { ent[stride - 1] = 0xffffffffu; continue; }    // padding: never wins
                             const std::vector<uint32_t>& row = rows[src[i] & 0xffffu];
                             for (size_t t = 0; t < row.size(); t++) ent[t] = row[t];
-                            ent[stride - 1] = (uint32_t)i | (src[i] & 0xffff0000u);              // place | run start << 16
+                            // tie-break word: the run start for a first row (runs are in shape order), the place for a second row
+                            ent[stride - 1] = unit & 1 ? (uint32_t)i : src[i] >> 16;
                         }
                         for (size_t cc = chunk; cc < chunk + padded / 32; cc++) dec[3 + 2 * n + 1 + cc] = (uint32_t)unit;
                         chunk += padded / 32;

@@ -596,7 +596,8 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
                     // class, and its index grows with p0's place in shape order first, p1's place in the list second.
                     // So within a class the first maximum is (first maximal p0, first maximal p1 of the list): two
                     // independent maxima.  One warp per chunk of 32 rows: each lane scores its row from the table
-                    // (at most max_row_terms products) and the chunk's best key score << 16 | (65535 - place) is kept.
+                    // (at most max_row_terms products) and the chunk's best key score << 16 | (65535 - tie-break word) is kept
+                    // (the word is the run start for a first row, the place in the list for a second row: both grow in shape order).
                     const int n_chunks = (int)decs[0], stride = (int)decs[1];
                     for (int c = warp; c < n_chunks; c += n_warps) {
                         const uint32_t* ent = decs + decs[2] + (size_t)(c * 32 + lane) * stride;
@@ -632,9 +633,7 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
                     uint64_t cand = 0;
                     if (lane < dec_n) {                          // (red[unit]: the best key of the unit's chunks)
                         const uint64_t k0 = (uint64_t)red[2 * lane], k1 = (uint64_t)red[2 * lane + 1];
-                        const uint32_t place0 = 65535u - (uint32_t)(k0 & 0xffffu);
-                        const uint32_t first = decs[decs[2] + (size_t)(decs[3 + 2 * lane] * 32 + place0) * decs[1] + decs[1] - 1] >> 16;
-                        const uint32_t shape = first + (65535u - (uint32_t)(k1 & 0xffffu));
+                        const uint32_t shape = (65535u - (uint32_t)(k0 & 0xffffu)) + (65535u - (uint32_t)(k1 & 0xffffu));   // run start + place
                         cand = ((k0 >> 16) + (k1 >> 16)) << 16 | (uint64_t)(65535u - shape);
                     }
                     bkey = big_warp_max64(cand);

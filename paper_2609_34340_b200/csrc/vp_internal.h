@@ -38,7 +38,7 @@ struct DevCat {
     // shape(p0, p1) = run_start(p0) + place of p1 in the list of p0's class.  Unit 2 cl holds the first rows of class cl,
     // unit 2 cl + 1 its second rows, each padded to whole chunks of 32 entries.  dec[0] = chunks, dec[1] = words per
     // entry, dec[2] = offset of the entries, dec[3 .. 3 + 2 n] = first chunk of every unit, then the unit of every chunk; an entry is the row's terms
-    // (table index | count << 16, zero padded) followed by place | run_start << 16 (all ones marks padding).  Null
+    // (table index | count << 16, zero padded) followed by its tie-break word: run_start for a first row, place for a second row (all ones marks padding).  Null
     // when the catalog has no such structure.
     const uint32_t* dec;
     int dec_classes, dec_words;
