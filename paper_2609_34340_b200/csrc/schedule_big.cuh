@@ -225,7 +225,10 @@ __global__ void __launch_bounds__(256) big_rank_kernel(const int* __restrict__ k
 #endif
 // DEC: the arg-max of Eq. (6) is taken class by class (see big_use_dec).
 template <int W, bool DEC>
-__global__ void __launch_bounds__(W == 2 ? 512 : 256, W == 2 ? 1 : VP_BIG_W1_CTAS)
+#ifndef BIG_W2_THREADS
+#define BIG_W2_THREADS 384             // 8 task warps + 4 others; 512 (8 others) measured 6 % slower, 320 5 % slower
+#endif
+__global__ void __launch_bounds__(W == 2 ? BIG_W2_THREADS : 256, W == 2 ? 1 : VP_BIG_W1_CTAS)
 vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand, const int64_t* __restrict__ tau_in, int B,
                        int32_t* __restrict__ n_steps, int32_t* __restrict__ chan_id, int16_t* __restrict__ lane_dst,
                        uint16_t* __restrict__ lane_inst, int64_t* __restrict__ lane_bytes, int64_t* __restrict__ send_off,
@@ -539,13 +542,14 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
             // warps, which has no task in Step 2 as a rule, copies them out during Step 2 of the next iteration.  (Plain
             // stores to global memory by the emitting warps, just before a CTA-wide barrier, made every iteration wait
             // for them: 6 % of the run time.)
-            const bool rows_async = N % 8 == 0 && kp.n_start * W <= (n_warps >> 1) &&
+            const int copy_warp0 = max(kp.n_start * W, (N + 31) >> 5);     // first warp with neither a task nor a slot to emit
+            const bool rows_async = N % 8 == 0 && copy_warp0 < n_warps &&
                 (((uintptr_t)lane_dst_b | (uintptr_t)lane_inst_b | (uintptr_t)lane_bytes_b | (uintptr_t)send_off_b |
                   (uintptr_t)(recv_off_b ? recv_off_b : send_off_b)) & 15) == 0;
             int copied = 0;                                  // activations copied out (upper warps)
             auto copy_row = [&](int kk) {
                 const unsigned char* sb = smem_raw + L.emit;
-                for (int e = tid - (NT >> 1); e < 28 * N / 16; e += NT >> 1) {
+                for (int e = tid - copy_warp0 * 32; e < 28 * N / 16; e += NT - copy_warp0 * 32) {
                     const int at = e * 16;
                     unsigned char* dst;
                     if (at < 4 * N) dst = at < 2 * N ? (unsigned char*)(lane_dst_b + (size_t)kk * N) + at
@@ -648,7 +652,7 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
                 VP_TICK(1);
 
                 if (W == 2 && warp == FILL_WARP && s_job_next < s_job_total) fill_step(1);   // (this warp has no task as a rule)
-                if (rows_async && warp >= (n_warps >> 1) && copied < k) copy_row(copied++);  // the last activation's rows
+                if (rows_async && warp >= copy_warp0 && copied < k) copy_row(copied++);      // the last activation's rows
 
                 // (B) MultiStartAA: W warps per (family, start), one lane per rank group
                 const int sub = W == 2 ? (warp & 1) : 0, wgroup = W == 2 ? (warp >> 1) : warp;
@@ -911,7 +915,7 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
                 __syncthreads();
                 VP_TICK(4);
             }
-            if (rows_async && warp >= (n_warps >> 1) && copied < k) copy_row(copied++);   // the last activation of the matrix
+            if (rows_async && warp >= copy_warp0 && copied < k) copy_row(copied++);       // the last activation of the matrix
         }
         __syncthreads();
         // ---- idle rows beyond n_steps; offset rows repeat the totals
