@@ -228,7 +228,10 @@ template <int W, bool DEC>
 #ifndef BIG_W2_THREADS
 #define BIG_W2_THREADS 384             // 8 task warps + 4 others; 512 (8 others) measured 6 % slower, 320 5 % slower
 #endif
-__global__ void __launch_bounds__(W == 2 ? BIG_W2_THREADS : 256, W == 2 ? 1 : VP_BIG_W1_CTAS)
+#ifndef BIG_W1_MAXT
+#define BIG_W1_MAXT 256
+#endif
+__global__ void __launch_bounds__(W == 2 ? BIG_W2_THREADS : BIG_W1_MAXT, W == 2 ? 1 : VP_BIG_W1_CTAS)
 vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand, const int64_t* __restrict__ tau_in, int B,
                        int32_t* __restrict__ n_steps, int32_t* __restrict__ chan_id, int16_t* __restrict__ lane_dst,
                        uint16_t* __restrict__ lane_inst, int64_t* __restrict__ lane_bytes, int64_t* __restrict__ send_off,

@@ -528,6 +528,47 @@ def test_status_codes_on_large_catalogs(vp, oracle_lib, granule):
                                       vp.ST_OVERFLOW_RISK, vp.ST_NEGATIVE, 0]
 
 
+@pytest.mark.parametrize("nodes,nic_bw", [(24, 64), (20, 50)])
+def test_class_wise_argmax_on_other_catalogs(vp, oracle_lib, nodes, nic_bw):
+    """Two-rail node-template catalogs of more than 1,024 shapes take Step 1 class by class (2,303 shapes at 24 nodes,
+    1,599 at 20 nodes with two path rates).  Matrices whose shape scores tie massively (every cell equal; equal cells
+    inside the switches only; equal cells between the two switches of a node only) check that the first maximum is
+    the same shape as in the oracle's scan; the others are random sparse, dense and flat, and a single cell."""
+    cat = node_template_catalog(tree_topology(nodes, pcie_bw=64, nic_bw=nic_bw))
+    N = cat.topology.N
+    assert cat.n_shapes >= 1024
+    rng = np.random.default_rng(nodes)
+    u = 256
+    B = 7
+    D = (rng.integers(0, 2000, size=(B, N, N)) * (rng.random((B, N, N)) < 0.4)).astype(np.int64)
+    D[1] = 1000                                              # every shape with the same lane count ties
+    D[2] = 0
+    D[3] = 0
+    for n in range(nodes):
+        lo = n * 8
+        for g0 in (lo, lo + 4):
+            D[2][g0:g0 + 4, g0:g0 + 4] = 700                 # inside the switches only
+        D[3][lo:lo + 4, lo + 4:lo + 8] = 500                 # between the two switches of a node only
+        D[3][lo + 4:lo + 8, lo:lo + 4] = 500
+    D[4] = rng.integers(0, 300, size=(N, N))                 # dense and flat
+    D[5] = 0
+    D[5][5, 9] = 77                                          # a single cell
+    D *= u
+    for b in range(B):
+        np.fill_diagonal(D[b], 0)
+    oc = oracle_lib.OracleCatalog(cat.topology.blob(), cat.blob())
+    dc = vp.load_catalog(cat.topology.blob(), cat.blob())
+    for extra in ({}, {"lambda_ns": 0, "k_target": N}):
+        w = WParams(granule_bytes=u, k_max=10 * N, **extra).resolved(N)
+        p = _params(vp, w)
+        plan = vp.schedule_batch(dc, p, torch.from_numpy(D).cuda())
+        torch.cuda.synchronize()
+        want = oc.schedule_batch(D, w, threads=B)
+        _assert_same(plan.cpu(), want)
+        assert (np.asarray(want["status"]) == 0).all()
+    assert vp.schedule_launch_info(dc, B, p)["kernel"] == "CTA per matrix, 16-bit credits"
+
+
 def test_plan_arrays_at_odd_addresses(vp, oracle_lib):
     """Plan arrays that are aligned to their element size only (2, 8 bytes), not to 16: the kernel for large catalogs
     then writes emit rows and idle rows with plain stores instead of staged 16-byte copies and bulk copies.  Also the
