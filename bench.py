@@ -183,7 +183,7 @@ class SchedRun:
         self.demand = sched["demand"].to(dev).contiguous()
         self.B, self.N = self.demand.shape[0], cat.topology.N
         per_matrix = w.k_max * self.N * 12 + 2 * (w.k_max + 1) * self.N * 8
-        fit = max(1, int(40e9 // per_matrix))                    # at most ~40 GB of plan buffers
+        fit = max(1, int(64e9 // per_matrix))                    # at most ~64 GB of plan buffers
         self.sub = min(self.B, sub_batch or self.B, fit)
         self.plan = vp.Plan.empty(self.sub, self.N, w.k_max, dev)
         self.ws = torch.empty(vp.schedule_workspace_bytes(self.dc, self.sub, self.params), dtype=torch.uint8, device=dev)
@@ -807,7 +807,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--sched-config", type=int, default=4, choices=[1, 2, 3, 4])
-    ap.add_argument("--sub-batch", type=int, default=1024,
+    ap.add_argument("--sub-batch", type=int, default=2048,
                     help="matrices per vp_schedule_batch call (the plan buffers are reused); the batch when smaller")
     ap.add_argument("--batch", type=int, default=None, help="truncate the scheduler batch (tests)")
     ap.add_argument("--sched-repeat", type=int, default=1,
