@@ -78,6 +78,11 @@ typedef struct vp_info {
     int32_t node_symmetric;       /* 1 if every shape is invariant under a shift of the node index:
                                      Eq. (6) is then evaluated on per-node-offset sums of D-hat   */
     int64_t rate_lcm;             /* lcm of all path rates (utilities are compared exactly)       */
+    int32_t row_patterns;         /* node-symmetric catalogs: distinct rows (terms of a shape that leave
+                                     one rail of node 0); 0 otherwise                              */
+    int32_t argmax_classes;       /* two-rail node-symmetric catalogs whose shapes decompose into classes
+                                     of first rows with a common list of second rows (see
+                                     vp_catalog_argmax_classes): the number of classes; 0 otherwise */
 } vp_info;
 
 /*
@@ -114,14 +119,32 @@ typedef struct vp_sched_params {
  * pair, repeats an instance beyond mult, or uses a directed resource twice
  * (Eq. 4).  A catalog that leaves a group pair uncovered loads (info.covered
  * = 0); demand on that pair ends with VP_ST_UNCOVERED.
- * device: CUDA device ordinal that will hold the image.  *out receives the
- * handle, to be released with vp_free_catalog.  Synchronous.
+ * device: CUDA device ordinal that will hold the image, or -1 for a host-only
+ * handle: the blobs are parsed, validated and analysed as usual, nothing is
+ * uploaded, vp_catalog_info and vp_catalog_argmax_classes work, and every call
+ * that would launch a kernel returns VP_E_BAD_ARG.  *out receives the handle,
+ * to be released with vp_free_catalog.  Synchronous.
  */
 int vp_load_catalog(const void* topology, size_t topology_bytes,
                     const void* channels, size_t channels_bytes,
                     int device, vp_catalog** out);
 void vp_free_catalog(vp_catalog* catalog);
 int vp_catalog_info(const vp_catalog* catalog, vp_info* out);
+
+/*
+ * The catalog's class decomposition of Eq. (6)'s arg-max, as the scheduler kernel for large catalogs uses it (host
+ * call; for tests and tools).  In a two-rail node-symmetric catalog a shape is a pair (first row, second row).  When
+ * the shapes that share a first row are consecutive and first rows fall into few classes with one common list of
+ * second rows, the shape of (first row p0, second row at place j of the list of p0's class) is run_start(p0) + j, and
+ * the first maximum over all shapes is the best of the classes' (first maximal p0, first maximal second row).
+ * out (host, capacity_words 32-bit words; may be NULL to query) receives: [0] chunks, [1] words per entry, [2] offset
+ * of the entries, [3 .. 3 + 2n] the first chunk of every unit (unit 2c = the first rows of class c, unit 2c + 1 its
+ * second rows; a chunk is 32 entries), then the unit of every chunk; an entry is the row's terms (table index |
+ * lane count << 16, zero padded; table index of (node offset delta, rail q, rail q') = (delta S + q) S + q') followed
+ * by its tie-break word: run_start for a first row, the place for a second row, all ones for padding.
+ * *words_needed receives the length; 0 when the catalog has no such structure.  VP_E_WORKSPACE if out is too small.
+ */
+int vp_catalog_argmax_classes(const vp_catalog* catalog, uint32_t* out, size_t capacity_words, size_t* words_needed);
 
 /*
  * vp_build_template_catalog - a node-symmetric catalog for many nodes (host code, no GPU work; no counterpart in the

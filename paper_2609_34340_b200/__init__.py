@@ -11,6 +11,7 @@ from .binding import (  # noqa: F401
     Plan,
     SchedParams,
     load_catalog,
+    catalog_argmax_classes,
     build_catalog,
     build_template_catalog,
     prune_paths,

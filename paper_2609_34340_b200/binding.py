@@ -31,7 +31,8 @@ class VpError(RuntimeError):
 class _Info(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("N", "G", "g", "groups_per_node", "n_resources", "n_instances",
                                           "n_shapes", "n_families", "max_nnz", "max_bucket", "covered",
-                                          "node_symmetric")] + [("rate_lcm", C.c_int64)]
+                                          "node_symmetric")] + [("rate_lcm", C.c_int64), ("row_patterns", C.c_int32),
+                                                                ("argmax_classes", C.c_int32)]
 
 
 class _Params(C.Structure):
@@ -74,6 +75,7 @@ def _load():
     lib.vp_free_catalog.argtypes = [vp]
     lib.vp_free_catalog.restype = None
     lib.vp_catalog_info.argtypes = [vp, C.POINTER(_Info)]
+    lib.vp_catalog_argmax_classes.argtypes = [vp, P, sz, C.POINTER(sz)]
     lib.vp_schedule_workspace_bytes.argtypes = [vp, i32, C.POINTER(_Params)]
     lib.vp_schedule_workspace_bytes.restype = sz
     sched_args = [vp, C.POINTER(_Params), P, P, i32] + [P] * 9
@@ -246,6 +248,18 @@ def load_catalog(topology: bytes, channels: bytes, device: int = 0) -> Catalog:
     _check(_load().vp_load_catalog(topology, len(topology), channels, len(channels), int(device), C.byref(h)),
            "vp_load_catalog")
     return Catalog(h.value, int(device))
+
+
+def catalog_argmax_classes(catalog: Catalog):
+    """``vp_catalog_argmax_classes``: the class decomposition of the arg-max as a numpy uint32 array (empty if none)."""
+    import numpy as np
+    need = C.c_size_t(0)
+    _check(_load().vp_catalog_argmax_classes(catalog._h, None, 0, C.byref(need)), "vp_catalog_argmax_classes")
+    out = np.zeros(need.value, dtype=np.uint32)
+    if need.value:
+        _check(_load().vp_catalog_argmax_classes(catalog._h, out.ctypes.data_as(C.c_void_p), need.value, C.byref(need)),
+               "vp_catalog_argmax_classes")
+    return out
 
 
 def build_catalog(topology: bytes):

@@ -42,6 +42,7 @@ int64_t gcd_i64(int64_t a, int64_t b) {
 
 template <typename T>
 int upload(vp_catalog* c, const std::vector<T>& v, const T** out) {
+    if (c->device < 0) { *out = nullptr; return VP_OK; }     // host-only handle: nothing is uploaded
     void* d = nullptr;
     // sizes are rounded up to 16 bytes (zero filled) so that the kernels may stage whole arrays with bulk copies
     size_t bytes = (std::max<size_t>(v.size(), 1) * sizeof(T) + 15) & ~(size_t)15;
@@ -59,7 +60,7 @@ extern "C" void vp_free_catalog(vp_catalog* c) {
     if (!c) return;
     int prev = -1;
     cudaGetDevice(&prev);
-    if (cudaSetDevice(c->device) == cudaSuccess) {
+    if (c->device >= 0 && cudaSetDevice(c->device) == cudaSuccess) {
         for (void* p : c->allocs) cudaFree(p);
         if (c->host_pipe_ready) {
             cudaStreamDestroy(c->copy_stream);
@@ -70,6 +71,15 @@ extern "C" void vp_free_catalog(vp_catalog* c) {
     delete c;
 }
 
+extern "C" int vp_catalog_argmax_classes(const vp_catalog* c, uint32_t* out, size_t capacity_words, size_t* words_needed) {
+    if (!c || !words_needed) return VP_E_BAD_ARG;
+    *words_needed = c->dec_host.size();
+    if (!out) return VP_OK;
+    if (capacity_words < c->dec_host.size()) return VP_E_WORKSPACE;
+    if (!c->dec_host.empty()) memcpy(out, c->dec_host.data(), c->dec_host.size() * sizeof(uint32_t));
+    return VP_OK;
+}
+
 extern "C" int vp_catalog_info(const vp_catalog* c, vp_info* out) {
     if (!c || !out) return VP_E_BAD_ARG;
     *out = c->info;
@@ -78,7 +88,7 @@ extern "C" int vp_catalog_info(const vp_catalog* c, vp_info* out) {
 
 extern "C" int vp_load_catalog(const void* topology, size_t topo_bytes, const void* channels, size_t chan_bytes,
                                int device, vp_catalog** out) {
-    if (!topology || !channels || !out || device < 0) return VP_E_BAD_ARG;
+    if (!topology || !channels || !out || device < -1) return VP_E_BAD_ARG;
     *out = nullptr;
     Reader t{(const uint8_t*)topology, topo_bytes}, h{(const uint8_t*)channels, chan_bytes};
     if (t.u32(0) != 0x50545056u || t.u32(4) != 1 || !t.ok) return VP_E_BAD_CATALOG;
@@ -258,12 +268,16 @@ extern "C" int vp_load_catalog(const void* topology, size_t topo_bytes, const vo
     c->memo_next = 0;
     c->host_pipe_ready = 0;
     int prev = -1;
-    cudaGetDevice(&prev);
-    if (cudaSetDevice(device) != cudaSuccess) { delete c; return VP_E_CUDA; }
-    cudaDeviceProp prop;
-    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete c; return VP_E_CUDA; }
-    c->sm_count = prop.multiProcessorCount;
-    c->max_smem_optin = (int)prop.sharedMemPerBlockOptin;
+    c->sm_count = 0;
+    c->max_smem_optin = 0;
+    if (device >= 0) {
+        cudaGetDevice(&prev);
+        if (cudaSetDevice(device) != cudaSuccess) { delete c; return VP_E_CUDA; }
+        cudaDeviceProp prop;
+        if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete c; return VP_E_CUDA; }
+        c->sm_count = prop.multiProcessorCount;
+        c->max_smem_optin = (int)prop.sharedMemPerBlockOptin;
+    }
     DevCat& dc = c->dc;
     memset(&dc, 0, sizeof(dc));
     dc.N = N; dc.G = G; dc.g = g; dc.S = S; dc.P = P;
@@ -382,6 +396,7 @@ extern "C" int vp_load_catalog(const void* topology, size_t topo_bytes, const vo
                     dec[3 + 2 * n] = (uint32_t)chunk;
                     dc.dec_classes = n;
                     dc.dec_words = (int)dec.size();
+                    c->dec_host = dec;
                     rc = upload(c, dec, &dc.dec);
                 }
             }
@@ -418,6 +433,7 @@ extern "C" int vp_load_catalog(const void* topology, size_t topo_bytes, const vo
     I.N = N; I.G = G; I.g = g; I.groups_per_node = S; I.n_resources = n_res; I.n_instances = n_inst;
     I.n_shapes = n_shapes; I.n_families = n_fam; I.max_nnz = max_nnz; I.max_bucket = max_bucket;
     I.covered = covered; I.node_symmetric = sym; I.rate_lcm = W;
+    I.row_patterns = dc.n_patterns; I.argmax_classes = dc.dec_classes;
     if (prev >= 0) cudaSetDevice(prev);
     *out = c;
     return VP_OK;

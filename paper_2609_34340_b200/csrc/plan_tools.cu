@@ -85,7 +85,7 @@ demand_kernel(const int32_t* __restrict__ idx, int n_src, long long per_src, int
 
 extern "C" int vp_plan_time(const vp_catalog* c, int B, int k_max, const int32_t* n_steps, const uint16_t* lane_inst,
                             const int64_t* lane_bytes, int64_t lambda_ns, int64_t* time_xw, void* cuda_stream) {
-    if (!c || B <= 0 || k_max <= 0 || !n_steps || !lane_inst || !lane_bytes || !time_xw) return VP_E_BAD_ARG;
+    if (!c || c->device < 0 || B <= 0 || k_max <= 0 || !n_steps || !lane_inst || !lane_bytes || !time_xw) return VP_E_BAD_ARG;
     if (lambda_ns < 0 || lambda_ns >= VP_ENTRY_LIMIT) return VP_E_BAD_ARG;
     int prev = -1;
     cudaGetDevice(&prev);

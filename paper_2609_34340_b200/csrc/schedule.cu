@@ -1176,7 +1176,7 @@ BigKernelFn pick_big_kernel(int w, bool dec) {
 }
 
 int resolve_params(const vp_catalog* c, const vp_sched_params* p, KParams* kp) {
-    if (!c || !p) return VP_E_BAD_ARG;
+    if (!c || !p || c->device < 0) return VP_E_BAD_ARG;         // (a host-only handle launches nothing)
     if (p->k_max <= 0 || p->granule_bytes <= 0 || p->lambda_ns < 0 || p->lambda_ns >= VP_ENTRY_LIMIT) return VP_E_BAD_ARG;
     if (p->k_target < 0 || p->n_start < 0 || p->i_aa < 0 || p->n_start > 64) return VP_E_BAD_ARG;
     kp->lambda_ns = p->lambda_ns; kp->granule = p->granule_bytes;

@@ -84,6 +84,7 @@ struct vp_catalog {
     vp_launch_memo memo[4];
     int memo_next;
     // the host-buffer scheduler call's own copy stream and events (created on first use, see host_api.cu)
+    std::vector<uint32_t> dec_host;   // host copy of DevCat::dec (vp_catalog_argmax_classes)
     cudaStream_t copy_stream;
     cudaEvent_t host_ev[4];
     int host_pipe_ready;

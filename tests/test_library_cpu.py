@@ -111,3 +111,76 @@ def test_status_bits_are_distinct_and_the_timeout_bit_is_declared():
     for name, v in values.items():
         assert getattr(vp, name[3:]) == v, name
     assert vp.ST_INTERNAL_TIMEOUT == 1 << 30 and vp.ST_INTERNAL_TIMEOUT & (vp.ST_PACK_MISMATCH | vp.ST_PACK_CAPACITY) == 0
+
+
+def test_host_only_handle_info_and_refusals():
+    """device = -1: the loader parses, validates and analyses without a GPU; calls that would launch refuse."""
+    import paper_2609_34340_b200 as vp
+    cat = complete_catalog(tree_topology(1))
+    dc = vp.load_catalog(cat.topology.blob(), cat.blob(), device=-1)
+    assert (dc.N, dc.G, dc.g, dc.n_shapes, dc.n_families, dc.covered, dc.node_symmetric) == (8, 2, 4, 3, 6, 1, 0)
+    assert dc.row_patterns == 0 and dc.argmax_classes == 0 and len(vp.catalog_argmax_classes(dc)) == 0
+    assert vp.schedule_workspace_bytes(dc, 4, vp.SchedParams()) == 0          # nothing can be launched from it
+    with pytest.raises(vp.VpError) as e:
+        vp.load_catalog(cat.topology.blob(), cat.blob()[:-2], device=-1)
+    assert e.value.code == vp.E_BAD_CATALOG
+    big = crossbar_catalog(crossbar_topology(6))
+    with pytest.raises(vp.VpError) as e:
+        vp.load_catalog(big.topology.blob(), big.blob(), device=-1)
+    assert e.value.code == vp.E_UNSUPPORTED
+    with pytest.raises(vp.VpError) as e:
+        vp.load_catalog(cat.topology.blob(), cat.blob(), device=-2)
+    assert e.value.code == vp.E_BAD_ARG
+    uncovered = type(cat)(cat.topology, [cat.shapes[-1]], [cat.buckets[-1]])   # the all-PIX shape only
+    assert vp.load_catalog(uncovered.topology.blob(), uncovered.blob(), device=-1).covered == 0
+
+
+@pytest.mark.parametrize("nodes,nic_bw", [(2, 64), (5, 50), (16, 64), (32, 64)])
+def test_argmax_classes_reproduce_every_shape(nodes, nic_bw):
+    """The loader's class decomposition of Eq. (6)'s arg-max, checked against the catalog itself: every shape of a
+    two-rail node-template catalog is (first row p0, second row p1); the decomposition claims that the shape of
+    (p0, the second row at place j of the list of p0's class) is run_start(p0) + j.  Rebuilt here from the shapes'
+    (a, d, count) lists alone: every claimed pair is that shape, and the claims cover every shape exactly once."""
+    import paper_2609_34340_b200 as vp
+    cat = node_template_catalog(tree_topology(nodes, pcie_bw=64, nic_bw=nic_bw))
+    S = cat.topology.groups_per_node
+    assert S == 2
+    dc = vp.load_catalog(cat.topology.blob(), cat.blob(), device=-1)
+    assert dc.node_symmetric == 1 and dc.argmax_classes > 0
+
+    def row(shape, q):                      # terms leaving rail q of node 0: (table index of (delta, q, q'), lanes), by destination
+        return tuple((((d // S) * S + q) * S + d % S, c) for (a, d, c) in shape if a == q)
+
+    rows_of_shape = [(row(s, 0), row(s, 1)) for s in cat.shapes]
+    assert dc.row_patterns == len({r for pair in rows_of_shape for r in pair})
+    d = vp.catalog_argmax_classes(dc)
+    n_chunks, stride, ent_off = int(d[0]), int(d[1]), int(d[2])
+    n = dc.argmax_classes
+    first = [int(x) for x in d[3:3 + 2 * n + 1]]
+    assert first[0] == 0 and first[-1] == n_chunks and first == sorted(first)
+    unit_of_chunk = [int(x) for x in d[3 + 2 * n + 1:3 + 2 * n + 1 + n_chunks]]
+    assert unit_of_chunk == [u for u in range(2 * n) for _ in range(first[u + 1] - first[u])]
+
+    def entries(unit):
+        out = []
+        for e in range(first[unit] * 32, first[unit + 1] * 32):
+            words = d[ent_off + e * stride: ent_off + (e + 1) * stride]
+            if int(words[-1]) == 0xFFFFFFFF:                     # padding comes last and scores nothing
+                assert not any(int(w) for w in words[:-1])
+                continue
+            assert len(out) == e - first[unit] * 32              # no padding in between
+            terms = tuple((int(w) & 0xFFFF, int(w) >> 16) for w in words[:-1] if int(w) >> 16)
+            out.append((terms, int(words[-1])))
+        return out
+
+    seen = np.zeros(cat.n_shapes, dtype=np.int64)
+    for cl in range(n):
+        members, second = entries(2 * cl), entries(2 * cl + 1)
+        assert members and second
+        assert [t for _, t in second] == list(range(len(second)))               # places count up
+        assert [t for _, t in members] == sorted({t for _, t in members})       # run starts in shape order
+        for p0, run_start in members:
+            for p1, place in second:
+                assert rows_of_shape[run_start + place] == (p0, p1), (cl, run_start, place)
+                seen[run_start + place] += 1
+    assert (seen == 1).all()
