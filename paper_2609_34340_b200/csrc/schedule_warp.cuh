@@ -95,14 +95,16 @@ __device__ __forceinline__ void decompose_warp(const DevCat& dc, const KParams& 
     // Plain score tables of at most 16 D-hat cells and at most 128 shapes: a lane keeps the lane counts of its (up to
     // four) shapes in registers, four bits per cell, and scoring needs no term loads.
     const bool dense = dc.tbl_size <= 16 && dc.n_shapes <= 128;
-    unsigned long long smask[4] = {0ull, 0ull, 0ull, 0ull};
+    const int n_rounds = (dc.n_shapes + 31) >> 5;         // shapes per lane (dense: at most four)
+    uint32_t smask[4][2] = {{0u, 0u}, {0u, 0u}, {0u, 0u}, {0u, 0u}};     // cells 0..7, cells 8..15
     if (dense)
         for (int u = 0; u < 4; u++) {
             const int s = lane + 32 * u;
             if (s < dc.n_shapes)
                 for (int e = 0; e < dc.max_terms; e++) {
                     const uint32_t w = ws<uint32_t>(c.o_term)[e * ns_pad + s];
-                    smask[u] |= (unsigned long long)(w >> 16) << (4 * ((w & 0xffffu) >> 3));
+                    const uint32_t cell = (w & 0xffffu) >> 3;
+                    smask[u][cell >> 3] |= (w >> 16) << (4 * (cell & 7));
                 }
         }
 
@@ -121,7 +123,8 @@ __device__ __forceinline__ void decompose_warp(const DevCat& dc, const KParams& 
                     if (cell < dc.tbl_size) {
                         const uint32_t d = (uint32_t)Dhat[cell];
 #pragma unroll
-                        for (int u = 0; u < 4; u++) sc[u] += d * (uint32_t)((smask[u] >> (4 * cell)) & 15ull);
+                        for (int u = 0; u < 4; u++)
+                            if (u < n_rounds) sc[u] += d * ((smask[u][cell >> 3] >> (4 * (cell & 7))) & 15u);
                     }
                 }
 #pragma unroll
@@ -134,7 +137,8 @@ __device__ __forceinline__ void decompose_warp(const DevCat& dc, const KParams& 
                     if (cell < dc.tbl_size) {
                         const int64_t d = Dhat[cell];
 #pragma unroll
-                        for (int u = 0; u < 4; u++) sc[u] += d * (int64_t)((smask[u] >> (4 * cell)) & 15ull);
+                        for (int u = 0; u < 4; u++)
+                            if (u < n_rounds) sc[u] += d * (int64_t)((smask[u][cell >> 3] >> (4 * (cell & 7))) & 15u);
                     }
                 }
 #pragma unroll
@@ -246,6 +250,18 @@ __device__ __forceinline__ void decompose_warp(const DevCat& dc, const KParams& 
                 den = F_new > 0 ? kp.lambda_ns * dc.W + tmax : 1;
             }
             if (has && a == 0) cnt.tasks++;
+            if (H == 1 && n_tasks <= 8) {
+                // one family, one round: the best start is the largest F, the lowest start among equals -- one maximum of
+                // F << 3 | (7 - start) over the warp (F is below 2^42)
+                const uint64_t key = has && a == 0 ? (uint64_t)F_new << 3 | (uint64_t)(7 - team) : 0ull;
+                const uint32_t hi = (uint32_t)(key >> 32), lo = (uint32_t)key;
+                const uint32_t mhi = __reduce_max_sync(0xffffffffu, hi);
+                const uint32_t mlo = __reduce_max_sync(0xffffffffu, hi == mhi ? lo : 0u);
+                const uint64_t mkey = (uint64_t)mhi << 32 | mlo;
+                bf = (int64_t)(mkey >> 3); bd = 1; bt = 7 - (int)(mkey & 7u);
+                cur_h = -1;                                       // (settled)
+                break;
+            }
             // the teams' results in task order (every lane follows along)
             const int in_round = min(8, n_tasks - task0);
             for (int t = 0; t < in_round; t++) {
