@@ -483,8 +483,9 @@ int vp_unpack_tokens(const int32_t* n_steps_b, const int16_t* lane_dst_b, const 
 /*
  * How vp_schedule_batch would launch for a batch of B matrices (for benchmarks and tests): out4 (host) receives
  * {kernel, CTAs, threads per CTA, dynamic shared memory bytes}.  kernel 0 = one CTA per matrix; kernel 1 = one
- * warp per matrix, chosen for topologies of at most four groups of four ranks once B exceeds the number of CTAs
- * that fit the GPU at once; kernel 2 = one CTA per matrix with 16-bit saturating credits in shared memory, chosen
+ * warp per matrix (one, two or four warps per CTA as B grows), chosen for topologies of at most four groups of four
+ * ranks when granule_bytes >= 256, and with smaller granules once B exceeds the number of CTAs that fit the GPU at
+ * once; kernel 2 = one CTA per matrix with 16-bit saturating credits in shared memory, chosen
  * for node-symmetric catalogs of more than sixteen groups of four ranks (a second launch of kernel 0 then takes the
  * matrices whose capacities or totals do not fit that representation).  All kernels produce identical plans.
  * CTAs is also the number of matrices in flight at once: a caller that splits a large batch into sub-batches

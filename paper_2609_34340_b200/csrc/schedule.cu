@@ -1251,11 +1251,13 @@ int plan_launch_uncached(const vp_catalog* c, int B, const vp_sched_params* p, L
     }
 #endif
 #ifndef VP_NO_WARP_KERNEL
-    // Small topologies (groups of four, at most four groups, plain D-hat scores) and more matrices than the
-    // CTAs of one wave: one warp per matrix gives up latency per matrix for three to four times as many
-    // matrices in flight, which is what counts once the batch no longer fits the GPU at once.
-    if (dc.g == 4 && dc.G <= 4 && !dc.sym && B > cap) {
-        const int warps = 4;
+    // Small topologies (groups of four, at most four groups, plain D-hat scores): one warp per matrix.  It has no block
+    // barriers and less work per activation than a CTA per matrix, and wins at every batch size once the matrices run
+    // in 32-bit granule units (granule >= 256 bytes; the choice between units and bytes is made per matrix, so the
+    // granule decides here); with smaller granules only when the batch exceeds the CTAs of one wave.  Up to four
+    // matrices per SM get a CTA of one warp each (a scheduler to themselves), larger batches two or four warps per CTA.
+    if (dc.g == 4 && dc.G <= 4 && !dc.sym && (B > cap || p->granule_bytes >= 256)) {
+        const int warps = B <= 4 * c->sm_count ? 1 : (B <= 8 * c->sm_count ? 2 : 4);
         const size_t smem = (size_t)warp_smem_layout(dc, L.kp, warps).total;
         if (smem + 2048 <= (size_t)c->max_smem_optin) {
             if (cudaFuncSetAttribute(vp_schedule_warp_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)

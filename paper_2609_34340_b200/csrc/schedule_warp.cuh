@@ -77,11 +77,39 @@ __device__ __forceinline__ int64_t team_max(int64_t v) {
     return max_v(v, __shfl_xor_sync(0xffffffffu, v, 2));
 }
 
+// Eq. (6) for the R shapes of a lane (shape lane + 32 u) from their lane counts, four bits per D-hat cell (cells 0..7 in
+// the first word, 8..15 in the second), against the cells themselves; S is the score type (32 bits while scores stay
+// below 2^31).  Cells are taken four at a time (a table has 1, 4, 9 or 16 of them; a cell beyond the table has count 0
+// in every shape, so what is read there does not matter).  Leaves the lane's first maximum in (best, best_s).
+template <int R, typename S>
+__device__ __forceinline__ void score_dense(const int64_t* Dhat, int tbl_size, const uint32_t (&smask)[4][2], int lane, int n_shapes,
+                                            int64_t& best, int& best_s) {
+    S sc[R];
+#pragma unroll
+    for (int u = 0; u < R; u++) sc[u] = 0;
+#pragma unroll
+    for (int quad = 0; quad < 4; quad++) {
+        if (quad * 4 < tbl_size) {
+#pragma unroll
+            for (int m = 0; m < 4; m++) {
+                const int cell = quad * 4 + m;
+                const S d = (S)Dhat[cell];
+#pragma unroll
+                for (int u = 0; u < R; u++) sc[u] += d * (S)((smask[u][cell >> 3] >> (4 * (cell & 7))) & 15u);
+            }
+        }
+    }
+#pragma unroll
+    for (int u = 0; u < R; u++)
+        if (lane + 32 * u < n_shapes && (int64_t)sc[u] > best) { best = (int64_t)sc[u]; best_s = lane + 32 * u; }
+}
+
 template <typename V>
 __device__ __forceinline__ void decompose_warp(const DevCat& dc, const KParams& kp, const WCtx& c, int64_t unit, int64_t left,
                                                int& k, int& st, Counters& cnt) {
     const int N = c.N, G = c.G, lane = c.lane;
-    const int ld = N + 1;                                // row stride of D_rem
+    // row stride of D_rem: N for 32-bit granules (a row's four credits of a group are one 16-byte load), N + 1 for bytes
+    const int ld = sizeof(V) == 4 ? N : N + 1;
     const int ns_pad = (dc.n_shapes + 31) & ~31;         // row stride of the transposed term table
     // Step 2 runs eight (family, start) tasks at a time: a team of four lanes per task, one lane per rank group, which
     // solves its group's exact 4 x 4 assignments on its own (best_assignment) -- no credit tiles, no hand-overs
@@ -114,36 +142,18 @@ __device__ __forceinline__ void decompose_warp(const DevCat& dc, const KParams& 
         // (A) Eq. (6): shape scores, first maximum
         int64_t best = -1;
         int best_s = 0x7fffffff;
+        const bool narrow_now = left < ((int64_t)1 << 31);       // every D-hat cell fits 32 bits
         if (dense) {
             const bool narrow = left * 4 < ((int64_t)1 << 31);   // a score is at most g x (what is left)
-            if (narrow) {
-                uint32_t sc[4] = {0u, 0u, 0u, 0u};
-#pragma unroll
-                for (int cell = 0; cell < 16; cell++) {
-                    if (cell < dc.tbl_size) {
-                        const uint32_t d = (uint32_t)Dhat[cell];
-#pragma unroll
-                        for (int u = 0; u < 4; u++)
-                            if (u < n_rounds) sc[u] += d * ((smask[u][cell >> 3] >> (4 * (cell & 7))) & 15u);
-                    }
-                }
-#pragma unroll
-                for (int u = 0; u < 4; u++)
-                    if (lane + 32 * u < dc.n_shapes && (int64_t)sc[u] > best) { best = (int64_t)sc[u]; best_s = lane + 32 * u; }
-            } else {
-                int64_t sc[4] = {0, 0, 0, 0};
-#pragma unroll
-                for (int cell = 0; cell < 16; cell++) {
-                    if (cell < dc.tbl_size) {
-                        const int64_t d = Dhat[cell];
-#pragma unroll
-                        for (int u = 0; u < 4; u++)
-                            if (u < n_rounds) sc[u] += d * (int64_t)((smask[u][cell >> 3] >> (4 * (cell & 7))) & 15u);
-                    }
-                }
-#pragma unroll
-                for (int u = 0; u < 4; u++)
-                    if (lane + 32 * u < dc.n_shapes && sc[u] > best) { best = sc[u]; best_s = lane + 32 * u; }
+            switch (n_rounds * 2 + (narrow ? 1 : 0)) {
+                case 3: score_dense<1, uint32_t>(Dhat, dc.tbl_size, smask, lane, dc.n_shapes, best, best_s); break;
+                case 5: score_dense<2, uint32_t>(Dhat, dc.tbl_size, smask, lane, dc.n_shapes, best, best_s); break;
+                case 7: score_dense<3, uint32_t>(Dhat, dc.tbl_size, smask, lane, dc.n_shapes, best, best_s); break;
+                case 9: score_dense<4, uint32_t>(Dhat, dc.tbl_size, smask, lane, dc.n_shapes, best, best_s); break;
+                case 2: score_dense<1, int64_t>(Dhat, dc.tbl_size, smask, lane, dc.n_shapes, best, best_s); break;
+                case 4: score_dense<2, int64_t>(Dhat, dc.tbl_size, smask, lane, dc.n_shapes, best, best_s); break;
+                case 6: score_dense<3, int64_t>(Dhat, dc.tbl_size, smask, lane, dc.n_shapes, best, best_s); break;
+                default: score_dense<4, int64_t>(Dhat, dc.tbl_size, smask, lane, dc.n_shapes, best, best_s); break;
             }
         } else {
             for (int s0 = lane; s0 < dc.n_shapes; s0 += 128) {     // four shapes per lane in flight
@@ -166,10 +176,12 @@ __device__ __forceinline__ void decompose_warp(const DevCat& dc, const KParams& 
                     if (s0 + 32 * u < dc.n_shapes && score[u] > best) { best = score[u]; best_s = s0 + 32 * u; }
             }
         }
+        VP_TICK(0);
         warp_argmax_first(best, best_s);
         if (best <= 0) { st |= VP_ST_UNCOVERED; break; }
         const int f0 = (int)ws<uint32_t>(c.o_bucket)[best_s], H = (int)ws<uint32_t>(c.o_bucket)[best_s + 1] - f0;
         const int n_tasks = H * kp.n_start;
+        VP_TICK(1);
 
         // (B) MultiStartAA, eight (family, start) tasks at a time; (C) best start per family, best family
         int64_t bf = -1, bd = 1, ff = -1, fd = 1;        // best family so far; best start of the current family
@@ -183,16 +195,19 @@ __device__ __forceinline__ void decompose_warp(const DevCat& dc, const KParams& 
             V cap_out[4], cap_in[4];
             int rq[4], cls_in[4];
             const int ag = active ? a : 0;                   // (spare lanes read group 0's tables and write nothing)
+            const uint2 fin4 = *(const uint2*)(ws<uint16_t>(c.o_fam_in) + f * N + ag * 4);        // four in-slots, 16 bits each
+            const uint32_t fcls4 = *(const uint32_t*)(ws<uint8_t>(c.o_fam_cls) + f * N + ag * 4);  // four out-slot classes
 #pragma unroll
             for (int q = 0; q < 4; q++) {
-                const unsigned w = ws<uint16_t>(c.o_fam_in)[f * N + ag * 4 + q];
-                cap_out[q] = cap[ws<uint8_t>(c.o_fam_cls)[f * N + ag * 4 + q]];
+                const unsigned w = ((q < 2 ? fin4.x : fin4.y) >> (16 * (q & 1))) & 0xffffu;
+                cap_out[q] = cap[(fcls4 >> (8 * q)) & 0xffu];
                 rq[q] = (int)(w & 0xffu);
                 cls_in[q] = (int)(w >> 8);
                 cap_in[q] = cap[cls_in[q]];
                 if (has) dstb[rq[q]] = (uint8_t)(a * 4 + ((q + tt) & 3));     // start t rotates the in-slots of every group
             }
             __syncwarp();
+            VP_TICK(2);
             int64_t F_old = -1, F_new = -1;
             bool alive = has;
             for (int sweep = 0; sweep < kp.i_aa && __any_sync(0xffffffffu, alive); sweep++) {
@@ -217,8 +232,14 @@ __device__ __forceinline__ void decompose_warp(const DevCat& dc, const KParams& 
 #pragma unroll
                     for (int q = 0; q < 4; q++) {
                         const V* row = Drem + (int)srcb[rq[q]] * ld + a * 4;
+                        if constexpr (sizeof(V) == 4) {
+                            const uint4 r4 = *(const uint4*)row;
+                            cm[0][q] = min_v((V)r4.x, cap_in[q]); cm[1][q] = min_v((V)r4.y, cap_in[q]);
+                            cm[2][q] = min_v((V)r4.z, cap_in[q]); cm[3][q] = min_v((V)r4.w, cap_in[q]);
+                        } else {
 #pragma unroll
-                        for (int i = 0; i < 4; i++) cm[i][q] = min_v(row[i], cap_in[q]);
+                            for (int i = 0; i < 4; i++) cm[i][q] = min_v(row[i], cap_in[q]);
+                        }
                     }
                     unsigned bpk;
                     part = best_assignment<4, V>(cm, bpk);
@@ -234,6 +255,7 @@ __device__ __forceinline__ void decompose_warp(const DevCat& dc, const KParams& 
                 }
                 __syncwarp();
             }
+            VP_TICK(3);
             // Evaluate (Eq. 9, 10), needed only when several families compete: the volume of every in-slot of this
             // lane's group under the final bindings, the slowest lane over the team
             int64_t den = 1;
@@ -276,6 +298,7 @@ __device__ __forceinline__ void decompose_warp(const DevCat& dc, const KParams& 
         }
         if (cur_h >= 0 && (bt < 0 || util_greater(ff, fd, bf, bd))) { bf = ff; bd = fd; bt = ft; }   // lowest family on ties
         if (bf <= 0) { st |= VP_ST_NO_PROGRESS; break; }
+        VP_TICK(4);
 
         // (D) emit activation k, D_rem -= X(E), write offset row k+1, re-sum D-hat
         {
@@ -294,6 +317,11 @@ __device__ __forceinline__ void decompose_warp(const DevCat& dc, const KParams& 
                 c.lane_inst_b[row + i] = busy ? (uint16_t)(w & 0xffffu) : (uint16_t)0xFFFF;
                 c.lane_bytes_b[row + i] = bytes;
                 Drem[i * ld + j] -= x;
+                if (busy) {                                   // Eq. (5): the volume leaves its group pair's cell of D-hat
+                    int64_t* cell = &Dhat[(i >> 2) * G + (j >> 2)];
+                    if (narrow_now) atomicSub((unsigned int*)cell, (unsigned int)x);     // high word is zero, low word >= x
+                    else atomicAdd((unsigned long long*)cell, (unsigned long long)(-(int64_t)x));
+                }
                 ws<int64_t>(c.o_send_acc)[i] = sa;
                 ws<int64_t>(c.o_recv_acc)[j] = ra;
                 c.send_off_b[orow + i] = sa;
@@ -302,22 +330,10 @@ __device__ __forceinline__ void decompose_warp(const DevCat& dc, const KParams& 
             if (lane == 0) c.chan_id_b[k] = f0 + h;
             left -= bf;
             __syncwarp();
-            {   // Eq. (5): two lanes per cell, eight entries each
-                const int cell = lane >> 1, half = lane & 1;
-                int64_t s = 0;
-                if (cell < G * G) {
-                    const int ga = cell / G, gd = cell - ga * G;
-#pragma unroll
-                    for (int ii = 0; ii < 2; ii++)
-#pragma unroll
-                        for (int jj = 0; jj < 4; jj++) s += (int64_t)Drem[(ga * 4 + half * 2 + ii) * ld + gd * 4 + jj];
-                }
-                s += __shfl_xor_sync(0xffffffffu, s, 1);
-                if (cell < G * G && half == 0) Dhat[cell] = s;
-            }
         }
         k++;
         __syncwarp();
+        VP_TICK(5);
     }
 }
 
@@ -393,6 +409,7 @@ vp_schedule_warp_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ deman
     unsigned long long n_act = 0;
     Counters cnt;
     cnt.tasks = 0; cnt.sweeps = 0; cnt.t_mark = 0;
+    for (int i = 0; i < 6; i++) cnt.cyc[i] = 0;
 
     for (;;) {
         int b = 0;
@@ -431,6 +448,9 @@ vp_schedule_warp_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ deman
         __syncwarp();
         int st = flags, k = 0;
         int64_t tau = 0;
+#ifdef VP_PHASE_TIMING
+        cnt.t_mark = clock64();
+#endif
         if (st == 0) {
             // ---- row / column sums, group sums (Eq. 5), quantum (Section 5)
             int64_t est = 0, tot = 0;
@@ -483,7 +503,7 @@ vp_schedule_warp_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ deman
             if (units) {
                 // the byte copy is no longer needed: overwrite it with the demand in granules
                 uint32_t* Drem32 = (uint32_t*)Drem;
-                for (int e = lane; e < N * N; e += 32) Drem32[(e / N) * ld + e % N] = (uint32_t)(D[e] / kp.granule);
+                for (int e = lane; e < N * N; e += 32) Drem32[e] = (uint32_t)(D[e] / kp.granule);   // (row stride N)
                 for (int cell = lane; cell < G * G; cell += 32) Dhat[cell] /= kp.granule;
                 __syncwarp();
                 c.o_cap = base + L.cap32;
@@ -518,6 +538,9 @@ vp_schedule_warp_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ deman
     if (lane == 0) {
         if (n_act) atomicAdd(&stats[0], n_act);
         if (cnt.tasks) { atomicAdd(&stats[1], cnt.tasks); atomicAdd(&stats[2], cnt.sweeps); }
+#ifdef VP_PHASE_TIMING
+        for (int i = 0; i < 6; i++) atomicAdd(&stats[3 + i], (unsigned long long)cnt.cyc[i]);
+#endif
     }
 }
 

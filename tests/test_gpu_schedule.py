@@ -607,24 +607,32 @@ def test_plan_arrays_at_odd_addresses(vp, oracle_lib):
 
 
 def test_batches_around_one_wave(vp, oracle_lib):
-    """Batch sizes just below and above the number of resident CTAs: the kernel changes, the plans do not."""
+    """Batch sizes just below and above the number of resident CTAs: the launch changes (a warp or a CTA per matrix, one
+    to four warps per CTA), the plans do not.  With the configuration's own granule every batch takes the warp kernel;
+    with a granule below 256 bytes the small batches take a CTA per matrix."""
     c = build_config(2)
-    cat, w = c["catalog"], c["params"]
+    cat, w0 = c["catalog"], c["params"]
     oc = oracle_lib.OracleCatalog(cat.topology.blob(), cat.blob())
     dc = vp.load_catalog(cat.topology.blob(), cat.blob())
     base = c["demand"][:37]
-    want = oc.schedule_batch(base.numpy(), w, threads=8)
-    p = _params(vp, w)
-    kernels = set()
-    for B in (591, 592, 593, 1187):
-        D = base.repeat((B + 36) // 37, 1, 1)[:B].contiguous()
-        kernels.add(vp.schedule_launch_info(dc, B, p)["kernel"])
-        got = vp.schedule_batch(dc, p, D.cuda()).cpu()
-        for key in KEYS:
-            for r0 in range(0, B, 37):
-                n = min(37, B - r0)
-                assert np.array_equal(got[key][r0:r0 + n], want[key][:n]), (B, key, r0)
-    assert kernels == {"CTA per matrix", "warp per matrix"}
+    for granule, expect in ((w0.granule_bytes, {"warp per matrix"}), (64, {"CTA per matrix", "warp per matrix"})):
+        w = WParams(granule_bytes=granule, k_max=w0.k_max).resolved(cat.topology.N)
+        want = oc.schedule_batch(base.numpy(), w, threads=8)
+        p = _params(vp, w)
+        kernels, threads = set(), set()
+        for B in (147, 591, 592, 593, 1187, 1190):
+            D = base.repeat((B + 36) // 37, 1, 1)[:B].contiguous()
+            info = vp.schedule_launch_info(dc, B, p)
+            kernels.add(info["kernel"])
+            threads.add(info["threads"])
+            got = vp.schedule_batch(dc, p, D.cuda()).cpu()
+            for key in KEYS:
+                for r0 in range(0, B, 37):
+                    n = min(37, B - r0)
+                    assert np.array_equal(got[key][r0:r0 + n], want[key][:n]), (granule, B, key, r0)
+        assert kernels == expect
+        if granule >= 256:
+            assert threads == {32, 64, 128}            # one, two and four warps per CTA
 
 
 def test_randomised_topologies_and_parameters(vp, oracle_lib):
