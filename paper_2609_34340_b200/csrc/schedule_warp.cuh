@@ -17,7 +17,7 @@ namespace {
 
 
 struct WarpSmem {                           // byte offsets; the per-warp block comes first, once per warp
-    int drem, dhat, send_acc, recv_acc, cred, cap64, tscale, cap32, bind_src, bind_dst, per_warp;
+    int drem, dremT, dhat, send_acc, recv_acc, cred, cap64, tscale, cap32, bind_src, bind_dst, per_warp;
     int term, fam_in, fam_cls, fam_slot, bucket, lut, total;
 };
 
@@ -25,6 +25,7 @@ __host__ __device__ inline WarpSmem warp_smem_layout(const DevCat& dc, const KPa
     WarpSmem L;
     int o = 0;
     L.drem = o;      o += align16(dc.N * (dc.N + 1) * 8);      // rows padded by one element: no bank conflicts down a column
+    L.dremT = o;     o += align16(dc.N * dc.N * 4);            // 32-bit granules: the transpose (a column's four credits of a group in 16 bytes)
     L.dhat = o;      o += align16(dc.G * dc.G * 8);
     L.send_acc = o;  o += dc.N * 8;
     L.recv_acc = o;  o += dc.N * 8;
@@ -53,7 +54,7 @@ extern __shared__ __align__(16) unsigned char vp_wsmem[];   // the CTA's dynamic
 // pointers: every access is then provably a shared-memory access with a 32-bit address.
 struct WCtx {
     int N, G, lane;
-    unsigned o_drem, o_dhat, o_send_acc, o_recv_acc, o_cred, o_cap, o_tscale, o_bind_src, o_bind_dst;
+    unsigned o_drem, o_dremT, o_dhat, o_send_acc, o_recv_acc, o_cred, o_cap, o_tscale, o_bind_src, o_bind_dst;
     unsigned o_term, o_fam_slot, o_fam_in, o_fam_cls, o_bucket, o_lut;
     int32_t* chan_id_b;
     int16_t* lane_dst_b;
@@ -118,6 +119,7 @@ __device__ __forceinline__ void decompose_warp(const DevCat& dc, const KParams& 
     const bool active = a < G;
     const int ns_shift = (kp.n_start & (kp.n_start - 1)) == 0 ? 31 - __clz(kp.n_start) : -1;
     V* const Drem = ws<V>(c.o_drem);
+    uint32_t* const DremT = ws<uint32_t>(c.o_dremT);      // (32-bit granules only) DremT[j * N + i] = Drem[i * N + j]
     const V* const cap = ws<V>(c.o_cap);
     int64_t* const Dhat = ws<int64_t>(c.o_dhat);
     // Plain score tables of at most 16 D-hat cells and at most 128 shapes: a lane keeps the lane counts of its (up to
@@ -216,9 +218,16 @@ __device__ __forceinline__ void decompose_warp(const DevCat& dc, const KParams& 
                     V cm[4][4];
 #pragma unroll
                     for (int q = 0; q < 4; q++) {
-                        const V* col = Drem + (a * 4) * ld + ((d4 >> (8 * q)) & 0xffu);
+                        const int dq = (int)((d4 >> (8 * q)) & 0xffu);
+                        if constexpr (sizeof(V) == 4) {
+                            const uint4 c4 = *(const uint4*)(DremT + dq * N + a * 4);
+                            cm[0][q] = min_v((V)c4.x, cap_out[q]); cm[1][q] = min_v((V)c4.y, cap_out[q]);
+                            cm[2][q] = min_v((V)c4.z, cap_out[q]); cm[3][q] = min_v((V)c4.w, cap_out[q]);
+                        } else {
+                            const V* col = Drem + (a * 4) * ld + dq;
 #pragma unroll
-                        for (int i = 0; i < 4; i++) cm[i][q] = min_v(col[i * ld], cap_out[q]);
+                            for (int i = 0; i < 4; i++) cm[i][q] = min_v(col[i * ld], cap_out[q]);
+                        }
                     }
                     unsigned bpk;
                     best_assignment<4, V>(cm, bpk);
@@ -317,6 +326,7 @@ __device__ __forceinline__ void decompose_warp(const DevCat& dc, const KParams& 
                 c.lane_inst_b[row + i] = busy ? (uint16_t)(w & 0xffffu) : (uint16_t)0xFFFF;
                 c.lane_bytes_b[row + i] = bytes;
                 Drem[i * ld + j] -= x;
+                if constexpr (sizeof(V) == 4) DremT[j * N + i] -= (uint32_t)x;
                 if (busy) {                                   // Eq. (5): the volume leaves its group pair's cell of D-hat
                     int64_t* cell = &Dhat[(i >> 2) * G + (j >> 2)];
                     if (narrow_now) atomicSub((unsigned int*)cell, (unsigned int)x);     // high word is zero, low word >= x
@@ -394,7 +404,7 @@ vp_schedule_warp_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ deman
     WCtx c;
     c.N = N; c.G = G; c.lane = lane;
     const unsigned base = (unsigned)warp * (unsigned)L.per_warp;
-    c.o_drem = base + L.drem; c.o_dhat = base + L.dhat; c.o_send_acc = base + L.send_acc; c.o_recv_acc = base + L.recv_acc;
+    c.o_drem = base + L.drem; c.o_dremT = base + L.dremT; c.o_dhat = base + L.dhat; c.o_send_acc = base + L.send_acc; c.o_recv_acc = base + L.recv_acc;
     c.o_cred = base + L.cred; c.o_tscale = base + L.tscale; c.o_bind_src = base + L.bind_src; c.o_bind_dst = base + L.bind_dst;
     c.o_cap = base + L.cap64;
     c.o_term = L.term; c.o_fam_slot = L.fam_slot; c.o_fam_in = L.fam_in; c.o_fam_cls = L.fam_cls; c.o_bucket = L.bucket;
@@ -503,7 +513,13 @@ vp_schedule_warp_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ deman
             if (units) {
                 // the byte copy is no longer needed: overwrite it with the demand in granules
                 uint32_t* Drem32 = (uint32_t*)Drem;
-                for (int e = lane; e < N * N; e += 32) Drem32[e] = (uint32_t)(D[e] / kp.granule);   // (row stride N)
+                uint32_t* DremT32 = ws<uint32_t>(c.o_dremT);
+                for (int e = lane; e < N * N; e += 32) {                                            // (row stride N, and the transpose)
+                    const uint32_t v = (uint32_t)(D[e] / kp.granule);
+                    const int i = e / N, j = e - i * N;
+                    Drem32[e] = v;
+                    DremT32[j * N + i] = v;
+                }
                 for (int cell = lane; cell < G * G; cell += 32) Dhat[cell] /= kp.granule;
                 __syncwarp();
                 c.o_cap = base + L.cap32;
