@@ -1129,8 +1129,8 @@ vp_schedule_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand, co
 
 }  // namespace
 
-#include "schedule_warp.cuh"
 #include "schedule_big.cuh"
+#include "schedule_warp.cuh"
 
 #ifndef VP_BIG_MIN_GROUPS
 #define VP_BIG_MIN_GROUPS 16      // node-symmetric catalogs with at least this many groups of four take vp_schedule_big_kernel

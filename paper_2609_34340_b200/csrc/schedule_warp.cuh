@@ -229,10 +229,21 @@ __device__ __forceinline__ void decompose_warp(const DevCat& dc, const KParams& 
                             for (int i = 0; i < 4; i++) cm[i][q] = min_v(col[i * ld], cap_out[q]);
                         }
                     }
-                    unsigned bpk;
-                    best_assignment<4, V>(cm, bpk);
-                    *(uint32_t*)(srcb + a * 4) = (uint32_t)(a * 4) * 0x01010101u +
-                        ((bpk & 3u) | ((bpk >> 2) & 3u) << 8 | ((bpk >> 4) & 3u) << 16 | ((bpk >> 6) & 3u) << 24);
+                    uint32_t rows4;                          // the row bound to position q, in byte q
+                    if constexpr (sizeof(V) == 4) {
+                        uint32_t v[4][4];
+#pragma unroll
+                        for (int i = 0; i < 4; i++)
+#pragma unroll
+                            for (int q = 0; q < 4; q++) v[i][q] = (uint32_t)cm[i][q] * 256u + big_tag(i, q);
+                        const uint32_t pb = ~big_best_key(v) & 255u;      // position 0 in the two highest bits
+                        rows4 = ((pb >> 6) & 3u) | ((pb << 4) & 0x300u) | ((pb << 14) & 0x30000u) | ((pb << 24) & 0x3000000u);
+                    } else {
+                        unsigned bpk;
+                        best_assignment<4, V>(cm, bpk);
+                        rows4 = (bpk & 3u) | ((bpk >> 2) & 3u) << 8 | ((bpk >> 4) & 3u) << 16 | ((bpk >> 6) & 3u) << 24;
+                    }
+                    *(uint32_t*)(srcb + a * 4) = (uint32_t)(a * 4) * 0x01010101u + rows4;
                 }
                 __syncwarp();
                 V part = 0;
@@ -250,10 +261,22 @@ __device__ __forceinline__ void decompose_warp(const DevCat& dc, const KParams& 
                             for (int i = 0; i < 4; i++) cm[i][q] = min_v(row[i], cap_in[q]);
                         }
                     }
-                    unsigned bpk;
-                    part = best_assignment<4, V>(cm, bpk);
+                    if constexpr (sizeof(V) == 4) {
+                        uint32_t v[4][4];
 #pragma unroll
-                    for (int q = 0; q < 4; q++) dstb[rq[q]] = (uint8_t)(a * 4 + ((bpk >> (2 * q)) & 3u));
+                        for (int i = 0; i < 4; i++)
+#pragma unroll
+                            for (int q = 0; q < 4; q++) v[i][q] = (uint32_t)cm[i][q] * 256u + big_tag(i, q);
+                        const uint32_t key = big_best_key(v), pb = ~key & 255u;
+                        part = (V)(key >> 8);
+#pragma unroll
+                        for (int q = 0; q < 4; q++) dstb[rq[q]] = (uint8_t)(a * 4 + ((pb >> (6 - 2 * q)) & 3u));
+                    } else {
+                        unsigned bpk;
+                        part = best_assignment<4, V>(cm, bpk);
+#pragma unroll
+                        for (int q = 0; q < 4; q++) dstb[rq[q]] = (uint8_t)(a * 4 + ((bpk >> (2 * q)) & 3u));
+                    }
                 }
                 const int64_t Fn = (int64_t)team_sum(part);   // Eq. (8)
                 if (alive) {
