@@ -31,6 +31,7 @@
 #include <cuda_runtime.h>
 
 #include <cstring>
+#include <mutex>
 #include <utility>
 
 #include "bulk_copy.cuh"
@@ -1175,6 +1176,27 @@ BigKernelFn pick_big_kernel(int w, bool dec) {
     return w == 2 ? vp_schedule_big_kernel<2, false> : vp_schedule_big_kernel<1, false>;
 }
 
+// Raises a kernel's limit of dynamic shared memory on the current device to `bytes` if it is lower.  The limit belongs
+// to the function, not to a launch: launches are planned once and replayed from a memo, several catalogs share the
+// kernels, and one kernel is launched with different sizes, so the limit must never be lowered by a later plan.
+int raise_dynamic_smem(const void* fn, size_t bytes) {
+    struct Mark { int device; const void* fn; size_t bytes; };
+    static Mark marks[64];
+    static int n_marks = 0;
+    static std::mutex lock;
+    std::lock_guard<std::mutex> hold(lock);
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return VP_E_CUDA;
+    Mark* m = nullptr;
+    for (int i = 0; i < n_marks; i++)
+        if (marks[i].device == dev && marks[i].fn == fn) m = &marks[i];
+    if (m && m->bytes >= bytes) return VP_OK;
+    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess) return VP_E_CUDA;
+    if (m) m->bytes = bytes;
+    else if (n_marks < 64) marks[n_marks++] = Mark{dev, fn, bytes};
+    return VP_OK;
+}
+
 int resolve_params(const vp_catalog* c, const vp_sched_params* p, KParams* kp) {
     if (!c || !p || c->device < 0) return VP_E_BAD_ARG;         // (a host-only handle launches nothing)
     if (p->k_max <= 0 || p->granule_bytes <= 0 || p->lambda_ns < 0 || p->lambda_ns >= VP_ENTRY_LIMIT) return VP_E_BAD_ARG;
@@ -1221,7 +1243,7 @@ int plan_launch_uncached(const vp_catalog* c, int B, const vp_sched_params* p, L
     if (L.smem + 2048 > (size_t)c->max_smem_optin) return VP_E_UNSUPPORTED;
     KernelFn fn = pick_kernel(dc.g, L.lpg);
     if (!fn) return VP_E_UNSUPPORTED;
-    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.smem) != cudaSuccess) return VP_E_CUDA;
+    if (raise_dynamic_smem((const void*)fn, L.smem) != VP_OK) return VP_E_CUDA;
     int per_sm = 0;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, L.threads, L.smem) != cudaSuccess || per_sm < 1)
         return VP_E_CUDA;
@@ -1240,7 +1262,7 @@ int plan_launch_uncached(const vp_catalog* c, int B, const vp_sched_params* p, L
             const int w = dc.G > 32 ? 2 : 1;
             const int threads = w == 2 ? BIG_W2_THREADS : (dc.G > 16 ? 256 : 128);
             BigKernelFn bf = pick_big_kernel(w, big_use_dec(dc));
-            if (cudaFuncSetAttribute(bf, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return VP_E_CUDA;
+            if (raise_dynamic_smem((const void*)bf, smem) != VP_OK) return VP_E_CUDA;
             int bper_sm = 0;
             if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&bper_sm, bf, threads, smem) != cudaSuccess || bper_sm < 1) return VP_E_CUDA;
             const long long bcap = (long long)bper_sm * c->sm_count;
@@ -1260,8 +1282,7 @@ int plan_launch_uncached(const vp_catalog* c, int B, const vp_sched_params* p, L
         const int warps = B <= 4 * c->sm_count ? 1 : (B <= 8 * c->sm_count ? 2 : 4);
         const size_t smem = (size_t)warp_smem_layout(dc, L.kp, warps).total;
         if (smem + 2048 <= (size_t)c->max_smem_optin) {
-            if (cudaFuncSetAttribute(vp_schedule_warp_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-                return VP_E_CUDA;
+            if (raise_dynamic_smem((const void*)vp_schedule_warp_kernel, smem) != VP_OK) return VP_E_CUDA;
             int wper_sm = 0;
             if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&wper_sm, vp_schedule_warp_kernel, warps * 32, smem) != cudaSuccess || wper_sm < 1)
                 return VP_E_CUDA;

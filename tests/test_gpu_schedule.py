@@ -635,6 +635,29 @@ def test_batches_around_one_wave(vp, oracle_lib):
             assert threads == {32, 64, 128}            # one, two and four warps per CTA
 
 
+def test_launches_of_different_sizes_interleaved(vp, oracle_lib):
+    """A large batch, a single matrix and the large batch again, on two catalogs that share a kernel: launches are
+    replayed from a memo with different amounts of dynamic shared memory, and a later, smaller plan must not shrink
+    what an earlier one needs."""
+    c2, c1 = build_config(2), build_config(1)
+    oc = oracle_lib.OracleCatalog(c2["catalog"].topology.blob(), c2["catalog"].blob())
+    dc2 = vp.load_catalog(c2["catalog"].topology.blob(), c2["catalog"].blob())
+    dc1 = vp.load_catalog(c1["catalog"].topology.blob(), c1["catalog"].blob())
+    p2, p1 = _params(vp, c2["params"]), _params(vp, c1["params"])
+    base = c2["demand"][:16]
+    want = oc.schedule_batch(base.numpy(), c2["params"], threads=8)
+    big = base.repeat(80, 1, 1).contiguous().cuda()            # 1280 matrices: four warps per CTA, the most shared memory
+    for B in (1280, 1, 1280, 300, 1280):
+        if B == 300:
+            vp.schedule_batch(dc1, p1, c1["demand"][:8].cuda())    # another catalog plans the same kernel with less
+        got = vp.schedule_batch(dc2, p2, big[:B].contiguous()).cpu()
+        torch.cuda.synchronize()
+        for key in KEYS:
+            for r0 in range(0, B, 16):
+                n = min(16, B - r0)
+                assert np.array_equal(got[key][r0:r0 + n], want[key][:n]), (B, key, r0)
+
+
 def test_randomised_topologies_and_parameters(vp, oracle_lib):
     """A seeded sweep over group sizes 1..4, complete and node-template catalogs, mixed rates, granules, densities,
     AA parameters, tau overrides and batch sizes on both sides of one wave: every plan equals the oracle's."""
