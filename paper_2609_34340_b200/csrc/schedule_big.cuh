@@ -324,6 +324,7 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
         __syncthreads();
     }
     const int ns_shift = (kp.n_start & (kp.n_start - 1)) == 0 ? 31 - __clz(kp.n_start) : -1;
+    const bool tpw2 = W == 1 && G <= 16;                 // two tasks per warp in Step 2 (see there)
     // Issues up to `batches` x 32 of the pending copies (one per lane) and commits them; FILL_WARP only.
     auto fill_step = [&](int batches) {
         const int R = L.fill_rows, rows = s_job_rows, total = s_job_total;
@@ -545,7 +546,8 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
             // warps, which has no task in Step 2 as a rule, copies them out during Step 2 of the next iteration.  (Plain
             // stores to global memory by the emitting warps, just before a CTA-wide barrier, made every iteration wait
             // for them: 6 % of the run time.)
-            const int copy_warp0 = max(kp.n_start * W, (N + 31) >> 5);     // first warp with neither a task nor a slot to emit
+            // first warp with neither a task nor a slot to emit
+            const int copy_warp0 = max(tpw2 ? (kp.n_start + 1) >> 1 : kp.n_start * W, (N + 31) >> 5);
             const bool rows_async = N % 8 == 0 && copy_warp0 < n_warps &&
                 (((uintptr_t)lane_dst_b | (uintptr_t)lane_inst_b | (uintptr_t)lane_bytes_b | (uintptr_t)send_off_b |
                   (uintptr_t)(recv_off_b ? recv_off_b : send_off_b)) & 15) == 0;
@@ -665,6 +667,162 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
                     if (W == 2) asm volatile("bar.sync %0, 64;" ::"r"(1 + wgroup) : "memory");
                     else __syncwarp();
                 };
+                if (tpw2) {
+                    // Up to sixteen groups: two tasks share a warp, sixteen lanes each (half the warps then carry Step 2 and
+                    // half the instructions are issued for it).  A task that ends is switched off lane by lane; votes and
+                    // sums run over the task's half of the warp.
+                    const int half = lane >> 4, a2 = lane & 15;
+                    const unsigned hmask = half ? 0xffff0000u : 0x0000ffffu;
+                    for (int task0 = warp * 2; task0 < n_tasks; task0 += n_warps * 2) {
+                        const bool has = task0 + half < n_tasks && a2 < G;
+                        const int task = min(task0 + half, n_tasks - 1);
+                        const int h = ns_shift >= 0 ? task >> ns_shift : task / kp.n_start, f = f0 + h, t = task - h * kp.n_start;
+                        uint8_t* srcb = bind_src + (size_t)task * N;
+                        uint8_t* dstb = bind_dst + (size_t)task * N;
+                        const int ag = a2 < G ? a2 : 0;
+                        uint32_t cap_out[4], cap_in[4];
+                        int rq[4], cls_in[4];
+                        uint32_t my_dst = 0, my_src = 0;
+                        uint32_t hot_in = 0xffffffffu;
+                        if (hot_mode && has) hot_in = *((const uint32_t*)colmap + a2);
+                        {
+                            const uint32_t co = __ldg((const uint32_t*)(dc.fam_cls + (size_t)f * N) + ag);
+                            const uint2 fi = __ldg((const uint2*)(dc.fam_in + (size_t)f * N) + ag);
+                            if (t == 0 && has) {                  // the family's slot words, parked for step (D)
+                                const uint4 sw = __ldg((const uint4*)(dc.fam_slot + (size_t)f * N) + a2);
+                                *((uint4*)(slotw + h * N) + a2) = sw;
+                            }
+                            const uint32_t fw[4] = {fi.x & 0xffffu, fi.x >> 16, fi.y & 0xffffu, fi.y >> 16};
+#pragma unroll
+                            for (int q = 0; q < 4; q++) {
+                                cap_out[q] = s_cap[(co >> (8 * q)) & 0xffu];
+                                rq[q] = (int)(fw[q] & 0xffu);
+                                cls_in[q] = (int)(fw[q] >> 8);
+                                cap_in[q] = s_cap[cls_in[q]];
+                                const uint32_t d = (uint32_t)(a2 * 4 + ((q + t) & 3));
+                                if (has) dstb[rq[q]] = (uint8_t)d;
+                                my_dst |= d << (8 * q);
+                            }
+                        }
+                        __syncwarp();
+                        int64_t F_old = -1, F_new = -1;
+                        bool alive = has;
+                        for (int sweep = 0; sweep < kp.i_aa && __any_sync(0xffffffffu, alive); sweep++) {
+                            bool moved = false;
+                            if (alive) {                          // source half
+                                const uint32_t d4 = *((const uint32_t*)dstb + a2);
+                                uint32_t v[4][4];
+#pragma unroll
+                                for (int q = 0; q < 4; q++) {
+                                    const uint16_t* colp = Cs + (a2 * 4) * CS + ((d4 >> (8 * q)) & 0xffu);
+#pragma unroll
+                                    for (int i = 0; i < 4; i++) v[i][q] = min_v((uint32_t)colp[i * CS], cap_out[q]) * 256u + big_tag(i, q);
+                                }
+                                if (hot_mode) {
+#pragma unroll
+                                    for (int q = 0; q < 4; q++) {
+                                        const int dq = (int)((d4 >> (8 * q)) & 0xffu), hc = colmap[dq];
+                                        if (hc != 0xFF) {
+#pragma unroll
+                                            for (int i = 0; i < 4; i++) {
+                                                const uint32_t val = (uint32_t)Cs[(a2 * 4 + i) * CS + dq] | (uint32_t)Hi[hc * N + a2 * 4 + i] << 16;
+                                                v[i][q] = min_v(val, cap_out[q]) * 256u + big_tag(i, q);
+                                            }
+                                        }
+                                    }
+                                }
+                                const uint32_t pb = ~big_best_key(v) & 255u;
+                                const uint32_t word = (uint32_t)(a2 * 4) * 0x01010101u +
+                                                      (((pb >> 6) & 3u) | (((pb >> 4) & 3u) << 8) | (((pb >> 2) & 3u) << 16) | ((pb & 3u) << 24));
+                                moved = sweep == 0 || word != my_src;
+                                my_src = word;
+                                *((uint32_t*)srcb + a2) = word;
+                            }
+                            __syncwarp();
+                            // no source binding of the task moved: the destination half would repeat itself (see below)
+                            const bool any_moved = __any_sync(hmask, moved);
+                            if (alive && !any_moved) {
+                                if (a2 == 0) n_sweeps++;
+                                F_new = F_old;
+                                alive = false;
+                            }
+                            uint32_t part = 0;
+                            moved = false;
+                            if (alive) {                          // destination half
+                                uint32_t v[4][4];
+#pragma unroll
+                                for (int q = 0; q < 4; q++) {
+                                    const uint32_t* rowp = (const uint32_t*)(Cs + (int)srcb[rq[q]] * CS + a2 * 4);
+                                    const uint32_t c2 = min_v(cap_in[q], 65535u) * 0x00010001u;
+                                    const uint32_t lo = __vminu2(rowp[0], c2), hi = __vminu2(rowp[1], c2);
+                                    v[0][q] = __byte_perm(lo, big_tag(0, q), 0x5104);
+                                    v[1][q] = __byte_perm(lo, big_tag(1, q), 0x5324);
+                                    v[2][q] = __byte_perm(hi, big_tag(2, q), 0x5104);
+                                    v[3][q] = __byte_perm(hi, big_tag(3, q), 0x5324);
+                                }
+                                if (hot_in != 0xffffffffu) {
+#pragma unroll
+                                    for (int j = 0; j < 4; j++) {
+                                        const int hc = (int)((hot_in >> (8 * j)) & 0xffu);
+                                        if (hc != 0xFF) {
+#pragma unroll
+                                            for (int q = 0; q < 4; q++) {
+                                                const int sq = srcb[rq[q]];
+                                                const uint32_t val = (uint32_t)Cs[sq * CS + a2 * 4 + j] | (uint32_t)Hi[hc * N + sq] << 16;
+                                                v[j][q] = min_v(val, cap_in[q]) * 256u + big_tag(j, q);
+                                            }
+                                        }
+                                    }
+                                }
+                                const uint32_t key = big_best_key(v);
+                                const uint32_t pb = ~key & 255u;
+                                part = key >> 8;
+                                uint32_t word = 0;
+#pragma unroll
+                                for (int q = 0; q < 4; q++) {
+                                    const uint32_t d = (uint32_t)(a2 * 4) + ((pb >> (6 - 2 * q)) & 3u);
+                                    dstb[rq[q]] = (uint8_t)d;
+                                    word |= d << (8 * q);
+                                }
+                                moved = word != my_dst;
+                                my_dst = word;
+                            }
+                            const uint32_t fm = __reduce_add_sync(hmask, part) << 1 | (uint32_t)__any_sync(hmask, moved);
+                            __syncwarp();
+                            if (alive) {
+                                F_new = (int64_t)(fm >> 1);
+                                if (a2 == 0) n_sweeps++;
+                                if (F_new <= F_old) alive = false;
+                                else {
+                                    F_old = F_new;
+                                    if (!(fm & 1u) && sweep + 1 < kp.i_aa) {   // no destination binding moved: the next sweep would repeat this one
+                                        if (a2 == 0) n_sweeps++;
+                                        alive = false;
+                                    }
+                                }
+                            }
+                        }
+                        int64_t tmax = 0;
+                        if (H > 1) {                              // Eq. (9), (10) over the task's sixteen lanes
+                            if (has) {
+#pragma unroll 1
+                                for (int q = 0; q < 4; q++) {
+                                    const int sq = srcb[rq[q]], dq = dstb[rq[q]];
+                                    uint32_t val = Cs[sq * CS + dq];
+                                    if (hot_mode && colmap[dq] != 0xFF) val |= (uint32_t)Hi[(int)colmap[dq] * N + sq] << 16;
+                                    tmax = max_v(tmax, (int64_t)min_v(val, cap_in[q]) * s_tscale[cls_in[q]]);
+                                }
+                            }
+#pragma unroll
+                            for (int o = 8; o; o >>= 1) tmax = max_v(tmax, __shfl_xor_sync(0xffffffffu, tmax, o));
+                        }
+                        if (has && a2 == 0) {
+                            n_tasks_done++;
+                            task_f[task] = F_new;
+                            task_den[task] = F_new > 0 ? kp.lambda_ns * dc.W + tmax : 1;
+                        }
+                    }
+                } else
                 for (int task = wgroup; task < n_tasks; task += n_warps / W) {
                     const int h = ns_shift >= 0 ? task >> ns_shift : task / kp.n_start, f = f0 + h, t = task - h * kp.n_start;
                     uint8_t* srcb = bind_src + (size_t)task * N;
@@ -985,6 +1143,8 @@ vp_schedule_big_kernel(DevCat dc, KParams kp, const int64_t* __restrict__ demand
     bulk_wait_all();
     unsigned long long* stats = (unsigned long long*)(counter + 4);
     if (tid == 0 && n_act) atomicAdd(&stats[0], n_act);
+    n_tasks_done = (unsigned long long)warp_sum_i64((int64_t)n_tasks_done);    // (counted by the first lane of every task)
+    n_sweeps = (unsigned long long)warp_sum_i64((int64_t)n_sweeps);
     if (lane == 0 && n_tasks_done) { atomicAdd(&stats[1], n_tasks_done); atomicAdd(&stats[2], n_sweeps); }
 #ifdef VP_PHASE_TIMING
     if (tid == 0) for (int i = 0; i < 6; i++) atomicAdd(&stats[3 + i], (unsigned long long)cnt.cyc[i]);
