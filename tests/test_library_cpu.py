@@ -39,7 +39,7 @@ def _load(lib, topo, chan):
     h = ctypes.c_void_p()
     lib.vp_load_catalog.argtypes = [ctypes.c_char_p, ctypes.c_size_t, ctypes.c_char_p, ctypes.c_size_t,
                                     ctypes.c_int, ctypes.POINTER(ctypes.c_void_p)]
-    rc = lib.vp_load_catalog(topo, len(topo), chan, len(chan), 0, ctypes.byref(h))
+    rc = lib.vp_load_catalog(topo, len(topo), chan, len(chan), -1, ctypes.byref(h))     # host-only handle: no GPU needed
     if rc == 0:
         lib.vp_free_catalog.argtypes = [ctypes.c_void_p]
         lib.vp_free_catalog(h)
@@ -49,8 +49,10 @@ def _load(lib, topo, chan):
 def test_loader_validates_before_using_the_device(lib):
     cat = complete_catalog(tree_topology(1))
     topo, chan = cat.topology.blob(), cat.blob()
-    ok = _load(lib, topo, chan)
-    assert ok in (0, -4)                     # -4 (no CUDA device) only on a CPU-only box
+    assert _load(lib, topo, chan) == 0
+    for other in (complete_catalog(tree_topology(2, pcie_bw=64, nic_bw=50)), node_template_catalog(tree_topology(9, nic_bw=50)),
+                  complete_catalog(tree_topology(1, g=3)), crossbar_catalog(crossbar_topology(4))):
+        assert _load(lib, other.topology.blob(), other.blob()) == 0
     n_shapes, n_fam, nnz = struct.unpack_from("<3I", chan, 12)
     nnz_off = 24 + 4 * (n_shapes + 1)
     fam_off = nnz_off + 8 * nnz + 4 * (n_shapes + 1)
