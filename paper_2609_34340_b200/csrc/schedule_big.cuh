@@ -219,7 +219,9 @@ __global__ void __launch_bounds__(256) big_rank_kernel(const int* __restrict__ k
     order[before] = b;
 }
 
-// W = warps per (family, start) task: one lane per rank group, 32 W >= G.
+// W = warps per (family, start) task: one lane per rank group, 32 W >= G.  With at most sixteen groups two tasks share a
+// warp (W = 1, launched with two warps per CTA); with 17 to 32 groups a CTA is four warps, a task each; with more, W = 2
+// and a CTA is twelve warps, eight of which hold the four tasks of Step 2.
 #ifndef VP_BIG_W1_CTAS
 #define VP_BIG_W1_CTAS 2
 #endif
